@@ -1,0 +1,161 @@
+"""ctypes front end of the CPU oracle (oracle.c).
+
+TEST INFRASTRUCTURE ONLY.  Imported by tests, by the smoke check and by the
+benchmark's CPU-baseline leg; the product package never imports it.  Inputs and
+outputs are numpy arrays; fp32 entry points take float32, fp64 ones take float64.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SO = os.path.join(_HERE, "liboracle.so")
+_SRC = [os.path.join(_HERE, "oracle.c"), os.path.join(_HERE, "oracle_attn.inc")]
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile oracle.c into liboracle.so next to it (gcc, OpenMP, no fast-math)."""
+    stale = force or not os.path.exists(_SO) or any(
+        os.path.getmtime(s) > os.path.getmtime(_SO) for s in _SRC)
+    if stale:
+        tmp = _SO + f".tmp{os.getpid()}"
+        subprocess.check_call(["gcc", "-O3", "-march=native", "-fopenmp", "-shared", "-fPIC",
+                               "-std=c11", _SRC[0], "-o", tmp, "-lm"])
+        os.replace(tmp, _SO)
+    return _SO
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        _lib = ctypes.CDLL(_SO)
+        _lib.oracle_plan_num_blocks.restype = ctypes.c_int64
+    return _lib
+
+
+def _p(a):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _real(prec):
+    return {"f32": np.float32, "f64": np.float64}[prec]
+
+
+def _arr(x, dt):
+    return np.ascontiguousarray(np.asarray(x), dtype=dt)
+
+
+def _check(rc, what):
+    if rc != 0:
+        raise RuntimeError(f"{what} failed with code {rc}")
+
+
+def attn_fwd(q, k, v, cu, scale=None, prec="f32"):
+    """Full forward.  q [T,Hq,d], k/v [T,Hkv,d] -> (out [T,Hq,d], lse [Hq,T])."""
+    dt = _real(prec)
+    q, k, v = _arr(q, dt), _arr(k, dt), _arr(v, dt)
+    cu = _arr(cu, np.int32)
+    T, hq, d = q.shape
+    hkv = k.shape[1]
+    assert cu[-1] == T and k.shape == v.shape == (T, hkv, d)
+    scale = 1.0 / np.sqrt(d) if scale is None else scale
+    out = np.empty_like(q)
+    lse = np.empty((hq, T), dtype=dt)
+    fn = getattr(_load(), f"oracle_attn_fwd_{prec}")
+    _check(fn(_p(q), _p(k), _p(v), _p(cu), ctypes.c_int(len(cu) - 1), ctypes.c_int(hq),
+              ctypes.c_int(hkv), ctypes.c_int(d), ctypes.c_double(scale), _p(out), _p(lse)),
+           "oracle_attn_fwd")
+    return out, lse
+
+
+def attn_bwd(q, k, v, out, lse, dout, cu, scale=None, prec="f32"):
+    """Full backward from the given out/lse -> (dq, dk, dv)."""
+    dt = _real(prec)
+    q, k, v, out, lse, dout = (_arr(x, dt) for x in (q, k, v, out, lse, dout))
+    cu = _arr(cu, np.int32)
+    T, hq, d = q.shape
+    hkv = k.shape[1]
+    scale = 1.0 / np.sqrt(d) if scale is None else scale
+    dq, dk, dv = np.empty_like(q), np.empty_like(k), np.empty_like(v)
+    fn = getattr(_load(), f"oracle_attn_bwd_{prec}")
+    _check(fn(_p(q), _p(k), _p(v), _p(out), _p(lse), _p(dout), _p(cu), ctypes.c_int(len(cu) - 1),
+              ctypes.c_int(hq), ctypes.c_int(hkv), ctypes.c_int(d), ctypes.c_double(scale),
+              _p(dq), _p(dk), _p(dv)), "oracle_attn_bwd")
+    return dq, dk, dv
+
+
+def attn_fwd_rows(q, k, v, cu, rows, heads, scale=None, prec="f32"):
+    """Forward of selected (global row, q head) pairs -> (out_rows [nr,d], lse_rows [nr])."""
+    dt = _real(prec)
+    q, k, v = _arr(q, dt), _arr(k, dt), _arr(v, dt)
+    cu, rows, heads = _arr(cu, np.int32), _arr(rows, np.int64), _arr(heads, np.int32)
+    T, hq, d = q.shape
+    hkv = k.shape[1]
+    scale = 1.0 / np.sqrt(d) if scale is None else scale
+    out = np.empty((len(rows), d), dtype=dt)
+    lse = np.empty(len(rows), dtype=dt)
+    fn = getattr(_load(), f"oracle_attn_fwd_rows_{prec}")
+    _check(fn(_p(q), _p(k), _p(v), _p(cu), ctypes.c_int(len(cu) - 1), ctypes.c_int(hq),
+              ctypes.c_int(hkv), ctypes.c_int(d), ctypes.c_double(scale), ctypes.c_int(len(rows)),
+              _p(rows), _p(heads), _p(out), _p(lse)), "oracle_attn_fwd_rows")
+    return out, lse
+
+
+def attn_dq_rows(q, k, v, dout, cu, rows, heads, scale=None, prec="f32"):
+    """dQ of selected (global row, q head) pairs (O and LSE recomputed inside) -> [nr,d]."""
+    dt = _real(prec)
+    q, k, v, dout = (_arr(x, dt) for x in (q, k, v, dout))
+    cu, rows, heads = _arr(cu, np.int32), _arr(rows, np.int64), _arr(heads, np.int32)
+    T, hq, d = q.shape
+    hkv = k.shape[1]
+    scale = 1.0 / np.sqrt(d) if scale is None else scale
+    dq = np.empty((len(rows), d), dtype=dt)
+    fn = getattr(_load(), f"oracle_attn_dq_rows_{prec}")
+    _check(fn(_p(q), _p(k), _p(v), _p(dout), _p(cu), ctypes.c_int(len(cu) - 1), ctypes.c_int(hq),
+              ctypes.c_int(hkv), ctypes.c_int(d), ctypes.c_double(scale), ctypes.c_int(len(rows)),
+              _p(rows), _p(heads), _p(dq)), "oracle_attn_dq_rows")
+    return dq
+
+
+def attn_dkv_cols(q, k, v, out, lse, dout, cu, cols, kvheads, scale=None, prec="f32"):
+    """dK, dV of selected (global key column, kv head) pairs from the given out/lse."""
+    dt = _real(prec)
+    q, k, v, out, lse, dout = (_arr(x, dt) for x in (q, k, v, out, lse, dout))
+    cu, cols, kvheads = _arr(cu, np.int32), _arr(cols, np.int64), _arr(kvheads, np.int32)
+    T, hq, d = q.shape
+    hkv = k.shape[1]
+    scale = 1.0 / np.sqrt(d) if scale is None else scale
+    dk = np.empty((len(cols), d), dtype=dt)
+    dv = np.empty((len(cols), d), dtype=dt)
+    fn = getattr(_load(), f"oracle_attn_dkv_cols_{prec}")
+    _check(fn(_p(q), _p(k), _p(v), _p(out), _p(lse), _p(dout), _p(cu), ctypes.c_int(len(cu) - 1),
+              ctypes.c_int(hq), ctypes.c_int(hkv), ctypes.c_int(d), ctypes.c_double(scale),
+              ctypes.c_int(len(cols)), _p(cols), _p(kvheads), _p(dk), _p(dv)),
+           "oracle_attn_dkv_cols")
+    return dk, dv
+
+
+def plan(cu, n_heads, tile, n_workers, direction=0):
+    """SH-Tile plan -> dict(weight, order, cta_of_tile, cta_offsets, cta_tiles, loads)."""
+    cu = _arr(cu, np.int32)
+    lib = _load()
+    n = len(cu) - 1
+    nb = lib.oracle_plan_num_blocks(_p(cu), ctypes.c_int(n), ctypes.c_int(tile))
+    if nb < 0:
+        raise RuntimeError("oracle_plan: bad arguments")
+    nt = nb * n_heads
+    res = dict(weight=np.empty(nt, np.int64), order=np.empty(nt, np.int32),
+               cta_of_tile=np.empty(nt, np.int32), cta_offsets=np.empty(n_workers + 1, np.int32),
+               cta_tiles=np.empty(nt, np.int32), loads=np.empty(n_workers, np.int64))
+    _check(lib.oracle_plan(_p(cu), ctypes.c_int(n), ctypes.c_int(n_heads), ctypes.c_int(tile),
+                           ctypes.c_int(n_workers), ctypes.c_int(direction), _p(res["weight"]),
+                           _p(res["order"]), _p(res["cta_of_tile"]), _p(res["cta_offsets"]),
+                           _p(res["cta_tiles"]), _p(res["loads"])), "oracle_plan")
+    res["n_blocks"] = int(nb)
+    return res

@@ -1,0 +1,136 @@
+/* CPU oracle for pool attention and for the SH-Tile plan.
+ *
+ * TEST INFRASTRUCTURE ONLY: a plain, slow, obviously correct restatement of the
+ * definitions, used by the tests, the smoke check and the benchmark's CPU-baseline
+ * leg.  The CUDA library never calls it and shares no code with it.
+ *
+ * Attention: see oracle_attn.inc (instantiated for float and double).
+ * Plan: oracle_plan() below, following the paper's SH-Tile construction (Section
+ * 4.3.1, Eq. 5), tile weight (Eq. 6) and heaviest-first placement (Algorithm 2) with
+ * no communication term, step by step.
+ *
+ * Build: gcc -O3 -march=native -fopenmp -shared -fPIC oracle.c -o liboracle.so -lm
+ * (no -ffast-math).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define CAT_(a, b) a##b
+#define CAT(a, b) CAT_(a, b)
+
+#define REAL float
+#define REAL_EXP expf
+#define REAL_LOG logf
+#define FN(name) CAT(name, _f32)
+#include "oracle_attn.inc"
+#undef REAL
+#undef REAL_EXP
+#undef REAL_LOG
+#undef FN
+
+#define REAL double
+#define REAL_EXP exp
+#define REAL_LOG log
+#define FN(name) CAT(name, _f64)
+#include "oracle_attn.inc"
+#undef REAL
+#undef REAL_EXP
+#undef REAL_LOG
+#undef FN
+
+/* ------------------------------------------------------------------------------------
+ * Plan.
+ *
+ * Step 1 (Eq. 5): the pool's token axis [0, T) is cut at multiples of `tile` into
+ *   NB = ceil(T / tile) blocks (the last may be short; no cut at sample boundaries);
+ *   the heads are split in H shards; tile id t = b * H + h.
+ * Step 2 (Eq. 6): weight of block b = number of causal (query, key) pairs it covers.
+ *   Query-major (direction 0): block b holds queries; a query at sample-local position
+ *   p attends p + 1 keys, so for every sample j the block intersects, with local range
+ *   [a, e):  sum_{p=a}^{e-1} (p + 1).
+ *   Key-major (direction 1): block b holds keys; a key at local position p of a sample
+ *   of length len is attended by len - p queries:  sum_{p=a}^{e-1} (len - p).
+ *   The sums are written out as loops (the closed forms are what the tests pin them to).
+ *   All H shards of a block weigh the same (the common factor Hq/H is dropped).
+ * Step 3 (Algorithm 2, ordering): tiles sorted by decreasing weight, then tile id.
+ * Step 4 (Algorithm 2, placement with Delta_comm = 0): each tile in that order goes to
+ *   the worker with the smallest load, lowest index on ties; its load grows by the weight.
+ *   With no communication term both branches of the algorithm's choice reduce to this
+ *   rule and the soft cap drops out.
+ * Step 5: per-worker tile lists in assignment order, as CSR.
+ * ------------------------------------------------------------------------------------ */
+
+typedef struct { int64_t w; int32_t id; } tile_key;
+
+static int cmp_tiles(const void* a, const void* b) {
+    const tile_key* x = (const tile_key*)a;
+    const tile_key* y = (const tile_key*)b;
+    if (x->w != y->w) return x->w > y->w ? -1 : 1;
+    return x->id < y->id ? -1 : (x->id > y->id ? 1 : 0);
+}
+
+int64_t oracle_plan_num_blocks(const int32_t* cu, int n, int tile) {
+    if (!cu || n <= 0 || tile <= 0) return -1;
+    const int64_t T = cu[n];
+    return (T + tile - 1) / tile;
+}
+
+int oracle_plan(const int32_t* cu, int n, int H, int tile, int W, int direction,
+                int64_t* weight /*[NB*H]*/, int32_t* order /*[NB*H]*/, int32_t* cta_of_tile /*[NB*H]*/,
+                int32_t* cta_offsets /*[W+1]*/, int32_t* cta_tiles /*[NB*H]*/, int64_t* loads /*[W]*/) {
+    if (!cu || n <= 0 || H <= 0 || tile <= 0 || W <= 0) return -1;
+    if (cu[0] != 0) return -1;
+    for (int j = 0; j < n; ++j) if (cu[j + 1] < cu[j]) return -1;
+    const int64_t T = cu[n];
+    const int64_t NB = (T + tile - 1) / tile;
+    const int64_t NT = NB * H;
+
+    /* steps 1-2 */
+    for (int64_t b = 0; b < NB; ++b) {
+        const int64_t q0 = b * tile, q1 = (b + 1) * tile < T ? (b + 1) * tile : T;
+        int64_t w = 0;
+        for (int j = 0; j < n; ++j) {
+            const int64_t s = cu[j], t = cu[j + 1], len = t - s;
+            const int64_t lo = q0 > s ? q0 : s, hi = q1 < t ? q1 : t;
+            for (int64_t g = lo; g < hi; ++g) {
+                const int64_t p = g - s;
+                w += direction == 0 ? (p + 1) : (len - p);
+            }
+        }
+        for (int h = 0; h < H; ++h) weight[b * H + h] = w;
+    }
+
+    /* step 3 */
+    tile_key* keys = (tile_key*)malloc(sizeof(tile_key) * (size_t)NT);
+    if (!keys) return -2;
+    for (int64_t t = 0; t < NT; ++t) { keys[t].w = weight[t]; keys[t].id = (int32_t)t; }
+    qsort(keys, (size_t)NT, sizeof(tile_key), cmp_tiles);
+    for (int64_t t = 0; t < NT; ++t) order[t] = keys[t].id;
+    free(keys);
+
+    /* step 4 */
+    for (int r = 0; r < W; ++r) loads[r] = 0;
+    for (int64_t x = 0; x < NT; ++x) {
+        const int32_t t = order[x];
+        int best = 0;
+        for (int r = 1; r < W; ++r) if (loads[r] < loads[best]) best = r;
+        cta_of_tile[t] = best;
+        loads[best] += weight[t];
+    }
+
+    /* step 5 */
+    for (int r = 0; r <= W; ++r) cta_offsets[r] = 0;
+    for (int64_t t = 0; t < NT; ++t) cta_offsets[cta_of_tile[t] + 1] += 1;
+    for (int r = 0; r < W; ++r) cta_offsets[r + 1] += cta_offsets[r];
+    int32_t* fill = (int32_t*)calloc((size_t)W, sizeof(int32_t));
+    if (!fill) return -2;
+    for (int64_t x = 0; x < NT; ++x) {
+        const int32_t t = order[x];
+        const int r = cta_of_tile[t];
+        cta_tiles[cta_offsets[r] + fill[r]++] = t;
+    }
+    free(fill);
+    return 0;
+}
