@@ -1,0 +1,163 @@
+/* libra.h — C ABI of the B200 pool-attention library (liblibra.so).
+ *
+ * The library computes causal, sample-masked ("document-masked") attention forward and
+ * backward over a pool of packed sequences on one GPU, with the work cut into
+ * sequence-block x head-shard tiles (SH-Tiles) that are weighted by the causal
+ * query-key pairs they cover and placed heaviest-first on persistent CTAs.
+ *
+ * Conventions for every entry point
+ *   - returns 0 on success, a negative LIBRA_ERR_* code otherwise; never throws, aborts
+ *     or prints;
+ *   - pointers named *_dev are DEVICE pointers owned by the caller, pointers named
+ *     *_host are HOST pointers owned by the caller; nothing is retained after the call
+ *     returns except inside a libra_plan_t;
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream);
+ *     work is enqueued on it and the call returns without synchronising unless stated;
+ *   - tensors are contiguous bf16 in the packed "thd" layout: q, out, dout, dq are
+ *     [T, Hq, d]; k, v, dk, dv are [T, Hkv, d]; lse is fp32 [Hq, T]; T = cu_seqlens[n];
+ *     query head h reads kv head h / (Hq / Hkv);
+ *   - cu_seqlens is int32 [n_samples + 1], starts at 0, non-decreasing (repeated offsets
+ *     = empty samples are allowed), ends at T.
+ *
+ * Citations name the paper's section, equation or algorithm that defines the operation.
+ */
+#ifndef LIBRA_H_
+#define LIBRA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define LIBRA_OK                 0
+#define LIBRA_ERR_INVALID_ARG   (-1)  /* null pointer, non-positive size, H does not divide Hq, ... */
+#define LIBRA_ERR_UNSUPPORTED   (-2)  /* head_dim not in {64,128}, tile size the kernels cannot run */
+#define LIBRA_ERR_PLAN_MISMATCH (-3)  /* plan was built for another T / head count / direction      */
+#define LIBRA_ERR_CUDA          (-4)  /* a CUDA runtime or driver call failed                        */
+#define LIBRA_ERR_OVERFLOW      (-5)  /* tile ids or loads would not fit their integer types         */
+#define LIBRA_ERR_TIMEOUT       (-6)  /* a bounded device-side wait gave up (reported by libra_status)*/
+#define LIBRA_ERR_BAD_SEQLENS   (-7)  /* cu_seqlens failed the device-side check                      */
+#define LIBRA_ERR_NO_DEVICE     (-8)  /* no CUDA device / not an sm_100 device                        */
+
+#define LIBRA_DIR_Q   1   /* query-major tiles (forward)  */
+#define LIBRA_DIR_KV  2   /* key-major tiles   (backward) */
+
+typedef struct libra_plan libra_plan_t;   /* opaque, library-owned */
+
+typedef struct {
+    int     n_workers;     /* persistent CTAs to place onto; 0 = one per SM of the current device */
+    int     directions;    /* LIBRA_DIR_Q | LIBRA_DIR_KV; 0 = both                                  */
+    int     tile_kv;       /* key-major block size in tokens; 0 = 128                              */
+    int     n_heads_kv;    /* key-major head shards; 0 = same as n_heads                           */
+    int64_t total_tokens;  /* T if the caller knows it; 0 = read cu_seqlens[n] back (one 4-byte
+                              synchronous copy on `stream`)                                         */
+} libra_plan_opts;
+
+typedef struct {
+    int64_t total_tokens;  /* T */
+    int     n_samples;     /* n */
+    int     hq, hkv;       /* query / kv heads, hkv divides hq */
+    int     head_dim;      /* 64 or 128 */
+    float   softmax_scale; /* 0 = 1/sqrt(head_dim) */
+} libra_dims;
+
+/* ---- planning ------------------------------------------------------------------------
+ * SH-Tile construction (Section 4.3.1, Eq. 5), tile weights (Eq. 6) and heaviest-first
+ * placement (Algorithm 2 with the communication term identically zero, which makes both
+ * of its branches "least-loaded worker, lowest index on ties" and removes the soft cap).
+ *
+ *   blocks : the token axis [0, T) cut at multiples of the tile size (last block may be
+ *            short; no cuts at sample boundaries); NB = ceil(T / tile)
+ *   tiles  : id t = b * H + h for block b and head shard h (H = n_heads shards)
+ *   weight : LIBRA_DIR_Q  - block b holds queries: sum over its tokens of (p + 1), p the
+ *                           token's position inside its sample (= keys it attends)
+ *            LIBRA_DIR_KV - block b holds keys: sum over its tokens of (len - p)
+ *                           (= queries that attend the key); same for every h
+ *   order  : tiles by decreasing weight, then increasing id
+ *   place  : each tile in that order to the worker with the smallest load so far
+ *   lists  : per-worker tile lists in placement order, CSR (cta_offsets, cta_tiles)
+ *
+ * All planning runs in device kernels on `stream`; results stay on the device inside the
+ * plan and are reused by every forward and backward call on the same layout (the paper
+ * builds one plan per pool and reuses it across layers and for the backward pass,
+ * Sections 4.1 and 4.3.3).  cu_seqlens_dev is read during the call only.
+ * Errors: INVALID_ARG (null, n_samples <= 0, n_heads <= 0, tile_q <= 0), OVERFLOW
+ * (NB * H >= 2^31), CUDA; a malformed cu_seqlens is detected on the device and reported
+ * by libra_plan_status as BAD_SEQLENS.
+ */
+int libra_plan_tiles(const int32_t* cu_seqlens_dev, int n_samples, int n_heads, int tile_q,
+                     const libra_plan_opts* opts /* nullable */, void* stream,
+                     libra_plan_t** plan_out);
+
+/* Sizes of a plan direction (host values, no synchronisation). */
+int libra_plan_info(const libra_plan_t* plan, int direction, int64_t* n_tiles, int* n_workers,
+                    int64_t* n_blocks, int* tile, int* n_heads);
+
+/* Synchronises `stream` of the plan's creation and returns the device status word:
+ * LIBRA_OK, LIBRA_ERR_BAD_SEQLENS or LIBRA_ERR_TIMEOUT. */
+int libra_plan_status(const libra_plan_t* plan);
+
+/* Copies one direction of the plan to caller-allocated HOST arrays (any may be NULL):
+ * weight int64[n_tiles], order int32[n_tiles], cta_of_tile int32[n_tiles],
+ * cta_offsets int32[n_workers+1], cta_tiles int32[n_tiles], loads int64[n_workers].
+ * Synchronises the plan's stream. */
+int libra_plan_export(const libra_plan_t* plan, int direction, int64_t* weight_host,
+                      int32_t* order_host, int32_t* cta_of_tile_host, int32_t* cta_offsets_host,
+                      int32_t* cta_tiles_host, int64_t* loads_host);
+
+/* Frees the plan's device and host memory (synchronises the device first). NULL is OK. */
+int libra_plan_destroy(libra_plan_t* plan);
+
+/* ---- attention -----------------------------------------------------------------------
+ * Forward (Section 2.2, Eq. 1 applied inside each sample under the block-diagonal causal
+ * mask of Section 2.3):  for row i of a sample starting at s, with keys s..i,
+ *     out_i = sum_k softmax_k(scale * <q_i, k_k>) v_k,   lse_i = ln sum_k exp(scale * <q_i, k_k>)
+ * bf16 inputs, fp32 accumulation and softmax, bf16 out (round to nearest even), fp32 lse
+ * (natural log).  One persistent kernel walks the plan's query-major tile lists.
+ * Requires a plan with LIBRA_DIR_Q, tile_q == 256 and n_heads dividing hq.
+ * Errors: INVALID_ARG, UNSUPPORTED, PLAN_MISMATCH (plan T != dims->total_tokens), CUDA.
+ */
+int libra_attn_pool_fwd(const void* q_dev, const void* k_dev, const void* v_dev,
+                        const int32_t* cu_seqlens_dev, const libra_plan_t* plan,
+                        void* out_dev, float* lse_dev, const libra_dims* dims, void* stream);
+
+/* Bytes of caller-owned device scratch libra_attn_pool_bwd needs (fp32 dQ accumulator and
+ * the row statistic D); 0 on bad arguments. */
+size_t libra_attn_pool_bwd_workspace_bytes(const libra_plan_t* plan, const libra_dims* dims);
+
+/* Backward: the gradient of <dout, out> with respect to q, k, v, given out and lse from the
+ * forward call (Section 4.3.3 states that the backward pass reuses the forward plan's
+ * structure; the arithmetic is the derivative of Eq. 1):
+ *     P_ik = exp(scale <q_i,k_k> - lse_i), D_i = <dout_i, out_i>, dS_ik = P_ik (<dout_i,v_k> - D_i)
+ *     dq_i = scale sum_k dS_ik k_k;  dk_k = scale sum_{h,i} dS_ik q_i;  dv_k = sum_{h,i} P_ik dout_i
+ * (sums over the query heads h of the kv head's group and the rows i >= k of the sample).
+ * Walks the plan's key-major tile lists; needs LIBRA_DIR_KV with tile_kv == 128 and
+ * n_heads_kv == hkv.  `workspace_dev` must hold libra_attn_pool_bwd_workspace_bytes bytes,
+ * 256-byte aligned; it is fully initialised inside the call.  dq accumulates through fp32
+ * atomics, so its low bits may differ from run to run.
+ */
+int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const void* v_dev,
+                        const void* out_dev, const float* lse_dev, const void* dout_dev,
+                        const int32_t* cu_seqlens_dev, const libra_plan_t* plan,
+                        void* dq_dev, void* dk_dev, void* dv_dev, void* workspace_dev,
+                        const libra_dims* dims, void* stream);
+
+/* ---- instrumentation -------------------------------------------------------------------
+ * Per-CTA busy time of the most recent forward (which = LIBRA_DIR_Q) or backward
+ * (LIBRA_DIR_KV) call that used this plan: nanoseconds between the CTA picking up its
+ * first tile and finishing its last, read with the GPU's global timer.  Copies n_workers
+ * values to ns_host and synchronises the device.  Also returns the kernel status
+ * (LIBRA_ERR_TIMEOUT if a bounded wait gave up). */
+int libra_busy_times(const libra_plan_t* plan, int which, uint64_t* ns_host);
+
+/* Number of kernels this library has launched in the calling process (for accounting). */
+int64_t libra_launch_count(void);
+
+const char* libra_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LIBRA_H_ */

@@ -1,0 +1,174 @@
+"""ctypes binding of liblibra.so: the same entry points as include/libra.h, argument
+marshalling only.  Tensors are torch CUDA tensors (device memory and streams come from
+torch); every computation runs in the library's kernels.
+
+Importing this module loads the library and raises if it has not been built — there is
+no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SO = os.path.join(_HERE, "liblibra.so")
+if not os.path.exists(_SO):
+    raise ImportError(f"{_SO} is missing: run `python -m paper_2607_23250_b200.build` (needs nvcc)")
+_lib = ctypes.CDLL(_SO)
+
+LIBRA_DIR_Q, LIBRA_DIR_KV = 1, 2
+ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_PLAN_MISMATCH, ERR_CUDA = -1, -2, -3, -4
+ERR_OVERFLOW, ERR_TIMEOUT, ERR_BAD_SEQLENS, ERR_NO_DEVICE = -5, -6, -7, -8
+
+EXPORTS = ["libra_plan_tiles", "libra_plan_info", "libra_plan_status", "libra_plan_export",
+           "libra_plan_destroy", "libra_attn_pool_fwd", "libra_attn_pool_bwd_workspace_bytes",
+           "libra_attn_pool_bwd", "libra_busy_times", "libra_launch_count", "libra_strerror"]
+
+
+class PlanOpts(ctypes.Structure):
+    _fields_ = [("n_workers", ctypes.c_int), ("directions", ctypes.c_int), ("tile_kv", ctypes.c_int),
+                ("n_heads_kv", ctypes.c_int), ("total_tokens", ctypes.c_int64)]
+
+
+class Dims(ctypes.Structure):
+    _fields_ = [("total_tokens", ctypes.c_int64), ("n_samples", ctypes.c_int), ("hq", ctypes.c_int),
+                ("hkv", ctypes.c_int), ("head_dim", ctypes.c_int), ("softmax_scale", ctypes.c_float)]
+
+
+_lib.libra_strerror.restype = ctypes.c_char_p
+_lib.libra_launch_count.restype = ctypes.c_int64
+_lib.libra_attn_pool_bwd_workspace_bytes.restype = ctypes.c_size_t
+_vp = ctypes.c_void_p
+
+
+class LibraError(RuntimeError):
+    def __init__(self, code, what):
+        self.code = code
+        super().__init__(f"{what}: {_lib.libra_strerror(code).decode()} ({code})")
+
+
+def _check(code, what):
+    if code != 0:
+        raise LibraError(code, what)
+
+
+def _ptr(t):
+    return _vp(t.data_ptr()) if t is not None else _vp(0)
+
+
+def _np(a):
+    return a.ctypes.data_as(_vp) if a is not None else _vp(0)
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return _vp(s.cuda_stream)
+
+
+def launch_count() -> int:
+    return int(_lib.libra_launch_count())
+
+
+class Plan:
+    """Owner of a libra_plan_t."""
+
+    def __init__(self, handle, cu_seqlens):
+        self._h = handle
+        self.cu_seqlens = cu_seqlens  # kept alive for the attention calls
+
+    def info(self, direction=LIBRA_DIR_Q):
+        nt, nb = ctypes.c_int64(), ctypes.c_int64()
+        w, tile, h = ctypes.c_int(), ctypes.c_int(), ctypes.c_int()
+        _check(_lib.libra_plan_info(self._h, direction, ctypes.byref(nt), ctypes.byref(w), ctypes.byref(nb),
+                                    ctypes.byref(tile), ctypes.byref(h)), "libra_plan_info")
+        return dict(n_tiles=nt.value, n_workers=w.value, n_blocks=nb.value, tile=tile.value, n_heads=h.value)
+
+    def status(self) -> int:
+        return int(_lib.libra_plan_status(self._h))
+
+    def export(self, direction=LIBRA_DIR_Q):
+        i = self.info(direction)
+        nt, w = i["n_tiles"], i["n_workers"]
+        res = dict(weight=np.empty(nt, np.int64), order=np.empty(nt, np.int32), cta_of_tile=np.empty(nt, np.int32),
+                   cta_offsets=np.empty(w + 1, np.int32), cta_tiles=np.empty(nt, np.int32),
+                   loads=np.empty(w, np.int64))
+        _check(_lib.libra_plan_export(self._h, direction, _np(res["weight"]), _np(res["order"]),
+                                      _np(res["cta_of_tile"]), _np(res["cta_offsets"]), _np(res["cta_tiles"]),
+                                      _np(res["loads"])), "libra_plan_export")
+        res["n_blocks"] = i["n_blocks"]
+        return res
+
+    def busy_times(self, which=LIBRA_DIR_Q):
+        w = self.info(which)["n_workers"]
+        out = np.zeros(w, np.uint64)
+        _check(_lib.libra_busy_times(self._h, which, _np(out)), "libra_busy_times")
+        return out
+
+    def destroy(self):
+        if self._h:
+            _lib.libra_plan_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+
+def libra_plan_tiles(cu_seqlens: torch.Tensor, n_heads: int, tile_q: int, n_workers: int = 0,
+                     directions: int = 0, tile_kv: int = 0, n_heads_kv: int = 0, total_tokens: int = 0,
+                     stream=None) -> Plan:
+    assert cu_seqlens.is_cuda and cu_seqlens.dtype == torch.int32 and cu_seqlens.is_contiguous()
+    opts = PlanOpts(n_workers, directions, tile_kv, n_heads_kv, total_tokens)
+    h = _vp()
+    _check(_lib.libra_plan_tiles(_ptr(cu_seqlens), ctypes.c_int(cu_seqlens.numel() - 1), ctypes.c_int(n_heads),
+                                 ctypes.c_int(tile_q), ctypes.byref(opts), _stream(stream), ctypes.byref(h)),
+           "libra_plan_tiles")
+    return Plan(h, cu_seqlens)
+
+
+def _dims(q, k, plan, scale):
+    T, hq, d = q.shape
+    return Dims(T, plan.cu_seqlens.numel() - 1, hq, k.shape[1], d, 0.0 if scale is None else float(scale))
+
+
+def _chk(*ts):
+    for t in ts:
+        assert t.is_cuda and t.is_contiguous(), "expected contiguous CUDA tensors"
+
+
+def libra_attn_pool_fwd(q, k, v, plan: Plan, out=None, lse=None, scale=None, stream=None):
+    """out [T,Hq,d] bf16, lse [Hq,T] fp32 (allocated with torch when not given)."""
+    _chk(q, k, v)
+    assert q.dtype == k.dtype == v.dtype == torch.bfloat16
+    T, hq, d = q.shape
+    out = torch.empty_like(q) if out is None else out
+    lse = torch.empty((hq, T), dtype=torch.float32, device=q.device) if lse is None else lse
+    dims = _dims(q, k, plan, scale)
+    _check(_lib.libra_attn_pool_fwd(_ptr(q), _ptr(k), _ptr(v), _ptr(plan.cu_seqlens), plan._h, _ptr(out), _ptr(lse),
+                                    ctypes.byref(dims), _stream(stream)), "libra_attn_pool_fwd")
+    return out, lse
+
+
+def libra_attn_pool_bwd_workspace_bytes(plan: Plan, q, k) -> int:
+    dims = _dims(q, k, plan, None)
+    return int(_lib.libra_attn_pool_bwd_workspace_bytes(plan._h, ctypes.byref(dims)))
+
+
+def libra_attn_pool_bwd(q, k, v, out, lse, dout, plan: Plan, dq=None, dk=None, dv=None, workspace=None,
+                        scale=None, stream=None):
+    _chk(q, k, v, out, lse, dout)
+    dq = torch.empty_like(q) if dq is None else dq
+    dk = torch.empty_like(k) if dk is None else dk
+    dv = torch.empty_like(v) if dv is None else dv
+    if workspace is None:
+        workspace = torch.empty(libra_attn_pool_bwd_workspace_bytes(plan, q, k), dtype=torch.uint8, device=q.device)
+    dims = _dims(q, k, plan, scale)
+    _check(_lib.libra_attn_pool_bwd(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), _ptr(dout),
+                                    _ptr(plan.cu_seqlens), plan._h, _ptr(dq), _ptr(dk), _ptr(dv), _ptr(workspace),
+                                    ctypes.byref(dims), _stream(stream)), "libra_attn_pool_bwd")
+    return dq, dk, dv

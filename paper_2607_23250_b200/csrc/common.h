@@ -1,0 +1,54 @@
+// Host-side structures shared by the library's translation units.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <atomic>
+
+#include "../../include/libra.h"
+
+namespace libra {
+
+// One direction (query-major or key-major) of a plan.  All d_* pointers are device memory.
+struct PlanDir {
+    int enabled = 0;
+    int tile = 0;        // tokens per block
+    int H = 0;           // head shards
+    int W = 0;           // workers (persistent CTAs)
+    int64_t NB = 0;      // blocks
+    int64_t NT = 0;      // tiles = NB * H
+    int64_t* d_weight_blk = nullptr;   // [NB]  weight of block b (every shard of it)
+    int32_t* d_blk_order = nullptr;    // [NB]  blocks by (weight desc, index asc)
+    int32_t* d_cta_of_tile = nullptr;  // [NT]
+    int32_t* d_pos = nullptr;          // [NT]  position of the tile in its worker's list
+    int32_t* d_cta_offsets = nullptr;  // [W+1]
+    int32_t* d_cta_tiles = nullptr;    // [NT]
+    int64_t* d_loads = nullptr;        // [W]
+    uint64_t* d_busy = nullptr;        // [2*W] (start, end) global-timer stamps of the last run
+};
+
+}  // namespace libra
+
+struct libra_plan {
+    int64_t T = 0;
+    int n = 0;
+    int device = 0;
+    int sm_count = 0;
+    cudaStream_t stream = nullptr;
+    int32_t* d_tok_start = nullptr;  // [T] first token of the sample that holds token t
+    int32_t* d_tok_end = nullptr;    // [T] one past the last token of that sample
+    int* d_status = nullptr;         // [4] word 0: plan status; word 1: fwd; word 2: bwd
+    libra::PlanDir dir[2];           // 0 = query-major, 1 = key-major
+};
+
+namespace libra {
+extern std::atomic<int64_t> g_launches;
+inline void count_launch(int n = 1) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+}  // namespace libra
+
+namespace libra {
+// bf16 [T, H, d] tensor viewed as (d, H, T); TMA box = 64 columns x 1 head x box_rows tokens,
+// 128-byte swizzle, out-of-range rows read as zero.  Defined in attn_fwd.cu.
+int make_thd_map(CUtensorMap* m, const void* base, int64_t T, int H, int d, int box_rows);
+}  // namespace libra

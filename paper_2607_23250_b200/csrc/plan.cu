@@ -1,0 +1,380 @@
+// Device tile planner: SH-Tile construction (Section 4.3.1, Eq. 5), tile weights (Eq. 6) and
+// heaviest-first placement (Algorithm 2 with a zero communication term) as CUDA kernels.
+//
+// Integer work only; every result must equal the step-by-step definition bit for bit.
+#include <stdio.h>
+
+#include <new>
+
+#include "common.h"
+
+namespace libra {
+
+std::atomic<int64_t> g_launches{0};
+
+// ---- kernels --------------------------------------------------------------------------------
+
+// cu_seqlens checks: starts at 0, non-decreasing, ends at T.
+__global__ void k_validate(const int32_t* __restrict__ cu, int n, int64_t T, int* status) {
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j > n) return;
+    bool bad = false;
+    if (j == 0 && cu[0] != 0) bad = true;
+    if (j == n && cu[n] != T) bad = true;
+    if (j < n && cu[j + 1] < cu[j]) bad = true;
+    if (bad) atomicExch(status, LIBRA_ERR_BAD_SEQLENS);
+}
+
+// For every token: the bounds [start, end) of the sample that holds it.
+// upper_bound keeps every index inside [0, n] whatever cu contains.
+__global__ void k_token_bounds(const int32_t* __restrict__ cu, int n, int64_t T, int32_t* __restrict__ tok_start,
+                               int32_t* __restrict__ tok_end) {
+    const int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (t >= T) return;
+    int lo = 0, hi = n;  // find the last j in [0, n) with cu[j] <= t
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (cu[mid] <= t) lo = mid; else hi = mid;
+    }
+    tok_start[t] = cu[lo];
+    tok_end[t] = cu[lo + 1];
+}
+
+// Weight of block b (Eq. 6): a token at position p of a sample of length len contributes
+// p + 1 pairs as a query (keys 0..p) and len - p pairs as a key (queries p..len-1).
+__global__ void k_block_weights(const int32_t* __restrict__ tok_start, const int32_t* __restrict__ tok_end,
+                                int64_t T, int tile, int64_t NB, int key_major, int64_t* __restrict__ weight_blk) {
+    const int64_t b = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (b >= NB) return;
+    const int64_t t0 = b * tile;
+    const int64_t t1 = (t0 + tile < T) ? t0 + tile : T;
+    int64_t w = 0;
+    for (int64_t t = t0; t < t1; ++t) w += key_major ? (int64_t)tok_end[t] - t : t - (int64_t)tok_start[t] + 1;
+    weight_blk[b] = w;
+}
+
+// Order of Algorithm 2: decreasing weight, then increasing id.  All H shards of a block weigh
+// the same and their ids b*H+h are consecutive, so ordering the blocks orders the tiles.
+// rank(b) = number of blocks that precede b; one thread per block, O(NB) each.
+__global__ void k_rank_blocks(const int64_t* __restrict__ weight_blk, int64_t NB, int32_t* __restrict__ blk_order) {
+    __shared__ int64_t sw[256];
+    const int64_t b = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    const int64_t wb = b < NB ? weight_blk[b] : 0;
+    int64_t rank = 0;
+    for (int64_t base = 0; base < NB; base += 256) {
+        const int64_t o = base + threadIdx.x;
+        sw[threadIdx.x] = o < NB ? weight_blk[o] : -1;
+        __syncthreads();
+        const int lim = (int)((NB - base < 256) ? NB - base : 256);
+        for (int i = 0; i < lim; ++i) {
+            const int64_t w = sw[i];
+            rank += (w > wb) || (w == wb && base + i < b);
+        }
+        __syncthreads();
+    }
+    if (b < NB) blk_order[rank] = (int32_t)b;
+}
+
+// Sequential placement by one warp.  Worker r's load lives in lane r % 32, register r / 32.
+// Per tile: every lane finds its lightest worker, a shuffle tree finds the warp's
+// (load, index) minimum, the owning lane adds the weight.  Ties go to the lowest index
+// because the comparison is lexicographic on (load, index).
+template <int PER>
+__global__ void __launch_bounds__(32) k_place(const int64_t* __restrict__ weight_blk,
+                                              const int32_t* __restrict__ blk_order, int64_t NT, int H, int W,
+                                              int32_t* __restrict__ cta_of_tile, int32_t* __restrict__ pos,
+                                              int32_t* __restrict__ cta_offsets, int64_t* __restrict__ loads) {
+    const int lane = threadIdx.x;
+    int64_t load[PER];
+    int32_t cnt[PER];
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+        load[i] = (lane + 32 * i < W) ? 0 : INT64_MAX;
+        cnt[i] = 0;
+    }
+    for (int64_t x0 = 0; x0 < NT; x0 += 32) {
+        // each lane fetches one upcoming tile, then they are broadcast one by one
+        const int64_t xl = x0 + lane;
+        int64_t w_l = 0;
+        int32_t t_l = 0;
+        if (xl < NT) {
+            const int32_t blk = blk_order[xl / H];
+            w_l = weight_blk[blk];
+            t_l = (int32_t)((int64_t)blk * H + xl % H);
+        }
+        const int lim = (int)((NT - x0 < 32) ? NT - x0 : 32);
+        for (int i = 0; i < lim; ++i) {
+            const int64_t w = __shfl_sync(0xffffffffu, w_l, i);
+            const int32_t t = __shfl_sync(0xffffffffu, t_l, i);
+            int64_t best = load[0];
+            int32_t bidx = lane;
+#pragma unroll
+            for (int k = 1; k < PER; ++k) {
+                if (load[k] < best) { best = load[k]; bidx = lane + 32 * k; }
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                const int64_t ob = __shfl_xor_sync(0xffffffffu, best, off);
+                const int32_t oi = __shfl_xor_sync(0xffffffffu, bidx, off);
+                if (ob < best || (ob == best && oi < bidx)) { best = ob; bidx = oi; }
+            }
+            int32_t my_pos = 0;
+            if ((bidx & 31) == lane) {
+#pragma unroll
+                for (int k = 0; k < PER; ++k) {
+                    if (k == (bidx >> 5)) { load[k] += w; my_pos = cnt[k]++; }
+                }
+                cta_of_tile[t] = bidx;
+                pos[t] = my_pos;
+            }
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < PER; ++i) {
+        const int r = lane + 32 * i;
+        if (r < W) { loads[r] = load[i]; cta_offsets[r + 1] = cnt[i]; }
+    }
+    __syncwarp();
+    if (lane == 0) {  // counts -> offsets
+        cta_offsets[0] = 0;
+        int32_t run = 0;
+        for (int r = 0; r < W; ++r) { run += cta_offsets[r + 1]; cta_offsets[r + 1] = run; }
+    }
+}
+
+__global__ void k_scatter_lists(const int32_t* __restrict__ cta_of_tile, const int32_t* __restrict__ pos,
+                                const int32_t* __restrict__ cta_offsets, int64_t NT, int32_t* __restrict__ cta_tiles) {
+    const int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (t >= NT) return;
+    cta_tiles[cta_offsets[cta_of_tile[t]] + pos[t]] = (int32_t)t;
+}
+
+// Expanders used by libra_plan_export.
+__global__ void k_expand_weight(const int64_t* __restrict__ weight_blk, int64_t NT, int H, int64_t* __restrict__ out) {
+    const int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (t < NT) out[t] = weight_blk[t / H];
+}
+__global__ void k_expand_order(const int32_t* __restrict__ blk_order, int64_t NT, int H, int32_t* __restrict__ out) {
+    const int64_t x = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (x < NT) out[x] = (int32_t)((int64_t)blk_order[x / H] * H + x % H);
+}
+
+// ---- host ---------------------------------------------------------------------------------
+
+static inline unsigned grid_for(int64_t n, int block) { return (unsigned)((n + block - 1) / block); }
+
+static void free_dir(PlanDir& d) {
+    cudaFree(d.d_weight_blk); cudaFree(d.d_blk_order); cudaFree(d.d_cta_of_tile); cudaFree(d.d_pos);
+    cudaFree(d.d_cta_offsets); cudaFree(d.d_cta_tiles); cudaFree(d.d_loads); cudaFree(d.d_busy);
+    d = PlanDir();
+}
+
+static int build_dir(libra_plan* p, PlanDir& d, int key_major) {
+    const int64_t T = p->T;
+    d.NB = (T + d.tile - 1) / d.tile;
+    if (d.NB * (int64_t)d.H >= (int64_t)INT32_MAX) return LIBRA_ERR_OVERFLOW;
+    if (d.NB > 65536) return LIBRA_ERR_UNSUPPORTED;  // the rank sort is quadratic in blocks
+    if (d.W > 1024) return LIBRA_ERR_UNSUPPORTED;
+    d.NT = d.NB * d.H;
+    cudaError_t e = cudaSuccess;
+    auto A = [&](void** ptr, size_t bytes) { if (e == cudaSuccess) e = cudaMalloc(ptr, bytes ? bytes : 1); };
+    A((void**)&d.d_weight_blk, sizeof(int64_t) * d.NB);
+    A((void**)&d.d_blk_order, sizeof(int32_t) * d.NB);
+    A((void**)&d.d_cta_of_tile, sizeof(int32_t) * d.NT);
+    A((void**)&d.d_pos, sizeof(int32_t) * d.NT);
+    A((void**)&d.d_cta_offsets, sizeof(int32_t) * (d.W + 1));
+    A((void**)&d.d_cta_tiles, sizeof(int32_t) * d.NT);
+    A((void**)&d.d_loads, sizeof(int64_t) * d.W);
+    A((void**)&d.d_busy, sizeof(uint64_t) * 2 * d.W);
+    if (e != cudaSuccess) return LIBRA_ERR_CUDA;
+    cudaStream_t s = p->stream;
+    cudaMemsetAsync(d.d_busy, 0, sizeof(uint64_t) * 2 * d.W, s);
+    k_block_weights<<<grid_for(d.NB, 128), 128, 0, s>>>(p->d_tok_start, p->d_tok_end, T, d.tile, d.NB, key_major,
+                                                        d.d_weight_blk);
+    k_rank_blocks<<<grid_for(d.NB, 256), 256, 0, s>>>(d.d_weight_blk, d.NB, d.d_blk_order);
+    if (d.W <= 160)
+        k_place<5><<<1, 32, 0, s>>>(d.d_weight_blk, d.d_blk_order, d.NT, d.H, d.W, d.d_cta_of_tile, d.d_pos,
+                                    d.d_cta_offsets, d.d_loads);
+    else if (d.W <= 320)
+        k_place<10><<<1, 32, 0, s>>>(d.d_weight_blk, d.d_blk_order, d.NT, d.H, d.W, d.d_cta_of_tile, d.d_pos,
+                                     d.d_cta_offsets, d.d_loads);
+    else
+        k_place<32><<<1, 32, 0, s>>>(d.d_weight_blk, d.d_blk_order, d.NT, d.H, d.W, d.d_cta_of_tile, d.d_pos,
+                                     d.d_cta_offsets, d.d_loads);
+    k_scatter_lists<<<grid_for(d.NT, 256), 256, 0, s>>>(d.d_cta_of_tile, d.d_pos, d.d_cta_offsets, d.NT,
+                                                        d.d_cta_tiles);
+    count_launch(4);
+    d.enabled = 1;
+    return cudaGetLastError() == cudaSuccess ? LIBRA_OK : LIBRA_ERR_CUDA;
+}
+
+}  // namespace libra
+
+using namespace libra;
+
+extern "C" int libra_plan_tiles(const int32_t* cu_seqlens_dev, int n_samples, int n_heads, int tile_q,
+                                const libra_plan_opts* opts, void* stream, libra_plan_t** plan_out) {
+    if (!cu_seqlens_dev || !plan_out || n_samples <= 0 || n_heads <= 0 || tile_q <= 0) return LIBRA_ERR_INVALID_ARG;
+    *plan_out = nullptr;
+    libra_plan_opts o = {0, 0, 0, 0, 0};
+    if (opts) o = *opts;
+    if (o.n_workers < 0 || o.tile_kv < 0 || o.n_heads_kv < 0 || o.total_tokens < 0) return LIBRA_ERR_INVALID_ARG;
+    if (o.directions & ~(LIBRA_DIR_Q | LIBRA_DIR_KV)) return LIBRA_ERR_INVALID_ARG;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return LIBRA_ERR_NO_DEVICE;
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return LIBRA_ERR_CUDA;
+    cudaStream_t s = (cudaStream_t)stream;
+    int64_t T = o.total_tokens;
+    if (T == 0) {
+        int32_t last = 0;
+        if (cudaMemcpyAsync(&last, cu_seqlens_dev + n_samples, sizeof(int32_t), cudaMemcpyDeviceToHost, s) !=
+                cudaSuccess ||
+            cudaStreamSynchronize(s) != cudaSuccess)
+            return LIBRA_ERR_CUDA;
+        T = last;
+    }
+    if (T <= 0 || T >= (int64_t)INT32_MAX) return LIBRA_ERR_INVALID_ARG;
+
+    libra_plan* p = new (std::nothrow) libra_plan();
+    if (!p) return LIBRA_ERR_CUDA;
+    p->T = T; p->n = n_samples; p->device = dev; p->sm_count = sms; p->stream = s;
+    int rc = LIBRA_OK;
+    if (cudaMalloc((void**)&p->d_tok_start, sizeof(int32_t) * T) != cudaSuccess ||
+        cudaMalloc((void**)&p->d_tok_end, sizeof(int32_t) * T) != cudaSuccess ||
+        cudaMalloc((void**)&p->d_status, sizeof(int) * 4) != cudaSuccess)
+        rc = LIBRA_ERR_CUDA;
+    if (rc == LIBRA_OK) {
+        cudaMemsetAsync(p->d_status, 0, sizeof(int) * 4, s);
+        k_validate<<<grid_for(n_samples + 1, 128), 128, 0, s>>>(cu_seqlens_dev, n_samples, T, p->d_status);
+        k_token_bounds<<<grid_for(T, 256), 256, 0, s>>>(cu_seqlens_dev, n_samples, T, p->d_tok_start, p->d_tok_end);
+        count_launch(2);
+        const int dirs = o.directions ? o.directions : (LIBRA_DIR_Q | LIBRA_DIR_KV);
+        const int W = o.n_workers ? o.n_workers : sms;
+        if (dirs & LIBRA_DIR_Q) {
+            PlanDir& d = p->dir[0];
+            d.tile = tile_q; d.H = n_heads; d.W = W;
+            rc = build_dir(p, d, 0);
+        }
+        if (rc == LIBRA_OK && (dirs & LIBRA_DIR_KV)) {
+            PlanDir& d = p->dir[1];
+            d.tile = o.tile_kv ? o.tile_kv : 128; d.H = o.n_heads_kv ? o.n_heads_kv : n_heads; d.W = W;
+            rc = build_dir(p, d, 1);
+        }
+    }
+    if (rc != LIBRA_OK) {
+        libra_plan_destroy(p);
+        return rc;
+    }
+    *plan_out = p;
+    return LIBRA_OK;
+}
+
+static PlanDir* dir_of(const libra_plan_t* plan, int direction) {
+    if (!plan) return nullptr;
+    if (direction == LIBRA_DIR_Q) return plan->dir[0].enabled ? const_cast<PlanDir*>(&plan->dir[0]) : nullptr;
+    if (direction == LIBRA_DIR_KV) return plan->dir[1].enabled ? const_cast<PlanDir*>(&plan->dir[1]) : nullptr;
+    return nullptr;
+}
+
+extern "C" int libra_plan_info(const libra_plan_t* plan, int direction, int64_t* n_tiles, int* n_workers,
+                               int64_t* n_blocks, int* tile, int* n_heads) {
+    if (!plan) return LIBRA_ERR_INVALID_ARG;
+    PlanDir* d = dir_of(plan, direction);
+    if (!d) return LIBRA_ERR_PLAN_MISMATCH;
+    if (n_tiles) *n_tiles = d->NT;
+    if (n_workers) *n_workers = d->W;
+    if (n_blocks) *n_blocks = d->NB;
+    if (tile) *tile = d->tile;
+    if (n_heads) *n_heads = d->H;
+    return LIBRA_OK;
+}
+
+extern "C" int libra_plan_status(const libra_plan_t* plan) {
+    if (!plan) return LIBRA_ERR_INVALID_ARG;
+    int st[4] = {0, 0, 0, 0};
+    if (cudaStreamSynchronize(plan->stream) != cudaSuccess) return LIBRA_ERR_CUDA;
+    if (cudaMemcpy(st, plan->d_status, sizeof(st), cudaMemcpyDeviceToHost) != cudaSuccess) return LIBRA_ERR_CUDA;
+    return st[0];
+}
+
+extern "C" int libra_plan_export(const libra_plan_t* plan, int direction, int64_t* weight_host, int32_t* order_host,
+                                 int32_t* cta_of_tile_host, int32_t* cta_offsets_host, int32_t* cta_tiles_host,
+                                 int64_t* loads_host) {
+    if (!plan) return LIBRA_ERR_INVALID_ARG;
+    PlanDir* d = dir_of(plan, direction);
+    if (!d) return LIBRA_ERR_PLAN_MISMATCH;
+    cudaStream_t s = plan->stream;
+    cudaError_t e = cudaSuccess;
+    auto ok = [&](cudaError_t x) { if (e == cudaSuccess) e = x; };
+    void* tmp = nullptr;
+    if (weight_host || order_host) ok(cudaMalloc(&tmp, sizeof(int64_t) * (d->NT ? d->NT : 1)));
+    if (e != cudaSuccess) return LIBRA_ERR_CUDA;
+    if (weight_host) {
+        k_expand_weight<<<grid_for(d->NT, 256), 256, 0, s>>>(d->d_weight_blk, d->NT, d->H, (int64_t*)tmp);
+        count_launch();
+        ok(cudaMemcpyAsync(weight_host, tmp, sizeof(int64_t) * d->NT, cudaMemcpyDeviceToHost, s));
+        ok(cudaStreamSynchronize(s));
+    }
+    if (order_host) {
+        k_expand_order<<<grid_for(d->NT, 256), 256, 0, s>>>(d->d_blk_order, d->NT, d->H, (int32_t*)tmp);
+        count_launch();
+        ok(cudaMemcpyAsync(order_host, tmp, sizeof(int32_t) * d->NT, cudaMemcpyDeviceToHost, s));
+        ok(cudaStreamSynchronize(s));
+    }
+    if (cta_of_tile_host)
+        ok(cudaMemcpyAsync(cta_of_tile_host, d->d_cta_of_tile, sizeof(int32_t) * d->NT, cudaMemcpyDeviceToHost, s));
+    if (cta_offsets_host)
+        ok(cudaMemcpyAsync(cta_offsets_host, d->d_cta_offsets, sizeof(int32_t) * (d->W + 1), cudaMemcpyDeviceToHost, s));
+    if (cta_tiles_host)
+        ok(cudaMemcpyAsync(cta_tiles_host, d->d_cta_tiles, sizeof(int32_t) * d->NT, cudaMemcpyDeviceToHost, s));
+    if (loads_host) ok(cudaMemcpyAsync(loads_host, d->d_loads, sizeof(int64_t) * d->W, cudaMemcpyDeviceToHost, s));
+    ok(cudaStreamSynchronize(s));
+    cudaFree(tmp);
+    return e == cudaSuccess ? LIBRA_OK : LIBRA_ERR_CUDA;
+}
+
+extern "C" int libra_plan_destroy(libra_plan_t* plan) {
+    if (!plan) return LIBRA_OK;
+    cudaDeviceSynchronize();
+    free_dir(plan->dir[0]);
+    free_dir(plan->dir[1]);
+    cudaFree(plan->d_tok_start);
+    cudaFree(plan->d_tok_end);
+    cudaFree(plan->d_status);
+    delete plan;
+    return LIBRA_OK;
+}
+
+extern "C" int libra_busy_times(const libra_plan_t* plan, int which, uint64_t* ns_host) {
+    if (!plan || !ns_host) return LIBRA_ERR_INVALID_ARG;
+    PlanDir* d = dir_of(plan, which);
+    if (!d) return LIBRA_ERR_PLAN_MISMATCH;
+    if (cudaDeviceSynchronize() != cudaSuccess) return LIBRA_ERR_CUDA;
+    uint64_t* tmp = new (std::nothrow) uint64_t[2 * (size_t)d->W];
+    if (!tmp) return LIBRA_ERR_CUDA;
+    int st[4] = {0, 0, 0, 0};
+    cudaError_t e = cudaMemcpy(tmp, d->d_busy, sizeof(uint64_t) * 2 * d->W, cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess) e = cudaMemcpy(st, plan->d_status, sizeof(st), cudaMemcpyDeviceToHost);
+    for (int r = 0; r < d->W; ++r) ns_host[r] = tmp[2 * r + 1] >= tmp[2 * r] ? tmp[2 * r + 1] - tmp[2 * r] : 0;
+    delete[] tmp;
+    if (e != cudaSuccess) return LIBRA_ERR_CUDA;
+    return st[which == LIBRA_DIR_Q ? 1 : 2];
+}
+
+extern "C" int64_t libra_launch_count(void) { return g_launches.load(); }
+
+extern "C" const char* libra_strerror(int code) {
+    switch (code) {
+        case LIBRA_OK: return "ok";
+        case LIBRA_ERR_INVALID_ARG: return "invalid argument";
+        case LIBRA_ERR_UNSUPPORTED: return "unsupported configuration";
+        case LIBRA_ERR_PLAN_MISMATCH: return "plan does not match the call";
+        case LIBRA_ERR_CUDA: return "CUDA call failed";
+        case LIBRA_ERR_OVERFLOW: return "integer overflow in plan sizes";
+        case LIBRA_ERR_TIMEOUT: return "a bounded device-side wait timed out";
+        case LIBRA_ERR_BAD_SEQLENS: return "cu_seqlens is malformed";
+        case LIBRA_ERR_NO_DEVICE: return "no usable CUDA device";
+        default: return "unknown error";
+    }
+}
