@@ -152,6 +152,14 @@ int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const void* v_dev,
  * (LIBRA_ERR_TIMEOUT if a bounded wait gave up). */
 int libra_busy_times(const libra_plan_t* plan, int which, uint64_t* ns_host);
 
+/* Kernel timing: when enabled, every forward / backward call records CUDA events on its
+ * stream around its main persistent kernel (not around the memset / prep / convert
+ * launches).  libra_kernel_time_ms synchronises on the closing event of the most recent call
+ * of direction `which` (LIBRA_DIR_Q = forward kernel, LIBRA_DIR_KV = backward main kernel)
+ * and returns its duration in milliseconds.  Off by default. */
+int libra_plan_set_timing(libra_plan_t* plan, int enabled);
+int libra_kernel_time_ms(const libra_plan_t* plan, int which, float* ms_host);
+
 /* Number of kernels this library has launched in the calling process (for accounting). */
 int64_t libra_launch_count(void);
 

@@ -25,7 +25,8 @@ ERR_OVERFLOW, ERR_TIMEOUT, ERR_BAD_SEQLENS, ERR_NO_DEVICE = -5, -6, -7, -8
 
 EXPORTS = ["libra_plan_tiles", "libra_plan_info", "libra_plan_status", "libra_plan_export",
            "libra_plan_destroy", "libra_attn_pool_fwd", "libra_attn_pool_bwd_workspace_bytes",
-           "libra_attn_pool_bwd", "libra_busy_times", "libra_launch_count", "libra_strerror"]
+           "libra_attn_pool_bwd", "libra_busy_times", "libra_plan_set_timing", "libra_kernel_time_ms", "libra_launch_count",
+           "libra_strerror"]
 
 
 class PlanOpts(ctypes.Structure):
@@ -106,6 +107,14 @@ class Plan:
         out = np.zeros(w, np.uint64)
         _check(_lib.libra_busy_times(self._h, which, _np(out)), "libra_busy_times")
         return out
+
+    def set_timing(self, enabled=True):
+        _check(_lib.libra_plan_set_timing(self._h, 1 if enabled else 0), "libra_plan_set_timing")
+
+    def kernel_time_ms(self, which=LIBRA_DIR_Q) -> float:
+        ms = ctypes.c_float()
+        _check(_lib.libra_kernel_time_ms(self._h, which, ctypes.byref(ms)), "libra_kernel_time_ms")
+        return float(ms.value)
 
     def destroy(self):
         if self._h:

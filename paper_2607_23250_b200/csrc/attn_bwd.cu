@@ -616,7 +616,10 @@ extern "C" int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const v
     prm.scale_log2 = scale * 1.4426950408889634f;
     prm.status = plan->d_status + 2;
     prm.busy = d.d_busy;
+    libra_plan_t* mp = const_cast<libra_plan_t*>(plan);
+    if (mp->timing) cudaEventRecord(mp->ev[1][0], s);
     rc = D == 128 ? launch_bwd<128>(tq, tk, tv, tdo, prm, d.W, s) : launch_bwd<64>(tq, tk, tv, tdo, prm, d.W, s);
+    if (mp->timing) { cudaEventRecord(mp->ev[1][1], s); mp->ev_valid[1] = 1; }
     if (rc != LIBRA_OK) return rc;
     {
         const int64_t n4 = T * dims->hq * D / 4;

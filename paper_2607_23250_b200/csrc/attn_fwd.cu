@@ -470,5 +470,9 @@ extern "C" int libra_attn_pool_fwd(const void* q_dev, const void* k_dev, const v
     prm.status = plan->d_status + 1;
     prm.busy = d.d_busy;
     cudaStream_t s = (cudaStream_t)stream;
-    return dims->head_dim == 128 ? launch_fwd<128>(tq, tk, tv, prm, d.W, s) : launch_fwd<64>(tq, tk, tv, prm, d.W, s);
+    libra_plan_t* mp = const_cast<libra_plan_t*>(plan);
+    if (mp->timing) cudaEventRecord(mp->ev[0][0], s);
+    rc = dims->head_dim == 128 ? launch_fwd<128>(tq, tk, tv, prm, d.W, s) : launch_fwd<64>(tq, tk, tv, prm, d.W, s);
+    if (mp->timing) { cudaEventRecord(mp->ev[0][1], s); mp->ev_valid[0] = 1; }
+    return rc;
 }

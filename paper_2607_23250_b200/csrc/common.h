@@ -40,6 +40,9 @@ struct libra_plan {
     int32_t* d_tok_end = nullptr;    // [T] one past the last token of that sample
     int* d_status = nullptr;         // [4] word 0: plan status; word 1: fwd; word 2: bwd
     libra::PlanDir dir[2];           // 0 = query-major, 1 = key-major
+    int timing = 0;                  // record events around the main kernels
+    cudaEvent_t ev[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};  // [direction][begin, end]
+    int ev_valid[2] = {0, 0};
 };
 
 namespace libra {

@@ -342,6 +342,9 @@ extern "C" int libra_plan_destroy(libra_plan_t* plan) {
     cudaFree(plan->d_tok_start);
     cudaFree(plan->d_tok_end);
     cudaFree(plan->d_status);
+    for (int a = 0; a < 2; ++a)
+        for (int b = 0; b < 2; ++b)
+            if (plan->ev[a][b]) cudaEventDestroy(plan->ev[a][b]);
     delete plan;
     return LIBRA_OK;
 }
@@ -360,6 +363,27 @@ extern "C" int libra_busy_times(const libra_plan_t* plan, int which, uint64_t* n
     delete[] tmp;
     if (e != cudaSuccess) return LIBRA_ERR_CUDA;
     return st[which == LIBRA_DIR_Q ? 1 : 2];
+}
+
+extern "C" int libra_plan_set_timing(libra_plan_t* plan, int enabled) {
+    if (!plan) return LIBRA_ERR_INVALID_ARG;
+    if (enabled) {
+        for (int a = 0; a < 2; ++a)
+            for (int b = 0; b < 2; ++b)
+                if (!plan->ev[a][b] && cudaEventCreate(&plan->ev[a][b]) != cudaSuccess) return LIBRA_ERR_CUDA;
+    }
+    plan->timing = enabled ? 1 : 0;
+    return LIBRA_OK;
+}
+
+extern "C" int libra_kernel_time_ms(const libra_plan_t* plan, int which, float* ms_host) {
+    if (!plan || !ms_host) return LIBRA_ERR_INVALID_ARG;
+    const int a = which == LIBRA_DIR_Q ? 0 : (which == LIBRA_DIR_KV ? 1 : -1);
+    if (a < 0) return LIBRA_ERR_INVALID_ARG;
+    if (!plan->ev_valid[a]) return LIBRA_ERR_PLAN_MISMATCH;
+    if (cudaEventSynchronize(plan->ev[a][1]) != cudaSuccess) return LIBRA_ERR_CUDA;
+    if (cudaEventElapsedTime(ms_host, plan->ev[a][0], plan->ev[a][1]) != cudaSuccess) return LIBRA_ERR_CUDA;
+    return LIBRA_OK;
 }
 
 extern "C" int64_t libra_launch_count(void) { return g_launches.load(); }
