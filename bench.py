@@ -161,6 +161,9 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     spec = pools.config(args.config, args.skew, seed=rank)       # every rank its own pool
+    if args.seqs:
+        import dataclasses
+        spec = dataclasses.replace(spec, n_seqs=args.seqs, name=f"{spec.name}[{args.seqs} seqs]")
     lengths = pools.pool_lengths(spec)
     cu_np = pools.cu_seqlens(lengths)
     T, hq, hkv, d = spec.total_tokens, spec.hq, spec.hkv, spec.head_dim
@@ -221,13 +224,24 @@ def run_ours(args):
     ms_per_step = float(ms.item())
     value = world * (ff + fb) / (ms_per_step * 1e-3) / 1e12
 
+    e2e = None
+    if not args.skip_e2e:
+        e2e = run_e2e(args, step, barrier, dict(q=q, k=k, v=v, dout=dout),
+                      dict(out=out, lse=lse, dq=dq, dk=dk, dv=dv), world, dev, ff + fb)
+    finish(args, rank, world, spec, lengths, plan, value, ms_per_step, kern_f, kern_b, busy_f, busy_b, clocks,
+           launches, e2e, ff, fb, q)
+    plan.destroy()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_e2e(args, step, barrier, dev_in, dev_out, world, dev, flops):
+    import torch
+    import torch.distributed as dist
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     # ---- end to end: pinned host inputs -> H2D -> fwd+bwd -> D2H of the results, every step
-    host_in = {n: torch.empty(x.shape, dtype=x.dtype).pin_memory().copy_(x) for n, x in
-               (("q", q), ("k", k), ("v", v), ("dout", dout))}
-    host_out = {n: torch.empty(x.shape, dtype=x.dtype).pin_memory() for n, x in
-                (("out", out), ("lse", lse), ("dq", dq), ("dk", dk), ("dv", dv))}
-    dev_in = {"q": q, "k": k, "v": v, "dout": dout}
-    dev_out = {"out": out, "lse": lse, "dq": dq, "dk": dk, "dv": dv}
+    host_in = {n: torch.empty(x.shape, dtype=x.dtype).pin_memory().copy_(x) for n, x in dev_in.items()}
+    host_out = {n: torch.empty(x.shape, dtype=x.dtype).pin_memory() for n, x in dev_out.items()}
     h2d = sum(x.numel() * x.element_size() for x in host_in.values())
     d2h = sum(x.numel() * x.element_size() for x in host_out.values())
 
@@ -249,8 +263,15 @@ def run_ours(args):
     e2e_ms = torch.tensor([e0.elapsed_time(e1) / n_e2e], device=dev, dtype=torch.float64)
     if world > 1:
         dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
-    e2e_value = world * (ff + fb) / (float(e2e_ms.item()) * 1e-3) / 1e12
+    e2e_value = world * flops / (float(e2e_ms.item()) * 1e-3) / 1e12
+    return {"value": round(e2e_value, 2), "unit": "TFLOP/s", "h2d_bytes_per_step": h2d,
+            "d2h_bytes_per_step": d2h, "ms_per_step": round(float(e2e_ms.item()), 3)}
 
+
+def finish(args, rank, world, spec, lengths, plan, value, ms_per_step, kern_f, kern_b, busy_f, busy_b, clocks,
+           launches, e2e, ff, fb, q):
+    from paper_2607_23250_b200 import binding as lb  # noqa: F401
+    T, hq, hkv, d = spec.total_tokens, spec.hq, spec.hkv, spec.head_dim
     if rank == 0:
         peaks = measured_peaks()
         kb = statistics.mean(kern_b)
@@ -285,21 +306,17 @@ def run_ours(args):
             "busy_max_over_mean": {"fwd": round(float(busy_f.max() / busy_f.mean()), 4),
                                    "bwd": round(float(busy_b.max() / busy_b.mean()), 4)},
             "clocks": clocks,
-            "e2e": {"value": round(e2e_value, 2), "unit": "TFLOP/s", "h2d_bytes_per_step": h2d,
-                    "d2h_bytes_per_step": d2h, "ms_per_step": round(float(e2e_ms.item()), 3)},
+            "e2e": e2e,
             "gpu_launches": int(launches),
             "roofline": {"bound": "tensor", "kernel": "k_attn_bwd", "achieved": round(ach, 1),
                          "peak": peaks["sustained"], "unit": "TFLOP/s", "frac": round(ach / peaks["sustained"], 4),
                          "peak_kind": f"bf16 sustained, {peaks['source']}", "traffic": traffic,
                          "frac_of_burst": round(ach / peaks["burst"], 4)},
         }
-        if world == 1:
+        if world == 1 and not args.skip_cpu:
             cb = time_oracle(spec, lengths)
             line["cpu_baseline"] = {k2: (round(v2, 6) if isinstance(v2, float) else v2) for k2, v2 in cb.items()}
         print(json.dumps(line), flush=True)
-    plan.destroy()
-    if world > 1:
-        dist.destroy_process_group()
 
 
 def run_reference(args):
@@ -331,6 +348,9 @@ def main():
     ap.add_argument("--config", type=int, default=2)
     ap.add_argument("--skew", type=float, default=0.0)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--seqs", type=int, default=0, help="override the number of packed sequences (profiling runs)")
+    ap.add_argument("--skip-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
+    ap.add_argument("--skip-cpu", action="store_true", help="skip the CPU oracle leg (profiling runs)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -26,13 +26,14 @@ def build(force: bool = False, verbose: bool = False) -> str:
     if not stale:
         return SO
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    extra = os.environ.get("LIBRA_NVCC_EXTRA", "").split()
     objs = []
     procs = []
     for s in srcs:
         o = os.path.join(HERE, "build", os.path.basename(s) + ".o")
         os.makedirs(os.path.dirname(o), exist_ok=True)
         objs.append(o)
-        procs.append((s, subprocess.Popen([nvcc, *NVCC_FLAGS, "-c", s, "-o", o], stdout=subprocess.PIPE,
+        procs.append((s, subprocess.Popen([nvcc, *NVCC_FLAGS, *extra, "-c", s, "-o", o], stdout=subprocess.PIPE,
                                           stderr=subprocess.STDOUT, text=True)))
     for s, p in procs:
         log, _ = p.communicate()

@@ -31,18 +31,21 @@ template <int D>
 struct BwdSmem {
     static constexpr int kHalfBytes = 128 * 128;
     static constexpr int kTileBytes = kHalfBytes * (D / 64);  // 128 x D bf16
+    static constexpr int kDoStages = (D == 128) ? 1 : 2;      // shared memory is full at D = 128
     static constexpr int kKOff = 0;
     static constexpr int kVOff = kTileBytes;
-    static constexpr int kQOff = 2 * kTileBytes;              // 2 stages
-    static constexpr int kDoOff = 4 * kTileBytes;             // 2 stages
-    static constexpr int kDsOff = 6 * kTileBytes;             // 128 keys x 128 queries bf16
-    static constexpr int kStatOff = kDsOff + 2 * kHalfBytes;  // per Q stage: lse2[128], dvec[128]
+    static constexpr int kQOff = 2 * kTileBytes;                    // 2 stages
+    static constexpr int kDoOff = 4 * kTileBytes;                   // kDoStages stages
+    static constexpr int kDsOff = kDoOff + kDoStages * kTileBytes;  // 128 keys x 128 queries bf16
+    static constexpr int kStageOff = kDsOff + 2 * kHalfBytes;       // 2 x (128 rows x 32 fp32) dQ staging
+    static constexpr int kStatOff = kStageOff + 2 * kHalfBytes;     // per Q stage: lse2[128], dvec[128]
     static constexpr int kBarOff = kStatOff + 2 * 1024;
     // kv_full, kv_empty, q_full[2], q_empty[2], do_full[2], do_empty[2], s_full, p_ready, dp_full,
     // ds_ready, dq_full, dq_empty, dkv_full, dkv_empty
     static constexpr int kNumBars = 18;
     static constexpr int kMiscOff = kBarOff + kNumBars * 8;
     static constexpr int kBytes = kMiscOff + 16;
+    static_assert(kBytes <= 232448, "exceeds the 227 KB shared memory of an sm_100 CTA");
 };
 
 struct BwdParams {
@@ -82,10 +85,30 @@ __device__ __forceinline__ int last_q_block(const int32_t* tok_end, int64_t T, i
     return (tok_end[last_key] - 1) / kBlk;
 }
 
+#ifdef LIBRA_PROF
+// Profiling build only: per-CTA cycle sums of the phases of one thread per role.
+__device__ unsigned long long g_bwd_prof[1024 * 24];
+struct Prof {
+    long long last;
+    unsigned long long acc[8];
+    __device__ void start() { last = clock64(); for (int i = 0; i < 8; ++i) acc[i] = 0; }
+    __device__ void mark(int k) { const long long now = clock64(); acc[k] += now - last; last = now; }
+    __device__ void flush(int cta, int base) { for (int i = 0; i < 8; ++i) g_bwd_prof[cta * 24 + base + i] = acc[i]; }
+};
+#define PROF_DECL Prof prof; prof.start();
+#define PROF(k) prof.mark(k);
+#define PROF_FLUSH(cond, base) if (cond) prof.flush(cta, base);
+#else
+#define PROF_DECL
+#define PROF(k)
+#define PROF_FLUSH(cond, base)
+#endif
+
 template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 k_attn_bwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-           const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do, const BwdParams p) {
+           const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do, const __grid_constant__ CUtensorMap tm_dq,
+           const BwdParams p) {
     using L = BwdSmem<D>;
     extern __shared__ __align__(1024) uint8_t smem[];
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBarOff);
@@ -144,6 +167,7 @@ k_attn_bwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         prefetch_tmap(&tm_k);
         prefetch_tmap(&tm_v);
         prefetch_tmap(&tm_do);
+        prefetch_tmap(&tm_dq);
     }
     tc_fence_before();
     __syncthreads();
@@ -191,13 +215,14 @@ k_attn_bwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                     bulk_load_1d(smem + L::kStatOff + st * 1024 + 512, p.dvec + (size_t)h * p.Tpad + qb, 512,
                                  &bar_qfull[st]);
                 }
-                ok = warp_wait_b(&bar_doempty[st], par, abort_flag);
+                const uint32_t dst = it_all % L::kDoStages, dpar = ((it_all / L::kDoStages) & 1) ^ 1;
+                ok = warp_wait_b(&bar_doempty[dst], dpar, abort_flag);
                 if (!ok) break;
                 if (lane == 0) {
-                    mbar_arrive_expect_tx(&bar_dofull[st], L::kTileBytes);
+                    mbar_arrive_expect_tx(&bar_dofull[dst], L::kTileBytes);
                     for (int half = 0; half < D / 64; ++half)
-                        tma_load_3d(smem + L::kDoOff + st * L::kTileBytes + half * L::kHalfBytes, &tm_do,
-                                    &bar_dofull[st], half * 64, h, qb);
+                        tma_load_3d(smem + L::kDoOff + dst * L::kTileBytes + half * L::kHalfBytes, &tm_do,
+                                    &bar_dofull[dst], half * 64, h, qb);
                 }
             }
         }
@@ -210,6 +235,7 @@ k_attn_bwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         const uint32_t sb = smem_u32(smem);
         uint32_t ucnt = 0, it_all = 0;
         bool ok = true;
+        PROF_DECL
         // C[tmem] = A(K-major tile) * B(K-major tile)^T over the head dimension
         auto issue_kmajor = [&](uint32_t d_col, uint32_t a_addr, uint32_t b_addr) {
 #pragma unroll
@@ -238,46 +264,56 @@ k_attn_bwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             for (int it = 0; it < n_it && ok; ++it, ++it_all) {
                 const uint32_t st = it_all & 1, par = (it_all >> 1) & 1;
                 // dP(it): needs dO and the dP/dQ columns drained of dQ(it-1)
-                ok = warp_wait_b(&bar_dofull[st], par, abort_flag);
+                const uint32_t dst = it_all % L::kDoStages, dpar = (it_all / L::kDoStages) & 1;
+                PROF(7)
+                ok = warp_wait_b(&bar_dofull[dst], dpar, abort_flag);
                 if (!ok) break;
+                PROF(0)
                 if (it_all > 0) {
                     ok = warp_wait_b(bar_dqempty, (it_all - 1) & 1, abort_flag);
                     if (!ok) break;
                 }
+                PROF(1)
                 tc_fence_after();
                 if (lane == 0) {
-                    issue_kmajor(kColDP, sb + L::kVOff, sb + L::kDoOff + st * L::kTileBytes);
+                    issue_kmajor(kColDP, sb + L::kVOff, sb + L::kDoOff + dst * L::kTileBytes);
                     tc_commit(bar_dpfull);
                 }
                 // dV(it) += P^T dO
+                PROF(7)
                 ok = warp_wait_b(bar_pready, it_all & 1, abort_flag);
                 if (!ok) break;
+                PROF(2)
                 if (it == 0 && ucnt > 0) {  // previous unit's dK/dV must have been read out
                     ok = warp_wait_b(bar_dkvempty, (ucnt - 1) & 1, abort_flag);
                     if (!ok) break;
                 }
                 tc_fence_after();
                 if (lane == 0) {
-                    const uint32_t doa = sb + L::kDoOff + st * L::kTileBytes;
+                    const uint32_t doa = sb + L::kDoOff + dst * L::kTileBytes;
 #pragma unroll
                     for (int kk = 0; kk < 8; ++kk)  // 16 queries per step; P^T of columns 64c.. lives at 64c + ..
                         mma_ts(tmem_base + kColDV, tmem_base + kColS + (kk / 4) * 64 + (kk % 4) * 8,
                                make_sdesc(doa + kk * 2048, L::kHalfBytes, 1024), idesc_dv, (it > 0 || kk > 0) ? 1u : 0u);
-                    tc_commit(&bar_doempty[st]);
+                    tc_commit(&bar_doempty[dst]);
                 }
                 // S(it+1)
                 if (it + 1 < n_it) {
                     const uint32_t nx = it_all + 1;
+                    PROF(7)
                     ok = warp_wait_b(&bar_qfull[nx & 1], (nx >> 1) & 1, abort_flag);
                     if (!ok) break;
+                    PROF(3)
                     if (lane == 0) {
                         issue_kmajor(kColS, sb + L::kKOff, sb + L::kQOff + (nx & 1) * L::kTileBytes);
                         tc_commit(bar_sfull);
                     }
                 }
                 // dK(it) += dS^T Q ; dQ(it) = dS K
+                PROF(7)
                 ok = warp_wait_b(bar_dsready, it_all & 1, abort_flag);
                 if (!ok) break;
+                PROF(4)
                 tc_fence_after();
                 if (lane == 0) {
                     const uint32_t dsa = sb + L::kDsOff;
@@ -302,12 +338,20 @@ k_attn_bwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             __syncwarp();
             ++ucnt;
         }
+        PROF_FLUSH(lane == 0, 8)
+    } else if (warp >= 12) {
+        // warps 14-15: nothing to do
     } else if (warp >= 8) {
         // ---------------- dQ reduce group ----------------
+        // TMEM -> registers (whole tile, frees the columns at once) -> 32-column chunks through two
+        // staging buffers -> TMA reduce-add into the fp32 accumulator (full 128-byte lines).
         const int r = (warp & 3) * 32 + lane;
+        const bool leader = (threadIdx.x == 8 * 32);
         const uint32_t t_dq = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + kColDP;
+        uint8_t* stage_row = smem + L::kStageOff + r * 128;
         uint32_t it_all = 0;
         bool ok = true;
+        PROF_DECL
         for (int idx = unit_begin; idx < unit_end && ok; ++idx) {
             const int t = p.cta_tiles[idx];
             const int kvh = t % p.hkv;
@@ -317,30 +361,49 @@ k_attn_bwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             const int n_it = G * nblk;
             for (int it = 0; it < n_it && ok; ++it, ++it_all) {
                 const int h = kvh * G + it / nblk;
-                const int64_t q = (int64_t)(i_lo + it % nblk) * kBlk + r;
+                const int qb = (i_lo + it % nblk) * kBlk;
                 ok = mbar_wait(bar_dqfull, it_all & 1, abort_flag);
                 if (!ok) break;
+                PROF(0)
                 tc_fence_after();
-                float* dst = p.dq_acc + ((size_t)q * p.hq + h) * D;
+                uint32_t v[D];
 #pragma unroll
-                for (int c = 0; c < D; c += 64) {
-                    uint32_t v[64];
-                    tmem_ld32(t_dq + c, v);
-                    tmem_ld32(t_dq + c + 32, v + 32);
-                    tmem_ld_wait();
-                    if (c + 64 >= D) {  // last read of the tile: the columns may be overwritten now
-                        tc_fence_before();
-                        mbar_arrive(bar_dqempty);
+                for (int c = 0; c < D; c += 32) tmem_ld32(t_dq + c, v + c);
+                tmem_ld_wait();
+                tc_fence_before();
+                mbar_arrive(bar_dqempty);  // the dP/dQ columns may be overwritten now
+                PROF(1)
+#pragma unroll
+                for (int c = 0; c < D / 32; ++c) {
+                    uint8_t* dst = stage_row + (c & 1) * L::kHalfBytes;
+                    // the buffer may still be read by the reduce issued two chunks ago
+                    if (leader) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) {
+                        uint4 w;
+                        w.x = v[c * 32 + k * 4]; w.y = v[c * 32 + k * 4 + 1];
+                        w.z = v[c * 32 + k * 4 + 2]; w.w = v[c * 32 + k * 4 + 3];
+                        *reinterpret_cast<uint4*>(dst + ((k ^ (r & 7)) << 4)) = w;
                     }
-                    if (q < p.T) {
-#pragma unroll
-                        for (int i = 0; i < 64; i += 4)
-                            red_add_v4(dst + c + i, __uint_as_float(v[i]), __uint_as_float(v[i + 1]),
-                                       __uint_as_float(v[i + 2]), __uint_as_float(v[i + 3]));
+                    fence_proxy_async_smem();
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    if (leader) {
+#ifndef LIBRA_DBG_NO_RED
+                        asm volatile(
+                            "cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];"
+                            ::"l"(reinterpret_cast<uint64_t>(&tm_dq)), "r"(h * D + c * 32), "r"(qb),
+                            "r"(smem_u32(smem + L::kStageOff + (c & 1) * L::kHalfBytes))
+                            : "memory");
+#endif
+                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                     }
                 }
+                PROF(2)
             }
         }
+        if (leader) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // all reduce-adds done before exit
+        PROF_FLUSH(leader, 16)
     } else {
         // ---------------- compute groups ----------------
         const int c = warp >> 2;  // query-column half of each key row
@@ -351,6 +414,7 @@ k_attn_bwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         uint8_t* ds_row = smem + L::kDsOff + c * L::kHalfBytes + r * 128;
         uint32_t ucnt = 0, it_all = 0;
         bool ok = true;
+        PROF_DECL
         for (int idx = unit_begin; idx < unit_end && ok; ++idx) {
             const int t = p.cta_tiles[idx];
             const int kvh = t % p.hkv;
@@ -374,6 +438,7 @@ k_attn_bwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 // ---- exp phase: P^T = exp2(S^T * c - LSE) ----
                 ok = mbar_wait(&bar_qfull[st], par, abort_flag) && mbar_wait(bar_sfull, it_all & 1, abort_flag);
                 if (!ok) break;
+                PROF(0)
                 tc_fence_after();
                 uint32_t sv[64];
                 tmem_ld32(t_s, sv);
@@ -402,14 +467,18 @@ k_attn_bwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 tmem_st_wait();
                 tc_fence_before();
                 mbar_arrive(bar_pready);
+                PROF(1)
                 // ---- dS phase: dS^T = P^T o (dP^T - D) ----
                 ok = mbar_wait(bar_dpfull, it_all & 1, abort_flag);
                 if (!ok) break;
+                PROF(2)
                 tc_fence_after();
                 uint32_t dpv[64];
                 tmem_ld32(t_dp, dpv);
                 tmem_ld32(t_dp + 32, dpv + 32);
                 tmem_ld_wait();
+                PROF(3)
+                PROF(4)
 #pragma unroll
                 for (int ch = 0; ch < 8; ++ch) {
                     const float4 d0 = *reinterpret_cast<const float4*>(dvec + ch * 8);
@@ -422,9 +491,11 @@ k_attn_bwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                     w.w = pack_bf16x2(pf[j + 6] * (__uint_as_float(dpv[j + 6]) - d1.z), pf[j + 7] * (__uint_as_float(dpv[j + 7]) - d1.w));
                     *reinterpret_cast<uint4*>(ds_row + ((ch ^ (r & 7)) << 4)) = w;
                 }
+                PROF(5)
                 fence_proxy_async_smem();
                 tc_fence_before();
                 mbar_arrive(bar_dsready);
+                PROF(7)
             }
             if (!ok) break;
             // ---- unit epilogue: dK * scale and dV to global ----
@@ -460,7 +531,9 @@ k_attn_bwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             tc_fence_before();
             mbar_arrive(bar_dkvempty);
             ++ucnt;
+            PROF(6)
         }
+        PROF_FLUSH(threadIdx.x == 0, 0)
     }
 
     // ---------------- teardown ----------------
@@ -530,7 +603,7 @@ static BwdWorkspace bwd_workspace(int64_t T, int hq, int d) {
 
 template <int D>
 static int launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tdo,
-                      const BwdParams& prm, int W, cudaStream_t s) {
+                      const CUtensorMap& tdq, const BwdParams& prm, int W, cudaStream_t s) {
     using L = BwdSmem<D>;
     static bool configured = false;
     if (!configured) {
@@ -538,7 +611,7 @@ static int launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtens
             return LIBRA_ERR_CUDA;
         configured = true;
     }
-    k_attn_bwd<D><<<W, kBwdThreads, L::kBytes, s>>>(tq, tk, tv, tdo, prm);
+    k_attn_bwd<D><<<W, kBwdThreads, L::kBytes, s>>>(tq, tk, tv, tdo, tdq, prm);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? LIBRA_OK : LIBRA_ERR_CUDA;
 }
@@ -546,6 +619,12 @@ static int launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtens
 }  // namespace libra
 
 using namespace libra;
+
+#ifdef LIBRA_PROF
+extern "C" int libra_debug_bwd_prof(unsigned long long* host, int n) {
+    return cudaMemcpyFromSymbol(host, libra::g_bwd_prof, sizeof(unsigned long long) * n) == cudaSuccess ? 0 : -4;
+}
+#endif
 
 extern "C" size_t libra_attn_pool_bwd_workspace_bytes(const libra_plan_t* plan, const libra_dims* dims) {
     if (!plan || !dims || dims->hq <= 0 || (dims->head_dim != 64 && dims->head_dim != 128)) return 0;
@@ -579,8 +658,9 @@ extern "C" int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const v
     float* lse2 = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(workspace_dev) + ws.dq_acc_bytes + ws.stat_bytes);
     cudaStream_t s = (cudaStream_t)stream;
 
-    CUtensorMap tq, tk, tv, tdo;
-    int rc = make_thd_map(&tq, q_dev, T, dims->hq, D, kBlk);
+    CUtensorMap tq, tk, tv, tdo, tdq;
+    int rc = make_f32_2d_map(&tdq, dq_acc, T, (int64_t)dims->hq * D, 32, kBlk);
+    if (rc == LIBRA_OK) rc = make_thd_map(&tq, q_dev, T, dims->hq, D, kBlk);
     if (rc == LIBRA_OK) rc = make_thd_map(&tk, k_dev, T, dims->hkv, D, kBlk);
     if (rc == LIBRA_OK) rc = make_thd_map(&tv, v_dev, T, dims->hkv, D, kBlk);
     if (rc == LIBRA_OK) rc = make_thd_map(&tdo, dout_dev, T, dims->hq, D, kBlk);
@@ -606,7 +686,7 @@ extern "C" int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const v
     prm.lse2 = lse2;
     prm.dvec = dvec;
     prm.cta_offsets = d.d_cta_offsets;
-    prm.cta_tiles = d.d_cta_tiles;
+    prm.cta_tiles = d.d_cta_exec;
     prm.tok_end = plan->d_tok_end;
     prm.T = T;
     prm.Tpad = ws.Tpad;
@@ -618,7 +698,7 @@ extern "C" int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const v
     prm.busy = d.d_busy;
     libra_plan_t* mp = const_cast<libra_plan_t*>(plan);
     if (mp->timing) cudaEventRecord(mp->ev[1][0], s);
-    rc = D == 128 ? launch_bwd<128>(tq, tk, tv, tdo, prm, d.W, s) : launch_bwd<64>(tq, tk, tv, tdo, prm, d.W, s);
+    rc = D == 128 ? launch_bwd<128>(tq, tk, tv, tdo, tdq, prm, d.W, s) : launch_bwd<64>(tq, tk, tv, tdo, tdq, prm, d.W, s);
     if (mp->timing) { cudaEventRecord(mp->ev[1][1], s); mp->ev_valid[1] = 1; }
     if (rc != LIBRA_OK) return rc;
     {

@@ -416,6 +416,19 @@ int make_thd_map(CUtensorMap* m, const void* base, int64_t T, int H, int d, int 
     return r == CUDA_SUCCESS ? LIBRA_OK : LIBRA_ERR_CUDA;
 }
 
+int make_f32_2d_map(CUtensorMap* m, const void* base, int64_t rows, int64_t cols, int box_cols, int box_rows) {
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return LIBRA_ERR_CUDA;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)cols * 4};
+    cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? LIBRA_OK : LIBRA_ERR_CUDA;
+}
+
 template <int D>
 static int launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& prm, int W,
                       cudaStream_t s) {
@@ -459,7 +472,7 @@ extern "C" int libra_attn_pool_fwd(const void* q_dev, const void* k_dev, const v
     prm.out = reinterpret_cast<__nv_bfloat16*>(out_dev);
     prm.lse = lse_dev;
     prm.cta_offsets = d.d_cta_offsets;
-    prm.cta_tiles = d.d_cta_tiles;
+    prm.cta_tiles = d.d_cta_exec;
     prm.tok_start = plan->d_tok_start;
     prm.T = plan->T;
     prm.hq = dims->hq;

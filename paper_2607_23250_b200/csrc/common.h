@@ -23,7 +23,8 @@ struct PlanDir {
     int32_t* d_cta_of_tile = nullptr;  // [NT]
     int32_t* d_pos = nullptr;          // [NT]  position of the tile in its worker's list
     int32_t* d_cta_offsets = nullptr;  // [W+1]
-    int32_t* d_cta_tiles = nullptr;    // [NT]
+    int32_t* d_cta_tiles = nullptr;    // [NT]  per-worker lists in placement order (the plan proper)
+    int32_t* d_cta_exec = nullptr;     // [NT]  the same lists, each re-ordered for execution (head-major)
     int64_t* d_loads = nullptr;        // [W]
     uint64_t* d_busy = nullptr;        // [2*W] (start, end) global-timer stamps of the last run
 };
@@ -54,4 +55,6 @@ namespace libra {
 // bf16 [T, H, d] tensor viewed as (d, H, T); TMA box = 64 columns x 1 head x box_rows tokens,
 // 128-byte swizzle, out-of-range rows read as zero.  Defined in attn_fwd.cu.
 int make_thd_map(CUtensorMap* m, const void* base, int64_t T, int H, int d, int box_rows);
+// fp32 matrix [rows, cols] (cols contiguous); box = box_cols x box_rows, 128-byte swizzle.
+int make_f32_2d_map(CUtensorMap* m, const void* base, int64_t rows, int64_t cols, int box_cols, int box_rows);
 }  // namespace libra

@@ -149,6 +149,30 @@ __global__ void k_scatter_lists(const int32_t* __restrict__ cta_of_tile, const i
     cta_tiles[cta_offsets[cta_of_tile[t]] + pos[t]] = (int32_t)t;
 }
 
+// Execution order inside a worker's list.  The placement fixes WHICH tiles a worker runs; the order
+// it runs them in is free.  Sorting every list by (head shard, block) makes all workers sweep
+// the same head and neighbouring blocks at about the same time, so K/V re-reads and the
+// backward's dQ atomics hit L2 instead of DRAM.  One thread block per worker, rank sort.
+__global__ void k_exec_order(const int32_t* __restrict__ cta_offsets, const int32_t* __restrict__ cta_tiles, int H,
+                             int64_t NB, int32_t* __restrict__ cta_exec) {
+    const int r = blockIdx.x;
+    const int beg = cta_offsets[r], n = cta_offsets[r + 1] - beg;
+    if (n > 16384) {  // quadratic sort too slow: keep placement order
+        for (int i = threadIdx.x; i < n; i += blockDim.x) cta_exec[beg + i] = cta_tiles[beg + i];
+        return;
+    }
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        const int32_t t = cta_tiles[beg + i];
+        const int64_t key = (int64_t)(t % H) * NB + t / H;
+        int rank = 0;
+        for (int j = 0; j < n; ++j) {
+            const int32_t u = cta_tiles[beg + j];
+            rank += ((int64_t)(u % H) * NB + u / H) < key;
+        }
+        cta_exec[beg + rank] = t;
+    }
+}
+
 // Expanders used by libra_plan_export.
 __global__ void k_expand_weight(const int64_t* __restrict__ weight_blk, int64_t NT, int H, int64_t* __restrict__ out) {
     const int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
@@ -165,7 +189,7 @@ static inline unsigned grid_for(int64_t n, int block) { return (unsigned)((n + b
 
 static void free_dir(PlanDir& d) {
     cudaFree(d.d_weight_blk); cudaFree(d.d_blk_order); cudaFree(d.d_cta_of_tile); cudaFree(d.d_pos);
-    cudaFree(d.d_cta_offsets); cudaFree(d.d_cta_tiles); cudaFree(d.d_loads); cudaFree(d.d_busy);
+    cudaFree(d.d_cta_offsets); cudaFree(d.d_cta_tiles); cudaFree(d.d_cta_exec); cudaFree(d.d_loads); cudaFree(d.d_busy);
     d = PlanDir();
 }
 
@@ -184,6 +208,7 @@ static int build_dir(libra_plan* p, PlanDir& d, int key_major) {
     A((void**)&d.d_pos, sizeof(int32_t) * d.NT);
     A((void**)&d.d_cta_offsets, sizeof(int32_t) * (d.W + 1));
     A((void**)&d.d_cta_tiles, sizeof(int32_t) * d.NT);
+    A((void**)&d.d_cta_exec, sizeof(int32_t) * d.NT);
     A((void**)&d.d_loads, sizeof(int64_t) * d.W);
     A((void**)&d.d_busy, sizeof(uint64_t) * 2 * d.W);
     if (e != cudaSuccess) return LIBRA_ERR_CUDA;
@@ -203,7 +228,8 @@ static int build_dir(libra_plan* p, PlanDir& d, int key_major) {
                                      d.d_cta_offsets, d.d_loads);
     k_scatter_lists<<<grid_for(d.NT, 256), 256, 0, s>>>(d.d_cta_of_tile, d.d_pos, d.d_cta_offsets, d.NT,
                                                         d.d_cta_tiles);
-    count_launch(4);
+    k_exec_order<<<d.W, 256, 0, s>>>(d.d_cta_offsets, d.d_cta_tiles, d.H, d.NB, d.d_cta_exec);
+    count_launch(5);
     d.enabled = 1;
     return cudaGetLastError() == cudaSuccess ? LIBRA_OK : LIBRA_ERR_CUDA;
 }
