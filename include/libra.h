@@ -44,6 +44,11 @@ extern "C" {
 #define LIBRA_DIR_Q   1   /* query-major tiles (forward)  */
 #define LIBRA_DIR_KV  2   /* key-major tiles   (backward) */
 
+/* kernels, for libra_busy_times / libra_kernel_time_ms */
+#define LIBRA_KERNEL_FWD       1   /* forward kernel (walks the query-major lists)            */
+#define LIBRA_KERNEL_BWD_DKDV  2   /* backward dK/dV kernel (walks the key-major lists)       */
+#define LIBRA_KERNEL_BWD_DQ    3   /* backward dQ kernel (walks the query-major lists)        */
+
 typedef struct libra_plan libra_plan_t;   /* opaque, library-owned */
 
 typedef struct {
@@ -123,8 +128,8 @@ int libra_attn_pool_fwd(const void* q_dev, const void* k_dev, const void* v_dev,
                         const int32_t* cu_seqlens_dev, const libra_plan_t* plan,
                         void* out_dev, float* lse_dev, const libra_dims* dims, void* stream);
 
-/* Bytes of caller-owned device scratch libra_attn_pool_bwd needs (fp32 dQ accumulator and
- * the row statistic D); 0 on bad arguments. */
+/* Bytes of caller-owned device scratch libra_attn_pool_bwd needs (the row statistics D and
+ * LSE in log2 units, padded to a multiple of 128 rows); 0 on bad arguments. */
 size_t libra_attn_pool_bwd_workspace_bytes(const libra_plan_t* plan, const libra_dims* dims);
 
 /* Backward: the gradient of <dout, out> with respect to q, k, v, given out and lse from the
@@ -133,10 +138,12 @@ size_t libra_attn_pool_bwd_workspace_bytes(const libra_plan_t* plan, const libra
  *     P_ik = exp(scale <q_i,k_k> - lse_i), D_i = <dout_i, out_i>, dS_ik = P_ik (<dout_i,v_k> - D_i)
  *     dq_i = scale sum_k dS_ik k_k;  dk_k = scale sum_{h,i} dS_ik q_i;  dv_k = sum_{h,i} P_ik dout_i
  * (sums over the query heads h of the kv head's group and the rows i >= k of the sample).
- * Walks the plan's key-major tile lists; needs LIBRA_DIR_KV with tile_kv == 128 and
- * n_heads_kv == hkv.  `workspace_dev` must hold libra_attn_pool_bwd_workspace_bytes bytes,
- * 256-byte aligned; it is fully initialised inside the call.  dq accumulates through fp32
- * atomics, so its low bits may differ from run to run.
+ * Three launches: row statistics, a dK/dV kernel that walks the plan's key-major lists, and a
+ * dQ kernel that walks its query-major lists; no atomics, so results are run-to-run identical.
+ * Needs a plan with both directions: LIBRA_DIR_KV with tile_kv == 128 and n_heads_kv == hkv,
+ * LIBRA_DIR_Q with tile_q == 256 and n_heads dividing hq.  `workspace_dev` must hold
+ * libra_attn_pool_bwd_workspace_bytes bytes, 256-byte aligned; it is fully written inside the
+ * call.  Errors: INVALID_ARG, UNSUPPORTED, PLAN_MISMATCH, CUDA.
  */
 int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const void* v_dev,
                         const void* out_dev, const float* lse_dev, const void* dout_dev,
@@ -145,18 +152,16 @@ int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const void* v_dev,
                         const libra_dims* dims, void* stream);
 
 /* ---- instrumentation -------------------------------------------------------------------
- * Per-CTA busy time of the most recent forward (which = LIBRA_DIR_Q) or backward
- * (LIBRA_DIR_KV) call that used this plan: nanoseconds between the CTA picking up its
- * first tile and finishing its last, read with the GPU's global timer.  Copies n_workers
- * values to ns_host and synchronises the device.  Also returns the kernel status
- * (LIBRA_ERR_TIMEOUT if a bounded wait gave up). */
+ * Per-CTA busy time of the most recent launch of kernel `which` (LIBRA_KERNEL_*) that used this
+ * plan: nanoseconds between the CTA starting and finishing its tile list, read with the GPU's
+ * global timer.  Copies n_workers values to ns_host and synchronises the device.  Returns the
+ * kernel status (LIBRA_ERR_TIMEOUT if a bounded wait gave up). */
 int libra_busy_times(const libra_plan_t* plan, int which, uint64_t* ns_host);
 
 /* Kernel timing: when enabled, every forward / backward call records CUDA events on its
- * stream around its main persistent kernel (not around the memset / prep / convert
- * launches).  libra_kernel_time_ms synchronises on the closing event of the most recent call
- * of direction `which` (LIBRA_DIR_Q = forward kernel, LIBRA_DIR_KV = backward main kernel)
- * and returns its duration in milliseconds.  Off by default. */
+ * stream around each persistent kernel (not around the row-statistics launch).
+ * libra_kernel_time_ms synchronises on the closing event of the most recent launch of kernel
+ * `which` (LIBRA_KERNEL_*) and returns its duration in milliseconds.  Off by default. */
 int libra_plan_set_timing(libra_plan_t* plan, int enabled);
 int libra_kernel_time_ms(const libra_plan_t* plan, int which, float* ms_host);
 

@@ -20,6 +20,7 @@ if not os.path.exists(_SO):
 _lib = ctypes.CDLL(_SO)
 
 LIBRA_DIR_Q, LIBRA_DIR_KV = 1, 2
+KERNEL_FWD, KERNEL_BWD_DKDV, KERNEL_BWD_DQ = 1, 2, 3
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_PLAN_MISMATCH, ERR_CUDA = -1, -2, -3, -4
 ERR_OVERFLOW, ERR_TIMEOUT, ERR_BAD_SEQLENS, ERR_NO_DEVICE = -5, -6, -7, -8
 
@@ -102,8 +103,8 @@ class Plan:
         res["n_blocks"] = i["n_blocks"]
         return res
 
-    def busy_times(self, which=LIBRA_DIR_Q):
-        w = self.info(which)["n_workers"]
+    def busy_times(self, which=KERNEL_FWD):
+        w = self.info(LIBRA_DIR_KV if which == KERNEL_BWD_DKDV else LIBRA_DIR_Q)["n_workers"]
         out = np.zeros(w, np.uint64)
         _check(_lib.libra_busy_times(self._h, which, _np(out)), "libra_busy_times")
         return out
@@ -111,7 +112,7 @@ class Plan:
     def set_timing(self, enabled=True):
         _check(_lib.libra_plan_set_timing(self._h, 1 if enabled else 0), "libra_plan_set_timing")
 
-    def kernel_time_ms(self, which=LIBRA_DIR_Q) -> float:
+    def kernel_time_ms(self, which=KERNEL_FWD) -> float:
         ms = ctypes.c_float()
         _check(_lib.libra_kernel_time_ms(self._h, which, ctypes.byref(ms)), "libra_kernel_time_ms")
         return float(ms.value)

@@ -1,22 +1,21 @@
 // Backward pool attention for sm_100a.
 //
-// Three kernels: (1) prep: D_i = <dO_i, O_i> and LSE in log2 units, both padded to a multiple
-// of 128 rows; (2) the persistent main kernel; (3) dQ fp32 -> bf16 with the softmax scale.
+// Three launches: (1) prep: D_i = <dO_i, O_i> and LSE in log2 units, padded to a multiple of 128
+// rows; (2) the dK/dV kernel over key-major tiles; (3) the dQ kernel over query-major tiles.
+// Splitting dQ off costs two extra GEMMs per block pair (S and dP are recomputed) but needs no
+// cross-CTA reduction at all: no fp32 dQ accumulator, no atomics, no shared-memory staging, and
+// the result is deterministic.  Both kernels are persistent and warp-specialised (320 threads:
+// warps 0-3 / 4-7 compute groups, warp 8 TMA, warp 9 MMA) and keep their accumulators in TMEM.
 //
-// Main kernel.  A work unit is a key-major tile: 128 keys x one kv head.  K and V of the unit
-// stay in shared memory; dK and dV stay in TMEM for the whole unit while the CTA streams every
-// (query head of the group, 128-row query block) that can see the keys, from the diagonal
-// block up to the block holding the end of the last key's sample.  Keys sit in TMEM lanes:
-//   S^T  = K Q^T          (SS)      P^T = exp2(S^T * c - LSE)   written over S^T as bf16
-//   dP^T = V dO^T         (SS)      dS^T = P^T o (dP^T - D)     written to shared memory
-//   dV  += P^T dO         (A from TMEM)
-//   dK  += dS^T Q         (SS, A K-major)
-//   dQ   = dS K           (SS, A and B MN-major; dQ reuses dP^T's TMEM columns)
-// dQ tiles are drained by a reduce group and added to an fp32 accumulator with vector atomics.
-// Roles (448 threads): warps 0-3 / 4-7 compute groups (query columns 0-63 / 64-127 of each key
-// row), warps 8-11 dQ reduce, warp 12 TMA, warp 13 MMA.
-// Tensor-pipe order per iteration i:  dP(i) | dV(i) S(i+1) | dK(i) dQ(i), so the exp phase of
-// iteration i+1 overlaps dK/dQ/dP and the dS phase overlaps dV/S.
+// dK/dV kernel: a unit is 128 keys x one kv head; K and V stay in shared memory, dK and dV in
+// TMEM, while the CTA streams every (query head of the group, 128-row query block) that sees the
+// keys.  Keys sit in TMEM lanes:
+//   S^T  = K Q^T   (SS)   P^T  = exp2(S^T c - LSE)   -> bf16 over S^T     dV += P^T dO   (A in TMEM)
+//   dP^T = V dO^T  (SS)   dS^T = P^T o (dP^T - D)    -> bf16 over dP^T    dK += dS^T Q   (A in TMEM)
+// dQ kernel: a unit is 128 query rows x one head; Q and dO stay in shared memory, dQ in TMEM, the
+// CTA streams the key blocks the rows see (as the forward does).  Queries sit in TMEM lanes:
+//   S  = Q K^T (SS, double-buffered)   dP = dO V^T (SS)   dS = P o (dP - D) -> bf16 over S
+//   dQ += dS K (A in TMEM)
 #include <math.h>
 
 #include "common.h"
@@ -24,45 +23,9 @@
 
 namespace libra {
 
-constexpr int kBwdThreads = 448;
+constexpr int kBwdThreads = 320;
 constexpr int kBlk = 128;
-
-template <int D>
-struct BwdSmem {
-    static constexpr int kHalfBytes = 128 * 128;
-    static constexpr int kTileBytes = kHalfBytes * (D / 64);  // 128 x D bf16
-    static constexpr int kDoStages = (D == 128) ? 1 : 2;      // shared memory is full at D = 128
-    static constexpr int kKOff = 0;
-    static constexpr int kVOff = kTileBytes;
-    static constexpr int kQOff = 2 * kTileBytes;                    // 2 stages
-    static constexpr int kDoOff = 4 * kTileBytes;                   // kDoStages stages
-    static constexpr int kDsOff = kDoOff + kDoStages * kTileBytes;  // 128 keys x 128 queries bf16
-    static constexpr int kStageOff = kDsOff + 2 * kHalfBytes;       // 2 x (128 rows x 32 fp32) dQ staging
-    static constexpr int kStatOff = kStageOff + 2 * kHalfBytes;     // per Q stage: lse2[128], dvec[128]
-    static constexpr int kBarOff = kStatOff + 2 * 1024;
-    // kv_full, kv_empty, q_full[2], q_empty[2], do_full[2], do_empty[2], s_full, p_ready, dp_full,
-    // ds_ready, dq_full, dq_empty, dkv_full, dkv_empty
-    static constexpr int kNumBars = 18;
-    static constexpr int kMiscOff = kBarOff + kNumBars * 8;
-    static constexpr int kBytes = kMiscOff + 16;
-    static_assert(kBytes <= 232448, "exceeds the 227 KB shared memory of an sm_100 CTA");
-};
-
-struct BwdParams {
-    float* dq_acc;            // [T, Hq, D] fp32, zeroed before the launch
-    __nv_bfloat16* dk;
-    __nv_bfloat16* dv;
-    const float* lse2;        // [Hq, Tpad]  LSE * log2(e)
-    const float* dvec;        // [Hq, Tpad]  D_i
-    const int32_t* cta_offsets;
-    const int32_t* cta_tiles;
-    const int32_t* tok_end;
-    int64_t T, Tpad;
-    int hq, hkv;
-    float scale, scale_log2;
-    int* status;
-    uint64_t* busy;
-};
+constexpr int kSmemMax = 232448;  // 227 KB per CTA on sm_100
 
 __device__ __forceinline__ void bulk_load_1d(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
@@ -70,19 +33,10 @@ __device__ __forceinline__ void bulk_load_1d(void* smem_dst, const void* gsrc, u
                  "l"(reinterpret_cast<uint64_t>(gsrc)), "r"(bytes), "r"(smem_u32(bar))
                  : "memory");
 }
-__device__ __forceinline__ void red_add_v4(float* gptr, float a, float b, float c, float d) {
-    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(gptr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
-}
 __device__ __forceinline__ bool warp_wait_b(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
     int ok = 1;
     if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag) ? 1 : 0;
     return __shfl_sync(0xffffffffu, ok, 0) != 0;
-}
-
-// Query blocks a key block [k0, k0+128) is seen by: diagonal .. block of (end of last key's sample - 1).
-__device__ __forceinline__ int last_q_block(const int32_t* tok_end, int64_t T, int64_t k0) {
-    const int64_t last_key = (k0 + kBlk <= T ? k0 + kBlk : T) - 1;
-    return (tok_end[last_key] - 1) / kBlk;
 }
 
 #ifdef LIBRA_PROF
@@ -104,12 +58,55 @@ struct Prof {
 #define PROF_FLUSH(cond, base)
 #endif
 
+// =================================================================================================
+// dK / dV kernel
+// =================================================================================================
+
+template <int D>
+struct DkvSmem {
+    static constexpr int kHalfBytes = 128 * 128;
+    static constexpr int kTileBytes = kHalfBytes * (D / 64);  // 128 x D bf16
+    static constexpr int kKOff = 0;
+    static constexpr int kVOff = kTileBytes;
+    static constexpr int kQOff = 2 * kTileBytes;   // 2 stages
+    static constexpr int kDoOff = 4 * kTileBytes;  // 2 stages
+    static constexpr int kStatOff = 6 * kTileBytes;  // per Q stage: lse2[128], dvec[128]
+    static constexpr int kBarOff = kStatOff + 2 * 1024;
+    // kv_full, kv_empty, q_full[2], q_empty[2], do_full[2], do_empty[2], s_full, p_ready, dp_full,
+    // ds_ready, dkv_full, dkv_empty
+    static constexpr int kNumBars = 16;
+    static constexpr int kMiscOff = kBarOff + kNumBars * 8;
+    static constexpr int kBytes = kMiscOff + 16;
+    static_assert(kBytes <= kSmemMax, "exceeds the shared memory of an sm_100 CTA");
+};
+
+struct DkvParams {
+    __nv_bfloat16* dk;
+    __nv_bfloat16* dv;
+    const float* lse2;  // [Hq, Tpad]  LSE * log2(e)
+    const float* dvec;  // [Hq, Tpad]  D_i
+    const int32_t* cta_offsets;
+    const int32_t* cta_tiles;
+    const int32_t* tok_end;
+    int64_t T, Tpad;
+    int hq, hkv;
+    float scale, scale_log2;
+    int* status;
+    uint64_t* busy;
+};
+
+// Query blocks a key block [k0, k0+128) is seen by: diagonal .. block of (end of last key's sample - 1).
+__device__ __forceinline__ int last_q_block(const int32_t* tok_end, int64_t T, int64_t k0) {
+    const int64_t last_key = (k0 + kBlk <= T ? k0 + kBlk : T) - 1;
+    return (tok_end[last_key] - 1) / kBlk;
+}
+
 template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 1)
-k_attn_bwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-           const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do, const __grid_constant__ CUtensorMap tm_dq,
-           const BwdParams p) {
-    using L = BwdSmem<D>;
+k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
+                const DkvParams p) {
+    using L = DkvSmem<D>;
     extern __shared__ __align__(1024) uint8_t smem[];
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBarOff);
     uint64_t* bar_kvfull = bars + 0;
@@ -122,10 +119,8 @@ k_attn_bwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     uint64_t* bar_pready = bars + 11;
     uint64_t* bar_dpfull = bars + 12;
     uint64_t* bar_dsready = bars + 13;
-    uint64_t* bar_dqfull = bars + 14;
-    uint64_t* bar_dqempty = bars + 15;
-    uint64_t* bar_dkvfull = bars + 16;
-    uint64_t* bar_dkvempty = bars + 17;
+    uint64_t* bar_dkvfull = bars + 14;
+    uint64_t* bar_dkvempty = bars + 15;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::kMiscOff);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kMiscOff + 4);
 
@@ -150,24 +145,21 @@ k_attn_bwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         mbar_init(bar_pready, 256);
         mbar_init(bar_dpfull, 1);
         mbar_init(bar_dsready, 256);
-        mbar_init(bar_dqfull, 1);
-        mbar_init(bar_dqempty, 128);
         mbar_init(bar_dkvfull, 1);
         mbar_init(bar_dkvempty, 256);
         *abort_flag = 0;
         fence_mbar_init();
         p.busy[2 * cta] = globaltimer_ns();
     }
-    if (warp == 13) {
+    if (warp == 9) {
         tmem_alloc(tmem_slot, 512);
         tmem_relinquish();
     }
-    if (warp == 12 && lane == 0) {
+    if (warp == 8 && lane == 0) {
         prefetch_tmap(&tm_q);
         prefetch_tmap(&tm_k);
         prefetch_tmap(&tm_v);
         prefetch_tmap(&tm_do);
-        prefetch_tmap(&tm_dq);
     }
     tc_fence_before();
     __syncthreads();
@@ -179,7 +171,7 @@ k_attn_bwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     const int unit_end = p.cta_offsets[cta + 1];
     const int G = p.hq / p.hkv;
 
-    if (warp == 12) {
+    if (warp == 8) {
         // ---------------- TMA producer ----------------
         uint32_t ucnt = 0, it_all = 0;
         bool ok = true;
@@ -215,23 +207,20 @@ k_attn_bwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                     bulk_load_1d(smem + L::kStatOff + st * 1024 + 512, p.dvec + (size_t)h * p.Tpad + qb, 512,
                                  &bar_qfull[st]);
                 }
-                const uint32_t dst = it_all % L::kDoStages, dpar = ((it_all / L::kDoStages) & 1) ^ 1;
-                ok = warp_wait_b(&bar_doempty[dst], dpar, abort_flag);
+                ok = warp_wait_b(&bar_doempty[st], par, abort_flag);
                 if (!ok) break;
                 if (lane == 0) {
-                    mbar_arrive_expect_tx(&bar_dofull[dst], L::kTileBytes);
+                    mbar_arrive_expect_tx(&bar_dofull[st], L::kTileBytes);
                     for (int half = 0; half < D / 64; ++half)
-                        tma_load_3d(smem + L::kDoOff + dst * L::kTileBytes + half * L::kHalfBytes, &tm_do,
-                                    &bar_dofull[dst], half * 64, h, qb);
+                        tma_load_3d(smem + L::kDoOff + st * L::kTileBytes + half * L::kHalfBytes, &tm_do,
+                                    &bar_dofull[st], half * 64, h, qb);
                 }
             }
         }
-    } else if (warp == 13) {
+    } else if (warp == 9) {
         // ---------------- MMA issuer ----------------
-        constexpr uint32_t idesc_s = make_idesc(128, 128, 0, 0);   // S^T, dP^T: both operands K-major
-        constexpr uint32_t idesc_dv = make_idesc(128, D, 0, 1);    // A from TMEM, B = dO MN-major
-        constexpr uint32_t idesc_dk = make_idesc(128, D, 0, 1);    // A = dS^T K-major, B = Q MN-major
-        constexpr uint32_t idesc_dq = make_idesc(128, D, 1, 1);    // A = dS MN-major, B = K MN-major
+        constexpr uint32_t idesc_s = make_idesc(128, 128, 0, 0);  // S^T, dP^T: both operands K-major
+        constexpr uint32_t idesc_acc = make_idesc(128, D, 0, 1);  // dV, dK: A from TMEM, B MN-major
         const uint32_t sb = smem_u32(smem);
         uint32_t ucnt = 0, it_all = 0;
         bool ok = true;
@@ -245,6 +234,13 @@ k_attn_bwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                        idesc_s, kk > 0);
             }
         };
+        // C[tmem] (+)= A(TMEM, bf16 packed: queries 64c.. at columns a_col + 64c ..) * B(MN-major tile)
+        auto issue_acc = [&](uint32_t d_col, uint32_t a_col, uint32_t b_addr, bool accumulate) {
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk)  // 16 queries per step
+                mma_ts(tmem_base + d_col, tmem_base + a_col + (kk / 4) * 64 + (kk % 4) * 8,
+                       make_sdesc(b_addr + kk * 2048, L::kHalfBytes, 1024), idesc_acc, (accumulate || kk > 0) ? 1u : 0u);
+        };
         for (int idx = unit_begin; idx < unit_end && ok; ++idx) {
             const int t = p.cta_tiles[idx];
             const int64_t k0 = (int64_t)(t / p.hkv) * kBlk;
@@ -253,7 +249,7 @@ k_attn_bwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             const int n_it = G * nblk;
             ok = warp_wait_b(bar_kvfull, ucnt & 1, abort_flag);
             if (!ok) break;
-            // S(0)
+            // S(0), dP(0)
             ok = warp_wait_b(&bar_qfull[it_all & 1], (it_all >> 1) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
@@ -261,73 +257,61 @@ k_attn_bwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 issue_kmajor(kColS, sb + L::kKOff, sb + L::kQOff + (it_all & 1) * L::kTileBytes);
                 tc_commit(bar_sfull);
             }
+            ok = warp_wait_b(&bar_dofull[it_all & 1], (it_all >> 1) & 1, abort_flag);
+            if (!ok) break;
+            if (lane == 0) {
+                issue_kmajor(kColDP, sb + L::kVOff, sb + L::kDoOff + (it_all & 1) * L::kTileBytes);
+                tc_commit(bar_dpfull);
+            }
             for (int it = 0; it < n_it && ok; ++it, ++it_all) {
-                const uint32_t st = it_all & 1, par = (it_all >> 1) & 1;
-                // dP(it): needs dO and the dP/dQ columns drained of dQ(it-1)
-                const uint32_t dst = it_all % L::kDoStages, dpar = (it_all / L::kDoStages) & 1;
-                PROF(7)
-                ok = warp_wait_b(&bar_dofull[dst], dpar, abort_flag);
-                if (!ok) break;
-                PROF(0)
-                if (it_all > 0) {
-                    ok = warp_wait_b(bar_dqempty, (it_all - 1) & 1, abort_flag);
-                    if (!ok) break;
-                }
-                PROF(1)
-                tc_fence_after();
-                if (lane == 0) {
-                    issue_kmajor(kColDP, sb + L::kVOff, sb + L::kDoOff + dst * L::kTileBytes);
-                    tc_commit(bar_dpfull);
-                }
+                const uint32_t st = it_all & 1;
+                const uint32_t nx = it_all + 1;
+                const bool more = it + 1 < n_it;
                 // dV(it) += P^T dO
                 PROF(7)
                 ok = warp_wait_b(bar_pready, it_all & 1, abort_flag);
                 if (!ok) break;
-                PROF(2)
+                PROF(0)
                 if (it == 0 && ucnt > 0) {  // previous unit's dK/dV must have been read out
                     ok = warp_wait_b(bar_dkvempty, (ucnt - 1) & 1, abort_flag);
                     if (!ok) break;
                 }
                 tc_fence_after();
                 if (lane == 0) {
-                    const uint32_t doa = sb + L::kDoOff + dst * L::kTileBytes;
-#pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)  // 16 queries per step; P^T of columns 64c.. lives at 64c + ..
-                        mma_ts(tmem_base + kColDV, tmem_base + kColS + (kk / 4) * 64 + (kk % 4) * 8,
-                               make_sdesc(doa + kk * 2048, L::kHalfBytes, 1024), idesc_dv, (it > 0 || kk > 0) ? 1u : 0u);
-                    tc_commit(&bar_doempty[dst]);
+                    issue_acc(kColDV, kColS, sb + L::kDoOff + st * L::kTileBytes, it > 0);
+                    tc_commit(&bar_doempty[st]);
                 }
                 // S(it+1)
-                if (it + 1 < n_it) {
-                    const uint32_t nx = it_all + 1;
+                if (more) {
                     PROF(7)
                     ok = warp_wait_b(&bar_qfull[nx & 1], (nx >> 1) & 1, abort_flag);
                     if (!ok) break;
-                    PROF(3)
+                    PROF(1)
                     if (lane == 0) {
                         issue_kmajor(kColS, sb + L::kKOff, sb + L::kQOff + (nx & 1) * L::kTileBytes);
                         tc_commit(bar_sfull);
                     }
                 }
-                // dK(it) += dS^T Q ; dQ(it) = dS K
+                // dK(it) += dS^T Q
                 PROF(7)
                 ok = warp_wait_b(bar_dsready, it_all & 1, abort_flag);
                 if (!ok) break;
-                PROF(4)
+                PROF(2)
                 tc_fence_after();
                 if (lane == 0) {
-                    const uint32_t dsa = sb + L::kDsOff;
-                    const uint32_t qa = sb + L::kQOff + st * L::kTileBytes;
-#pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)  // over 16 queries
-                        mma_ss(tmem_base + kColDK, make_sdesc(dsa + (kk / 4) * L::kHalfBytes + (kk % 4) * 32, 16, 1024),
-                               make_sdesc(qa + kk * 2048, L::kHalfBytes, 1024), idesc_dk, (it > 0 || kk > 0) ? 1u : 0u);
+                    issue_acc(kColDK, kColDP, sb + L::kQOff + st * L::kTileBytes, it > 0);
                     tc_commit(&bar_qempty[st]);
-#pragma unroll
-                    for (int kk = 0; kk < 8; ++kk)  // over 16 keys
-                        mma_ss(tmem_base + kColDP, make_sdesc(dsa + kk * 2048, L::kHalfBytes, 1024),
-                               make_sdesc(sb + L::kKOff + kk * 2048, L::kHalfBytes, 1024), idesc_dq, kk > 0);
-                    tc_commit(bar_dqfull);
+                }
+                // dP(it+1)
+                if (more) {
+                    PROF(7)
+                    ok = warp_wait_b(&bar_dofull[nx & 1], (nx >> 1) & 1, abort_flag);
+                    if (!ok) break;
+                    PROF(3)
+                    if (lane == 0) {
+                        issue_kmajor(kColDP, sb + L::kVOff, sb + L::kDoOff + (nx & 1) * L::kTileBytes);
+                        tc_commit(bar_dpfull);
+                    }
                 }
                 __syncwarp();
             }
@@ -339,71 +323,6 @@ k_attn_bwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             ++ucnt;
         }
         PROF_FLUSH(lane == 0, 8)
-    } else if (warp >= 12) {
-        // warps 14-15: nothing to do
-    } else if (warp >= 8) {
-        // ---------------- dQ reduce group ----------------
-        // TMEM -> registers (whole tile, frees the columns at once) -> 32-column chunks through two
-        // staging buffers -> TMA reduce-add into the fp32 accumulator (full 128-byte lines).
-        const int r = (warp & 3) * 32 + lane;
-        const bool leader = (threadIdx.x == 8 * 32);
-        const uint32_t t_dq = tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + kColDP;
-        uint8_t* stage_row = smem + L::kStageOff + r * 128;
-        uint32_t it_all = 0;
-        bool ok = true;
-        PROF_DECL
-        for (int idx = unit_begin; idx < unit_end && ok; ++idx) {
-            const int t = p.cta_tiles[idx];
-            const int kvh = t % p.hkv;
-            const int64_t k0 = (int64_t)(t / p.hkv) * kBlk;
-            const int i_lo = (int)(k0 / kBlk);
-            const int nblk = last_q_block(p.tok_end, p.T, k0) - i_lo + 1;
-            const int n_it = G * nblk;
-            for (int it = 0; it < n_it && ok; ++it, ++it_all) {
-                const int h = kvh * G + it / nblk;
-                const int qb = (i_lo + it % nblk) * kBlk;
-                ok = mbar_wait(bar_dqfull, it_all & 1, abort_flag);
-                if (!ok) break;
-                PROF(0)
-                tc_fence_after();
-                uint32_t v[D];
-#pragma unroll
-                for (int c = 0; c < D; c += 32) tmem_ld32(t_dq + c, v + c);
-                tmem_ld_wait();
-                tc_fence_before();
-                mbar_arrive(bar_dqempty);  // the dP/dQ columns may be overwritten now
-                PROF(1)
-#pragma unroll
-                for (int c = 0; c < D / 32; ++c) {
-                    uint8_t* dst = stage_row + (c & 1) * L::kHalfBytes;
-                    // the buffer may still be read by the reduce issued two chunks ago
-                    if (leader) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-                    asm volatile("bar.sync 1, 128;" ::: "memory");
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) {
-                        uint4 w;
-                        w.x = v[c * 32 + k * 4]; w.y = v[c * 32 + k * 4 + 1];
-                        w.z = v[c * 32 + k * 4 + 2]; w.w = v[c * 32 + k * 4 + 3];
-                        *reinterpret_cast<uint4*>(dst + ((k ^ (r & 7)) << 4)) = w;
-                    }
-                    fence_proxy_async_smem();
-                    asm volatile("bar.sync 1, 128;" ::: "memory");
-                    if (leader) {
-#ifndef LIBRA_DBG_NO_RED
-                        asm volatile(
-                            "cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];"
-                            ::"l"(reinterpret_cast<uint64_t>(&tm_dq)), "r"(h * D + c * 32), "r"(qb),
-                            "r"(smem_u32(smem + L::kStageOff + (c & 1) * L::kHalfBytes))
-                            : "memory");
-#endif
-                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                    }
-                }
-                PROF(2)
-            }
-        }
-        if (leader) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // all reduce-adds done before exit
-        PROF_FLUSH(leader, 16)
     } else {
         // ---------------- compute groups ----------------
         const int c = warp >> 2;  // query-column half of each key row
@@ -411,7 +330,6 @@ k_attn_bwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t t_s = tmem_base + lane_addr + kColS + 64 * c;
         const uint32_t t_dp = tmem_base + lane_addr + kColDP + 64 * c;
-        uint8_t* ds_row = smem + L::kDsOff + c * L::kHalfBytes + r * 128;
         uint32_t ucnt = 0, it_all = 0;
         bool ok = true;
         PROF_DECL
@@ -433,8 +351,8 @@ k_attn_bwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 const float* lse2 = reinterpret_cast<const float*>(smem + L::kStatOff + st * 1024) + 64 * c;
                 const float* dvec = lse2 + 128;
                 const bool need_mask = (qb == k0) || (qb + kBlk - 1 >= min_kend) || partial;
-                const int j_lo = (int)(key - qb) - 64 * c;       // first visible column of this half
-                const int j_hi = kend - 1 - qb - 64 * c;         // last visible column
+                const int j_lo = (int)(key - qb) - 64 * c;  // first visible column of this half
+                const int j_hi = kend - 1 - qb - 64 * c;    // last visible column
                 // ---- exp phase: P^T = exp2(S^T * c - LSE) ----
                 ok = mbar_wait(&bar_qfull[st], par, abort_flag) && mbar_wait(bar_sfull, it_all & 1, abort_flag);
                 if (!ok) break;
@@ -468,7 +386,7 @@ k_attn_bwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 tc_fence_before();
                 mbar_arrive(bar_pready);
                 PROF(1)
-                // ---- dS phase: dS^T = P^T o (dP^T - D) ----
+                // ---- dS phase: dS^T = P^T o (dP^T - D), packed over this half's own dP^T columns ----
                 ok = mbar_wait(bar_dpfull, it_all & 1, abort_flag);
                 if (!ok) break;
                 PROF(2)
@@ -477,25 +395,22 @@ k_attn_bwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 tmem_ld32(t_dp, dpv);
                 tmem_ld32(t_dp + 32, dpv + 32);
                 tmem_ld_wait();
-                PROF(3)
-                PROF(4)
+                {
+                    uint32_t pk[32];
 #pragma unroll
-                for (int ch = 0; ch < 8; ++ch) {
-                    const float4 d0 = *reinterpret_cast<const float4*>(dvec + ch * 8);
-                    const float4 d1 = *reinterpret_cast<const float4*>(dvec + ch * 8 + 4);
-                    const int j = ch * 8;
-                    uint4 w;
-                    w.x = pack_bf16x2(pf[j] * (__uint_as_float(dpv[j]) - d0.x), pf[j + 1] * (__uint_as_float(dpv[j + 1]) - d0.y));
-                    w.y = pack_bf16x2(pf[j + 2] * (__uint_as_float(dpv[j + 2]) - d0.z), pf[j + 3] * (__uint_as_float(dpv[j + 3]) - d0.w));
-                    w.z = pack_bf16x2(pf[j + 4] * (__uint_as_float(dpv[j + 4]) - d1.x), pf[j + 5] * (__uint_as_float(dpv[j + 5]) - d1.y));
-                    w.w = pack_bf16x2(pf[j + 6] * (__uint_as_float(dpv[j + 6]) - d1.z), pf[j + 7] * (__uint_as_float(dpv[j + 7]) - d1.w));
-                    *reinterpret_cast<uint4*>(ds_row + ((ch ^ (r & 7)) << 4)) = w;
+                    for (int j = 0; j < 64; j += 4) {
+                        const float4 d4 = *reinterpret_cast<const float4*>(dvec + j);
+                        pk[j >> 1] = pack_bf16x2(pf[j] * (__uint_as_float(dpv[j]) - d4.x),
+                                                 pf[j + 1] * (__uint_as_float(dpv[j + 1]) - d4.y));
+                        pk[(j >> 1) + 1] = pack_bf16x2(pf[j + 2] * (__uint_as_float(dpv[j + 2]) - d4.z),
+                                                       pf[j + 3] * (__uint_as_float(dpv[j + 3]) - d4.w));
+                    }
+                    tmem_st32(t_dp, pk);
                 }
-                PROF(5)
-                fence_proxy_async_smem();
+                tmem_st_wait();
                 tc_fence_before();
                 mbar_arrive(bar_dsready);
-                PROF(7)
+                PROF(3)
             }
             if (!ok) break;
             // ---- unit epilogue: dK * scale and dV to global ----
@@ -531,7 +446,7 @@ k_attn_bwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             tc_fence_before();
             mbar_arrive(bar_dkvempty);
             ++ucnt;
-            PROF(6)
+            PROF(4)
         }
         PROF_FLUSH(threadIdx.x == 0, 0)
     }
@@ -539,14 +454,367 @@ k_attn_bwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     // ---------------- teardown ----------------
     tc_fence_before();
     __syncthreads();
-    if (warp == 13) tmem_dealloc(tmem_base, 512);
+    if (warp == 9) tmem_dealloc(tmem_base, 512);
     if (threadIdx.x == 0) {
         if (*abort_flag) atomicExch(p.status, LIBRA_ERR_TIMEOUT);
         p.busy[2 * cta + 1] = globaltimer_ns();
     }
 }
 
-// ---- prep and post kernels --------------------------------------------------------------------
+// =================================================================================================
+// dQ kernel
+// =================================================================================================
+
+template <int D>
+struct DqSmem {
+    static constexpr int kHalfBytes = 128 * 128;
+    static constexpr int kTileBytes = kHalfBytes * (D / 64);
+    static constexpr int kKStages = 3;  // K_j lives from S(j) (issued two blocks ahead) to dQ(j)
+    static constexpr int kVStages = 2;
+    static constexpr int kQOff = 0;
+    static constexpr int kDoOff = kTileBytes;
+    static constexpr int kKOff = 2 * kTileBytes;
+    static constexpr int kVOff = kKOff + kKStages * kTileBytes;
+    static constexpr int kBarOff = kVOff + kVStages * kTileBytes;
+    // q_full, q_empty, k_full[3], k_empty[3], v_full[2], v_empty[2], s_full[2], dp_full, ds_ready, dq_full,
+    // do_full, do_empty
+    static constexpr int kNumBars = 19;
+    static constexpr int kMiscOff = kBarOff + kNumBars * 8;
+    static constexpr int kBytes = kMiscOff + 16;
+    static_assert(kBytes <= kSmemMax, "exceeds the shared memory of an sm_100 CTA");
+};
+
+struct DqParams {
+    __nv_bfloat16* dq;
+    const float* lse2;
+    const float* dvec;
+    const int32_t* cta_offsets;
+    const int32_t* cta_tiles;
+    const int32_t* tok_start;
+    int64_t T, Tpad;
+    int hq, hkv, H;
+    float scale, scale_log2;
+    int* status;
+    uint64_t* busy;
+};
+
+template <int D>
+__global__ void __launch_bounds__(kBwdThreads, 1)
+k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+              const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do, const DqParams p) {
+    using L = DqSmem<D>;
+    extern __shared__ __align__(1024) uint8_t smem[];
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBarOff);
+    uint64_t* bar_qfull = bars + 0;
+    uint64_t* bar_qempty = bars + 1;
+    uint64_t* bar_dofull = bars + 17;
+    uint64_t* bar_doempty = bars + 18;
+    uint64_t* bar_kfull = bars + 2;    // [3]
+    uint64_t* bar_kempty = bars + 5;   // [3]
+    uint64_t* bar_vfull = bars + 8;    // [2]
+    uint64_t* bar_vempty = bars + 10;  // [2]
+    uint64_t* bar_sfull = bars + 12;   // [2]
+    uint64_t* bar_dpfull = bars + 14;
+    uint64_t* bar_dsready = bars + 15;
+    uint64_t* bar_dqfull = bars + 16;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::kMiscOff);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kMiscOff + 4);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int cta = blockIdx.x;
+
+    if ((smem_u32(smem) & 1023u) != 0) {
+        if (threadIdx.x == 0) atomicExch(p.status, LIBRA_ERR_CUDA);
+        return;
+    }
+    if (threadIdx.x == 0) {
+        mbar_init(bar_qfull, 1);
+        mbar_init(bar_qempty, 1);
+        mbar_init(bar_dofull, 1);
+        mbar_init(bar_doempty, 1);
+        for (int s = 0; s < L::kKStages; ++s) { mbar_init(&bar_kfull[s], 1); mbar_init(&bar_kempty[s], 1); }
+        for (int s = 0; s < L::kVStages; ++s) { mbar_init(&bar_vfull[s], 1); mbar_init(&bar_vempty[s], 1); }
+        mbar_init(&bar_sfull[0], 1);
+        mbar_init(&bar_sfull[1], 1);
+        mbar_init(bar_dpfull, 1);
+        mbar_init(bar_dsready, 256);
+        mbar_init(bar_dqfull, 1);
+        *abort_flag = 0;
+        fence_mbar_init();
+        p.busy[2 * cta] = globaltimer_ns();
+    }
+    if (warp == 9) {
+        tmem_alloc(tmem_slot, 512);
+        tmem_relinquish();
+    }
+    if (warp == 8 && lane == 0) {
+        prefetch_tmap(&tm_q);
+        prefetch_tmap(&tm_k);
+        prefetch_tmap(&tm_v);
+        prefetch_tmap(&tm_do);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    constexpr uint32_t kColS = 0 /* two buffers: 0 and 128 */, kColDP = 256, kColDQ = 384;
+
+    const int tile_begin = p.cta_offsets[cta];
+    const int tile_end = p.cta_offsets[cta + 1];
+    const int heads_per_shard = p.hq / p.H;
+    const int G = p.hq / p.hkv;
+
+    // All roles walk the same sequence of sub-blocks: (tile, sub-block of 128 rows, head of the shard).
+    // A sub-block past the end of the pool is skipped by every role.
+    if (warp == 8) {
+        // ---------------- TMA producer ----------------
+        uint32_t bcnt = 0, kcnt = 0, vcnt = 0;
+        bool ok = true;
+        for (int idx = tile_begin; idx < tile_end && ok; ++idx) {
+            const int t = p.cta_tiles[idx];
+            for (int sub = 0; sub < 2 && ok; ++sub) {
+                const int64_t q0 = (int64_t)(t / p.H) * (2 * kBlk) + sub * kBlk;
+                if (q0 >= p.T) continue;
+                const int lo = p.tok_start[q0] / kBlk, hi = (int)(q0 / kBlk);
+                for (int hh = 0; hh < heads_per_shard && ok; ++hh) {
+                    const int h = (t % p.H) * heads_per_shard + hh;
+                    const int kvh = h / G;
+                    ok = warp_wait_b(bar_qempty, (bcnt & 1) ^ 1, abort_flag);
+                    if (!ok) break;
+                    if (lane == 0) {
+                        mbar_arrive_expect_tx(bar_qfull, L::kTileBytes);
+                        for (int half = 0; half < D / 64; ++half)
+                            tma_load_3d(smem + L::kQOff + half * L::kHalfBytes, &tm_q, bar_qfull, half * 64, h, (int)q0);
+                    }
+                    ok = warp_wait_b(bar_doempty, (bcnt & 1) ^ 1, abort_flag);
+                    if (!ok) break;
+                    if (lane == 0) {
+                        mbar_arrive_expect_tx(bar_dofull, L::kTileBytes);
+                        for (int half = 0; half < D / 64; ++half)
+                            tma_load_3d(smem + L::kDoOff + half * L::kHalfBytes, &tm_do, bar_dofull, half * 64, h, (int)q0);
+                    }
+                    ++bcnt;
+                    for (int j = lo; j <= hi && ok; ++j) {
+                        const uint32_t ks = kcnt % L::kKStages;
+                        ok = warp_wait_b(&bar_kempty[ks], ((kcnt / L::kKStages) & 1) ^ 1, abort_flag);
+                        if (!ok) break;
+                        if (lane == 0) {
+                            mbar_arrive_expect_tx(&bar_kfull[ks], L::kTileBytes);
+                            for (int half = 0; half < D / 64; ++half)
+                                tma_load_3d(smem + L::kKOff + ks * L::kTileBytes + half * L::kHalfBytes, &tm_k,
+                                            &bar_kfull[ks], half * 64, kvh, j * kBlk);
+                        }
+                        ++kcnt;
+                        const uint32_t vs = vcnt % L::kVStages;
+                        ok = warp_wait_b(&bar_vempty[vs], ((vcnt / L::kVStages) & 1) ^ 1, abort_flag);
+                        if (!ok) break;
+                        if (lane == 0) {
+                            mbar_arrive_expect_tx(&bar_vfull[vs], L::kTileBytes);
+                            for (int half = 0; half < D / 64; ++half)
+                                tma_load_3d(smem + L::kVOff + vs * L::kTileBytes + half * L::kHalfBytes, &tm_v,
+                                            &bar_vfull[vs], half * 64, kvh, j * kBlk);
+                        }
+                        ++vcnt;
+                    }
+                }
+            }
+        }
+    } else if (warp == 9) {
+        // ---------------- MMA issuer ----------------
+        constexpr uint32_t idesc_s = make_idesc(128, 128, 0, 0);  // S, dP: both operands K-major
+        constexpr uint32_t idesc_dq = make_idesc(128, D, 0, 1);   // dQ: A from TMEM, B = K MN-major
+        const uint32_t sb = smem_u32(smem);
+        uint32_t bcnt = 0, kcnt = 0, vcnt = 0, scnt = 0, dscnt = 0;
+        bool ok = true;
+        auto issue_kmajor = [&](uint32_t d_col, uint32_t a_addr, uint32_t b_addr) {
+#pragma unroll
+            for (int kk = 0; kk < D / 16; ++kk) {
+                const uint32_t off = (kk / 4) * L::kHalfBytes + (kk % 4) * 32;
+                mma_ss(tmem_base + d_col, make_sdesc(a_addr + off, 16, 1024), make_sdesc(b_addr + off, 16, 1024),
+                       idesc_s, kk > 0);
+            }
+        };
+        // S(j) into buffer scnt & 1 from K ring entry kidx; waits for the K tile first.  `last`: no later
+        // MMA of this sub-block reads Q, so the Q buffer is handed back for the next load.
+        auto do_s = [&](uint32_t kidx, bool last) -> bool {
+            if (!warp_wait_b(&bar_kfull[kidx % L::kKStages], (kidx / L::kKStages) & 1, abort_flag)) return false;
+            if (lane == 0) {
+                issue_kmajor(kColS + (scnt & 1) * 128, sb + L::kQOff, sb + L::kKOff + (kidx % L::kKStages) * L::kTileBytes);
+                tc_commit(&bar_sfull[scnt & 1]);
+                if (last) tc_commit(bar_qempty);
+            }
+            ++scnt;
+            return true;
+        };
+        auto do_dp = [&](bool last) -> bool {
+            const uint32_t vs = vcnt % L::kVStages;
+            if (!warp_wait_b(&bar_vfull[vs], (vcnt / L::kVStages) & 1, abort_flag)) return false;
+            if (lane == 0) {
+                issue_kmajor(kColDP, sb + L::kDoOff, sb + L::kVOff + vs * L::kTileBytes);
+                tc_commit(bar_dpfull);
+                tc_commit(&bar_vempty[vs]);
+                if (last) tc_commit(bar_doempty);
+            }
+            ++vcnt;
+            return true;
+        };
+        for (int idx = tile_begin; idx < tile_end && ok; ++idx) {
+            const int t = p.cta_tiles[idx];
+            for (int sub = 0; sub < 2 && ok; ++sub) {
+                const int64_t q0 = (int64_t)(t / p.H) * (2 * kBlk) + sub * kBlk;
+                if (q0 >= p.T) continue;
+                const int lo = p.tok_start[q0] / kBlk, hi = (int)(q0 / kBlk);
+                for (int hh = 0; hh < heads_per_shard && ok; ++hh) {
+                    ok = warp_wait_b(bar_qfull, bcnt & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t kbase = kcnt;  // ring index of K_lo
+                    ok = do_s(kbase, lo == hi);                                      // S(lo)
+                    if (ok) ok = warp_wait_b(bar_dofull, bcnt & 1, abort_flag);
+                    ++bcnt;
+                    if (ok) ok = do_dp(lo == hi);                                    // dP(lo)
+                    if (ok && lo + 1 <= hi) ok = do_s(kbase + 1, lo + 1 == hi);      // S(lo+1)
+                    if (!ok) break;
+                    for (int j = lo; j <= hi && ok; ++j) {
+                        // dQ += dS(j) K_j
+                        ok = warp_wait_b(bar_dsready, dscnt & 1, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint32_t kidx = kbase + (j - lo);
+                        if (lane == 0) {
+                            const uint32_t ka = sb + L::kKOff + (kidx % L::kKStages) * L::kTileBytes;
+                            const uint32_t a_col = kColS + (dscnt & 1) * 128;  // dS(j) sits in S(j)'s buffer
+#pragma unroll
+                            for (int kk = 0; kk < 8; ++kk)  // 16 keys per step
+                                mma_ts(tmem_base + kColDQ, tmem_base + a_col + (kk / 4) * 64 + (kk % 4) * 8,
+                                       make_sdesc(ka + kk * 2048, L::kHalfBytes, 1024), idesc_dq,
+                                       (j > lo || kk > 0) ? 1u : 0u);
+                            tc_commit(&bar_kempty[kidx % L::kKStages]);
+                        }
+                        ++dscnt;
+                        if (j + 1 <= hi) ok = do_dp(j + 1 == hi);                              // dP(j+1)
+                        if (ok && j + 2 <= hi) ok = do_s(kbase + (j + 2 - lo), j + 2 == hi);  // S(j+2) into dS(j)'s buffer
+                        __syncwarp();
+                    }
+                    if (!ok) break;
+                    kcnt = kbase + (hi - lo + 1);
+                    if (lane == 0) tc_commit(bar_dqfull);
+                    __syncwarp();
+                }
+            }
+        }
+    } else {
+        // ---------------- compute groups ----------------
+        const int c = warp >> 2;  // key-column half of each query row
+        const int r = (warp & 3) * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+        uint32_t scnt = 0, dpcnt = 0, bcnt = 0;
+        bool ok = true;
+        for (int idx = tile_begin; idx < tile_end && ok; ++idx) {
+            const int t = p.cta_tiles[idx];
+            for (int sub = 0; sub < 2 && ok; ++sub) {
+                const int64_t q0 = (int64_t)(t / p.H) * (2 * kBlk) + sub * kBlk;
+                if (q0 >= p.T) continue;
+                const int lo = p.tok_start[q0] / kBlk, hi = (int)(q0 / kBlk);
+                const int64_t row = q0 + r;
+                const bool row_ok = row < p.T;
+                const int kstart = row_ok ? p.tok_start[row] : 0;
+                const int64_t last_row = (q0 + kBlk <= p.T ? q0 + kBlk : p.T) - 1;
+                const int max_kstart = p.tok_start[last_row];
+                for (int hh = 0; hh < heads_per_shard && ok; ++hh) {
+                    const int h = (t % p.H) * heads_per_shard + hh;
+                    const float lse2 = p.lse2[(size_t)h * p.Tpad + row];  // padded rows hold zeros
+                    const float dsum = p.dvec[(size_t)h * p.Tpad + row];
+                    for (int j = lo; j <= hi && ok; ++j) {
+                        const uint32_t buf = scnt & 1;
+                        const uint32_t t_s = tmem_base + lane_addr + kColS + buf * 128 + 64 * c;
+                        const uint32_t t_dp = tmem_base + lane_addr + kColDP + 64 * c;
+                        const int k0 = j * kBlk;
+                        const bool need_mask = (j == hi) || (k0 < max_kstart) || !row_ok;
+                        const int c_lo = (row_ok ? kstart - k0 : kBlk) - 64 * c;    // first visible column of this half
+                        const int c_hi = (row_ok ? (int)(row - k0) : -1) - 64 * c;  // last visible column
+                        // ---- P = exp2(S c - LSE) ----
+                        ok = mbar_wait(&bar_sfull[buf], (scnt >> 1) & 1, abort_flag);
+                        if (!ok) break;
+                        ++scnt;
+                        tc_fence_after();
+                        uint32_t sv[64];
+                        tmem_ld32(t_s, sv);
+                        tmem_ld32(t_s + 32, sv + 32);
+                        tmem_ld_wait();
+                        float pf[64];
+#pragma unroll
+                        for (int i = 0; i < 64; ++i) pf[i] = ex2_approx(fmaf(__uint_as_float(sv[i]), p.scale_log2, -lse2));
+                        if (need_mask) {
+#pragma unroll
+                            for (int i = 0; i < 64; ++i)
+                                if (i < c_lo || i > c_hi) pf[i] = 0.f;
+                        }
+                        // ---- dS = P o (dP - D), packed over this half's own S columns ----
+                        ok = mbar_wait(bar_dpfull, dpcnt & 1, abort_flag);
+                        if (!ok) break;
+                        ++dpcnt;
+                        tc_fence_after();
+                        uint32_t dpv[64];
+                        tmem_ld32(t_dp, dpv);
+                        tmem_ld32(t_dp + 32, dpv + 32);
+                        tmem_ld_wait();
+                        {
+                            uint32_t pk[32];
+#pragma unroll
+                            for (int i = 0; i < 64; i += 2)
+                                pk[i >> 1] = pack_bf16x2(pf[i] * (__uint_as_float(dpv[i]) - dsum),
+                                                         pf[i + 1] * (__uint_as_float(dpv[i + 1]) - dsum));
+                            tmem_st32(t_s, pk);
+                        }
+                        tmem_st_wait();
+                        tc_fence_before();
+                        mbar_arrive(bar_dsready);
+                    }
+                    if (!ok) break;
+                    // ---- epilogue: dQ * scale to global ----
+                    ok = mbar_wait(bar_dqfull, bcnt & 1, abort_flag);
+                    if (!ok) break;
+                    ++bcnt;
+                    tc_fence_after();
+                    constexpr int kCols = D / 2;
+                    const uint32_t t_dq = tmem_base + lane_addr + kColDQ + c * kCols;
+                    __nv_bfloat16* gdst = p.dq + ((size_t)row * p.hq + h) * D + c * kCols;
+#pragma unroll
+                    for (int cc = 0; cc < kCols; cc += 32) {
+                        uint32_t v[32];
+                        tmem_ld32(t_dq + cc, v);
+                        tmem_ld_wait();
+                        if (row_ok) {
+#pragma unroll
+                            for (int i = 0; i < 32; i += 8) {
+                                uint4 w;
+                                w.x = pack_bf16x2(__uint_as_float(v[i]) * p.scale, __uint_as_float(v[i + 1]) * p.scale);
+                                w.y = pack_bf16x2(__uint_as_float(v[i + 2]) * p.scale, __uint_as_float(v[i + 3]) * p.scale);
+                                w.z = pack_bf16x2(__uint_as_float(v[i + 4]) * p.scale, __uint_as_float(v[i + 5]) * p.scale);
+                                w.w = pack_bf16x2(__uint_as_float(v[i + 6]) * p.scale, __uint_as_float(v[i + 7]) * p.scale);
+                                *reinterpret_cast<uint4*>(gdst + cc + i) = w;
+                            }
+                        }
+                    }
+                    tc_fence_before();  // the next dQ MMA follows this group's next ds_ready arrival
+                }
+            }
+        }
+    }
+
+    // ---------------- teardown ----------------
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 9) tmem_dealloc(tmem_base, 512);
+    if (threadIdx.x == 0) {
+        if (*abort_flag) atomicExch(p.status, LIBRA_ERR_TIMEOUT);
+        p.busy[2 * cta + 1] = globaltimer_ns();
+    }
+}
+
+// ---- prep kernel ------------------------------------------------------------------------------
 
 // One warp per (token, head): D = <dO, O>; LSE to log2 units; rows in [T, Tpad) get zeros.
 template <int D>
@@ -578,41 +846,39 @@ __global__ void k_bwd_prep(const __nv_bfloat16* __restrict__ out, const __nv_bfl
     }
 }
 
-__global__ void k_bwd_dq_convert(const float* __restrict__ acc, int64_t n4, float scale, __nv_bfloat16* __restrict__ dq) {
-    const int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-    if (i >= n4) return;
-    const float4 v = reinterpret_cast<const float4*>(acc)[i];
-    uint2 w;
-    w.x = pack_bf16x2(v.x * scale, v.y * scale);
-    w.y = pack_bf16x2(v.z * scale, v.w * scale);
-    reinterpret_cast<uint2*>(dq)[i] = w;
-}
-
 struct BwdWorkspace {
-    size_t dq_acc_bytes, stat_bytes, total;
+    size_t stat_bytes, total;
     int64_t Tpad;
 };
-static BwdWorkspace bwd_workspace(int64_t T, int hq, int d) {
+static BwdWorkspace bwd_workspace(int64_t T, int hq) {
     BwdWorkspace w;
     w.Tpad = (T + 127) / 128 * 128;
-    w.dq_acc_bytes = ((size_t)T * hq * d * sizeof(float) + 255) & ~(size_t)255;
     w.stat_bytes = ((size_t)hq * w.Tpad * sizeof(float) + 255) & ~(size_t)255;
-    w.total = w.dq_acc_bytes + 2 * w.stat_bytes;
+    w.total = 2 * w.stat_bytes;
     return w;
+}
+
+template <typename Kernel>
+static int set_smem(Kernel k, int bytes) {
+    return cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) == cudaSuccess ? LIBRA_OK
+                                                                                                      : LIBRA_ERR_CUDA;
 }
 
 template <int D>
 static int launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tdo,
-                      const CUtensorMap& tdq, const BwdParams& prm, int W, cudaStream_t s) {
-    using L = BwdSmem<D>;
+                      const DkvParams& pa, int Wa, const DqParams& pb, int Wb, libra_plan_t* mp, cudaStream_t s) {
     static bool configured = false;
     if (!configured) {
-        if (cudaFuncSetAttribute(k_attn_bwd<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kBytes) != cudaSuccess)
-            return LIBRA_ERR_CUDA;
+        if (set_smem(k_attn_bwd_dkdv<D>, DkvSmem<D>::kBytes) != LIBRA_OK) return LIBRA_ERR_CUDA;
+        if (set_smem(k_attn_bwd_dq<D>, DqSmem<D>::kBytes) != LIBRA_OK) return LIBRA_ERR_CUDA;
         configured = true;
     }
-    k_attn_bwd<D><<<W, kBwdThreads, L::kBytes, s>>>(tq, tk, tv, tdo, tdq, prm);
-    count_launch();
+    if (mp->timing) cudaEventRecord(mp->ev[1][0], s);
+    k_attn_bwd_dkdv<D><<<Wa, kBwdThreads, DkvSmem<D>::kBytes, s>>>(tq, tk, tv, tdo, pa);
+    if (mp->timing) { cudaEventRecord(mp->ev[1][1], s); mp->ev_valid[1] = 1; cudaEventRecord(mp->ev[2][0], s); }
+    k_attn_bwd_dq<D><<<Wb, kBwdThreads, DqSmem<D>::kBytes, s>>>(tq, tk, tv, tdo, pb);
+    if (mp->timing) { cudaEventRecord(mp->ev[2][1], s); mp->ev_valid[2] = 1; }
+    count_launch(2);
     return cudaGetLastError() == cudaSuccess ? LIBRA_OK : LIBRA_ERR_CUDA;
 }
 
@@ -628,7 +894,7 @@ extern "C" int libra_debug_bwd_prof(unsigned long long* host, int n) {
 
 extern "C" size_t libra_attn_pool_bwd_workspace_bytes(const libra_plan_t* plan, const libra_dims* dims) {
     if (!plan || !dims || dims->hq <= 0 || (dims->head_dim != 64 && dims->head_dim != 128)) return 0;
-    return bwd_workspace(plan->T, dims->hq, dims->head_dim).total;
+    return bwd_workspace(plan->T, dims->hq).total;
 }
 
 extern "C" int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const void* v_dev, const void* out_dev,
@@ -640,11 +906,13 @@ extern "C" int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const v
         return LIBRA_ERR_INVALID_ARG;
     if (dims->hq <= 0 || dims->hkv <= 0 || dims->hq % dims->hkv) return LIBRA_ERR_INVALID_ARG;
     if (dims->head_dim != 64 && dims->head_dim != 128) return LIBRA_ERR_UNSUPPORTED;
-    const PlanDir& d = plan->dir[1];
-    if (!d.enabled || plan->T != dims->total_tokens) return LIBRA_ERR_PLAN_MISMATCH;
-    if (d.tile != kBlk) return LIBRA_ERR_UNSUPPORTED;
-    if (d.H != dims->hkv) return LIBRA_ERR_PLAN_MISMATCH;
-    if (d.W > plan->sm_count) return LIBRA_ERR_UNSUPPORTED;
+    const PlanDir& dq_dir = plan->dir[0];
+    const PlanDir& dkv_dir = plan->dir[1];
+    if (!dq_dir.enabled || !dkv_dir.enabled || plan->T != dims->total_tokens) return LIBRA_ERR_PLAN_MISMATCH;
+    if (dkv_dir.tile != kBlk || dq_dir.tile != 2 * kBlk) return LIBRA_ERR_UNSUPPORTED;
+    if (dkv_dir.H != dims->hkv) return LIBRA_ERR_PLAN_MISMATCH;
+    if (dims->hq % dq_dir.H) return LIBRA_ERR_INVALID_ARG;
+    if (dkv_dir.W > plan->sm_count || dq_dir.W > plan->sm_count) return LIBRA_ERR_UNSUPPORTED;
     if (((uintptr_t)q_dev | (uintptr_t)k_dev | (uintptr_t)v_dev | (uintptr_t)out_dev | (uintptr_t)dout_dev |
          (uintptr_t)dq_dev | (uintptr_t)dk_dev | (uintptr_t)dv_dev) & 15)
         return LIBRA_ERR_INVALID_ARG;
@@ -652,21 +920,18 @@ extern "C" int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const v
 
     const int D = dims->head_dim;
     const int64_t T = plan->T;
-    const BwdWorkspace ws = bwd_workspace(T, dims->hq, D);
-    float* dq_acc = reinterpret_cast<float*>(workspace_dev);
-    float* dvec = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(workspace_dev) + ws.dq_acc_bytes);
-    float* lse2 = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(workspace_dev) + ws.dq_acc_bytes + ws.stat_bytes);
+    const BwdWorkspace ws = bwd_workspace(T, dims->hq);
+    float* dvec = reinterpret_cast<float*>(workspace_dev);
+    float* lse2 = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(workspace_dev) + ws.stat_bytes);
     cudaStream_t s = (cudaStream_t)stream;
 
-    CUtensorMap tq, tk, tv, tdo, tdq;
-    int rc = make_f32_2d_map(&tdq, dq_acc, T, (int64_t)dims->hq * D, 32, kBlk);
-    if (rc == LIBRA_OK) rc = make_thd_map(&tq, q_dev, T, dims->hq, D, kBlk);
+    CUtensorMap tq, tk, tv, tdo;
+    int rc = make_thd_map(&tq, q_dev, T, dims->hq, D, kBlk);
     if (rc == LIBRA_OK) rc = make_thd_map(&tk, k_dev, T, dims->hkv, D, kBlk);
     if (rc == LIBRA_OK) rc = make_thd_map(&tv, v_dev, T, dims->hkv, D, kBlk);
     if (rc == LIBRA_OK) rc = make_thd_map(&tdo, dout_dev, T, dims->hq, D, kBlk);
     if (rc != LIBRA_OK) return rc;
 
-    if (cudaMemsetAsync(dq_acc, 0, (size_t)T * dims->hq * D * sizeof(float), s) != cudaSuccess) return LIBRA_ERR_CUDA;
     {
         const int64_t warps = ws.Tpad * dims->hq;
         const unsigned grid = (unsigned)((warps * 32 + 255) / 256);
@@ -679,32 +944,39 @@ extern "C" int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const v
         count_launch();
     }
     const float scale = dims->softmax_scale > 0.f ? dims->softmax_scale : 1.0f / sqrtf((float)D);
-    BwdParams prm;
-    prm.dq_acc = dq_acc;
-    prm.dk = reinterpret_cast<__nv_bfloat16*>(dk_dev);
-    prm.dv = reinterpret_cast<__nv_bfloat16*>(dv_dev);
-    prm.lse2 = lse2;
-    prm.dvec = dvec;
-    prm.cta_offsets = d.d_cta_offsets;
-    prm.cta_tiles = d.d_cta_exec;
-    prm.tok_end = plan->d_tok_end;
-    prm.T = T;
-    prm.Tpad = ws.Tpad;
-    prm.hq = dims->hq;
-    prm.hkv = dims->hkv;
-    prm.scale = scale;
-    prm.scale_log2 = scale * 1.4426950408889634f;
-    prm.status = plan->d_status + 2;
-    prm.busy = d.d_busy;
+    DkvParams pa;
+    pa.dk = reinterpret_cast<__nv_bfloat16*>(dk_dev);
+    pa.dv = reinterpret_cast<__nv_bfloat16*>(dv_dev);
+    pa.lse2 = lse2;
+    pa.dvec = dvec;
+    pa.cta_offsets = dkv_dir.d_cta_offsets;
+    pa.cta_tiles = dkv_dir.d_cta_exec;
+    pa.tok_end = plan->d_tok_end;
+    pa.T = T;
+    pa.Tpad = ws.Tpad;
+    pa.hq = dims->hq;
+    pa.hkv = dims->hkv;
+    pa.scale = scale;
+    pa.scale_log2 = scale * 1.4426950408889634f;
+    pa.status = plan->d_status + 2;
+    pa.busy = dkv_dir.d_busy;
+    DqParams pb;
+    pb.dq = reinterpret_cast<__nv_bfloat16*>(dq_dev);
+    pb.lse2 = lse2;
+    pb.dvec = dvec;
+    pb.cta_offsets = dq_dir.d_cta_offsets;
+    pb.cta_tiles = dq_dir.d_cta_exec;
+    pb.tok_start = plan->d_tok_start;
+    pb.T = T;
+    pb.Tpad = ws.Tpad;
+    pb.hq = dims->hq;
+    pb.hkv = dims->hkv;
+    pb.H = dq_dir.H;
+    pb.scale = scale;
+    pb.scale_log2 = scale * 1.4426950408889634f;
+    pb.status = plan->d_status + 2;
+    pb.busy = dq_dir.d_busy2;
     libra_plan_t* mp = const_cast<libra_plan_t*>(plan);
-    if (mp->timing) cudaEventRecord(mp->ev[1][0], s);
-    rc = D == 128 ? launch_bwd<128>(tq, tk, tv, tdo, tdq, prm, d.W, s) : launch_bwd<64>(tq, tk, tv, tdo, tdq, prm, d.W, s);
-    if (mp->timing) { cudaEventRecord(mp->ev[1][1], s); mp->ev_valid[1] = 1; }
-    if (rc != LIBRA_OK) return rc;
-    {
-        const int64_t n4 = T * dims->hq * D / 4;
-        k_bwd_dq_convert<<<(unsigned)((n4 + 255) / 256), 256, 0, s>>>(dq_acc, n4, scale, (__nv_bfloat16*)dq_dev);
-        count_launch();
-    }
-    return cudaGetLastError() == cudaSuccess ? LIBRA_OK : LIBRA_ERR_CUDA;
+    return D == 128 ? launch_bwd<128>(tq, tk, tv, tdo, pa, dkv_dir.W, pb, dq_dir.W, mp, s)
+                    : launch_bwd<64>(tq, tk, tv, tdo, pa, dkv_dir.W, pb, dq_dir.W, mp, s);
 }

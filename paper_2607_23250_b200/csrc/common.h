@@ -27,6 +27,7 @@ struct PlanDir {
     int32_t* d_cta_exec = nullptr;     // [NT]  the same lists, each re-ordered for execution (head-major)
     int64_t* d_loads = nullptr;        // [W]
     uint64_t* d_busy = nullptr;        // [2*W] (start, end) global-timer stamps of the last run
+    uint64_t* d_busy2 = nullptr;       // [2*W] same, for the second kernel that walks this direction (dQ)
 };
 
 }  // namespace libra
@@ -42,8 +43,8 @@ struct libra_plan {
     int* d_status = nullptr;         // [4] word 0: plan status; word 1: fwd; word 2: bwd
     libra::PlanDir dir[2];           // 0 = query-major, 1 = key-major
     int timing = 0;                  // record events around the main kernels
-    cudaEvent_t ev[2][2] = {{nullptr, nullptr}, {nullptr, nullptr}};  // [direction][begin, end]
-    int ev_valid[2] = {0, 0};
+    cudaEvent_t ev[3][2] = {{nullptr, nullptr}, {nullptr, nullptr}, {nullptr, nullptr}};  // [kernel][begin, end]
+    int ev_valid[3] = {0, 0, 0};
 };
 
 namespace libra {

@@ -189,7 +189,7 @@ static inline unsigned grid_for(int64_t n, int block) { return (unsigned)((n + b
 
 static void free_dir(PlanDir& d) {
     cudaFree(d.d_weight_blk); cudaFree(d.d_blk_order); cudaFree(d.d_cta_of_tile); cudaFree(d.d_pos);
-    cudaFree(d.d_cta_offsets); cudaFree(d.d_cta_tiles); cudaFree(d.d_cta_exec); cudaFree(d.d_loads); cudaFree(d.d_busy);
+    cudaFree(d.d_cta_offsets); cudaFree(d.d_cta_tiles); cudaFree(d.d_cta_exec); cudaFree(d.d_loads); cudaFree(d.d_busy); cudaFree(d.d_busy2);
     d = PlanDir();
 }
 
@@ -211,9 +211,11 @@ static int build_dir(libra_plan* p, PlanDir& d, int key_major) {
     A((void**)&d.d_cta_exec, sizeof(int32_t) * d.NT);
     A((void**)&d.d_loads, sizeof(int64_t) * d.W);
     A((void**)&d.d_busy, sizeof(uint64_t) * 2 * d.W);
+    A((void**)&d.d_busy2, sizeof(uint64_t) * 2 * d.W);
     if (e != cudaSuccess) return LIBRA_ERR_CUDA;
     cudaStream_t s = p->stream;
     cudaMemsetAsync(d.d_busy, 0, sizeof(uint64_t) * 2 * d.W, s);
+    cudaMemsetAsync(d.d_busy2, 0, sizeof(uint64_t) * 2 * d.W, s);
     k_block_weights<<<grid_for(d.NB, 128), 128, 0, s>>>(p->d_tok_start, p->d_tok_end, T, d.tile, d.NB, key_major,
                                                         d.d_weight_blk);
     k_rank_blocks<<<grid_for(d.NB, 256), 256, 0, s>>>(d.d_weight_blk, d.NB, d.d_blk_order);
@@ -368,7 +370,7 @@ extern "C" int libra_plan_destroy(libra_plan_t* plan) {
     cudaFree(plan->d_tok_start);
     cudaFree(plan->d_tok_end);
     cudaFree(plan->d_status);
-    for (int a = 0; a < 2; ++a)
+    for (int a = 0; a < 3; ++a)
         for (int b = 0; b < 2; ++b)
             if (plan->ev[a][b]) cudaEventDestroy(plan->ev[a][b]);
     delete plan;
@@ -377,24 +379,27 @@ extern "C" int libra_plan_destroy(libra_plan_t* plan) {
 
 extern "C" int libra_busy_times(const libra_plan_t* plan, int which, uint64_t* ns_host) {
     if (!plan || !ns_host) return LIBRA_ERR_INVALID_ARG;
-    PlanDir* d = dir_of(plan, which);
+    if (which < LIBRA_KERNEL_FWD || which > LIBRA_KERNEL_BWD_DQ) return LIBRA_ERR_INVALID_ARG;
+    // the forward and the dQ kernel walk the query-major lists, the dK/dV kernel the key-major ones
+    PlanDir* d = dir_of(plan, which == LIBRA_KERNEL_BWD_DKDV ? LIBRA_DIR_KV : LIBRA_DIR_Q);
     if (!d) return LIBRA_ERR_PLAN_MISMATCH;
     if (cudaDeviceSynchronize() != cudaSuccess) return LIBRA_ERR_CUDA;
     uint64_t* tmp = new (std::nothrow) uint64_t[2 * (size_t)d->W];
     if (!tmp) return LIBRA_ERR_CUDA;
     int st[4] = {0, 0, 0, 0};
-    cudaError_t e = cudaMemcpy(tmp, d->d_busy, sizeof(uint64_t) * 2 * d->W, cudaMemcpyDeviceToHost);
+    const uint64_t* src = which == LIBRA_KERNEL_BWD_DQ ? d->d_busy2 : d->d_busy;
+    cudaError_t e = cudaMemcpy(tmp, src, sizeof(uint64_t) * 2 * d->W, cudaMemcpyDeviceToHost);
     if (e == cudaSuccess) e = cudaMemcpy(st, plan->d_status, sizeof(st), cudaMemcpyDeviceToHost);
     for (int r = 0; r < d->W; ++r) ns_host[r] = tmp[2 * r + 1] >= tmp[2 * r] ? tmp[2 * r + 1] - tmp[2 * r] : 0;
     delete[] tmp;
     if (e != cudaSuccess) return LIBRA_ERR_CUDA;
-    return st[which == LIBRA_DIR_Q ? 1 : 2];
+    return st[which == LIBRA_KERNEL_FWD ? 1 : 2];
 }
 
 extern "C" int libra_plan_set_timing(libra_plan_t* plan, int enabled) {
     if (!plan) return LIBRA_ERR_INVALID_ARG;
     if (enabled) {
-        for (int a = 0; a < 2; ++a)
+        for (int a = 0; a < 3; ++a)
             for (int b = 0; b < 2; ++b)
                 if (!plan->ev[a][b] && cudaEventCreate(&plan->ev[a][b]) != cudaSuccess) return LIBRA_ERR_CUDA;
     }
@@ -404,8 +409,8 @@ extern "C" int libra_plan_set_timing(libra_plan_t* plan, int enabled) {
 
 extern "C" int libra_kernel_time_ms(const libra_plan_t* plan, int which, float* ms_host) {
     if (!plan || !ms_host) return LIBRA_ERR_INVALID_ARG;
-    const int a = which == LIBRA_DIR_Q ? 0 : (which == LIBRA_DIR_KV ? 1 : -1);
-    if (a < 0) return LIBRA_ERR_INVALID_ARG;
+    const int a = which - 1;  // LIBRA_KERNEL_FWD / _BWD_DKDV / _BWD_DQ
+    if (a < 0 || a > 2) return LIBRA_ERR_INVALID_ARG;
     if (!plan->ev_valid[a]) return LIBRA_ERR_PLAN_MISMATCH;
     if (cudaEventSynchronize(plan->ev[a][1]) != cudaSuccess) return LIBRA_ERR_CUDA;
     if (cudaEventElapsedTime(ms_host, plan->ev[a][0], plan->ev[a][1]) != cudaSuccess) return LIBRA_ERR_CUDA;

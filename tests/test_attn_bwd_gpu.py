@@ -23,7 +23,8 @@ def _run(lengths, hq, hkv, d, seed=0, W=0, qscale=1.0):
     out, lse = lb.libra_attn_pool_fwd(q, k, v, plan)
     dq, dk, dv = lb.libra_attn_pool_bwd(q, k, v, out, lse, dout, plan)
     torch.cuda.synchronize()
-    assert plan.busy_times(lb.LIBRA_DIR_KV) is not None      # raises on a kernel timeout status
+    plan.busy_times(lb.KERNEL_BWD_DKDV)                       # raises on a kernel timeout status
+    plan.busy_times(lb.KERNEL_BWD_DQ)
     f = {n: t[n].float().numpy() for n in t}
     o_ref, l_ref = oracle.attn_fwd(f["q"], f["k"], f["v"], cu_np)
     ref = oracle.attn_bwd(f["q"], f["k"], f["v"], o_ref, l_ref, f["dout"], cu_np)
