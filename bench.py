@@ -199,7 +199,7 @@ def run_ours(args):
     if rank == 0:
         sampler.start()
     n0 = lb.launch_count()
-    kern_f, kern_b = [], []
+    kern_f, kern_b, kern_q = [], [], []
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     e0.record()
@@ -212,11 +212,13 @@ def run_ours(args):
     # kernel-only durations (events recorded by the library on the launch stream), untimed extra steps
     for _ in range(min(args.steps, 5)):
         step()
-        kern_f.append(plan.kernel_time_ms(lb.LIBRA_DIR_Q))
-        kern_b.append(plan.kernel_time_ms(lb.LIBRA_DIR_KV))
+        kern_f.append(plan.kernel_time_ms(lb.KERNEL_FWD))
+        kern_b.append(plan.kernel_time_ms(lb.KERNEL_BWD_DKDV))
+        kern_q.append(plan.kernel_time_ms(lb.KERNEL_BWD_DQ))
     clocks = sampler.stop() if rank == 0 else None
-    busy_f = plan.busy_times(lb.LIBRA_DIR_Q).astype(np.float64)
-    busy_b = plan.busy_times(lb.LIBRA_DIR_KV).astype(np.float64)
+    busy_f = plan.busy_times(lb.KERNEL_FWD).astype(np.float64)
+    busy_b = plan.busy_times(lb.KERNEL_BWD_DKDV).astype(np.float64)
+    busy_q = plan.busy_times(lb.KERNEL_BWD_DQ).astype(np.float64)
 
     ms = torch.tensor([total_ms / args.steps], device=dev, dtype=torch.float64)
     if world > 1:
@@ -228,8 +230,8 @@ def run_ours(args):
     if not args.skip_e2e:
         e2e = run_e2e(args, step, barrier, dict(q=q, k=k, v=v, dout=dout),
                       dict(out=out, lse=lse, dq=dq, dk=dk, dv=dv), world, dev, ff + fb)
-    finish(args, rank, world, spec, lengths, plan, value, ms_per_step, kern_f, kern_b, busy_f, busy_b, clocks,
-           launches, e2e, ff, fb, q)
+    finish(args, rank, world, spec, lengths, plan, value, ms_per_step, (kern_f, kern_b, kern_q),
+           (busy_f, busy_b, busy_q), clocks, launches, e2e, ff, fb, q)
     plan.destroy()
     if world > 1:
         dist.destroy_process_group()
@@ -268,25 +270,21 @@ def run_e2e(args, step, barrier, dev_in, dev_out, world, dev, flops):
             "d2h_bytes_per_step": d2h, "ms_per_step": round(float(e2e_ms.item()), 3)}
 
 
-def finish(args, rank, world, spec, lengths, plan, value, ms_per_step, kern_f, kern_b, busy_f, busy_b, clocks,
-           launches, e2e, ff, fb, q):
+def finish(args, rank, world, spec, lengths, plan, value, ms_per_step, kern, busy, clocks, launches, e2e, ff, fb, q):
+    kern_f, kern_b, kern_q = kern
+    busy_f, busy_b, busy_q = busy
     from paper_2607_23250_b200 import binding as lb  # noqa: F401
     T, hq, hkv, d = spec.total_tokens, spec.hq, spec.hkv, spec.head_dim
     if rank == 0:
         peaks = measured_peaks()
         kb = statistics.mean(kern_b)
         kf = statistics.mean(kern_f)
-        # dominant kernel: the backward main kernel (10 d flops per causal pair per head per launch)
-        ach = fb / (kb * 1e-3) / 1e12
-        traffic = None
-        tr_path = os.path.join(ROOT, "profiles", "dram_traffic.json")
-        if os.path.exists(tr_path):
-            try:
-                tr = json.load(open(tr_path)).get("k_attn_bwd", {})
-                if tr.get("config") == args.config:
-                    traffic = tr.get("bytes_per_launch")
-            except Exception:
-                traffic = None
+        kq = statistics.mean(kern_q)
+        # Dominant kernel: the backward dK/dV kernel.  Algorithmic work per launch: the four GEMMs of
+        # the dK/dV gradient it owns (S, dP, dV, dK = 8 d flops per causal pair per query head).
+        fa = fb * 8 // 10
+        ach = fa / (kb * 1e-3) / 1e12
+        traffic = read_traffic("k_attn_bwd_dkdv", args)
         line = {
             "metric": METRIC, "value": round(value, 2), "unit": "TFLOP/s", "n_gpus": world,
             "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 4),
@@ -302,13 +300,16 @@ def finish(args, rank, world, spec, lengths, plan, value, ms_per_step, kern_f, k
                                  "sustained_measured": round(100 * value / world / peaks["sustained"], 2),
                                  "nominal_2250": round(100 * value / world / 2250.0, 2), "peaks": peaks["source"]},
             "fwd_kernel": {"ms": round(kf, 4), "tflops": round(ff / kf / 1e9, 1)},
-            "bwd_kernel": {"ms": round(kb, 4), "tflops": round(fb / kb / 1e9, 1)},
+            "bwd_dkdv_kernel": {"ms": round(kb, 4), "executed_tflops": round(fa / kb / 1e9, 1)},
+            "bwd_dq_kernel": {"ms": round(kq, 4), "executed_tflops": round(fb * 6 // 10 / kq / 1e9, 1)},
+            "bwd_useful_tflops": round(fb / (kb + kq) / 1e9, 1),
             "busy_max_over_mean": {"fwd": round(float(busy_f.max() / busy_f.mean()), 4),
-                                   "bwd": round(float(busy_b.max() / busy_b.mean()), 4)},
+                                   "bwd_dkdv": round(float(busy_b.max() / busy_b.mean()), 4),
+                                   "bwd_dq": round(float(busy_q.max() / busy_q.mean()), 4)},
             "clocks": clocks,
             "e2e": e2e,
             "gpu_launches": int(launches),
-            "roofline": {"bound": "tensor", "kernel": "k_attn_bwd", "achieved": round(ach, 1),
+            "roofline": {"bound": "tensor", "kernel": "k_attn_bwd_dkdv", "achieved": round(ach, 1),
                          "peak": peaks["sustained"], "unit": "TFLOP/s", "frac": round(ach / peaks["sustained"], 4),
                          "peak_kind": f"bf16 sustained, {peaks['source']}", "traffic": traffic,
                          "frac_of_burst": round(ach / peaks["burst"], 4)},
@@ -317,6 +318,20 @@ def finish(args, rank, world, spec, lengths, plan, value, ms_per_step, kern_f, k
             cb = time_oracle(spec, lengths)
             line["cpu_baseline"] = {k2: (round(v2, 6) if isinstance(v2, float) else v2) for k2, v2 in cb.items()}
         print(json.dumps(line), flush=True)
+
+
+def read_traffic(kernel, args):
+    """DRAM bytes per launch of `kernel` from the committed ncu summary (profiles/dram_traffic.txt:
+    lines `kernel config seqs bytes`), scaled by nothing: only an exact workload match is used."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+    try:
+        for line in open(path):
+            parts = line.split()
+            if len(parts) >= 4 and parts[0] == kernel and int(parts[1]) == args.config and int(parts[2]) == args.seqs:
+                return int(float(parts[3]))
+    except Exception:
+        pass
+    return None
 
 
 def run_reference(args):

@@ -225,21 +225,25 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         uint32_t ucnt = 0, it_all = 0;
         bool ok = true;
         PROF_DECL
-        // C[tmem] = A(K-major tile) * B(K-major tile)^T over the head dimension
-        auto issue_kmajor = [&](uint32_t d_col, uint32_t a_addr, uint32_t b_addr) {
+        // Base descriptors are built once; every MMA only adds a constant to them.
+        const uint64_t kdesc0 = make_sdesc(sb, 16, 1024);             // K-major view of a tile at offset 0
+        const uint64_t mdesc0 = make_sdesc(sb, L::kHalfBytes, 1024);  // MN-major view
+        // C[tmem] = A(K-major tile) * B(K-major tile)^T over the head dimension; offsets from smem base
+        auto issue_kmajor = [&](uint32_t d_col, uint32_t a_off, uint32_t b_off) {
+            const uint64_t da = sdesc_advance(kdesc0, a_off), db = sdesc_advance(kdesc0, b_off);
 #pragma unroll
             for (int kk = 0; kk < D / 16; ++kk) {
                 const uint32_t off = (kk / 4) * L::kHalfBytes + (kk % 4) * 32;
-                mma_ss(tmem_base + d_col, make_sdesc(a_addr + off, 16, 1024), make_sdesc(b_addr + off, 16, 1024),
-                       idesc_s, kk > 0);
+                mma_ss(tmem_base + d_col, sdesc_advance(da, off), sdesc_advance(db, off), idesc_s, kk > 0);
             }
         };
         // C[tmem] (+)= A(TMEM, bf16 packed: queries 64c.. at columns a_col + 64c ..) * B(MN-major tile)
-        auto issue_acc = [&](uint32_t d_col, uint32_t a_col, uint32_t b_addr, bool accumulate) {
+        auto issue_acc = [&](uint32_t d_col, uint32_t a_col, uint32_t b_off, bool accumulate) {
+            const uint64_t db = sdesc_advance(mdesc0, b_off);
 #pragma unroll
             for (int kk = 0; kk < 8; ++kk)  // 16 queries per step
-                mma_ts(tmem_base + d_col, tmem_base + a_col + (kk / 4) * 64 + (kk % 4) * 8,
-                       make_sdesc(b_addr + kk * 2048, L::kHalfBytes, 1024), idesc_acc, (accumulate || kk > 0) ? 1u : 0u);
+                mma_ts(tmem_base + d_col, tmem_base + a_col + (kk / 4) * 64 + (kk % 4) * 8, sdesc_advance(db, kk * 2048),
+                       idesc_acc, (accumulate || kk > 0) ? 1u : 0u);
         };
         for (int idx = unit_begin; idx < unit_end && ok; ++idx) {
             const int t = p.cta_tiles[idx];
@@ -254,13 +258,13 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             if (!ok) break;
             tc_fence_after();
             if (lane == 0) {
-                issue_kmajor(kColS, sb + L::kKOff, sb + L::kQOff + (it_all & 1) * L::kTileBytes);
+                issue_kmajor(kColS, L::kKOff, L::kQOff + (it_all & 1) * L::kTileBytes);
                 tc_commit(bar_sfull);
             }
             ok = warp_wait_b(&bar_dofull[it_all & 1], (it_all >> 1) & 1, abort_flag);
             if (!ok) break;
             if (lane == 0) {
-                issue_kmajor(kColDP, sb + L::kVOff, sb + L::kDoOff + (it_all & 1) * L::kTileBytes);
+                issue_kmajor(kColDP, L::kVOff, L::kDoOff + (it_all & 1) * L::kTileBytes);
                 tc_commit(bar_dpfull);
             }
             for (int it = 0; it < n_it && ok; ++it, ++it_all) {
@@ -269,16 +273,20 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const bool more = it + 1 < n_it;
                 // dV(it) += P^T dO
                 PROF(7)
+#ifndef LIBRA_DBG_FREE_MMA
                 ok = warp_wait_b(bar_pready, it_all & 1, abort_flag);
                 if (!ok) break;
+#endif
                 PROF(0)
+#ifndef LIBRA_DBG_FREE_MMA
                 if (it == 0 && ucnt > 0) {  // previous unit's dK/dV must have been read out
                     ok = warp_wait_b(bar_dkvempty, (ucnt - 1) & 1, abort_flag);
                     if (!ok) break;
                 }
+#endif
                 tc_fence_after();
                 if (lane == 0) {
-                    issue_acc(kColDV, kColS, sb + L::kDoOff + st * L::kTileBytes, it > 0);
+                    issue_acc(kColDV, kColS, L::kDoOff + st * L::kTileBytes, it > 0);
                     tc_commit(&bar_doempty[st]);
                 }
                 // S(it+1)
@@ -288,18 +296,20 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     if (!ok) break;
                     PROF(1)
                     if (lane == 0) {
-                        issue_kmajor(kColS, sb + L::kKOff, sb + L::kQOff + (nx & 1) * L::kTileBytes);
+                        issue_kmajor(kColS, L::kKOff, L::kQOff + (nx & 1) * L::kTileBytes);
                         tc_commit(bar_sfull);
                     }
                 }
                 // dK(it) += dS^T Q
                 PROF(7)
+#ifndef LIBRA_DBG_FREE_MMA
                 ok = warp_wait_b(bar_dsready, it_all & 1, abort_flag);
                 if (!ok) break;
+#endif
                 PROF(2)
                 tc_fence_after();
                 if (lane == 0) {
-                    issue_acc(kColDK, kColDP, sb + L::kQOff + st * L::kTileBytes, it > 0);
+                    issue_acc(kColDK, kColDP, L::kQOff + st * L::kTileBytes, it > 0);
                     tc_commit(&bar_qempty[st]);
                 }
                 // dP(it+1)
@@ -309,7 +319,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     if (!ok) break;
                     PROF(3)
                     if (lane == 0) {
-                        issue_kmajor(kColDP, sb + L::kVOff, sb + L::kDoOff + (nx & 1) * L::kTileBytes);
+                        issue_kmajor(kColDP, L::kVOff, L::kDoOff + (nx & 1) * L::kTileBytes);
                         tc_commit(bar_dpfull);
                     }
                 }
@@ -333,6 +343,9 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         uint32_t ucnt = 0, it_all = 0;
         bool ok = true;
         PROF_DECL
+#if defined(LIBRA_DBG_FREE_MMA) && !defined(LIBRA_DBG_FREE_MMA_COMPUTE_ON)
+        ok = false;
+#endif
         for (int idx = unit_begin; idx < unit_end && ok; ++idx) {
             const int t = p.cta_tiles[idx];
             const int kvh = t % p.hkv;
@@ -627,12 +640,14 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         const uint32_t sb = smem_u32(smem);
         uint32_t bcnt = 0, kcnt = 0, vcnt = 0, scnt = 0, dscnt = 0;
         bool ok = true;
-        auto issue_kmajor = [&](uint32_t d_col, uint32_t a_addr, uint32_t b_addr) {
+        const uint64_t kdesc0 = make_sdesc(sb, 16, 1024);             // K-major view of a tile at offset 0
+        const uint64_t mdesc0 = make_sdesc(sb, L::kHalfBytes, 1024);  // MN-major view
+        auto issue_kmajor = [&](uint32_t d_col, uint32_t a_off, uint32_t b_off) {
+            const uint64_t da = sdesc_advance(kdesc0, a_off), db = sdesc_advance(kdesc0, b_off);
 #pragma unroll
             for (int kk = 0; kk < D / 16; ++kk) {
                 const uint32_t off = (kk / 4) * L::kHalfBytes + (kk % 4) * 32;
-                mma_ss(tmem_base + d_col, make_sdesc(a_addr + off, 16, 1024), make_sdesc(b_addr + off, 16, 1024),
-                       idesc_s, kk > 0);
+                mma_ss(tmem_base + d_col, sdesc_advance(da, off), sdesc_advance(db, off), idesc_s, kk > 0);
             }
         };
         // S(j) into buffer scnt & 1 from K ring entry kidx; waits for the K tile first.  `last`: no later
@@ -640,7 +655,7 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         auto do_s = [&](uint32_t kidx, bool last) -> bool {
             if (!warp_wait_b(&bar_kfull[kidx % L::kKStages], (kidx / L::kKStages) & 1, abort_flag)) return false;
             if (lane == 0) {
-                issue_kmajor(kColS + (scnt & 1) * 128, sb + L::kQOff, sb + L::kKOff + (kidx % L::kKStages) * L::kTileBytes);
+                issue_kmajor(kColS + (scnt & 1) * 128, L::kQOff, L::kKOff + (kidx % L::kKStages) * L::kTileBytes);
                 tc_commit(&bar_sfull[scnt & 1]);
                 if (last) tc_commit(bar_qempty);
             }
@@ -651,7 +666,7 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             const uint32_t vs = vcnt % L::kVStages;
             if (!warp_wait_b(&bar_vfull[vs], (vcnt / L::kVStages) & 1, abort_flag)) return false;
             if (lane == 0) {
-                issue_kmajor(kColDP, sb + L::kDoOff, sb + L::kVOff + vs * L::kTileBytes);
+                issue_kmajor(kColDP, L::kDoOff, L::kVOff + vs * L::kTileBytes);
                 tc_commit(bar_dpfull);
                 tc_commit(&bar_vempty[vs]);
                 if (last) tc_commit(bar_doempty);
@@ -683,12 +698,12 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                         tc_fence_after();
                         const uint32_t kidx = kbase + (j - lo);
                         if (lane == 0) {
-                            const uint32_t ka = sb + L::kKOff + (kidx % L::kKStages) * L::kTileBytes;
+                            const uint64_t ka = sdesc_advance(mdesc0, L::kKOff + (kidx % L::kKStages) * L::kTileBytes);
                             const uint32_t a_col = kColS + (dscnt & 1) * 128;  // dS(j) sits in S(j)'s buffer
 #pragma unroll
                             for (int kk = 0; kk < 8; ++kk)  // 16 keys per step
                                 mma_ts(tmem_base + kColDQ, tmem_base + a_col + (kk / 4) * 64 + (kk % 4) * 8,
-                                       make_sdesc(ka + kk * 2048, L::kHalfBytes, 1024), idesc_dq,
+                                       sdesc_advance(ka, kk * 2048), idesc_dq,
                                        (j > lo || kk > 0) ? 1u : 0u);
                             tc_commit(&bar_kempty[kidx % L::kKStages]);
                         }

@@ -17,11 +17,16 @@
 #include "common.h"
 #include "ptx.cuh"
 
+#ifndef LIBRA_FWD_REG_DEC
+#define LIBRA_FWD_REG_DEC 56
+#define LIBRA_FWD_REG_INC 216
+#endif
+
 namespace libra {
 
 constexpr int kBM = 128;            // rows per slot
 constexpr int kBN = 128;            // keys per block
-constexpr int kFwdThreads = 320;
+constexpr int kFwdThreads = 384;  // warps 10-11 only donate registers
 constexpr float kRescaleThreshold = 8.0f;  // log2 units: O is rescaled only when the max grows by more
 
 template <int D>
@@ -69,6 +74,24 @@ __device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volati
     if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag) ? 1 : 0;
     return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
+
+#ifdef LIBRA_PROF
+__device__ unsigned long long g_fwd_prof[1024 * 24];
+struct FProf {
+    long long last;
+    unsigned long long acc[8];
+    __device__ void start() { last = clock64(); for (int i = 0; i < 8; ++i) acc[i] = 0; }
+    __device__ void mark(int k) { const long long now = clock64(); acc[k] += now - last; last = now; }
+    __device__ void flush(int cta, int base) { for (int i = 0; i < 8; ++i) g_fwd_prof[cta * 24 + base + i] = acc[i]; }
+};
+#define PROF_DECL FProf prof; prof.start();
+#define PROF(k) prof.mark(k);
+#define PROF_FLUSH(cond, base) if (cond) prof.flush(cta, base);
+#else
+#define PROF_DECL
+#define PROF(k)
+#define PROF_FLUSH(cond, base)
+#endif
 
 template <int D>
 __global__ void __launch_bounds__(kFwdThreads, 1)
@@ -124,8 +147,13 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     const int heads_per_shard = p.hq / p.H;
     const int G = p.hq / p.hkv;
 
-    if (warp == 8) {
+    // The softmax groups hold a whole 128-column row of S in registers; the producer / MMA
+    // warpgroup needs few registers and hands the rest over.
+    if (warp >= 10) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(LIBRA_FWD_REG_DEC));
+    } else if (warp == 8) {
         // ---------------- TMA producer ----------------
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(LIBRA_FWD_REG_DEC));
         uint32_t ring = 0, qcnt = 0;
         bool ok = true;
         for (int idx = tile_begin; idx < tile_end && ok; ++idx) {
@@ -166,29 +194,34 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         }
     } else if (warp == 9) {
         // ---------------- MMA issuer ----------------
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(LIBRA_FWD_REG_DEC));
         constexpr uint32_t idesc_s = make_idesc(kBM, kBN, 0, 0);
         constexpr uint32_t idesc_pv = make_idesc(kBM, D, 0, 1);
         const uint32_t smem_base = smem_u32(smem);
         uint32_t ring = 0, qcnt = 0;
         uint32_t pcnt[2] = {0, 0};
         bool ok = true;
+        PROF_DECL
+        // Base descriptors are built once; every MMA only adds a constant to them.
+        const uint64_t desc_q = make_sdesc(smem_base + L::kQOff, 16, 1024);                  // K-major Q slot 0
+        const uint64_t desc_k = make_sdesc(smem_base + L::kRingOff, 16, 1024);               // K-major ring stage 0
+        const uint64_t desc_v = make_sdesc(smem_base + L::kRingOff, L::kHalfBytes, 1024);    // MN-major ring stage 0
         auto issue_s = [&](int g, uint32_t stage) {
-            const uint32_t qa = smem_base + L::kQOff + g * L::kTileBytes;
-            const uint32_t ka = smem_base + L::kRingOff + stage * L::kTileBytes;
+            const uint64_t qa = sdesc_advance(desc_q, g * L::kTileBytes);
+            const uint64_t ka = sdesc_advance(desc_k, stage * L::kTileBytes);
 #pragma unroll
             for (int kk = 0; kk < D / 16; ++kk) {
                 const uint32_t off = (kk / 4) * L::kHalfBytes + (kk % 4) * 32;
-                mma_ss(tmem_base + g * kBN, make_sdesc(qa + off, 16, 1024), make_sdesc(ka + off, 16, 1024), idesc_s,
-                       kk > 0);
+                mma_ss(tmem_base + g * kBN, sdesc_advance(qa, off), sdesc_advance(ka, off), idesc_s, kk > 0);
             }
             tc_commit(&bar_sfull[g]);
         };
         auto issue_pv = [&](int g, uint32_t stage, bool accumulate) {
-            const uint32_t va = smem_base + L::kRingOff + stage * L::kTileBytes;
+            const uint64_t va = sdesc_advance(desc_v, stage * L::kTileBytes);
 #pragma unroll
             for (int kk = 0; kk < kBN / 16; ++kk) {
-                mma_ts(tmem_base + 2 * kBN + g * D, tmem_base + g * kBN + kk * 8,
-                       make_sdesc(va + kk * 2048, L::kHalfBytes, 1024), idesc_pv, (accumulate || kk > 0) ? 1u : 0u);
+                mma_ts(tmem_base + 2 * kBN + g * D, tmem_base + g * kBN + kk * 8, sdesc_advance(va, kk * 2048), idesc_pv,
+                       (accumulate || kk > 0) ? 1u : 0u);
             }
             tc_commit(&bar_odone[g]);
         };
@@ -199,8 +232,10 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             const bool act1 = r[1].lo <= r[1].hi;
             const int lo = r[0].lo, hi = act1 ? r[1].hi : r[0].hi;
             for (int hh = 0; hh < heads_per_shard && ok; ++hh) {
+                PROF(7)
                 ok = warp_wait(bar_qfull, qcnt & 1, abort_flag);
                 if (!ok) break;
+                PROF(0)
                 ++qcnt;
                 // prologue: S(lo)
                 uint32_t st = ring % L::kStages;
@@ -215,20 +250,25 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 ++ring;
                 for (int j = lo; j <= hi && ok; ++j) {
                     const uint32_t st_v = ring % L::kStages;
+                    PROF(7)
                     ok = warp_wait(&bar_full[st_v], (ring / L::kStages) & 1, abort_flag);
                     if (!ok) break;
+                    PROF(1)
                     ++ring;
                     uint32_t st_k = 0;
                     if (j + 1 <= hi) {
                         st_k = ring % L::kStages;
                         ok = warp_wait(&bar_full[st_k], (ring / L::kStages) & 1, abort_flag);
                         if (!ok) break;
+                        PROF(2)
                         ++ring;
                     }
                     for (int g = 0; g < 2 && ok; ++g) {
                         if (j >= r[g].lo && j <= r[g].hi) {
+                            PROF(7)
                             ok = warp_wait(&bar_pready[g], pcnt[g] & 1, abort_flag);
                             if (!ok) break;
+                            PROF(3 + g)
                             ++pcnt[g];
                             tc_fence_after();
                             if (lane == 0) issue_pv(g, st_v, j != r[g].lo);
@@ -248,8 +288,10 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 __syncwarp();
             }
         }
+        PROF_FLUSH(lane == 0, 8)
     } else {
         // ---------------- softmax groups ----------------
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(LIBRA_FWD_REG_INC));
         const int g = warp >> 2;
         const int row_in_tile = (warp & 3) * 32 + lane;
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
@@ -257,6 +299,7 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         const uint32_t t_o = tmem_base + lane_addr + 2 * kBN + g * D;
         uint32_t scnt = 0, ocnt = 0;
         bool ok = true;
+        PROF_DECL
         for (int idx = tile_begin; idx < tile_end && ok; ++idx) {
             const int t = p.cta_tiles[idx];
             const int64_t qs = (int64_t)(t / p.H) * (2 * kBM) + g * kBM;
@@ -272,8 +315,10 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 const int h = (t % p.H) * heads_per_shard + hh;
                 float m_ref = -INFINITY, l_sum = 0.f;
                 for (int j = rg.lo; j <= rg.hi && ok; ++j) {
+                    PROF(3)
                     ok = mbar_wait(&bar_sfull[g], scnt & 1, abort_flag);
                     if (!ok) break;
+                    PROF(0)
                     ++scnt;
                     tc_fence_after();
                     uint32_t sr[kBN];
@@ -282,6 +327,7 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                     tmem_ld32(t_s + 64, sr + 64);
                     tmem_ld32(t_s + 96, sr + 96);
                     tmem_ld_wait();
+                    PROF(4)
                     const int k0 = j * kBN;
                     const bool need_mask = (k0 + kBN - 1 > qs) || (k0 < max_kstart) || !row_ok;
                     if (need_mask) {
@@ -291,9 +337,9 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                         for (int i = 0; i < kBN; ++i)
                             if (i < c_lo || i > c_hi) sr[i] = 0xff800000u;  // -inf
                     }
-                    float mx = __uint_as_float(sr[0]);
+                    float mx = fmaxf(__uint_as_float(sr[0]), __uint_as_float(sr[1]));
 #pragma unroll
-                    for (int i = 1; i < kBN; ++i) mx = fmaxf(mx, __uint_as_float(sr[i]));
+                    for (int i = 2; i < kBN; i += 2) mx = max3(mx, __uint_as_float(sr[i]), __uint_as_float(sr[i + 1]));
                     mx *= p.scale_log2;  // scale > 0, so the max commutes with it
                     // lazy rescale: keep the old reference unless the max grew by > threshold
                     float m_new = m_ref;
@@ -319,32 +365,44 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                             tmem_st32(t_o + c, orow);
                         }
                     }
+                    PROF(5)
                     l_sum *= factor;
                     m_ref = m_new;
                     const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
-                    float psum = 0.f;
+                    const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2);
+                    const uint64_t negm2 = f2_pack(-m_use, -m_use);
+                    uint64_t psum2 = f2_pack(0.f, 0.f);
 #pragma unroll
                     for (int c = 0; c < kBN; c += 32) {
                         uint32_t pk[16];
 #pragma unroll
                         for (int i = 0; i < 32; i += 2) {
-                            const float p0 = ex2_approx(fmaf(__uint_as_float(sr[c + i]), p.scale_log2, -m_use));
-                            const float p1 = ex2_approx(fmaf(__uint_as_float(sr[c + i + 1]), p.scale_log2, -m_use));
-                            psum += p0 + p1;
+                            float x0, x1;
+                            f2_unpack(f2_fma(f2_pack(__uint_as_float(sr[c + i]), __uint_as_float(sr[c + i + 1])), scale2, negm2),
+                                      x0, x1);
+                            const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
+                            psum2 = f2_add(psum2, f2_pack(p0, p1));
                             pk[i >> 1] = pack_bf16x2(p0, p1);
                         }
                         tmem_st16(t_s + (c >> 1), pk);
                     }
-                    l_sum += psum;
+                    {
+                        float a, b;
+                        f2_unpack(psum2, a, b);
+                        l_sum += a + b;
+                    }
+                    PROF(6)
                     tmem_st_wait();
                     tc_fence_before();
                     mbar_arrive(&bar_pready[g]);
+                    PROF(1)
                     ++ocnt;
                 }
                 if (!ok) break;
                 // epilogue: wait for the last PV, normalise, store
                 ok = mbar_wait(&bar_odone[g], (ocnt - 1) & 1, abort_flag);
                 if (!ok) break;
+                PROF(2)
                 tc_fence_after();
                 const float inv_l = (l_sum > 0.f) ? 1.0f / l_sum : 0.f;
                 __nv_bfloat16* orow_ptr = p.out + ((size_t)row * p.hq + h) * D;
@@ -372,6 +430,8 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 tc_fence_before();
             }
         }
+        PROF_FLUSH(threadIdx.x == 0, 0)
+        PROF_FLUSH(threadIdx.x == 128, 16)
     }
 
     // ---------------- teardown ----------------
@@ -447,6 +507,12 @@ static int launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtens
 }  // namespace libra
 
 using namespace libra;
+
+#ifdef LIBRA_PROF
+extern "C" int libra_debug_fwd_prof(unsigned long long* host, int n) {
+    return cudaMemcpyFromSymbol(host, libra::g_fwd_prof, sizeof(unsigned long long) * n) == cudaSuccess ? 0 : -4;
+}
+#endif
 
 extern "C" int libra_attn_pool_fwd(const void* q_dev, const void* k_dev, const void* v_dev,
                                    const int32_t* cu_seqlens_dev, const libra_plan_t* plan, void* out_dev,
