@@ -33,7 +33,7 @@ template <int D>
 struct FwdSmem {
     static constexpr int kHalfBytes = 128 * 128;              // 128 rows x 64 bf16 (one swizzle column)
     static constexpr int kTileBytes = kHalfBytes * (D / 64);  // one 128 x D operand tile
-    static constexpr int kStages = (D == 128) ? 4 : 6;
+    static constexpr int kStages = (D == 128) ? 5 : 8;
     static constexpr int kQOff = 0;
     static constexpr int kRingOff = 2 * kTileBytes;
     static constexpr int kBarOff = kRingOff + kStages * kTileBytes;
@@ -337,9 +337,19 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                         for (int i = 0; i < kBN; ++i)
                             if (i < c_lo || i > c_hi) sr[i] = 0xff800000u;  // -inf
                     }
-                    float mx = fmaxf(__uint_as_float(sr[0]), __uint_as_float(sr[1]));
+                    float mx;
+                    {   // eight independent chains keep the 3-input max off the latency-bound path
+                        float pm[8];
 #pragma unroll
-                    for (int i = 2; i < kBN; i += 2) mx = max3(mx, __uint_as_float(sr[i]), __uint_as_float(sr[i + 1]));
+                        for (int u = 0; u < 8; ++u) pm[u] = fmaxf(__uint_as_float(sr[2 * u]), __uint_as_float(sr[2 * u + 1]));
+#pragma unroll
+                        for (int i = 16; i < kBN; i += 16)
+#pragma unroll
+                            for (int u = 0; u < 8; ++u)
+                                pm[u] = max3(pm[u], __uint_as_float(sr[i + 2 * u]), __uint_as_float(sr[i + 2 * u + 1]));
+                        mx = fmaxf(max3(pm[0], pm[1], pm[2]), max3(pm[3], pm[4], pm[5]));
+                        mx = max3(mx, pm[6], pm[7]);
+                    }
                     mx *= p.scale_log2;  // scale > 0, so the max commutes with it
                     // lazy rescale: keep the old reference unless the max grew by > threshold
                     float m_new = m_ref;
@@ -371,7 +381,7 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                     const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
                     const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2);
                     const uint64_t negm2 = f2_pack(-m_use, -m_use);
-                    uint64_t psum2 = f2_pack(0.f, 0.f);
+                    uint64_t psum2[4] = {f2_pack(0.f, 0.f), f2_pack(0.f, 0.f), f2_pack(0.f, 0.f), f2_pack(0.f, 0.f)};
 #pragma unroll
                     for (int c = 0; c < kBN; c += 32) {
                         uint32_t pk[16];
@@ -381,14 +391,14 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                             f2_unpack(f2_fma(f2_pack(__uint_as_float(sr[c + i]), __uint_as_float(sr[c + i + 1])), scale2, negm2),
                                       x0, x1);
                             const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
-                            psum2 = f2_add(psum2, f2_pack(p0, p1));
+                            psum2[(i >> 1) & 3] = f2_add(psum2[(i >> 1) & 3], f2_pack(p0, p1));
                             pk[i >> 1] = pack_bf16x2(p0, p1);
                         }
                         tmem_st16(t_s + (c >> 1), pk);
                     }
                     {
                         float a, b;
-                        f2_unpack(psum2, a, b);
+                        f2_unpack(f2_add(f2_add(psum2[0], psum2[1]), f2_add(psum2[2], psum2[3])), a, b);
                         l_sum += a + b;
                     }
                     PROF(6)
