@@ -28,7 +28,7 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-from paper_2607_23250_b200 import pools  # noqa: E402
+from paper_2607_23250_b200 import pools, sharding  # noqa: E402
 
 METRIC = "useful attention TFLOP/s fwd+bwd (sum of per-sample causal FLOPs)"
 
@@ -160,10 +160,7 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
-    spec = pools.config(args.config, args.skew, seed=rank)       # every rank its own pool
-    if args.seqs:
-        import dataclasses
-        spec = dataclasses.replace(spec, n_seqs=args.seqs, name=f"{spec.name}[{args.seqs} seqs]")
+    spec = sharding.rank_spec(args.config, args.skew, rank, args.seqs)       # every rank its own pool
     lengths = pools.pool_lengths(spec)
     cu_np = pools.cu_seqlens(lengths)
     T, hq, hkv, d = spec.total_tokens, spec.hq, spec.hkv, spec.head_dim
@@ -220,11 +217,8 @@ def run_ours(args):
     busy_b = plan.busy_times(lb.KERNEL_BWD_DKDV).astype(np.float64)
     busy_q = plan.busy_times(lb.KERNEL_BWD_DQ).astype(np.float64)
 
-    ms = torch.tensor([total_ms / args.steps], device=dev, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-    ms_per_step = float(ms.item())
-    value = world * (ff + fb) / (ms_per_step * 1e-3) / 1e12
+    ms_per_step, work = sharding.aggregate(total_ms / args.steps, float(ff + fb), device=dev)
+    value = work / (ms_per_step * 1e-3) / 1e12
 
     e2e = None
     if not args.skip_e2e:
@@ -262,12 +256,9 @@ def run_e2e(args, step, barrier, dev_in, dev_out, world, dev, flops):
         e2e_step()
     e1.record()
     barrier()
-    e2e_ms = torch.tensor([e0.elapsed_time(e1) / n_e2e], device=dev, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(e2e_ms, op=dist.ReduceOp.MAX)
-    e2e_value = world * flops / (float(e2e_ms.item()) * 1e-3) / 1e12
-    return {"value": round(e2e_value, 2), "unit": "TFLOP/s", "h2d_bytes_per_step": h2d,
-            "d2h_bytes_per_step": d2h, "ms_per_step": round(float(e2e_ms.item()), 3)}
+    e2e_ms, work = sharding.aggregate(e0.elapsed_time(e1) / n_e2e, float(flops), device=dev)
+    return {"value": round(work / (e2e_ms * 1e-3) / 1e12, 2), "unit": "TFLOP/s", "h2d_bytes_per_step": h2d,
+            "d2h_bytes_per_step": d2h, "ms_per_step": round(e2e_ms, 3)}
 
 
 def finish(args, rank, world, spec, lengths, plan, value, ms_per_step, kern, busy, clocks, launches, e2e, ff, fb, q):

@@ -1,0 +1,152 @@
+"""Full-size parity: the Qwen3-8B-shaped pool in the launch configuration the benchmark times.
+
+The whole oracle would take minutes here, so outputs are sampled: rows of O / LSE / dQ and
+columns of dK / dV are recomputed one by one by the CPU oracle on the (sample, kv-head group)
+sub-problem they belong to.  Short samples are checked with the oracle's own forward results
+(the mathematical gradient); key columns of long samples use the out / lse arrays that are the
+backward's inputs.  Properties that hold at any size are checked over the whole tensors.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2607_23250_b200 import pools
+
+pytestmark = pytest.mark.gpu
+
+TOL_O, TOL_G, TOL_LSE = 2e-2, 5e-2, 1e-3
+
+
+def _rel(got, want, floor=1e-3):
+    want = np.asarray(want, np.float64)
+    return float(np.abs(np.asarray(got, np.float64) - want).max() / max(np.abs(want).max(), floor))
+
+
+@pytest.fixture(scope="module")
+def run():
+    from paper_2607_23250_b200 import binding as lb
+    spec = pools.config(2)
+    lengths = pools.pool_lengths(spec)
+    cu_np = pools.cu_seqlens(lengths)
+    T, hq, hkv, d = spec.total_tokens, spec.hq, spec.hkv, spec.head_dim
+    t = pools.make_tensors(T, hq, hkv, d, seed=0, device="cuda")
+    cu = torch.from_numpy(cu_np).cuda()
+    plan = lb.libra_plan_tiles(cu, hq, 256, tile_kv=128, n_heads_kv=hkv, total_tokens=T)   # as bench.py
+    assert plan.status() == 0
+    out, lse = lb.libra_attn_pool_fwd(t["q"], t["k"], t["v"], plan)
+    dq, dk, dv = lb.libra_attn_pool_bwd(t["q"], t["k"], t["v"], out, lse, t["dout"], plan)
+    torch.cuda.synchronize()
+    for kern in (lb.KERNEL_FWD, lb.KERNEL_BWD_DKDV, lb.KERNEL_BWD_DQ):
+        plan.busy_times(kern)
+    res = dict(spec=spec, lengths=lengths, cu=cu_np, t=t, out=out, lse=lse, dq=dq, dk=dk, dv=dv, plan=plan, lb=lb)
+    yield res
+    plan.destroy()
+
+
+def _sub(run, j, kvh):
+    """Host copy (fp32) of sample j restricted to kv head kvh and its query-head group."""
+    spec, cu, t = run["spec"], run["cu"], run["t"]
+    G = spec.hq // spec.hkv
+    s, e = int(cu[j]), int(cu[j + 1])
+    hs = slice(kvh * G, (kvh + 1) * G)
+    f = lambda x: x.float().cpu().numpy()
+    return dict(q=f(t["q"][s:e, hs]), dout=f(t["dout"][s:e, hs]), k=f(t["k"][s:e, kvh:kvh + 1]),
+                v=f(t["v"][s:e, kvh:kvh + 1]), out=f(run["out"][s:e, hs]), lse=run["lse"][hs, s:e].cpu().numpy(),
+                dq=f(run["dq"][s:e, hs]), dk=f(run["dk"][s:e, kvh:kvh + 1]), dv=f(run["dv"][s:e, kvh:kvh + 1]),
+                n=e - s, G=G)
+
+
+def test_plan_matches_oracle_at_full_size(run):
+    lb, plan, spec = run["lb"], run["plan"], run["spec"]
+    for direction, d_or, tile, H in ((lb.LIBRA_DIR_Q, 0, 256, spec.hq), (lb.LIBRA_DIR_KV, 1, 128, spec.hkv)):
+        got = plan.export(direction)
+        want = oracle.plan(run["cu"], H, tile, plan.info(direction)["n_workers"], d_or)
+        for key in ("weight", "order", "cta_of_tile", "cta_offsets", "cta_tiles", "loads"):
+            assert np.array_equal(got[key], want[key]), (direction, key)
+
+
+def test_sampled_rows_forward_and_dq(run):
+    rng = np.random.default_rng(0)
+    lengths = np.asarray(run["lengths"])
+    order = np.argsort(-lengths)
+    picks = list(order[:3]) + list(rng.choice(len(lengths), 5, replace=False))     # long samples and random ones
+    worst = dict(o=0.0, lse=0.0, dq=0.0)
+    for j in picks:
+        kvh = int(rng.integers(0, run["spec"].hkv))
+        s = _sub(run, int(j), kvh)
+        n = s["n"]
+        cand = {0, n - 1, min(n - 1, 127), min(n - 1, 128), min(n - 1, 255), min(n - 1, 256), n // 2}
+        cand |= {int(x) for x in rng.integers(0, n, 4)}
+        # global tile boundaries that fall inside the sample
+        first = int(run["cu"][j])
+        cand |= {b - first for b in range((first // 256 + 1) * 256 - 1, first + n, 4096) if 0 <= b - first < n}
+        rows = np.array(sorted(cand), dtype=np.int64)
+        heads = rng.integers(0, s["G"], size=len(rows)).astype(np.int32)
+        o_ref, l_ref = oracle.attn_fwd_rows(s["q"], s["k"], s["v"], [0, n], rows, heads)
+        dq_ref = oracle.attn_dq_rows(s["q"], s["k"], s["v"], s["dout"], [0, n], rows, heads)
+        for x, (r, h) in enumerate(zip(rows, heads)):
+            worst["o"] = max(worst["o"], _rel(s["out"][r, h], o_ref[x]))
+            worst["lse"] = max(worst["lse"], abs(float(s["lse"][h, r]) - float(l_ref[x])))
+            worst["dq"] = max(worst["dq"], _rel(s["dq"][r, h], dq_ref[x], floor=1e-2))
+    assert worst["o"] <= TOL_O and worst["lse"] <= TOL_LSE and worst["dq"] <= TOL_G, worst
+
+
+def test_short_samples_full_gradient(run):
+    """Samples of at most 1500 tokens: the whole sample against the oracle's own forward + backward."""
+    rng = np.random.default_rng(1)
+    lengths = np.asarray(run["lengths"])
+    small = [j for j in range(len(lengths)) if 2 <= lengths[j] <= 1500]
+    for j in rng.choice(small, 4, replace=False):
+        kvh = int(rng.integers(0, run["spec"].hkv))
+        s = _sub(run, int(j), kvh)
+        cu = [0, s["n"]]
+        o_ref, l_ref = oracle.attn_fwd(s["q"], s["k"], s["v"], cu)
+        g_ref = oracle.attn_bwd(s["q"], s["k"], s["v"], o_ref, l_ref, s["dout"], cu)
+        assert _rel(s["out"], o_ref) <= TOL_O
+        assert np.abs(s["lse"] - l_ref).max() <= TOL_LSE
+        for name, ref in zip(("dq", "dk", "dv"), g_ref):
+            assert _rel(s[name], ref) <= TOL_G, (name, int(j))
+
+
+def test_sampled_key_columns_of_long_samples(run):
+    rng = np.random.default_rng(2)
+    lengths = np.asarray(run["lengths"])
+    for j in np.argsort(-lengths)[:2]:
+        kvh = int(rng.integers(0, run["spec"].hkv))
+        s = _sub(run, int(j), kvh)
+        n = s["n"]
+        cols = np.array(sorted({0, 1, 127, 128, n // 3, n // 2, n - 129, n - 2, n - 1} | {int(x) for x in rng.integers(0, n, 3)}),
+                        dtype=np.int64)
+        # the group's heads are heads 0..G-1 of the sub-problem, on its single kv head 0
+        dk_ref, dv_ref = oracle.attn_dkv_cols(s["q"], s["k"], s["v"], s["out"], s["lse"], s["dout"], [0, n], cols,
+                                              np.zeros(len(cols), np.int32))
+        for x, cidx in enumerate(cols):
+            assert _rel(s["dk"][cidx, 0], dk_ref[x], floor=1e-2) <= TOL_G, ("dk", int(cidx))
+            assert _rel(s["dv"][cidx, 0], dv_ref[x], floor=1e-2) <= TOL_G, ("dv", int(cidx))
+
+
+def test_whole_tensor_properties(run):
+    spec, cu, t = run["spec"], run["cu"], run["t"]
+    for name in ("out", "lse", "dq", "dk", "dv"):
+        assert bool(torch.isfinite(run[name]).all()), name
+    lengths = np.asarray(run["lengths"])
+    ones = [j for j in range(len(lengths)) if lengths[j] == 1]
+    G = spec.hq // spec.hkv
+    for j in ones[:8]:
+        r = int(cu[j])
+        # a one-token sample returns its V row, has zero dQ / dK, and dV = sum of the group's dO
+        v_rep = t["v"][r].float().repeat_interleave(G, dim=0)
+        assert torch.equal(run["out"][r].float(), v_rep)
+        assert float(run["dq"][r].float().abs().max()) < 1e-5 and float(run["dk"][r].float().abs().max()) < 1e-5
+        want = t["dout"][r].float().reshape(spec.hkv, G, -1).sum(1)
+        assert float((run["dv"][r].float() - want).abs().max()) <= 0.02 * float(want.abs().max())
+    # first row of every sample attends only itself
+    firsts = torch.from_numpy(cu[:-1].astype(np.int64)).cuda()
+    v_first = t["v"][firsts].float().repeat_interleave(G, dim=1)
+    assert torch.equal(run["out"][firsts].float(), v_first)
+    # same call again gives bit-identical results (no atomics anywhere on the path)
+    lb, plan = run["lb"], run["plan"]
+    dq2, dk2, dv2 = lb.libra_attn_pool_bwd(t["q"], t["k"], t["v"], run["out"], run["lse"], t["dout"], plan)
+    torch.cuda.synchronize()
+    assert torch.equal(dq2, run["dq"]) and torch.equal(dk2, run["dk"]) and torch.equal(dv2, run["dv"])
