@@ -379,10 +379,10 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
                 for (int j = 0; j < 64; j += 4) {
                     const float4 l4 = *reinterpret_cast<const float4*>(lse2 + j);
-                    pf[j] = ex2_approx(fmaf(__uint_as_float(sv[j]), p.scale_log2, -l4.x));
-                    pf[j + 1] = ex2_approx(fmaf(__uint_as_float(sv[j + 1]), p.scale_log2, -l4.y));
-                    pf[j + 2] = ex2_approx(fmaf(__uint_as_float(sv[j + 2]), p.scale_log2, -l4.z));
-                    pf[j + 3] = ex2_approx(fmaf(__uint_as_float(sv[j + 3]), p.scale_log2, -l4.w));
+                    pf[j] = ex2_mixed<0>(fmaf(__uint_as_float(sv[j]), p.scale_log2, -l4.x));
+                    pf[j + 1] = ex2_mixed<1>(fmaf(__uint_as_float(sv[j + 1]), p.scale_log2, -l4.y));
+                    pf[j + 2] = ex2_mixed<0>(fmaf(__uint_as_float(sv[j + 2]), p.scale_log2, -l4.z));
+                    pf[j + 3] = ex2_mixed<1>(fmaf(__uint_as_float(sv[j + 3]), p.scale_log2, -l4.w));
                 }
                 if (need_mask) {
 #pragma unroll

@@ -339,7 +339,10 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                         mbar_arrive(bar_sfree);  // S(j+1) may overwrite the columns
                         float pf[64];
 #pragma unroll
-                        for (int i = 0; i < 64; ++i) pf[i] = ex2_approx(fmaf(__uint_as_float(sv[i]), p.scale_log2, -lse2));
+                        for (int i = 0; i < 64; i += 2) {
+                            pf[i] = ex2_mixed<0>(fmaf(__uint_as_float(sv[i]), p.scale_log2, -lse2));
+                            pf[i + 1] = ex2_mixed<1>(fmaf(__uint_as_float(sv[i + 1]), p.scale_log2, -lse2));
+                        }
                         if (need_mask) {
 #pragma unroll
                             for (int i = 0; i < 64; ++i)

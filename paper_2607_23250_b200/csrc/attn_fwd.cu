@@ -246,6 +246,7 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                     for (int g = 0; g < 2; ++g)
                         if (lo >= r[g].lo && lo <= r[g].hi) issue_s(g, st);
                     tc_commit(&bar_empty[st]);
+                    if (lo == hi) tc_commit(bar_qempty);  // no later MMA of this tile reads Q
                 }
                 ++ring;
                 for (int j = lo; j <= hi && ok; ++j) {
@@ -281,10 +282,10 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                     if (lane == 0) {
                         tc_commit(&bar_empty[st_v]);
                         if (j + 1 <= hi) tc_commit(&bar_empty[st_k]);
-                    }
+                        if (j + 1 == hi) tc_commit(bar_qempty);  // S(hi) was the last reader of Q: the next
+                    }                                            // tile's Q load overlaps the last block
                     __syncwarp();
                 }
-                if (ok && lane == 0) tc_commit(bar_qempty);
                 __syncwarp();
             }
         }
@@ -390,7 +391,7 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                             float x0, x1;
                             f2_unpack(f2_fma(f2_pack(__uint_as_float(sr[c + i]), __uint_as_float(sr[c + i + 1])), scale2, negm2),
                                       x0, x1);
-                            const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
+                            const float p0 = ex2_mixed<0>(x0), p1 = ex2_mixed<1>(x1);
                             psum2[(i >> 1) & 3] = f2_add(psum2[(i >> 1) & 3], f2_pack(p0, p1));
                             pk[i >> 1] = pack_bf16x2(p0, p1);
                         }

@@ -37,7 +37,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
+#ifdef LIBRA_DBG_TEST_WAIT
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+#else
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+#endif
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
         : "r"(smem_u32(bar)), "r"(parity)
@@ -211,6 +215,36 @@ __device__ __forceinline__ float ex2_approx(float x) {
     return y;
 #endif
 }
+__device__ __forceinline__ float ex2_approx(float x);
+// 2^x without the special-function unit (the MUFU pipe does 16 exp2 per clock per SM, the FMA
+// pipes 128 flops): round x to the nearest integer n with the magic-number trick, evaluate 2^f on
+// f = x - n in [-0.5, 0.5] with a cubic (relative error < 1e-4, far below bf16 resolution),
+// then add n to the exponent field.  Valid for x in [-126, 126]; smaller x is clamped (result
+// 2^-126, which rounds to zero in every use here).
+__device__ __forceinline__ float ex2_emul(float x) {
+    x = fmaxf(x, -126.0f);
+    const float t = x + 12582912.0f;             // 1.5 * 2^23: low mantissa bits now hold n
+    const float f = x - (t - 12582912.0f);
+    float p = fmaf(f, 0.05550410866f, 0.2402265070f);
+    p = fmaf(p, f, 0.6931471806f);
+    p = fmaf(p, f, 1.0f);
+    return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+}
+// Alternate between the two units so neither is the bottleneck: even elements on MUFU, odd on FMA.
+// Measured on B200: with half of the exponentials on the FMA pipes all three kernels got slower
+// (issue slots, not the MUFU pipe, are what the softmax warps run out of), so this is off.
+#ifndef LIBRA_EX2_EMUL
+#define LIBRA_EX2_EMUL 0
+#endif
+template <int I>
+__device__ __forceinline__ float ex2_mixed(float x) {
+#if LIBRA_EX2_EMUL
+    return (I & 1) ? ex2_emul(x) : ex2_approx(x);
+#else
+    return ex2_approx(x);
+#endif
+}
+
 // Packed pairs of fp32 (sm_100 executes add/mul/fma on two floats per instruction).
 __device__ __forceinline__ uint64_t f2_pack(float lo, float hi) {
     uint64_t r;
