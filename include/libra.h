@@ -40,6 +40,7 @@ extern "C" {
 #define LIBRA_ERR_TIMEOUT       (-6)  /* a bounded device-side wait gave up (reported by libra_status)*/
 #define LIBRA_ERR_BAD_SEQLENS   (-7)  /* cu_seqlens failed the device-side check                      */
 #define LIBRA_ERR_NO_DEVICE     (-8)  /* no CUDA device / not an sm_100 device                        */
+#define LIBRA_ERR_SCRATCH_TOO_SMALL (-9) /* problem needs more than the library's built-in scratch    */
 
 #define LIBRA_DIR_Q   1   /* query-major tiles (forward)  */
 #define LIBRA_DIR_KV  2   /* key-major tiles   (backward) */
@@ -150,6 +151,30 @@ int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const void* v_dev,
                         const int32_t* cu_seqlens_dev, const libra_plan_t* plan,
                         void* dq_dev, void* dk_dev, void* dv_dev, void* workspace_dev,
                         const libra_dims* dims, void* stream);
+
+/* Backward without any allocation (no counterpart in the paper: this is a deployment aid).
+ * Same computation, arguments and results as libra_attn_pool_bwd, but the caller passes no
+ * workspace: the row-statistics scratch is a fixed 16 MiB array inside the library's device
+ * image (libra_attn_pool_bwd_noalloc_max_bytes reports its size).  It is meant for callers that
+ * cannot obtain device memory when they need the backward pass, for example while a stream is
+ * being captured, inside an allocator callback, or in a process that fixes its device memory at
+ * start-up.  The call performs no cudaMalloc / cudaFree and calls no allocating routine.
+ *   - Limit: libra_attn_pool_bwd_workspace_bytes(plan, dims) must not exceed the built-in size
+ *     (2 * hq * round_up(T, 128) floats <= 4 Mi floats); otherwise nothing is launched and
+ *     LIBRA_ERR_SCRATCH_TOO_SMALL is returned.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current); make that first call outside any stream capture.
+ *   - All calls on a device share the one array and it keeps the previous call's contents; the
+ *     call overwrites every element it later reads, so nothing needs clearing.  Two calls whose
+ *     GPU work overlaps (different streams, no dependency) race on it: serialise them.
+ *   - Every GPU that loads the library holds the 16 MiB until the process exits.
+ */
+size_t libra_attn_pool_bwd_noalloc_max_bytes(void);
+int libra_attn_pool_bwd_noalloc(const void* q_dev, const void* k_dev, const void* v_dev,
+                                const void* out_dev, const float* lse_dev, const void* dout_dev,
+                                const int32_t* cu_seqlens_dev, const libra_plan_t* plan,
+                                void* dq_dev, void* dk_dev, void* dv_dev,
+                                const libra_dims* dims, void* stream);
 
 /* ---- instrumentation -------------------------------------------------------------------
  * Per-CTA busy time of the most recent launch of kernel `which` (LIBRA_KERNEL_*) that used this

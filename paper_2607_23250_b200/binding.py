@@ -23,10 +23,12 @@ LIBRA_DIR_Q, LIBRA_DIR_KV = 1, 2
 KERNEL_FWD, KERNEL_BWD_DKDV, KERNEL_BWD_DQ = 1, 2, 3
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_PLAN_MISMATCH, ERR_CUDA = -1, -2, -3, -4
 ERR_OVERFLOW, ERR_TIMEOUT, ERR_BAD_SEQLENS, ERR_NO_DEVICE = -5, -6, -7, -8
+ERR_SCRATCH_TOO_SMALL = -9
 
 EXPORTS = ["libra_plan_tiles", "libra_plan_info", "libra_plan_status", "libra_plan_export",
            "libra_plan_destroy", "libra_attn_pool_fwd", "libra_attn_pool_bwd_workspace_bytes",
-           "libra_attn_pool_bwd", "libra_busy_times", "libra_plan_set_timing", "libra_kernel_time_ms", "libra_launch_count",
+           "libra_attn_pool_bwd", "libra_attn_pool_bwd_noalloc_max_bytes", "libra_attn_pool_bwd_noalloc",
+           "libra_busy_times", "libra_plan_set_timing", "libra_kernel_time_ms", "libra_launch_count",
            "libra_strerror"]
 
 
@@ -43,6 +45,7 @@ class Dims(ctypes.Structure):
 _lib.libra_strerror.restype = ctypes.c_char_p
 _lib.libra_launch_count.restype = ctypes.c_int64
 _lib.libra_attn_pool_bwd_workspace_bytes.restype = ctypes.c_size_t
+_lib.libra_attn_pool_bwd_noalloc_max_bytes.restype = ctypes.c_size_t
 _vp = ctypes.c_void_p
 
 
@@ -181,4 +184,19 @@ def libra_attn_pool_bwd(q, k, v, out, lse, dout, plan: Plan, dq=None, dk=None, d
     _check(_lib.libra_attn_pool_bwd(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), _ptr(dout),
                                     _ptr(plan.cu_seqlens), plan._h, _ptr(dq), _ptr(dk), _ptr(dv), _ptr(workspace),
                                     ctypes.byref(dims), _stream(stream)), "libra_attn_pool_bwd")
+    return dq, dk, dv
+
+
+def libra_attn_pool_bwd_noalloc_max_bytes() -> int:
+    return int(_lib.libra_attn_pool_bwd_noalloc_max_bytes())
+
+
+def libra_attn_pool_bwd_noalloc(q, k, v, out, lse, dout, plan: Plan, dq, dk, dv, scale=None, stream=None):
+    """Backward that takes no workspace and allocates nothing: dq, dk, dv must be passed in.
+    Raises LibraError(ERR_SCRATCH_TOO_SMALL) when the pool exceeds the library's built-in scratch."""
+    _chk(q, k, v, out, lse, dout, dq, dk, dv)
+    dims = _dims(q, k, plan, scale)
+    _check(_lib.libra_attn_pool_bwd_noalloc(_ptr(q), _ptr(k), _ptr(v), _ptr(out), _ptr(lse), _ptr(dout),
+                                            _ptr(plan.cu_seqlens), plan._h, _ptr(dq), _ptr(dk), _ptr(dv),
+                                            ctypes.byref(dims), _stream(stream)), "libra_attn_pool_bwd_noalloc")
     return dq, dk, dv

@@ -430,6 +430,7 @@ extern "C" const char* libra_strerror(int code) {
         case LIBRA_ERR_TIMEOUT: return "a bounded device-side wait timed out";
         case LIBRA_ERR_BAD_SEQLENS: return "cu_seqlens is malformed";
         case LIBRA_ERR_NO_DEVICE: return "no usable CUDA device";
+        case LIBRA_ERR_SCRATCH_TOO_SMALL: return "problem exceeds the library's built-in scratch (use libra_attn_pool_bwd with a caller workspace)";
         default: return "unknown error";
     }
 }
