@@ -33,10 +33,9 @@ __device__ __forceinline__ void bulk_load_1d(void* smem_dst, const void* gsrc, u
                  "l"(reinterpret_cast<uint64_t>(gsrc)), "r"(bytes), "r"(smem_u32(bar))
                  : "memory");
 }
+// Every lane polls the barrier itself (no elected lane + shuffle on the path between MMA groups).
 __device__ __forceinline__ bool warp_wait_b(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-    int ok = 1;
-    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag) ? 1 : 0;
-    return __shfl_sync(0xffffffffu, ok, 0) != 0;
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
 }
 
 #ifdef LIBRA_PROF
@@ -379,10 +378,10 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #pragma unroll
                 for (int j = 0; j < 64; j += 4) {
                     const float4 l4 = *reinterpret_cast<const float4*>(lse2 + j);
-                    pf[j] = ex2_mixed<0>(fmaf(__uint_as_float(sv[j]), p.scale_log2, -l4.x));
-                    pf[j + 1] = ex2_mixed<1>(fmaf(__uint_as_float(sv[j + 1]), p.scale_log2, -l4.y));
-                    pf[j + 2] = ex2_mixed<0>(fmaf(__uint_as_float(sv[j + 2]), p.scale_log2, -l4.z));
-                    pf[j + 3] = ex2_mixed<1>(fmaf(__uint_as_float(sv[j + 3]), p.scale_log2, -l4.w));
+                    pf[j] = ex2_sel(fmaf(__uint_as_float(sv[j]), p.scale_log2, -l4.x), j);
+                    pf[j + 1] = ex2_sel(fmaf(__uint_as_float(sv[j + 1]), p.scale_log2, -l4.y), j + 1);
+                    pf[j + 2] = ex2_sel(fmaf(__uint_as_float(sv[j + 2]), p.scale_log2, -l4.z), j + 2);
+                    pf[j + 3] = ex2_sel(fmaf(__uint_as_float(sv[j + 3]), p.scale_log2, -l4.w), j + 3);
                 }
                 if (need_mask) {
 #pragma unroll

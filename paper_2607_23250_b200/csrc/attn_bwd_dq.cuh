@@ -340,8 +340,8 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                         float pf[64];
 #pragma unroll
                         for (int i = 0; i < 64; i += 2) {
-                            pf[i] = ex2_mixed<0>(fmaf(__uint_as_float(sv[i]), p.scale_log2, -lse2));
-                            pf[i + 1] = ex2_mixed<1>(fmaf(__uint_as_float(sv[i + 1]), p.scale_log2, -lse2));
+                            pf[i] = ex2_sel(fmaf(__uint_as_float(sv[i]), p.scale_log2, -lse2), i);
+                            pf[i + 1] = ex2_sel(fmaf(__uint_as_float(sv[i + 1]), p.scale_log2, -lse2), i + 1);
                         }
                         if (need_mask) {
 #pragma unroll

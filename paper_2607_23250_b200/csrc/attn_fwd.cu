@@ -69,10 +69,11 @@ __device__ __forceinline__ SlotRange slot_range(const int32_t* tok_start, int64_
     return r;
 }
 
+// Every lane polls the barrier itself: electing one lane and broadcasting its result costs a
+// divergent branch plus a shuffle on the path between two MMA groups, which is enough silence for the
+// tensor pipe to drain (a wait on an already completed barrier measured ~230 cycles that way, ~100 so).
 __device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-    int ok = 1;
-    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag) ? 1 : 0;
-    return __shfl_sync(0xffffffffu, ok, 0) != 0;
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
 }
 
 #ifdef LIBRA_PROF
@@ -391,7 +392,7 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                             float x0, x1;
                             f2_unpack(f2_fma(f2_pack(__uint_as_float(sr[c + i]), __uint_as_float(sr[c + i + 1])), scale2, negm2),
                                       x0, x1);
-                            const float p0 = ex2_mixed<0>(x0), p1 = ex2_mixed<1>(x1);
+                            const float p0 = ex2_sel(x0, i), p1 = ex2_sel(x1, i + 1);
                             psum2[(i >> 1) & 3] = f2_add(psum2[(i >> 1) & 3], f2_pack(p0, p1));
                             pk[i >> 1] = pack_bf16x2(p0, p1);
                         }

@@ -86,6 +86,12 @@ __device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* m
         "l"(reinterpret_cast<uint64_t>(m)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
 }
+// Pull a tile into L2 ahead of the load that will need it (no shared memory, no barrier).
+__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap* m, int c0, int c1, int c2) {
+    asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(reinterpret_cast<uint64_t>(m)),
+                 "r"(c0), "r"(c1), "r"(c2)
+                 : "memory");
+}
 // Make generic-proxy shared-memory writes visible to the async proxy (TMA, tcgen05.mma).
 __device__ __forceinline__ void fence_proxy_async_smem() {
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -230,16 +236,14 @@ __device__ __forceinline__ float ex2_emul(float x) {
     p = fmaf(p, f, 1.0f);
     return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
 }
-// Alternate between the two units so neither is the bottleneck: even elements on MUFU, odd on FMA.
-// Measured on B200: with half of the exponentials on the FMA pipes all three kernels got slower
-// (issue slots, not the MUFU pipe, are what the softmax warps run out of), so this is off.
-#ifndef LIBRA_EX2_EMUL
-#define LIBRA_EX2_EMUL 0
+// Optionally move one exponential in every LIBRA_EX2_EMUL_MOD onto the FMA pipes (0 = never).  `idx`
+// must be a compile-time constant after unrolling so the choice folds away.
+#ifndef LIBRA_EX2_EMUL_MOD
+#define LIBRA_EX2_EMUL_MOD 0
 #endif
-template <int I>
-__device__ __forceinline__ float ex2_mixed(float x) {
-#if LIBRA_EX2_EMUL
-    return (I & 1) ? ex2_emul(x) : ex2_approx(x);
+__device__ __forceinline__ float ex2_sel(float x, int idx) {
+#if LIBRA_EX2_EMUL_MOD > 0
+    return (idx % LIBRA_EX2_EMUL_MOD) == (LIBRA_EX2_EMUL_MOD - 1) ? ex2_emul(x) : ex2_approx(x);
 #else
     return ex2_approx(x);
 #endif
