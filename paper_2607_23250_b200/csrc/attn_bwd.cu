@@ -172,6 +172,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
     if (warp == 8) {
         // ---------------- TMA producer ----------------
+        const bool leader = elect_one();
         uint32_t ucnt = 0, it_all = 0;
         bool ok = true;
         for (int idx = unit_begin; idx < unit_end && ok; ++idx) {
@@ -182,7 +183,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const int nblk = last_q_block(p.tok_end, p.T, k0) - i_lo + 1;
             ok = warp_wait_b(bar_kvempty, (ucnt & 1) ^ 1, abort_flag);
             if (!ok) break;
-            if (lane == 0) {
+            if (leader) {
                 mbar_arrive_expect_tx(bar_kvfull, 2 * L::kTileBytes);
                 for (int half = 0; half < D / 64; ++half) {
                     tma_load_3d(smem + L::kKOff + half * L::kHalfBytes, &tm_k, bar_kvfull, half * 64, kvh, (int)k0);
@@ -197,7 +198,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const uint32_t st = it_all & 1, par = ((it_all >> 1) & 1) ^ 1;
                 ok = warp_wait_b(&bar_qempty[st], par, abort_flag);
                 if (!ok) break;
-                if (lane == 0) {
+                if (leader) {
                     mbar_arrive_expect_tx(&bar_qfull[st], L::kTileBytes + 1024);
                     for (int half = 0; half < D / 64; ++half)
                         tma_load_3d(smem + L::kQOff + st * L::kTileBytes + half * L::kHalfBytes, &tm_q, &bar_qfull[st],
@@ -208,7 +209,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
                 ok = warp_wait_b(&bar_doempty[st], par, abort_flag);
                 if (!ok) break;
-                if (lane == 0) {
+                if (leader) {
                     mbar_arrive_expect_tx(&bar_dofull[st], L::kTileBytes);
                     for (int half = 0; half < D / 64; ++half)
                         tma_load_3d(smem + L::kDoOff + st * L::kTileBytes + half * L::kHalfBytes, &tm_do,
@@ -218,6 +219,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         }
     } else if (warp == 9) {
         // ---------------- MMA issuer ----------------
+        const bool leader = elect_one();
         constexpr uint32_t idesc_s = make_idesc(128, 128, 0, 0);  // S^T, dP^T: both operands K-major
         constexpr uint32_t idesc_acc = make_idesc(128, D, 0, 1);  // dV, dK: A from TMEM, B MN-major
         const uint32_t sb = smem_u32(smem);
@@ -256,13 +258,13 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             ok = warp_wait_b(&bar_qfull[it_all & 1], (it_all >> 1) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            if (lane == 0) {
+            if (leader) {
                 issue_kmajor(kColS, L::kKOff, L::kQOff + (it_all & 1) * L::kTileBytes);
                 tc_commit(bar_sfull);
             }
             ok = warp_wait_b(&bar_dofull[it_all & 1], (it_all >> 1) & 1, abort_flag);
             if (!ok) break;
-            if (lane == 0) {
+            if (leader) {
                 issue_kmajor(kColDP, L::kVOff, L::kDoOff + (it_all & 1) * L::kTileBytes);
                 tc_commit(bar_dpfull);
             }
@@ -284,7 +286,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
 #endif
                 tc_fence_after();
-                if (lane == 0) {
+                if (leader) {
                     issue_acc(kColDV, kColS, L::kDoOff + st * L::kTileBytes, it > 0);
                     tc_commit(&bar_doempty[st]);
                 }
@@ -294,7 +296,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     ok = warp_wait_b(&bar_qfull[nx & 1], (nx >> 1) & 1, abort_flag);
                     if (!ok) break;
                     PROF(1)
-                    if (lane == 0) {
+                    if (leader) {
                         issue_kmajor(kColS, L::kKOff, L::kQOff + (nx & 1) * L::kTileBytes);
                         tc_commit(bar_sfull);
                     }
@@ -307,7 +309,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 #endif
                 PROF(2)
                 tc_fence_after();
-                if (lane == 0) {
+                if (leader) {
                     issue_acc(kColDK, kColDP, L::kQOff + st * L::kTileBytes, it > 0);
                     tc_commit(&bar_qempty[st]);
                 }
@@ -317,14 +319,14 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     ok = warp_wait_b(&bar_dofull[nx & 1], (nx >> 1) & 1, abort_flag);
                     if (!ok) break;
                     PROF(3)
-                    if (lane == 0) {
+                    if (leader) {
                         issue_kmajor(kColDP, L::kVOff, L::kDoOff + (nx & 1) * L::kTileBytes);
                         tc_commit(bar_dpfull);
                     }
                 }
                 __syncwarp();
             }
-            if (ok && lane == 0) {
+            if (ok && leader) {
                 tc_commit(bar_dkvfull);
                 tc_commit(bar_kvempty);
             }
@@ -541,7 +543,7 @@ static int launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtens
     if (mp->timing) cudaEventRecord(mp->ev[1][0], s);
     k_attn_bwd_dkdv<D><<<Wa, kBwdThreads, DkvSmem<D>::kBytes, s>>>(tq, tk, tv, tdo, pa);
     if (mp->timing) { cudaEventRecord(mp->ev[1][1], s); mp->ev_valid[1] = 1; cudaEventRecord(mp->ev[2][0], s); }
-    k_attn_bwd_dq<D><<<Wb, kBwdThreads, DqSmem<D>::kBytes, s>>>(tq, tk, tv, tdo, pb);
+    k_attn_bwd_dq<D><<<Wb, kDqThreads, DqSmem<D>::kBytes, s>>>(tq, tk, tv, tdo, pb);
     if (mp->timing) { cudaEventRecord(mp->ev[2][1], s); mp->ev_valid[2] = 1; }
     count_launch(2);
     return cudaGetLastError() == cudaSuccess ? LIBRA_OK : LIBRA_ERR_CUDA;
@@ -550,6 +552,12 @@ static int launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtens
 }  // namespace libra
 
 using namespace libra;
+
+#ifdef LIBRA_TRACE
+extern "C" int libra_debug_trace(long long* host, int n) {
+    return cudaMemcpyFromSymbol(host, libra::g_trace, sizeof(long long) * n) == cudaSuccess ? 0 : -4;
+}
+#endif
 
 #ifdef LIBRA_PROF
 extern "C" int libra_debug_bwd_prof(unsigned long long* host, int n) {

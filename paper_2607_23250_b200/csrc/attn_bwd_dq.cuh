@@ -15,6 +15,11 @@
 
 namespace libra {
 
+constexpr int kDqGroups = 4;                      // compute warpgroups: each owns 128 / kDqGroups key columns
+constexpr int kDqCW = 128 / kDqGroups;            // S / dP columns per compute thread
+constexpr int kDqThreads = (4 * kDqGroups + 2) * 32;
+constexpr int kDqTmaWarp = 4 * kDqGroups, kDqMmaWarp = 4 * kDqGroups + 1;
+
 template <int D>
 struct DqSmem {
     static constexpr int kHalfBytes = 128 * 128;
@@ -49,7 +54,7 @@ struct DqParams {
 };
 
 template <int D>
-__global__ void __launch_bounds__(kBwdThreads, 1)
+__global__ void __launch_bounds__(kDqThreads, 1)
 k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
               const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do, const DqParams p) {
     using L = DqSmem<D>;
@@ -82,26 +87,26 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     }
     if (threadIdx.x == 0) {
         mbar_init(bar_qfull, 1);
-        mbar_init(bar_qempty, 128);
+        mbar_init(bar_qempty, 64 * kDqGroups);   // the groups that stage Q
         mbar_init(bar_dofull, 1);
-        mbar_init(bar_doempty, 128);
+        mbar_init(bar_doempty, 64 * kDqGroups);  // the groups that stage dO
         for (int s = 0; s < L::kKStages; ++s) { mbar_init(&bar_kfull[s], 1); mbar_init(&bar_kempty[s], 1); }
         for (int s = 0; s < L::kVStages; ++s) { mbar_init(&bar_vfull[s], 1); mbar_init(&bar_vempty[s], 1); }
-        mbar_init(bar_qtready, 256);
+        mbar_init(bar_qtready, 128 * kDqGroups);
         mbar_init(bar_sfull, 1);
-        mbar_init(bar_sfree, 256);
+        mbar_init(bar_sfree, 128 * kDqGroups);
         mbar_init(bar_dpfull, 1);
-        mbar_init(bar_dsready, 256);
+        mbar_init(bar_dsready, 128 * kDqGroups);
         mbar_init(bar_dqfull, 1);
         *abort_flag = 0;
         fence_mbar_init();
         p.busy[2 * cta] = globaltimer_ns();
     }
-    if (warp == 9) {
+    if (warp == kDqMmaWarp) {
         tmem_alloc(tmem_slot, 512);
         tmem_relinquish();
     }
-    if (warp == 8 && lane == 0) {
+    if (warp == kDqTmaWarp && lane == 0) {
         prefetch_tmap(&tm_q);
         prefetch_tmap(&tm_k);
         prefetch_tmap(&tm_v);
@@ -121,8 +126,9 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
 
     // All roles walk the same sequence of sub-blocks: (tile, sub-block of 128 rows, head of the shard).
     // A sub-block past the end of the pool is skipped by every role.
-    if (warp == 8) {
+    if (warp == kDqTmaWarp) {
         // ---------------- TMA producer ----------------
+        const bool leader = elect_one();
         uint32_t bcnt = 0, kcnt = 0, vcnt = 0;
         bool ok = true;
         for (int idx = tile_begin; idx < tile_end && ok; ++idx) {
@@ -136,14 +142,14 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     const int kvh = h / G;
                     ok = warp_wait_b(bar_qempty, (bcnt & 1) ^ 1, abort_flag);
                     if (!ok) break;
-                    if (lane == 0) {
+                    if (leader) {
                         mbar_arrive_expect_tx(bar_qfull, L::kTileBytes);
                         for (int half = 0; half < D / 64; ++half)
                             tma_load_3d(smem + L::kQOff + half * L::kHalfBytes, &tm_q, bar_qfull, half * 64, h, (int)q0);
                     }
                     ok = warp_wait_b(bar_doempty, (bcnt & 1) ^ 1, abort_flag);
                     if (!ok) break;
-                    if (lane == 0) {
+                    if (leader) {
                         mbar_arrive_expect_tx(bar_dofull, L::kTileBytes);
                         for (int half = 0; half < D / 64; ++half)
                             tma_load_3d(smem + L::kDoOff + half * L::kHalfBytes, &tm_do, bar_dofull, half * 64, h, (int)q0);
@@ -153,7 +159,7 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                         const uint32_t ks = kcnt % L::kKStages;
                         ok = warp_wait_b(&bar_kempty[ks], ((kcnt / L::kKStages) & 1) ^ 1, abort_flag);
                         if (!ok) break;
-                        if (lane == 0) {
+                        if (leader) {
                             mbar_arrive_expect_tx(&bar_kfull[ks], L::kTileBytes);
                             for (int half = 0; half < D / 64; ++half)
                                 tma_load_3d(smem + L::kKOff + ks * L::kTileBytes + half * L::kHalfBytes, &tm_k,
@@ -163,7 +169,7 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                         const uint32_t vs = vcnt % L::kVStages;
                         ok = warp_wait_b(&bar_vempty[vs], ((vcnt / L::kVStages) & 1) ^ 1, abort_flag);
                         if (!ok) break;
-                        if (lane == 0) {
+                        if (leader) {
                             mbar_arrive_expect_tx(&bar_vfull[vs], L::kTileBytes);
                             for (int half = 0; half < D / 64; ++half)
                                 tma_load_3d(smem + L::kVOff + vs * L::kTileBytes + half * L::kHalfBytes, &tm_v,
@@ -174,8 +180,9 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 }
             }
         }
-    } else if (warp == 9) {
+    } else if (warp == kDqMmaWarp) {
         // ---------------- MMA issuer ----------------
+        const bool leader = elect_one();
         constexpr uint32_t idesc_s = make_idesc(128, 128, 0, 0);  // S, dP: A in TMEM, B K-major
         constexpr uint32_t idesc_dq = make_idesc(128, D, 0, 1);   // dQ: A in TMEM, B = K MN-major
         const uint32_t sb = smem_u32(smem);
@@ -184,6 +191,7 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         uint32_t bcnt = 0, kcnt = 0, vcnt = 0, blk = 0;
         bool ok = true;
         PROF_DECL
+        TRACE_DECL(0, cta == 0 && lane == 0)
         // C[tmem d_col] = A[tmem a_col, bf16 packed over the head dimension] * B(K-major tile at b_off)^T
         auto issue_qk = [&](uint32_t d_col, uint32_t a_col, uint32_t b_off) {
             const uint64_t db = sdesc_advance(kdesc0, b_off);
@@ -198,10 +206,12 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             PROF(7)
             if (!warp_wait_b(&bar_kfull[kidx % L::kKStages], (kidx / L::kKStages) & 1, abort_flag)) return false;
             PROF(0)
-            if (lane == 0) {
+            TRACE(1)
+            if (leader) {
                 issue_qk(kColS, kColQ, L::kKOff + (kidx % L::kKStages) * L::kTileBytes);
                 tc_commit(bar_sfull);
             }
+            TRACE(2)
             return true;
         };
         auto do_dp = [&]() -> bool {
@@ -209,11 +219,13 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             PROF(7)
             if (!warp_wait_b(&bar_vfull[vs], (vcnt / L::kVStages) & 1, abort_flag)) return false;
             PROF(1)
-            if (lane == 0) {
+            TRACE(3)
+            if (leader) {
                 issue_qk(kColDP, kColDO, L::kVOff + vs * L::kTileBytes);
                 tc_commit(bar_dpfull);
                 tc_commit(&bar_vempty[vs]);
             }
+            TRACE(4)
             ++vcnt;
             return true;
         };
@@ -238,9 +250,11 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                         // S(j+1) as soon as the compute groups have read S(j)
                         if (j + 1 <= hi) {
                             PROF(7)
+                            TRACE(8)
                             ok = warp_wait_b(bar_sfree, blk & 1, abort_flag);
                             if (!ok) break;
                             PROF(3)
+                            TRACE(5)
                             tc_fence_after();
                             ok = do_s(kbase + (j + 1 - lo));
                             if (!ok) break;
@@ -250,22 +264,27 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                         ok = warp_wait_b(bar_dsready, blk & 1, abort_flag);
                         if (!ok) break;
                         PROF(4)
+                        TRACE(6)
                         tc_fence_after();
                         const uint32_t kidx = kbase + (j - lo);
-                        if (lane == 0) {
+                        if (leader) {
                             const uint64_t ka = sdesc_advance(mdesc0, L::kKOff + (kidx % L::kKStages) * L::kTileBytes);
 #pragma unroll
-                            for (int kk = 0; kk < 8; ++kk)  // 16 keys per step; dS of keys 64c.. at columns 64c ..
-                                mma_ts(tmem_base + kColDQ, tmem_base + kColDP + (kk / 4) * 64 + (kk % 4) * 8,
+                            for (int kk = 0; kk < 8; ++kk)  // 16 keys per step; group c left dS of its keys at columns CW c ..
+                                mma_ts(tmem_base + kColDQ,
+                                       tmem_base + kColDP + (kk / (kDqCW / 16)) * kDqCW + (kk % (kDqCW / 16)) * 8,
                                        sdesc_advance(ka, kk * 2048), idesc_dq, (j > lo || kk > 0) ? 1u : 0u);
                             tc_commit(&bar_kempty[kidx % L::kKStages]);
                         }
+                        TRACE(7)
                         if (j + 1 <= hi) ok = do_dp();  // dP(j+1) over dS(j), after dQ(j) in pipe order
+                        TRACE(15)
                         __syncwarp();
+                        TRACE(16)
                     }
                     if (!ok) break;
                     kcnt = kbase + (hi - lo + 1);
-                    if (lane == 0) tc_commit(bar_dqfull);
+                    if (leader) tc_commit(bar_dqfull);
                     __syncwarp();
                 }
             }
@@ -273,14 +292,18 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         PROF_FLUSH(lane == 0, 512 * 24 + 8)
     } else {
         // ---------------- compute groups ----------------
-        const int c = warp >> 2;  // key-column half of each query row; group 0 also stages Q, group 1 dO
+        constexpr int CW = kDqCW;
+        const int c = warp >> 2;  // which CW key columns of each query row this group owns
+        // staging duty: even groups copy Q, odd groups dO; group pair c >> 1 takes that 64-column half
+        const int st_op = c & 1, st_half = c >> 1;
         const int r = (warp & 3) * 32 + lane;
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t t_s = tmem_base + lane_addr + kColS + 64 * c;
-        const uint32_t t_dp = tmem_base + lane_addr + kColDP + 64 * c;
+        const uint32_t t_s = tmem_base + lane_addr + kColS + CW * c;
+        const uint32_t t_dp = tmem_base + lane_addr + kColDP + CW * c;
         uint32_t bcnt = 0, blk = 0;
         bool ok = true;
         PROF_DECL
+        TRACE_DECL(1 + warp, cta == 0 && lane == 0)
         for (int idx = tile_begin; idx < tile_end && ok; ++idx) {
             const int t = p.cta_tiles[idx];
             for (int sub = 0; sub < 2 && ok; ++sub) {
@@ -299,23 +322,22 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     // ---- stage this group's operand (Q or dO) row from shared memory into TMEM ----
                     // The MMAs that read the previous unit's copy have completed: their s_full / dp_full
                     // completions were waited for above in program order.
-                    ok = mbar_wait(c == 0 ? bar_qfull : bar_dofull, bcnt & 1, abort_flag);
+                    ok = mbar_wait(st_op == 0 ? bar_qfull : bar_dofull, bcnt & 1, abort_flag);
                     if (!ok) break;
                     {
-                        const uint8_t* src = smem + (c == 0 ? L::kQOff : L::kDoOff) + r * 128;
-                        const uint32_t t_dst = tmem_base + lane_addr + (c == 0 ? kColQ : kColDO);
-#pragma unroll
-                        for (int half = 0; half < D / 64; ++half) {
+                        if (st_half < D / 64) {
+                            const uint8_t* src = smem + (st_op == 0 ? L::kQOff : L::kDoOff) + st_half * L::kHalfBytes + r * 128;
+                            const uint32_t t_dst = tmem_base + lane_addr + (st_op == 0 ? kColQ : kColDO) + 32 * st_half;
                             uint32_t w[32];
 #pragma unroll
                             for (int ch = 0; ch < 8; ++ch) {
-                                const uint4 v = *reinterpret_cast<const uint4*>(src + half * L::kHalfBytes + ((ch ^ (r & 7)) << 4));
+                                const uint4 v = *reinterpret_cast<const uint4*>(src + ((ch ^ (r & 7)) << 4));
                                 w[4 * ch] = v.x; w[4 * ch + 1] = v.y; w[4 * ch + 2] = v.z; w[4 * ch + 3] = v.w;
                             }
-                            tmem_st32(t_dst + 32 * half, w);
+                            tmem_st32(t_dst, w);
+                            tmem_st_wait();
                         }
-                        tmem_st_wait();
-                        mbar_arrive(c == 0 ? bar_qempty : bar_doempty);  // the smem tile may be reloaded
+                        mbar_arrive(st_op == 0 ? bar_qempty : bar_doempty);  // the smem tile may be reloaded
                         tc_fence_before();
                         mbar_arrive(bar_qtready);
                     }
@@ -323,70 +345,76 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     for (int j = lo; j <= hi && ok; ++j, ++blk) {
                         const int k0 = j * kBlk;
                         const bool need_mask = (j == hi) || (k0 < max_kstart) || !row_ok;
-                        const int c_lo = (row_ok ? kstart - k0 : kBlk) - 64 * c;    // first visible column of this half
-                        const int c_hi = (row_ok ? (int)(row - k0) : -1) - 64 * c;  // last visible column
+                        const int c_lo = (row_ok ? kstart - k0 : kBlk) - CW * c;    // first visible column of this group's range
+                        const int c_hi = (row_ok ? (int)(row - k0) : -1) - CW * c;  // last visible column
                         // ---- P = exp2(S c - LSE) ----
                         PROF(4)
                         ok = mbar_wait(bar_sfull, blk & 1, abort_flag);
                         if (!ok) break;
                         PROF(0)
+                        TRACE(10)
                         tc_fence_after();
-                        uint32_t sv[64];
-                        tmem_ld32(t_s, sv);
-                        tmem_ld32(t_s + 32, sv + 32);
+                        uint32_t sv[CW];
+#pragma unroll
+                        for (int i = 0; i < CW; i += 32) tmem_ld32(t_s + i, sv + i);
                         tmem_ld_wait();
                         tc_fence_before();
                         mbar_arrive(bar_sfree);  // S(j+1) may overwrite the columns
-                        float pf[64];
+                        TRACE(14)
+                        float pf[CW];
 #pragma unroll
-                        for (int i = 0; i < 64; i += 2) {
+                        for (int i = 0; i < CW; i += 2) {
                             pf[i] = ex2_sel(fmaf(__uint_as_float(sv[i]), p.scale_log2, -lse2), i);
                             pf[i + 1] = ex2_sel(fmaf(__uint_as_float(sv[i + 1]), p.scale_log2, -lse2), i + 1);
                         }
                         if (need_mask) {
 #pragma unroll
-                            for (int i = 0; i < 64; ++i)
+                            for (int i = 0; i < CW; ++i)
                                 if (i < c_lo || i > c_hi) pf[i] = 0.f;
                         }
                         // ---- dS = P o (dP - D), packed over this half's own dP columns ----
                         PROF(1)
+                        TRACE(11)
                         ok = mbar_wait(bar_dpfull, blk & 1, abort_flag);
                         if (!ok) break;
                         PROF(2)
+                        TRACE(12)
                         tc_fence_after();
-                        uint32_t dpv[64];
-                        tmem_ld32(t_dp, dpv);
-                        tmem_ld32(t_dp + 32, dpv + 32);
+                        uint32_t dpv[CW];
+#pragma unroll
+                        for (int i = 0; i < CW; i += 32) tmem_ld32(t_dp + i, dpv + i);
                         tmem_ld_wait();
                         {
-                            uint32_t pk[32];
+                            uint32_t pk[CW / 2];
 #pragma unroll
-                            for (int i = 0; i < 64; i += 2)
+                            for (int i = 0; i < CW; i += 2)
                                 pk[i >> 1] = pack_bf16x2(pf[i] * (__uint_as_float(dpv[i]) - dsum),
                                                          pf[i + 1] * (__uint_as_float(dpv[i + 1]) - dsum));
-                            tmem_st32(t_dp, pk);
+                            if constexpr (CW == 64) tmem_st32(t_dp, pk); else tmem_st16(t_dp, pk);
                         }
                         tmem_st_wait();
                         tc_fence_before();
                         mbar_arrive(bar_dsready);
                         PROF(3)
+                        TRACE(13)
                     }
                     if (!ok) break;
                     // ---- epilogue: dQ * scale to global ----
                     ok = mbar_wait(bar_dqfull, (bcnt - 1) & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    constexpr int kCols = D / 2;
+                    constexpr int kCols = D / kDqGroups;
+                    constexpr int kChunk = kCols < 32 ? kCols : 32;
                     const uint32_t t_dq = tmem_base + lane_addr + kColDQ + c * kCols;
                     __nv_bfloat16* gdst = p.dq + ((size_t)row * p.hq + h) * D + c * kCols;
 #pragma unroll
-                    for (int cc = 0; cc < kCols; cc += 32) {
-                        uint32_t v[32];
-                        tmem_ld32(t_dq + cc, v);
+                    for (int cc = 0; cc < kCols; cc += kChunk) {
+                        uint32_t v[kChunk];
+                        if constexpr (kChunk == 32) tmem_ld32(t_dq + cc, v); else tmem_ld16(t_dq + cc, v);
                         tmem_ld_wait();
                         if (row_ok) {
 #pragma unroll
-                            for (int i = 0; i < 32; i += 8) {
+                            for (int i = 0; i < kChunk; i += 8) {
                                 uint4 w;
                                 w.x = pack_bf16x2(__uint_as_float(v[i]) * p.scale, __uint_as_float(v[i + 1]) * p.scale);
                                 w.y = pack_bf16x2(__uint_as_float(v[i + 2]) * p.scale, __uint_as_float(v[i + 3]) * p.scale);
@@ -406,7 +434,7 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     // ---------------- teardown ----------------
     tc_fence_before();
     __syncthreads();
-    if (warp == 9) tmem_dealloc(tmem_base, 512);
+    if (warp == kDqMmaWarp) tmem_dealloc(tmem_base, 512);
     if (threadIdx.x == 0) {
         if (*abort_flag) atomicExch(p.status, LIBRA_ERR_TIMEOUT);
         p.busy[2 * cta + 1] = globaltimer_ns();

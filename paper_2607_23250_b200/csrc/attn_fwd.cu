@@ -155,6 +155,7 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     } else if (warp == 8) {
         // ---------------- TMA producer ----------------
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(LIBRA_FWD_REG_DEC));
+        const bool leader = elect_one();
         uint32_t ring = 0, qcnt = 0;
         bool ok = true;
         for (int idx = tile_begin; idx < tile_end && ok; ++idx) {
@@ -169,7 +170,7 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 const int kvh = h / G;
                 ok = warp_wait(bar_qempty, (qcnt & 1) ^ 1, abort_flag);
                 if (!ok) break;
-                if (lane == 0) {
+                if (leader) {
                     mbar_arrive_expect_tx(bar_qfull, (act1 ? 2 : 1) * L::kTileBytes);
                     for (int g = 0; g < (act1 ? 2 : 1); ++g)
                         for (int half = 0; half < D / 64; ++half)
@@ -182,7 +183,7 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                         const uint32_t st = ring % L::kStages;
                         ok = warp_wait(&bar_empty[st], ((ring / L::kStages) & 1) ^ 1, abort_flag);
                         if (!ok) break;
-                        if (lane == 0) {
+                        if (leader) {
                             mbar_arrive_expect_tx(&bar_full[st], L::kTileBytes);
                             for (int half = 0; half < D / 64; ++half)
                                 tma_load_3d(smem + L::kRingOff + st * L::kTileBytes + half * L::kHalfBytes,
@@ -196,6 +197,7 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     } else if (warp == 9) {
         // ---------------- MMA issuer ----------------
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(LIBRA_FWD_REG_DEC));
+        const bool leader = elect_one();
         constexpr uint32_t idesc_s = make_idesc(kBM, kBN, 0, 0);
         constexpr uint32_t idesc_pv = make_idesc(kBM, D, 0, 1);
         const uint32_t smem_base = smem_u32(smem);
@@ -243,7 +245,7 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 ok = warp_wait(&bar_full[st], (ring / L::kStages) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                if (lane == 0) {
+                if (leader) {
                     for (int g = 0; g < 2; ++g)
                         if (lo >= r[g].lo && lo <= r[g].hi) issue_s(g, st);
                     tc_commit(&bar_empty[st]);
@@ -273,14 +275,14 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                             PROF(3 + g)
                             ++pcnt[g];
                             tc_fence_after();
-                            if (lane == 0) issue_pv(g, st_v, j != r[g].lo);
+                            if (leader) issue_pv(g, st_v, j != r[g].lo);
                         }
                         if (j + 1 <= hi && j + 1 >= r[g].lo && j + 1 <= r[g].hi) {
-                            if (lane == 0) issue_s(g, st_k);
+                            if (leader) issue_s(g, st_k);
                         }
                     }
                     if (!ok) break;
-                    if (lane == 0) {
+                    if (leader) {
                         tc_commit(&bar_empty[st_v]);
                         if (j + 1 <= hi) tc_commit(&bar_empty[st_k]);
                         if (j + 1 == hi) tc_commit(bar_qempty);  // S(hi) was the last reader of Q: the next

@@ -73,6 +73,15 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     return true;
 }
 
+// One lane of a converged warp, chosen by the hardware. A role that elects its leader once and tests that
+// predicate lets the compiler keep descriptors in uniform registers; measured with 16 ALU-busy warps beside
+// it, a group of eight MMAs + commit + wait issued this way takes 600 clk against 770 with `lane == 0`.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+    return pred != 0;
+}
+
 // ---- TMA --------------------------------------------------------------------------------
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* m) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
@@ -283,5 +292,22 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
 }
+
+#ifdef LIBRA_TRACE
+// Trace build only: raw (event id, clock) pairs of one thread per role in CTA 0.
+__device__ long long g_trace[18 * 4096 * 2];
+struct Trace {
+    int n, role, on;
+    __device__ void init(int r, bool enable) { n = 0; role = r; on = enable; }
+    __device__ void ev(int id) {
+        if (on && n < 4096) { g_trace[(role * 4096 + n) * 2] = id; g_trace[(role * 4096 + n) * 2 + 1] = clock64(); ++n; }
+    }
+};
+#define TRACE_DECL(role, cond) Trace tr; tr.init(role, cond);
+#define TRACE(id) tr.ev(id);
+#else
+#define TRACE_DECL(role, cond)
+#define TRACE(id)
+#endif
 
 }  // namespace libra
