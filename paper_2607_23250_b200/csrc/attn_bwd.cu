@@ -33,10 +33,6 @@ __device__ __forceinline__ void bulk_load_1d(void* smem_dst, const void* gsrc, u
                  "l"(reinterpret_cast<uint64_t>(gsrc)), "r"(bytes), "r"(smem_u32(bar))
                  : "memory");
 }
-// Every lane polls the barrier itself (no elected lane + shuffle on the path between MMA groups).
-__device__ __forceinline__ bool warp_wait_b(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
-}
 
 #ifdef LIBRA_PROF
 // Profiling build only: per-CTA cycle sums of the phases of one thread per role.
@@ -172,168 +168,170 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 
     if (warp == 8) {
         // ---------------- TMA producer ----------------
-        const bool leader = elect_one();
-        uint32_t ucnt = 0, it_all = 0;
-        bool ok = true;
-        for (int idx = unit_begin; idx < unit_end && ok; ++idx) {
-            const int t = p.cta_tiles[idx];
-            const int kvh = t % p.hkv;
-            const int64_t k0 = (int64_t)(t / p.hkv) * kBlk;
-            const int i_lo = (int)(k0 / kBlk);
-            const int nblk = last_q_block(p.tok_end, p.T, k0) - i_lo + 1;
-            ok = warp_wait_b(bar_kvempty, (ucnt & 1) ^ 1, abort_flag);
-            if (!ok) break;
-            if (leader) {
-                mbar_arrive_expect_tx(bar_kvfull, 2 * L::kTileBytes);
-                for (int half = 0; half < D / 64; ++half) {
-                    tma_load_3d(smem + L::kKOff + half * L::kHalfBytes, &tm_k, bar_kvfull, half * 64, kvh, (int)k0);
-                    tma_load_3d(smem + L::kVOff + half * L::kHalfBytes, &tm_v, bar_kvfull, half * 64, kvh, (int)k0);
-                }
-            }
-            ++ucnt;
-            const int n_it = G * nblk;
-            for (int it = 0; it < n_it && ok; ++it, ++it_all) {
-                const int h = kvh * G + it / nblk;
-                const int qb = (i_lo + it % nblk) * kBlk;
-                const uint32_t st = it_all & 1, par = ((it_all >> 1) & 1) ^ 1;
-                ok = warp_wait_b(&bar_qempty[st], par, abort_flag);
+        if (elect_one()) {  // one elected thread runs the whole role
+            uint32_t ucnt = 0, it_all = 0;
+            bool ok = true;
+            for (int idx = unit_begin; idx < unit_end && ok; ++idx) {
+                const int t = p.cta_tiles[idx];
+                const int kvh = t % p.hkv;
+                const int64_t k0 = (int64_t)(t / p.hkv) * kBlk;
+                const int i_lo = (int)(k0 / kBlk);
+                const int nblk = last_q_block(p.tok_end, p.T, k0) - i_lo + 1;
+                ok = mbar_wait(bar_kvempty, (ucnt & 1) ^ 1, abort_flag);
                 if (!ok) break;
-                if (leader) {
-                    mbar_arrive_expect_tx(&bar_qfull[st], L::kTileBytes + 1024);
-                    for (int half = 0; half < D / 64; ++half)
-                        tma_load_3d(smem + L::kQOff + st * L::kTileBytes + half * L::kHalfBytes, &tm_q, &bar_qfull[st],
-                                    half * 64, h, qb);
-                    bulk_load_1d(smem + L::kStatOff + st * 1024, p.lse2 + (size_t)h * p.Tpad + qb, 512, &bar_qfull[st]);
-                    bulk_load_1d(smem + L::kStatOff + st * 1024 + 512, p.dvec + (size_t)h * p.Tpad + qb, 512,
-                                 &bar_qfull[st]);
+                {
+                    mbar_arrive_expect_tx(bar_kvfull, 2 * L::kTileBytes);
+                    for (int half = 0; half < D / 64; ++half) {
+                        tma_load_3d(smem + L::kKOff + half * L::kHalfBytes, &tm_k, bar_kvfull, half * 64, kvh, (int)k0);
+                        tma_load_3d(smem + L::kVOff + half * L::kHalfBytes, &tm_v, bar_kvfull, half * 64, kvh, (int)k0);
+                    }
                 }
-                ok = warp_wait_b(&bar_doempty[st], par, abort_flag);
-                if (!ok) break;
-                if (leader) {
-                    mbar_arrive_expect_tx(&bar_dofull[st], L::kTileBytes);
-                    for (int half = 0; half < D / 64; ++half)
-                        tma_load_3d(smem + L::kDoOff + st * L::kTileBytes + half * L::kHalfBytes, &tm_do,
-                                    &bar_dofull[st], half * 64, h, qb);
+                ++ucnt;
+                const int n_it = G * nblk;
+                for (int it = 0; it < n_it && ok; ++it, ++it_all) {
+                    const int h = kvh * G + it / nblk;
+                    const int qb = (i_lo + it % nblk) * kBlk;
+                    const uint32_t st = it_all & 1, par = ((it_all >> 1) & 1) ^ 1;
+                    ok = mbar_wait(&bar_qempty[st], par, abort_flag);
+                    if (!ok) break;
+                    {
+                        mbar_arrive_expect_tx(&bar_qfull[st], L::kTileBytes + 1024);
+                        for (int half = 0; half < D / 64; ++half)
+                            tma_load_3d(smem + L::kQOff + st * L::kTileBytes + half * L::kHalfBytes, &tm_q, &bar_qfull[st],
+                                        half * 64, h, qb);
+                        bulk_load_1d(smem + L::kStatOff + st * 1024, p.lse2 + (size_t)h * p.Tpad + qb, 512, &bar_qfull[st]);
+                        bulk_load_1d(smem + L::kStatOff + st * 1024 + 512, p.dvec + (size_t)h * p.Tpad + qb, 512,
+                                     &bar_qfull[st]);
+                    }
+                    ok = mbar_wait(&bar_doempty[st], par, abort_flag);
+                    if (!ok) break;
+                    {
+                        mbar_arrive_expect_tx(&bar_dofull[st], L::kTileBytes);
+                        for (int half = 0; half < D / 64; ++half)
+                            tma_load_3d(smem + L::kDoOff + st * L::kTileBytes + half * L::kHalfBytes, &tm_do,
+                                        &bar_dofull[st], half * 64, h, qb);
+                    }
                 }
             }
         }
+        __syncwarp();
     } else if (warp == 9) {
         // ---------------- MMA issuer ----------------
-        const bool leader = elect_one();
-        constexpr uint32_t idesc_s = make_idesc(128, 128, 0, 0);  // S^T, dP^T: both operands K-major
-        constexpr uint32_t idesc_acc = make_idesc(128, D, 0, 1);  // dV, dK: A from TMEM, B MN-major
-        const uint32_t sb = smem_u32(smem);
-        uint32_t ucnt = 0, it_all = 0;
-        bool ok = true;
-        PROF_DECL
-        // Base descriptors are built once; every MMA only adds a constant to them.
-        const uint64_t kdesc0 = make_sdesc(sb, 16, 1024);             // K-major view of a tile at offset 0
-        const uint64_t mdesc0 = make_sdesc(sb, L::kHalfBytes, 1024);  // MN-major view
-        // C[tmem] = A(K-major tile) * B(K-major tile)^T over the head dimension; offsets from smem base
-        auto issue_kmajor = [&](uint32_t d_col, uint32_t a_off, uint32_t b_off) {
-            const uint64_t da = sdesc_advance(kdesc0, a_off), db = sdesc_advance(kdesc0, b_off);
-#pragma unroll
-            for (int kk = 0; kk < D / 16; ++kk) {
-                const uint32_t off = (kk / 4) * L::kHalfBytes + (kk % 4) * 32;
-                mma_ss(tmem_base + d_col, sdesc_advance(da, off), sdesc_advance(db, off), idesc_s, kk > 0);
-            }
-        };
-        // C[tmem] (+)= A(TMEM, bf16 packed: queries 64c.. at columns a_col + 64c ..) * B(MN-major tile)
-        auto issue_acc = [&](uint32_t d_col, uint32_t a_col, uint32_t b_off, bool accumulate) {
-            const uint64_t db = sdesc_advance(mdesc0, b_off);
-#pragma unroll
-            for (int kk = 0; kk < 8; ++kk)  // 16 queries per step
-                mma_ts(tmem_base + d_col, tmem_base + a_col + (kk / 4) * 64 + (kk % 4) * 8, sdesc_advance(db, kk * 2048),
-                       idesc_acc, (accumulate || kk > 0) ? 1u : 0u);
-        };
-        for (int idx = unit_begin; idx < unit_end && ok; ++idx) {
-            const int t = p.cta_tiles[idx];
-            const int64_t k0 = (int64_t)(t / p.hkv) * kBlk;
-            const int i_lo = (int)(k0 / kBlk);
-            const int nblk = last_q_block(p.tok_end, p.T, k0) - i_lo + 1;
-            const int n_it = G * nblk;
-            ok = warp_wait_b(bar_kvfull, ucnt & 1, abort_flag);
-            if (!ok) break;
-            // S(0), dP(0)
-            ok = warp_wait_b(&bar_qfull[it_all & 1], (it_all >> 1) & 1, abort_flag);
-            if (!ok) break;
-            tc_fence_after();
-            if (leader) {
-                issue_kmajor(kColS, L::kKOff, L::kQOff + (it_all & 1) * L::kTileBytes);
-                tc_commit(bar_sfull);
-            }
-            ok = warp_wait_b(&bar_dofull[it_all & 1], (it_all >> 1) & 1, abort_flag);
-            if (!ok) break;
-            if (leader) {
-                issue_kmajor(kColDP, L::kVOff, L::kDoOff + (it_all & 1) * L::kTileBytes);
-                tc_commit(bar_dpfull);
-            }
-            for (int it = 0; it < n_it && ok; ++it, ++it_all) {
-                const uint32_t st = it_all & 1;
-                const uint32_t nx = it_all + 1;
-                const bool more = it + 1 < n_it;
-                // dV(it) += P^T dO
-                PROF(7)
-#ifndef LIBRA_DBG_FREE_MMA
-                ok = warp_wait_b(bar_pready, it_all & 1, abort_flag);
+        if (elect_one()) {  // one elected thread runs the whole role
+            constexpr uint32_t idesc_s = make_idesc(128, 128, 0, 0);  // S^T, dP^T: both operands K-major
+            constexpr uint32_t idesc_acc = make_idesc(128, D, 0, 1);  // dV, dK: A from TMEM, B MN-major
+            const uint32_t sb = smem_u32(smem);
+            uint32_t ucnt = 0, it_all = 0;
+            bool ok = true;
+            PROF_DECL
+            // Base descriptors are built once; every MMA only adds a constant to them.
+            const uint64_t kdesc0 = make_sdesc(sb, 16, 1024);             // K-major view of a tile at offset 0
+            const uint64_t mdesc0 = make_sdesc(sb, L::kHalfBytes, 1024);  // MN-major view
+            // C[tmem] = A(K-major tile) * B(K-major tile)^T over the head dimension; offsets from smem base
+            auto issue_kmajor = [&](uint32_t d_col, uint32_t a_off, uint32_t b_off) {
+                const uint64_t da = sdesc_advance(kdesc0, a_off), db = sdesc_advance(kdesc0, b_off);
+    #pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = (kk / 4) * L::kHalfBytes + (kk % 4) * 32;
+                    mma_ss(tmem_base + d_col, sdesc_advance(da, off), sdesc_advance(db, off), idesc_s, kk > 0);
+                }
+            };
+            // C[tmem] (+)= A(TMEM, bf16 packed: queries 64c.. at columns a_col + 64c ..) * B(MN-major tile)
+            auto issue_acc = [&](uint32_t d_col, uint32_t a_col, uint32_t b_off, bool accumulate) {
+                const uint64_t db = sdesc_advance(mdesc0, b_off);
+    #pragma unroll
+                for (int kk = 0; kk < 8; ++kk)  // 16 queries per step
+                    mma_ts(tmem_base + d_col, tmem_base + a_col + (kk / 4) * 64 + (kk % 4) * 8, sdesc_advance(db, kk * 2048),
+                           idesc_acc, (accumulate || kk > 0) ? 1u : 0u);
+            };
+            for (int idx = unit_begin; idx < unit_end && ok; ++idx) {
+                const int t = p.cta_tiles[idx];
+                const int64_t k0 = (int64_t)(t / p.hkv) * kBlk;
+                const int i_lo = (int)(k0 / kBlk);
+                const int nblk = last_q_block(p.tok_end, p.T, k0) - i_lo + 1;
+                const int n_it = G * nblk;
+                ok = mbar_wait(bar_kvfull, ucnt & 1, abort_flag);
                 if (!ok) break;
-#endif
-                PROF(0)
-#ifndef LIBRA_DBG_FREE_MMA
-                if (it == 0 && ucnt > 0) {  // previous unit's dK/dV must have been read out
-                    ok = warp_wait_b(bar_dkvempty, (ucnt - 1) & 1, abort_flag);
-                    if (!ok) break;
-                }
-#endif
+                // S(0), dP(0)
+                ok = mbar_wait(&bar_qfull[it_all & 1], (it_all >> 1) & 1, abort_flag);
+                if (!ok) break;
                 tc_fence_after();
-                if (leader) {
-                    issue_acc(kColDV, kColS, L::kDoOff + st * L::kTileBytes, it > 0);
-                    tc_commit(&bar_doempty[st]);
+                {
+                    issue_kmajor(kColS, L::kKOff, L::kQOff + (it_all & 1) * L::kTileBytes);
+                    tc_commit(bar_sfull);
                 }
-                // S(it+1)
-                if (more) {
+                ok = mbar_wait(&bar_dofull[it_all & 1], (it_all >> 1) & 1, abort_flag);
+                if (!ok) break;
+                {
+                    issue_kmajor(kColDP, L::kVOff, L::kDoOff + (it_all & 1) * L::kTileBytes);
+                    tc_commit(bar_dpfull);
+                }
+                for (int it = 0; it < n_it && ok; ++it, ++it_all) {
+                    const uint32_t st = it_all & 1;
+                    const uint32_t nx = it_all + 1;
+                    const bool more = it + 1 < n_it;
+                    // dV(it) += P^T dO
                     PROF(7)
-                    ok = warp_wait_b(&bar_qfull[nx & 1], (nx >> 1) & 1, abort_flag);
+    #ifndef LIBRA_DBG_FREE_MMA
+                    ok = mbar_wait(bar_pready, it_all & 1, abort_flag);
                     if (!ok) break;
-                    PROF(1)
-                    if (leader) {
-                        issue_kmajor(kColS, L::kKOff, L::kQOff + (nx & 1) * L::kTileBytes);
-                        tc_commit(bar_sfull);
+    #endif
+                    PROF(0)
+    #ifndef LIBRA_DBG_FREE_MMA
+                    if (it == 0 && ucnt > 0) {  // previous unit's dK/dV must have been read out
+                        ok = mbar_wait(bar_dkvempty, (ucnt - 1) & 1, abort_flag);
+                        if (!ok) break;
+                    }
+    #endif
+                    tc_fence_after();
+                    {
+                        issue_acc(kColDV, kColS, L::kDoOff + st * L::kTileBytes, it > 0);
+                        tc_commit(&bar_doempty[st]);
+                    }
+                    // S(it+1)
+                    if (more) {
+                        PROF(7)
+                        ok = mbar_wait(&bar_qfull[nx & 1], (nx >> 1) & 1, abort_flag);
+                        if (!ok) break;
+                        PROF(1)
+                        {
+                            issue_kmajor(kColS, L::kKOff, L::kQOff + (nx & 1) * L::kTileBytes);
+                            tc_commit(bar_sfull);
+                        }
+                    }
+                    // dK(it) += dS^T Q
+                    PROF(7)
+    #ifndef LIBRA_DBG_FREE_MMA
+                    ok = mbar_wait(bar_dsready, it_all & 1, abort_flag);
+                    if (!ok) break;
+    #endif
+                    PROF(2)
+                    tc_fence_after();
+                    {
+                        issue_acc(kColDK, kColDP, L::kQOff + st * L::kTileBytes, it > 0);
+                        tc_commit(&bar_qempty[st]);
+                    }
+                    // dP(it+1)
+                    if (more) {
+                        PROF(7)
+                        ok = mbar_wait(&bar_dofull[nx & 1], (nx >> 1) & 1, abort_flag);
+                        if (!ok) break;
+                        PROF(3)
+                        {
+                            issue_kmajor(kColDP, L::kVOff, L::kDoOff + (nx & 1) * L::kTileBytes);
+                            tc_commit(bar_dpfull);
+                        }
                     }
                 }
-                // dK(it) += dS^T Q
-                PROF(7)
-#ifndef LIBRA_DBG_FREE_MMA
-                ok = warp_wait_b(bar_dsready, it_all & 1, abort_flag);
-                if (!ok) break;
-#endif
-                PROF(2)
-                tc_fence_after();
-                if (leader) {
-                    issue_acc(kColDK, kColDP, L::kQOff + st * L::kTileBytes, it > 0);
-                    tc_commit(&bar_qempty[st]);
+                if (ok) {
+                    tc_commit(bar_dkvfull);
+                    tc_commit(bar_kvempty);
                 }
-                // dP(it+1)
-                if (more) {
-                    PROF(7)
-                    ok = warp_wait_b(&bar_dofull[nx & 1], (nx >> 1) & 1, abort_flag);
-                    if (!ok) break;
-                    PROF(3)
-                    if (leader) {
-                        issue_kmajor(kColDP, L::kVOff, L::kDoOff + (nx & 1) * L::kTileBytes);
-                        tc_commit(bar_dpfull);
-                    }
-                }
-                __syncwarp();
+                ++ucnt;
             }
-            if (ok && leader) {
-                tc_commit(bar_dkvfull);
-                tc_commit(bar_kvempty);
-            }
-            __syncwarp();
-            ++ucnt;
+            PROF_FLUSH(true, 8)
         }
-        PROF_FLUSH(lane == 0, 8)
+        __syncwarp();
     } else {
         // ---------------- compute groups ----------------
         const int c = warp >> 2;  // query-column half of each key row

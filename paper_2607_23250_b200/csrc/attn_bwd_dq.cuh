@@ -128,168 +128,170 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     // A sub-block past the end of the pool is skipped by every role.
     if (warp == kDqTmaWarp) {
         // ---------------- TMA producer ----------------
-        const bool leader = elect_one();
-        uint32_t bcnt = 0, kcnt = 0, vcnt = 0;
-        bool ok = true;
-        for (int idx = tile_begin; idx < tile_end && ok; ++idx) {
-            const int t = p.cta_tiles[idx];
-            for (int sub = 0; sub < 2 && ok; ++sub) {
-                const int64_t q0 = (int64_t)(t / p.H) * (2 * kBlk) + sub * kBlk;
-                if (q0 >= p.T) continue;
-                const int lo = p.tok_start[q0] / kBlk, hi = (int)(q0 / kBlk);
-                for (int hh = 0; hh < heads_per_shard && ok; ++hh) {
-                    const int h = (t % p.H) * heads_per_shard + hh;
-                    const int kvh = h / G;
-                    ok = warp_wait_b(bar_qempty, (bcnt & 1) ^ 1, abort_flag);
-                    if (!ok) break;
-                    if (leader) {
-                        mbar_arrive_expect_tx(bar_qfull, L::kTileBytes);
-                        for (int half = 0; half < D / 64; ++half)
-                            tma_load_3d(smem + L::kQOff + half * L::kHalfBytes, &tm_q, bar_qfull, half * 64, h, (int)q0);
-                    }
-                    ok = warp_wait_b(bar_doempty, (bcnt & 1) ^ 1, abort_flag);
-                    if (!ok) break;
-                    if (leader) {
-                        mbar_arrive_expect_tx(bar_dofull, L::kTileBytes);
-                        for (int half = 0; half < D / 64; ++half)
-                            tma_load_3d(smem + L::kDoOff + half * L::kHalfBytes, &tm_do, bar_dofull, half * 64, h, (int)q0);
-                    }
-                    ++bcnt;
-                    for (int j = lo; j <= hi && ok; ++j) {
-                        const uint32_t ks = kcnt % L::kKStages;
-                        ok = warp_wait_b(&bar_kempty[ks], ((kcnt / L::kKStages) & 1) ^ 1, abort_flag);
+        if (elect_one()) {  // one elected thread runs the whole role
+            uint32_t bcnt = 0, kcnt = 0, vcnt = 0;
+            bool ok = true;
+            for (int idx = tile_begin; idx < tile_end && ok; ++idx) {
+                const int t = p.cta_tiles[idx];
+                for (int sub = 0; sub < 2 && ok; ++sub) {
+                    const int64_t q0 = (int64_t)(t / p.H) * (2 * kBlk) + sub * kBlk;
+                    if (q0 >= p.T) continue;
+                    const int lo = p.tok_start[q0] / kBlk, hi = (int)(q0 / kBlk);
+                    for (int hh = 0; hh < heads_per_shard && ok; ++hh) {
+                        const int h = (t % p.H) * heads_per_shard + hh;
+                        const int kvh = h / G;
+                        ok = mbar_wait(bar_qempty, (bcnt & 1) ^ 1, abort_flag);
                         if (!ok) break;
-                        if (leader) {
-                            mbar_arrive_expect_tx(&bar_kfull[ks], L::kTileBytes);
+                        {
+                            mbar_arrive_expect_tx(bar_qfull, L::kTileBytes);
                             for (int half = 0; half < D / 64; ++half)
-                                tma_load_3d(smem + L::kKOff + ks * L::kTileBytes + half * L::kHalfBytes, &tm_k,
-                                            &bar_kfull[ks], half * 64, kvh, j * kBlk);
+                                tma_load_3d(smem + L::kQOff + half * L::kHalfBytes, &tm_q, bar_qfull, half * 64, h, (int)q0);
                         }
-                        ++kcnt;
-                        const uint32_t vs = vcnt % L::kVStages;
-                        ok = warp_wait_b(&bar_vempty[vs], ((vcnt / L::kVStages) & 1) ^ 1, abort_flag);
+                        ok = mbar_wait(bar_doempty, (bcnt & 1) ^ 1, abort_flag);
                         if (!ok) break;
-                        if (leader) {
-                            mbar_arrive_expect_tx(&bar_vfull[vs], L::kTileBytes);
+                        {
+                            mbar_arrive_expect_tx(bar_dofull, L::kTileBytes);
                             for (int half = 0; half < D / 64; ++half)
-                                tma_load_3d(smem + L::kVOff + vs * L::kTileBytes + half * L::kHalfBytes, &tm_v,
-                                            &bar_vfull[vs], half * 64, kvh, j * kBlk);
+                                tma_load_3d(smem + L::kDoOff + half * L::kHalfBytes, &tm_do, bar_dofull, half * 64, h, (int)q0);
                         }
-                        ++vcnt;
+                        ++bcnt;
+                        for (int j = lo; j <= hi && ok; ++j) {
+                            const uint32_t ks = kcnt % L::kKStages;
+                            ok = mbar_wait(&bar_kempty[ks], ((kcnt / L::kKStages) & 1) ^ 1, abort_flag);
+                            if (!ok) break;
+                            {
+                                mbar_arrive_expect_tx(&bar_kfull[ks], L::kTileBytes);
+                                for (int half = 0; half < D / 64; ++half)
+                                    tma_load_3d(smem + L::kKOff + ks * L::kTileBytes + half * L::kHalfBytes, &tm_k,
+                                                &bar_kfull[ks], half * 64, kvh, j * kBlk);
+                            }
+                            ++kcnt;
+                            const uint32_t vs = vcnt % L::kVStages;
+                            ok = mbar_wait(&bar_vempty[vs], ((vcnt / L::kVStages) & 1) ^ 1, abort_flag);
+                            if (!ok) break;
+                            {
+                                mbar_arrive_expect_tx(&bar_vfull[vs], L::kTileBytes);
+                                for (int half = 0; half < D / 64; ++half)
+                                    tma_load_3d(smem + L::kVOff + vs * L::kTileBytes + half * L::kHalfBytes, &tm_v,
+                                                &bar_vfull[vs], half * 64, kvh, j * kBlk);
+                            }
+                            ++vcnt;
+                        }
                     }
                 }
             }
         }
+        __syncwarp();
     } else if (warp == kDqMmaWarp) {
         // ---------------- MMA issuer ----------------
-        const bool leader = elect_one();
-        constexpr uint32_t idesc_s = make_idesc(128, 128, 0, 0);  // S, dP: A in TMEM, B K-major
-        constexpr uint32_t idesc_dq = make_idesc(128, D, 0, 1);   // dQ: A in TMEM, B = K MN-major
-        const uint32_t sb = smem_u32(smem);
-        const uint64_t kdesc0 = make_sdesc(sb, 16, 1024);             // K-major view of a tile at offset 0
-        const uint64_t mdesc0 = make_sdesc(sb, L::kHalfBytes, 1024);  // MN-major view
-        uint32_t bcnt = 0, kcnt = 0, vcnt = 0, blk = 0;
-        bool ok = true;
-        PROF_DECL
-        TRACE_DECL(0, cta == 0 && lane == 0)
-        // C[tmem d_col] = A[tmem a_col, bf16 packed over the head dimension] * B(K-major tile at b_off)^T
-        auto issue_qk = [&](uint32_t d_col, uint32_t a_col, uint32_t b_off) {
-            const uint64_t db = sdesc_advance(kdesc0, b_off);
-#pragma unroll
-            for (int kk = 0; kk < D / 16; ++kk) {
-                const uint32_t off = (kk / 4) * L::kHalfBytes + (kk % 4) * 32;
-                mma_ts(tmem_base + d_col, tmem_base + a_col + kk * 8, sdesc_advance(db, off), idesc_s, kk > 0);
-            }
-        };
-        // S(j) from K ring entry kidx
-        auto do_s = [&](uint32_t kidx) -> bool {
-            PROF(7)
-            if (!warp_wait_b(&bar_kfull[kidx % L::kKStages], (kidx / L::kKStages) & 1, abort_flag)) return false;
-            PROF(0)
-            TRACE(1)
-            if (leader) {
-                issue_qk(kColS, kColQ, L::kKOff + (kidx % L::kKStages) * L::kTileBytes);
-                tc_commit(bar_sfull);
-            }
-            TRACE(2)
-            return true;
-        };
-        auto do_dp = [&]() -> bool {
-            const uint32_t vs = vcnt % L::kVStages;
-            PROF(7)
-            if (!warp_wait_b(&bar_vfull[vs], (vcnt / L::kVStages) & 1, abort_flag)) return false;
-            PROF(1)
-            TRACE(3)
-            if (leader) {
-                issue_qk(kColDP, kColDO, L::kVOff + vs * L::kTileBytes);
-                tc_commit(bar_dpfull);
-                tc_commit(&bar_vempty[vs]);
-            }
-            TRACE(4)
-            ++vcnt;
-            return true;
-        };
-        for (int idx = tile_begin; idx < tile_end && ok; ++idx) {
-            const int t = p.cta_tiles[idx];
-            for (int sub = 0; sub < 2 && ok; ++sub) {
-                const int64_t q0 = (int64_t)(t / p.H) * (2 * kBlk) + sub * kBlk;
-                if (q0 >= p.T) continue;
-                const int lo = p.tok_start[q0] / kBlk, hi = (int)(q0 / kBlk);
-                for (int hh = 0; hh < heads_per_shard && ok; ++hh) {
-                    PROF(7)
-                    ok = warp_wait_b(bar_qtready, bcnt & 1, abort_flag);  // Q and dO are in TMEM
-                    if (!ok) break;
-                    PROF(2)
-                    ++bcnt;
-                    tc_fence_after();
-                    const uint32_t kbase = kcnt;  // ring index of K_lo
-                    ok = do_s(kbase);             // S(lo)
-                    if (ok) ok = do_dp();         // dP(lo)
-                    if (!ok) break;
-                    for (int j = lo; j <= hi && ok; ++j, ++blk) {
-                        // S(j+1) as soon as the compute groups have read S(j)
-                        if (j + 1 <= hi) {
-                            PROF(7)
-                            TRACE(8)
-                            ok = warp_wait_b(bar_sfree, blk & 1, abort_flag);
-                            if (!ok) break;
-                            PROF(3)
-                            TRACE(5)
-                            tc_fence_after();
-                            ok = do_s(kbase + (j + 1 - lo));
-                            if (!ok) break;
-                        }
-                        // dQ += dS(j) K_j
+        if (elect_one()) {  // one elected thread runs the whole role
+            constexpr uint32_t idesc_s = make_idesc(128, 128, 0, 0);  // S, dP: A in TMEM, B K-major
+            constexpr uint32_t idesc_dq = make_idesc(128, D, 0, 1);   // dQ: A in TMEM, B = K MN-major
+            const uint32_t sb = smem_u32(smem);
+            const uint64_t kdesc0 = make_sdesc(sb, 16, 1024);             // K-major view of a tile at offset 0
+            const uint64_t mdesc0 = make_sdesc(sb, L::kHalfBytes, 1024);  // MN-major view
+            uint32_t bcnt = 0, kcnt = 0, vcnt = 0, blk = 0;
+            bool ok = true;
+            PROF_DECL
+            TRACE_DECL(0, cta == 0)
+            // C[tmem d_col] = A[tmem a_col, bf16 packed over the head dimension] * B(K-major tile at b_off)^T
+            auto issue_qk = [&](uint32_t d_col, uint32_t a_col, uint32_t b_off) {
+                const uint64_t db = sdesc_advance(kdesc0, b_off);
+    #pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = (kk / 4) * L::kHalfBytes + (kk % 4) * 32;
+                    mma_ts(tmem_base + d_col, tmem_base + a_col + kk * 8, sdesc_advance(db, off), idesc_s, kk > 0);
+                }
+            };
+            // S(j) from K ring entry kidx
+            auto do_s = [&](uint32_t kidx) -> bool {
+                PROF(7)
+                if (!mbar_wait(&bar_kfull[kidx % L::kKStages], (kidx / L::kKStages) & 1, abort_flag)) return false;
+                PROF(0)
+                TRACE(1)
+                {
+                    issue_qk(kColS, kColQ, L::kKOff + (kidx % L::kKStages) * L::kTileBytes);
+                    tc_commit(bar_sfull);
+                }
+                TRACE(2)
+                return true;
+            };
+            auto do_dp = [&]() -> bool {
+                const uint32_t vs = vcnt % L::kVStages;
+                PROF(7)
+                if (!mbar_wait(&bar_vfull[vs], (vcnt / L::kVStages) & 1, abort_flag)) return false;
+                PROF(1)
+                TRACE(3)
+                {
+                    issue_qk(kColDP, kColDO, L::kVOff + vs * L::kTileBytes);
+                    tc_commit(bar_dpfull);
+                    tc_commit(&bar_vempty[vs]);
+                }
+                TRACE(4)
+                ++vcnt;
+                return true;
+            };
+            for (int idx = tile_begin; idx < tile_end && ok; ++idx) {
+                const int t = p.cta_tiles[idx];
+                for (int sub = 0; sub < 2 && ok; ++sub) {
+                    const int64_t q0 = (int64_t)(t / p.H) * (2 * kBlk) + sub * kBlk;
+                    if (q0 >= p.T) continue;
+                    const int lo = p.tok_start[q0] / kBlk, hi = (int)(q0 / kBlk);
+                    for (int hh = 0; hh < heads_per_shard && ok; ++hh) {
                         PROF(7)
-                        ok = warp_wait_b(bar_dsready, blk & 1, abort_flag);
+                        ok = mbar_wait(bar_qtready, bcnt & 1, abort_flag);  // Q and dO are in TMEM
                         if (!ok) break;
-                        PROF(4)
-                        TRACE(6)
+                        PROF(2)
+                        ++bcnt;
                         tc_fence_after();
-                        const uint32_t kidx = kbase + (j - lo);
-                        if (leader) {
-                            const uint64_t ka = sdesc_advance(mdesc0, L::kKOff + (kidx % L::kKStages) * L::kTileBytes);
-#pragma unroll
-                            for (int kk = 0; kk < 8; ++kk)  // 16 keys per step; group c left dS of its keys at columns CW c ..
-                                mma_ts(tmem_base + kColDQ,
-                                       tmem_base + kColDP + (kk / (kDqCW / 16)) * kDqCW + (kk % (kDqCW / 16)) * 8,
-                                       sdesc_advance(ka, kk * 2048), idesc_dq, (j > lo || kk > 0) ? 1u : 0u);
-                            tc_commit(&bar_kempty[kidx % L::kKStages]);
+                        const uint32_t kbase = kcnt;  // ring index of K_lo
+                        ok = do_s(kbase);             // S(lo)
+                        if (ok) ok = do_dp();         // dP(lo)
+                        if (!ok) break;
+                        for (int j = lo; j <= hi && ok; ++j, ++blk) {
+                            // S(j+1) as soon as the compute groups have read S(j)
+                            if (j + 1 <= hi) {
+                                PROF(7)
+                                TRACE(8)
+                                ok = mbar_wait(bar_sfree, blk & 1, abort_flag);
+                                if (!ok) break;
+                                PROF(3)
+                                TRACE(5)
+                                tc_fence_after();
+                                ok = do_s(kbase + (j + 1 - lo));
+                                if (!ok) break;
+                            }
+                            // dQ += dS(j) K_j
+                            PROF(7)
+                            ok = mbar_wait(bar_dsready, blk & 1, abort_flag);
+                            if (!ok) break;
+                            PROF(4)
+                            TRACE(6)
+                            tc_fence_after();
+                            const uint32_t kidx = kbase + (j - lo);
+                            {
+                                const uint64_t ka = sdesc_advance(mdesc0, L::kKOff + (kidx % L::kKStages) * L::kTileBytes);
+    #pragma unroll
+                                for (int kk = 0; kk < 8; ++kk)  // 16 keys per step; group c left dS of its keys at columns CW c ..
+                                    mma_ts(tmem_base + kColDQ,
+                                           tmem_base + kColDP + (kk / (kDqCW / 16)) * kDqCW + (kk % (kDqCW / 16)) * 8,
+                                           sdesc_advance(ka, kk * 2048), idesc_dq, (j > lo || kk > 0) ? 1u : 0u);
+                                tc_commit(&bar_kempty[kidx % L::kKStages]);
+                            }
+                            TRACE(7)
+                            if (j + 1 <= hi) ok = do_dp();  // dP(j+1) over dS(j), after dQ(j) in pipe order
+                            TRACE(15)
+                            TRACE(16)
                         }
-                        TRACE(7)
-                        if (j + 1 <= hi) ok = do_dp();  // dP(j+1) over dS(j), after dQ(j) in pipe order
-                        TRACE(15)
-                        __syncwarp();
-                        TRACE(16)
+                        if (!ok) break;
+                        kcnt = kbase + (hi - lo + 1);
+                        tc_commit(bar_dqfull);
                     }
-                    if (!ok) break;
-                    kcnt = kbase + (hi - lo + 1);
-                    if (leader) tc_commit(bar_dqfull);
-                    __syncwarp();
                 }
             }
+            PROF_FLUSH(true, 512 * 24 + 8)
         }
-        PROF_FLUSH(lane == 0, 512 * 24 + 8)
+        __syncwarp();
     } else {
         // ---------------- compute groups ----------------
         constexpr int CW = kDqCW;

@@ -304,7 +304,10 @@ struct Trace {
     }
 };
 #define TRACE_DECL(role, cond) Trace tr; tr.init(role, cond);
-#define TRACE(id) tr.ev(id);
+#ifndef LIBRA_TRACE_MASK
+#define LIBRA_TRACE_MASK 0xffffffffu
+#endif
+#define TRACE(id) if ((LIBRA_TRACE_MASK >> (id)) & 1u) tr.ev(id);
 #else
 #define TRACE_DECL(role, cond)
 #define TRACE(id)
