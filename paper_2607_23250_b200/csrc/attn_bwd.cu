@@ -224,6 +224,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             uint32_t ucnt = 0, it_all = 0;
             bool ok = true;
             PROF_DECL
+            TRACE_DECL(17, cta == 0)
             // Base descriptors are built once; every MMA only adds a constant to them.
             const uint64_t kdesc0 = make_sdesc(sb, 16, 1024);             // K-major view of a tile at offset 0
             const uint64_t mdesc0 = make_sdesc(sb, L::kHalfBytes, 1024);  // MN-major view
@@ -267,6 +268,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     tc_commit(bar_dpfull);
                 }
                 for (int it = 0; it < n_it && ok; ++it, ++it_all) {
+                    TRACE(20)
                     const uint32_t st = it_all & 1;
                     const uint32_t nx = it_all + 1;
                     const bool more = it + 1 < n_it;

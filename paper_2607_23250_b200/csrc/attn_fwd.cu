@@ -205,6 +205,7 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         uint32_t pcnt[2] = {0, 0};
         bool ok = true;
         PROF_DECL
+        TRACE_DECL(0, cta == 0 && leader)
         // Base descriptors are built once; every MMA only adds a constant to them.
         const uint64_t desc_q = make_sdesc(smem_base + L::kQOff, 16, 1024);                  // K-major Q slot 0
         const uint64_t desc_k = make_sdesc(smem_base + L::kRingOff, 16, 1024);               // K-major ring stage 0
@@ -253,6 +254,7 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 }
                 ++ring;
                 for (int j = lo; j <= hi && ok; ++j) {
+                    TRACE(20)
                     const uint32_t st_v = ring % L::kStages;
                     PROF(7)
                     ok = warp_wait(&bar_full[st_v], (ring / L::kStages) & 1, abort_flag);
@@ -569,3 +571,9 @@ extern "C" int libra_attn_pool_fwd(const void* q_dev, const void* k_dev, const v
     if (mp->timing) { cudaEventRecord(mp->ev[0][1], s); mp->ev_valid[0] = 1; }
     return rc;
 }
+
+#ifdef LIBRA_TRACE
+extern "C" int libra_debug_trace_fwd(long long* host, int n) {
+    return cudaMemcpyFromSymbol(host, libra::g_trace, sizeof(long long) * n) == cudaSuccess ? 0 : -4;
+}
+#endif
