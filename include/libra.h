@@ -42,6 +42,20 @@ extern "C" {
 #define LIBRA_ERR_NO_DEVICE     (-8)  /* no CUDA device / not an sm_100 device                        */
 #define LIBRA_ERR_SCRATCH_TOO_SMALL (-9) /* problem needs more than the library's built-in scratch    */
 
+/* Tile weight used by the placement.
+ * PAIRS  : the paper's Eq. 6, the causal (query, key) pairs the tile covers.
+ * BLOCKS : a time proxy the paper does not have (it notes in Section 3.2 that a FLOPs-balanced
+ *          assignment need not be time-balanced): the kernels spend the same time on a
+ *          cost_block x cost_block block of the score matrix whether all of it or only a corner is
+ *          visible, so the weight counts blocks instead of pairs.  The token axis is cut into chunks
+ *          at multiples of cost_block; a query-major tile weighs, summed over the row chunks it
+ *          holds,  8 * (key chunks that hold a key some row of the chunk attends) + unit_cost_q;
+ *          a key-major tile, summed over its key chunks,
+ *          8 * (query chunks that hold a query attending some key of the chunk) + unit_cost_kv.
+ *          Ordering, placement and tie-breaks are those of Algorithm 2 in both models. */
+#define LIBRA_WEIGHT_PAIRS   0
+#define LIBRA_WEIGHT_BLOCKS  1
+
 #define LIBRA_DIR_Q   1   /* query-major tiles (forward)  */
 #define LIBRA_DIR_KV  2   /* key-major tiles   (backward) */
 
@@ -59,6 +73,11 @@ typedef struct {
     int     n_heads_kv;    /* key-major head shards; 0 = same as n_heads                           */
     int64_t total_tokens;  /* T if the caller knows it; 0 = read cu_seqlens[n] back (one 4-byte
                               synchronous copy on `stream`)                                         */
+    int     weight_model;  /* LIBRA_WEIGHT_PAIRS (0, Eq. 6) or LIBRA_WEIGHT_BLOCKS                  */
+    int     cost_block;    /* LIBRA_WEIGHT_BLOCKS: edge of the square blocks counted; 0 = 128      */
+    int     unit_cost_q;   /* LIBRA_WEIGHT_BLOCKS: added per row chunk of a query-major tile, in
+                              eighths of a block (>= 0)                                             */
+    int     unit_cost_kv;  /* same per key chunk of a key-major tile                                */
 } libra_plan_opts;
 
 typedef struct {
@@ -89,7 +108,10 @@ typedef struct {
  * plan and are reused by every forward and backward call on the same layout (the paper
  * builds one plan per pool and reuses it across layers and for the backward pass,
  * Sections 4.1 and 4.3.3).  cu_seqlens_dev is read during the call only.
- * Errors: INVALID_ARG (null, n_samples <= 0, n_heads <= 0, tile_q <= 0), OVERFLOW
+ * With opts->weight_model = LIBRA_WEIGHT_BLOCKS the weight is the block count described at
+ * LIBRA_WEIGHT_BLOCKS above; everything else is unchanged.
+ * Errors: INVALID_ARG (null, n_samples <= 0, n_heads <= 0, tile_q <= 0, a negative option,
+ * an unknown weight model), OVERFLOW
  * (NB * H >= 2^31), CUDA; a malformed cu_seqlens is detected on the device and reported
  * by libra_plan_status as BAD_SEQLENS.
  */

@@ -141,8 +141,10 @@ def attn_dkv_cols(q, k, v, out, lse, dout, cu, cols, kvheads, scale=None, prec="
     return dk, dv
 
 
-def plan(cu, n_heads, tile, n_workers, direction=0):
-    """SH-Tile plan -> dict(weight, order, cta_of_tile, cta_offsets, cta_tiles, loads)."""
+def plan(cu, n_heads, tile, n_workers, direction=0, weight_model=0, cost_block=128, unit_cost=0):
+    """SH-Tile plan -> dict(weight, order, cta_of_tile, cta_offsets, cta_tiles, loads).
+
+    weight_model 0: pair count (Eq. 6); 1: block count (cost_block, unit_cost), see oracle_plan_blocks."""
     cu = _arr(cu, np.int32)
     lib = _load()
     n = len(cu) - 1
@@ -153,9 +155,14 @@ def plan(cu, n_heads, tile, n_workers, direction=0):
     res = dict(weight=np.empty(nt, np.int64), order=np.empty(nt, np.int32),
                cta_of_tile=np.empty(nt, np.int32), cta_offsets=np.empty(n_workers + 1, np.int32),
                cta_tiles=np.empty(nt, np.int32), loads=np.empty(n_workers, np.int64))
-    _check(lib.oracle_plan(_p(cu), ctypes.c_int(n), ctypes.c_int(n_heads), ctypes.c_int(tile),
-                           ctypes.c_int(n_workers), ctypes.c_int(direction), _p(res["weight"]),
-                           _p(res["order"]), _p(res["cta_of_tile"]), _p(res["cta_offsets"]),
-                           _p(res["cta_tiles"]), _p(res["loads"])), "oracle_plan")
+    outs = (_p(res["weight"]), _p(res["order"]), _p(res["cta_of_tile"]), _p(res["cta_offsets"]),
+            _p(res["cta_tiles"]), _p(res["loads"]))
+    if weight_model == 0:
+        _check(lib.oracle_plan(_p(cu), ctypes.c_int(n), ctypes.c_int(n_heads), ctypes.c_int(tile),
+                               ctypes.c_int(n_workers), ctypes.c_int(direction), *outs), "oracle_plan")
+    else:
+        _check(lib.oracle_plan_blocks(_p(cu), ctypes.c_int(n), ctypes.c_int(n_heads), ctypes.c_int(tile),
+                                      ctypes.c_int(n_workers), ctypes.c_int(direction), ctypes.c_int(cost_block),
+                                      ctypes.c_int(unit_cost), *outs), "oracle_plan_blocks")
     res["n_blocks"] = int(nb)
     return res

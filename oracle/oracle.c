@@ -71,37 +71,9 @@ static int cmp_tiles(const void* a, const void* b) {
     return x->id < y->id ? -1 : (x->id > y->id ? 1 : 0);
 }
 
-int64_t oracle_plan_num_blocks(const int32_t* cu, int n, int tile) {
-    if (!cu || n <= 0 || tile <= 0) return -1;
-    const int64_t T = cu[n];
-    return (T + tile - 1) / tile;
-}
-
-int oracle_plan(const int32_t* cu, int n, int H, int tile, int W, int direction,
-                int64_t* weight /*[NB*H]*/, int32_t* order /*[NB*H]*/, int32_t* cta_of_tile /*[NB*H]*/,
-                int32_t* cta_offsets /*[W+1]*/, int32_t* cta_tiles /*[NB*H]*/, int64_t* loads /*[W]*/) {
-    if (!cu || n <= 0 || H <= 0 || tile <= 0 || W <= 0) return -1;
-    if (cu[0] != 0) return -1;
-    for (int j = 0; j < n; ++j) if (cu[j + 1] < cu[j]) return -1;
-    const int64_t T = cu[n];
-    const int64_t NB = (T + tile - 1) / tile;
-    const int64_t NT = NB * H;
-
-    /* steps 1-2 */
-    for (int64_t b = 0; b < NB; ++b) {
-        const int64_t q0 = b * tile, q1 = (b + 1) * tile < T ? (b + 1) * tile : T;
-        int64_t w = 0;
-        for (int j = 0; j < n; ++j) {
-            const int64_t s = cu[j], t = cu[j + 1], len = t - s;
-            const int64_t lo = q0 > s ? q0 : s, hi = q1 < t ? q1 : t;
-            for (int64_t g = lo; g < hi; ++g) {
-                const int64_t p = g - s;
-                w += direction == 0 ? (p + 1) : (len - p);
-            }
-        }
-        for (int h = 0; h < H; ++h) weight[b * H + h] = w;
-    }
-
+/* Steps 3-5, common to both weight models: order, place, list. */
+static int place_tiles(int64_t NT, int W, const int64_t* weight, int32_t* order, int32_t* cta_of_tile,
+                       int32_t* cta_offsets, int32_t* cta_tiles, int64_t* loads) {
     /* step 3 */
     tile_key* keys = (tile_key*)malloc(sizeof(tile_key) * (size_t)NT);
     if (!keys) return -2;
@@ -133,4 +105,89 @@ int oracle_plan(const int32_t* cu, int n, int H, int tile, int W, int direction,
     }
     free(fill);
     return 0;
+}
+
+int64_t oracle_plan_num_blocks(const int32_t* cu, int n, int tile) {
+    if (!cu || n <= 0 || tile <= 0) return -1;
+    const int64_t T = cu[n];
+    return (T + tile - 1) / tile;
+}
+
+int oracle_plan(const int32_t* cu, int n, int H, int tile, int W, int direction,
+                int64_t* weight /*[NB*H]*/, int32_t* order /*[NB*H]*/, int32_t* cta_of_tile /*[NB*H]*/,
+                int32_t* cta_offsets /*[W+1]*/, int32_t* cta_tiles /*[NB*H]*/, int64_t* loads /*[W]*/) {
+    if (!cu || n <= 0 || H <= 0 || tile <= 0 || W <= 0) return -1;
+    if (cu[0] != 0) return -1;
+    for (int j = 0; j < n; ++j) if (cu[j + 1] < cu[j]) return -1;
+    const int64_t T = cu[n];
+    const int64_t NB = (T + tile - 1) / tile;
+    const int64_t NT = NB * H;
+
+    /* steps 1-2 */
+    for (int64_t b = 0; b < NB; ++b) {
+        const int64_t q0 = b * tile, q1 = (b + 1) * tile < T ? (b + 1) * tile : T;
+        int64_t w = 0;
+        for (int j = 0; j < n; ++j) {
+            const int64_t s = cu[j], t = cu[j + 1], len = t - s;
+            const int64_t lo = q0 > s ? q0 : s, hi = q1 < t ? q1 : t;
+            for (int64_t g = lo; g < hi; ++g) {
+                const int64_t p = g - s;
+                w += direction == 0 ? (p + 1) : (len - p);
+            }
+        }
+        for (int h = 0; h < H; ++h) weight[b * H + h] = w;
+    }
+
+    return place_tiles(NT, W, weight, order, cta_of_tile, cta_offsets, cta_tiles, loads);
+}
+
+/* ------------------------------------------------------------------------------------
+ * Plan with the block-count weight (not in the paper; Section 3.2 only remarks that equal
+ * FLOPs need not mean equal time).  A kernel spends the same time on a g x g block of the
+ * score matrix whether one pair of it is visible or all, so this weight counts blocks.
+ *
+ * The token axis is cut into chunks at multiples of g.  A tile (block b of `tile` tokens,
+ * any head shard) is the union of the chunk pieces it intersects.  For each piece:
+ *   query-major: the piece holds query rows r0..r1.  The sample of r0 starts at s0.  Row r0
+ *     attends keys s0..r0, rows after it attend keys no earlier than s0 and no later than
+ *     r1, so the key chunks with a visible pair are floor(s0/g) .. floor(r1/g).
+ *   key-major: the piece holds keys c0..c1.  The sample of c1 ends at e1 (exclusive).  Key
+ *     c1 is attended by queries c1..e1-1, earlier keys of the piece by queries no earlier
+ *     than c0 and no later than e1-1, so the query chunks are floor(c0/g) .. floor((e1-1)/g).
+ * Weight of the tile = sum over its pieces of (8 * chunks + unit_cost).
+ * Steps 3-5 are those of oracle_plan.
+ * ------------------------------------------------------------------------------------ */
+int oracle_plan_blocks(const int32_t* cu, int n, int H, int tile, int W, int direction, int g, int unit_cost,
+                       int64_t* weight, int32_t* order, int32_t* cta_of_tile, int32_t* cta_offsets,
+                       int32_t* cta_tiles, int64_t* loads) {
+    if (!cu || n <= 0 || H <= 0 || tile <= 0 || W <= 0 || g <= 0 || unit_cost < 0) return -1;
+    if (cu[0] != 0) return -1;
+    for (int j = 0; j < n; ++j) if (cu[j + 1] < cu[j]) return -1;
+    const int64_t T = cu[n];
+    const int64_t NB = (T + tile - 1) / tile;
+    const int64_t NT = NB * H;
+    for (int64_t b = 0; b < NB; ++b) {
+        const int64_t t0 = b * tile, t1 = (b + 1) * tile < T ? (b + 1) * tile : T;
+        int64_t w = 0;
+        int64_t first = t0;
+        while (first < t1) {
+            int64_t end = (first / g + 1) * g;  /* the piece ends at the next multiple of g or at the tile end */
+            if (end > t1) end = t1;
+            const int64_t last = end - 1;
+            int64_t chunks;
+            if (direction == 0) {
+                int j = 0;
+                while (!(cu[j] <= first && first < cu[j + 1])) ++j;  /* sample of the first row */
+                chunks = last / g - cu[j] / g + 1;
+            } else {
+                int j = 0;
+                while (!(cu[j] <= last && last < cu[j + 1])) ++j;    /* sample of the last key */
+                chunks = (cu[j + 1] - 1) / g - first / g + 1;
+            }
+            w += 8 * chunks + unit_cost;
+            first = end;
+        }
+        for (int h = 0; h < H; ++h) weight[b * H + h] = w;
+    }
+    return place_tiles(NT, W, weight, order, cta_of_tile, cta_offsets, cta_tiles, loads);
 }

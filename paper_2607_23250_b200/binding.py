@@ -20,6 +20,7 @@ if not os.path.exists(_SO):
 _lib = ctypes.CDLL(_SO)
 
 LIBRA_DIR_Q, LIBRA_DIR_KV = 1, 2
+LIBRA_WEIGHT_PAIRS, LIBRA_WEIGHT_BLOCKS = 0, 1
 KERNEL_FWD, KERNEL_BWD_DKDV, KERNEL_BWD_DQ = 1, 2, 3
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_PLAN_MISMATCH, ERR_CUDA = -1, -2, -3, -4
 ERR_OVERFLOW, ERR_TIMEOUT, ERR_BAD_SEQLENS, ERR_NO_DEVICE = -5, -6, -7, -8
@@ -34,7 +35,8 @@ EXPORTS = ["libra_plan_tiles", "libra_plan_info", "libra_plan_status", "libra_pl
 
 class PlanOpts(ctypes.Structure):
     _fields_ = [("n_workers", ctypes.c_int), ("directions", ctypes.c_int), ("tile_kv", ctypes.c_int),
-                ("n_heads_kv", ctypes.c_int), ("total_tokens", ctypes.c_int64)]
+                ("n_heads_kv", ctypes.c_int), ("total_tokens", ctypes.c_int64), ("weight_model", ctypes.c_int),
+                ("cost_block", ctypes.c_int), ("unit_cost_q", ctypes.c_int), ("unit_cost_kv", ctypes.c_int)]
 
 
 class Dims(ctypes.Structure):
@@ -134,9 +136,11 @@ class Plan:
 
 def libra_plan_tiles(cu_seqlens: torch.Tensor, n_heads: int, tile_q: int, n_workers: int = 0,
                      directions: int = 0, tile_kv: int = 0, n_heads_kv: int = 0, total_tokens: int = 0,
-                     stream=None) -> Plan:
+                     stream=None, weight_model: int = 0, cost_block: int = 0, unit_cost_q: int = 0,
+                     unit_cost_kv: int = 0) -> Plan:
     assert cu_seqlens.is_cuda and cu_seqlens.dtype == torch.int32 and cu_seqlens.is_contiguous()
-    opts = PlanOpts(n_workers, directions, tile_kv, n_heads_kv, total_tokens)
+    opts = PlanOpts(n_workers, directions, tile_kv, n_heads_kv, total_tokens, weight_model, cost_block,
+                    unit_cost_q, unit_cost_kv)
     h = _vp()
     _check(_lib.libra_plan_tiles(_ptr(cu_seqlens), ctypes.c_int(cu_seqlens.numel() - 1), ctypes.c_int(n_heads),
                                  ctypes.c_int(tile_q), ctypes.byref(opts), _stream(stream), ctypes.byref(h)),

@@ -538,6 +538,7 @@ static int launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtens
     if (!configured) {
         if (set_smem(k_attn_bwd_dkdv<D>, DkvSmem<D>::kBytes) != LIBRA_OK) return LIBRA_ERR_CUDA;
         if (set_smem(k_attn_bwd_dq<D>, DqSmem<D>::kBytes) != LIBRA_OK) return LIBRA_ERR_CUDA;
+        if (!regs_pool_ok(k_attn_bwd_dq<D>, 128 * kDqGroups, kDqRegsCompute, 128, kDqRegsOther)) return LIBRA_ERR_UNSUPPORTED;
         configured = true;
     }
     if (mp->timing) cudaEventRecord(mp->ev[1][0], s);

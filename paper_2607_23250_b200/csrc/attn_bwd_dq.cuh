@@ -11,13 +11,22 @@
 // Queries sit in TMEM lanes, so LSE and D are per-thread scalars and the masks are the forward's.
 // Pipeline per key block j on the tensor pipe:  S(j+1) | dQ(j) dP(j+1); the exp phase of block
 // j+1 overlaps dQ(j) and dP(j+1), the dS phase overlaps S(j+2).
+// Units are chained the same way: once a thread has seen the last S and dP of a unit complete it copies
+// the next unit's Q / dO row over the old one, so S and dP of the next unit's first block are issued right
+// behind the last dQ of this one, and the dQ read-out overlaps them.
 #pragma once
 
 namespace libra {
 
+#ifndef LIBRA_DQ_PREFETCH
+#define LIBRA_DQ_PREFETCH 0
+#endif
 constexpr int kDqGroups = 4;                      // compute warpgroups: each owns 128 / kDqGroups key columns
 constexpr int kDqCW = 128 / kDqGroups;            // S / dP columns per compute thread
-constexpr int kDqThreads = (4 * kDqGroups + 2) * 32;
+// The producer / MMA warps sit in a warpgroup of their own (two of its warps idle) so that it can hand
+// registers to the compute groups with setmaxnreg.
+constexpr int kDqThreads = (4 * kDqGroups + 4) * 32;
+constexpr int kDqRegsCompute = 104, kDqRegsOther = 40;  // from 96 at launch: 4 x 128 x 8 asked, 128 x 56 released
 constexpr int kDqTmaWarp = 4 * kDqGroups, kDqMmaWarp = 4 * kDqGroups + 1;
 
 template <int D>
@@ -32,8 +41,8 @@ struct DqSmem {
     static constexpr int kVOff = kKOff + kKStages * kTileBytes;
     static constexpr int kBarOff = kVOff + kVStages * kTileBytes;
     // q_full, q_empty, do_full, do_empty, k_full[3], k_empty[3], v_full[2], v_empty[2], qt_ready,
-    // s_full, s_free, dp_full, ds_ready, dq_full
-    static constexpr int kNumBars = 20;
+    // s_full, s_free, dp_full, ds_ready, dq_full, dot_ready, dq_empty
+    static constexpr int kNumBars = 22;
     static constexpr int kMiscOff = kBarOff + kNumBars * 8;
     static constexpr int kBytes = kMiscOff + 16;
     static_assert(kBytes <= kSmemMax, "exceeds the shared memory of an sm_100 CTA");
@@ -51,6 +60,42 @@ struct DqParams {
     float scale, scale_log2;
     int* status;
     uint64_t* busy;
+};
+
+// Walks the units of one CTA in the order every role uses: tiles of the CTA's list x the two 128-row
+// sub-blocks of a tile x the heads of the shard.  A sub-block past the end of the pool is skipped.
+struct DqUnit {
+    int64_t q0;
+    int lo, hi, h;  // key blocks lo..hi, query head h
+    bool valid;
+};
+struct DqUnitIter {
+    const DqParams& p;
+    int idx, end, sub, hh, hps;
+    __device__ DqUnitIter(const DqParams& p_, int begin, int end_, int heads_per_shard)
+        : p(p_), idx(begin), end(end_), sub(0), hh(0), hps(heads_per_shard) {}
+    __device__ DqUnit next() {
+        DqUnit u;
+        u.valid = false;
+        while (idx < end) {
+            const int t = p.cta_tiles[idx];
+            const int64_t q0 = (int64_t)(t / p.H) * (2 * kBlk) + sub * kBlk;
+            const bool live = q0 < p.T;
+            if (live) {
+                u.q0 = q0;
+                u.lo = p.tok_start[q0] / kBlk;
+                u.hi = (int)(q0 / kBlk);
+                u.h = (t % p.H) * hps + hh;
+                u.valid = true;
+            }
+            if (!live || ++hh == hps) {
+                hh = 0;
+                if (++sub == 2) { sub = 0; ++idx; }
+            }
+            if (live) return u;
+        }
+        return u;
+    }
 };
 
 template <int D>
@@ -74,6 +119,8 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     uint64_t* bar_dpfull = bars + 17;
     uint64_t* bar_dsready = bars + 18;
     uint64_t* bar_dqfull = bars + 19;
+    uint64_t* bar_dotready = bars + 20;
+    uint64_t* bar_dqempty = bars + 21;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::kMiscOff);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kMiscOff + 4);
 
@@ -92,7 +139,9 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         mbar_init(bar_doempty, 64 * kDqGroups);  // the groups that stage dO
         for (int s = 0; s < L::kKStages; ++s) { mbar_init(&bar_kfull[s], 1); mbar_init(&bar_kempty[s], 1); }
         for (int s = 0; s < L::kVStages; ++s) { mbar_init(&bar_vfull[s], 1); mbar_init(&bar_vempty[s], 1); }
-        mbar_init(bar_qtready, 128 * kDqGroups);
+        mbar_init(bar_qtready, 64 * kDqGroups);   // the groups that stage Q
+        mbar_init(bar_dotready, 64 * kDqGroups);  // the groups that stage dO
+        mbar_init(bar_dqempty, 128 * kDqGroups);
         mbar_init(bar_sfull, 1);
         mbar_init(bar_sfree, 128 * kDqGroups);
         mbar_init(bar_dpfull, 1);
@@ -126,78 +175,97 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
 
     // All roles walk the same sequence of sub-blocks: (tile, sub-block of 128 rows, head of the shard).
     // A sub-block past the end of the pool is skipped by every role.
-    if (warp == kDqTmaWarp) {
+    if (warp > kDqMmaWarp) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kDqRegsOther));
+    } else if (warp == kDqTmaWarp) {
         // ---------------- TMA producer ----------------
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kDqRegsOther));
         if (elect_one()) {  // one elected thread runs the whole role
-            uint32_t bcnt = 0, kcnt = 0, vcnt = 0;
+            uint32_t ucnt = 0, kcnt = 0, vcnt = 0;
             bool ok = true;
-            for (int idx = tile_begin; idx < tile_end && ok; ++idx) {
-                const int t = p.cta_tiles[idx];
-                for (int sub = 0; sub < 2 && ok; ++sub) {
-                    const int64_t q0 = (int64_t)(t / p.H) * (2 * kBlk) + sub * kBlk;
-                    if (q0 >= p.T) continue;
-                    const int lo = p.tok_start[q0] / kBlk, hi = (int)(q0 / kBlk);
-                    for (int hh = 0; hh < heads_per_shard && ok; ++hh) {
-                        const int h = (t % p.H) * heads_per_shard + hh;
-                        const int kvh = h / G;
-                        ok = mbar_wait(bar_qempty, (bcnt & 1) ^ 1, abort_flag);
-                        if (!ok) break;
-                        {
-                            mbar_arrive_expect_tx(bar_qfull, L::kTileBytes);
-                            for (int half = 0; half < D / 64; ++half)
-                                tma_load_3d(smem + L::kQOff + half * L::kHalfBytes, &tm_q, bar_qfull, half * 64, h, (int)q0);
-                        }
-                        ok = mbar_wait(bar_doempty, (bcnt & 1) ^ 1, abort_flag);
-                        if (!ok) break;
-                        {
-                            mbar_arrive_expect_tx(bar_dofull, L::kTileBytes);
-                            for (int half = 0; half < D / 64; ++half)
-                                tma_load_3d(smem + L::kDoOff + half * L::kHalfBytes, &tm_do, bar_dofull, half * 64, h, (int)q0);
-                        }
-                        ++bcnt;
-                        for (int j = lo; j <= hi && ok; ++j) {
-                            const uint32_t ks = kcnt % L::kKStages;
-                            ok = mbar_wait(&bar_kempty[ks], ((kcnt / L::kKStages) & 1) ^ 1, abort_flag);
-                            if (!ok) break;
-                            {
-                                mbar_arrive_expect_tx(&bar_kfull[ks], L::kTileBytes);
-                                for (int half = 0; half < D / 64; ++half)
-                                    tma_load_3d(smem + L::kKOff + ks * L::kTileBytes + half * L::kHalfBytes, &tm_k,
-                                                &bar_kfull[ks], half * 64, kvh, j * kBlk);
+            // Tiles a unit will need are pulled into L2 this many key blocks ahead: the shared-memory rings
+            // hold one block of lead, which covers an L2 hit but not a first touch in DRAM.
+            constexpr int kAhead = LIBRA_DQ_PREFETCH;
+            auto prefetch_kv = [&](int kvh, int j) {
+                for (int half = 0; half < D / 64; ++half) {
+                    tma_prefetch_3d(&tm_k, half * 64, kvh, j * kBlk);
+                    tma_prefetch_3d(&tm_v, half * 64, kvh, j * kBlk);
+                }
+            };
+            DqUnitIter units(p, tile_begin, tile_end, heads_per_shard);
+            DqUnit u = units.next();
+            while (u.valid && ok) {
+                const DqUnit nx = units.next();
+                const int h = u.h, kvh = h / G, lo = u.lo, hi = u.hi;
+                ok = mbar_wait(bar_qempty, (ucnt & 1) ^ 1, abort_flag);
+                if (!ok) break;
+                {
+                    mbar_arrive_expect_tx(bar_qfull, L::kTileBytes);
+                    for (int half = 0; half < D / 64; ++half)
+                        tma_load_3d(smem + L::kQOff + half * L::kHalfBytes, &tm_q, bar_qfull, half * 64, h, (int)u.q0);
+                }
+                ok = mbar_wait(bar_doempty, (ucnt & 1) ^ 1, abort_flag);
+                if (!ok) break;
+                {
+                    mbar_arrive_expect_tx(bar_dofull, L::kTileBytes);
+                    for (int half = 0; half < D / 64; ++half)
+                        tma_load_3d(smem + L::kDoOff + half * L::kHalfBytes, &tm_do, bar_dofull, half * 64, h, (int)u.q0);
+                }
+                ++ucnt;
+                const int j_next = hi - kAhead > lo ? hi - kAhead : lo;  // where the next unit's first tiles are requested
+                for (int j = lo; j <= hi && ok; ++j) {
+                    if (kAhead > 0) {
+                        if (j + kAhead <= hi) prefetch_kv(kvh, j + kAhead);
+                        if (j == j_next && nx.valid) {
+                            for (int half = 0; half < D / 64; ++half) {
+                                tma_prefetch_3d(&tm_q, half * 64, nx.h, (int)nx.q0);
+                                tma_prefetch_3d(&tm_do, half * 64, nx.h, (int)nx.q0);
                             }
-                            ++kcnt;
-                            const uint32_t vs = vcnt % L::kVStages;
-                            ok = mbar_wait(&bar_vempty[vs], ((vcnt / L::kVStages) & 1) ^ 1, abort_flag);
-                            if (!ok) break;
-                            {
-                                mbar_arrive_expect_tx(&bar_vfull[vs], L::kTileBytes);
-                                for (int half = 0; half < D / 64; ++half)
-                                    tma_load_3d(smem + L::kVOff + vs * L::kTileBytes + half * L::kHalfBytes, &tm_v,
-                                                &bar_vfull[vs], half * 64, kvh, j * kBlk);
-                            }
-                            ++vcnt;
+                            for (int jj = nx.lo; jj <= nx.hi && jj < nx.lo + kAhead; ++jj) prefetch_kv(nx.h / G, jj);
                         }
                     }
+                    const uint32_t ks = kcnt % L::kKStages;
+                    ok = mbar_wait(&bar_kempty[ks], ((kcnt / L::kKStages) & 1) ^ 1, abort_flag);
+                    if (!ok) break;
+                    {
+                        mbar_arrive_expect_tx(&bar_kfull[ks], L::kTileBytes);
+                        for (int half = 0; half < D / 64; ++half)
+                            tma_load_3d(smem + L::kKOff + ks * L::kTileBytes + half * L::kHalfBytes, &tm_k,
+                                        &bar_kfull[ks], half * 64, kvh, j * kBlk);
+                    }
+                    ++kcnt;
+                    const uint32_t vs = vcnt % L::kVStages;
+                    ok = mbar_wait(&bar_vempty[vs], ((vcnt / L::kVStages) & 1) ^ 1, abort_flag);
+                    if (!ok) break;
+                    {
+                        mbar_arrive_expect_tx(&bar_vfull[vs], L::kTileBytes);
+                        for (int half = 0; half < D / 64; ++half)
+                            tma_load_3d(smem + L::kVOff + vs * L::kTileBytes + half * L::kHalfBytes, &tm_v,
+                                        &bar_vfull[vs], half * 64, kvh, j * kBlk);
+                    }
+                    ++vcnt;
                 }
+                u = nx;
             }
         }
         __syncwarp();
     } else if (warp == kDqMmaWarp) {
         // ---------------- MMA issuer ----------------
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kDqRegsOther));
         if (elect_one()) {  // one elected thread runs the whole role
             constexpr uint32_t idesc_s = make_idesc(128, 128, 0, 0);  // S, dP: A in TMEM, B K-major
             constexpr uint32_t idesc_dq = make_idesc(128, D, 0, 1);   // dQ: A in TMEM, B = K MN-major
             const uint32_t sb = smem_u32(smem);
             const uint64_t kdesc0 = make_sdesc(sb, 16, 1024);             // K-major view of a tile at offset 0
             const uint64_t mdesc0 = make_sdesc(sb, L::kHalfBytes, 1024);  // MN-major view
-            uint32_t bcnt = 0, kcnt = 0, vcnt = 0, blk = 0;
+            uint32_t kcnt = 0, vcnt = 0, blk = 0;
             bool ok = true;
             PROF_DECL
             TRACE_DECL(0, cta == 0)
             // C[tmem d_col] = A[tmem a_col, bf16 packed over the head dimension] * B(K-major tile at b_off)^T
             auto issue_qk = [&](uint32_t d_col, uint32_t a_col, uint32_t b_off) {
                 const uint64_t db = sdesc_advance(kdesc0, b_off);
-    #pragma unroll
+#pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
                     const uint32_t off = (kk / 4) * L::kHalfBytes + (kk % 4) * 32;
                     mma_ts(tmem_base + d_col, tmem_base + a_col + kk * 8, sdesc_advance(db, off), idesc_s, kk > 0);
@@ -231,69 +299,82 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 ++vcnt;
                 return true;
             };
-            for (int idx = tile_begin; idx < tile_end && ok; ++idx) {
-                const int t = p.cta_tiles[idx];
-                for (int sub = 0; sub < 2 && ok; ++sub) {
-                    const int64_t q0 = (int64_t)(t / p.H) * (2 * kBlk) + sub * kBlk;
-                    if (q0 >= p.T) continue;
-                    const int lo = p.tok_start[q0] / kBlk, hi = (int)(q0 / kBlk);
-                    for (int hh = 0; hh < heads_per_shard && ok; ++hh) {
+            DqUnitIter units(p, tile_begin, tile_end, heads_per_shard);
+            DqUnit u = units.next();
+            uint32_t ucnt = 0;
+            if (u.valid) {  // first unit: nothing to overlap its first S and dP with
+                ok = mbar_wait(bar_qtready, 0, abort_flag);
+                if (ok) { tc_fence_after(); ok = do_s(kcnt); }
+                if (ok) ok = mbar_wait(bar_dotready, 0, abort_flag);
+                if (ok) { tc_fence_after(); ok = do_dp(); }
+            }
+            while (u.valid && ok) {
+                const DqUnit nx = units.next();
+                const int lo = u.lo, hi = u.hi;
+                const uint32_t kbase = kcnt;  // ring index of K_lo
+                for (int j = lo; j <= hi && ok; ++j, ++blk) {
+                    const bool last = j == hi;
+                    // S(j+1) as soon as the compute groups have read S(j)
+                    if (!last) {
                         PROF(7)
-                        ok = mbar_wait(bar_qtready, bcnt & 1, abort_flag);  // Q and dO are in TMEM
+                        ok = mbar_wait(bar_sfree, blk & 1, abort_flag);
+                        if (!ok) break;
+                        PROF(3)
+                        tc_fence_after();
+                        ok = do_s(kbase + (j + 1 - lo));
+                        if (!ok) break;
+                    }
+                    // dQ += dS(j) K_j
+                    PROF(7)
+                    ok = mbar_wait(bar_dsready, blk & 1, abort_flag);
+                    if (ok && j == lo && ucnt > 0) ok = mbar_wait(bar_dqempty, (ucnt - 1) & 1, abort_flag);  // dQ read out
+                    if (!ok) break;
+                    PROF(4)
+                    tc_fence_after();
+                    const uint32_t kidx = kbase + (j - lo);
+                    {
+                        const uint64_t ka = sdesc_advance(mdesc0, L::kKOff + (kidx % L::kKStages) * L::kTileBytes);
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk)  // 16 keys per step; group c left dS of its keys at columns CW c ..
+                            mma_ts(tmem_base + kColDQ,
+                                   tmem_base + kColDP + (kk / (kDqCW / 16)) * kDqCW + (kk % (kDqCW / 16)) * 8,
+                                   sdesc_advance(ka, kk * 2048), idesc_dq, (j > lo || kk > 0) ? 1u : 0u);
+                        tc_commit(&bar_kempty[kidx % L::kKStages]);
+                        if (last) tc_commit(bar_dqfull);
+                    }
+                    if (!last) {
+                        ok = do_dp();  // dP(j+1) over dS(j), after dQ(j) in pipe order
+                    } else if (nx.valid) {
+                        // first block of the next unit, behind the last dQ of this one: its Q and dO rows
+                        // were copied into TMEM while that dQ ran
+                        PROF(7)
+                        TRACE(21)
+                        ok = mbar_wait(bar_sfree, blk & 1, abort_flag);
+                        if (ok) ok = mbar_wait(bar_qtready, (ucnt + 1) & 1, abort_flag);
                         if (!ok) break;
                         PROF(2)
-                        ++bcnt;
+                        TRACE(22)
                         tc_fence_after();
-                        const uint32_t kbase = kcnt;  // ring index of K_lo
-                        ok = do_s(kbase);             // S(lo)
-                        if (ok) ok = do_dp();         // dP(lo)
+                        ok = do_s(kbase + (hi - lo + 1));
+                        TRACE(23)
+                        if (ok) ok = mbar_wait(bar_dotready, (ucnt + 1) & 1, abort_flag);
                         if (!ok) break;
-                        for (int j = lo; j <= hi && ok; ++j, ++blk) {
-                            // S(j+1) as soon as the compute groups have read S(j)
-                            if (j + 1 <= hi) {
-                                PROF(7)
-                                TRACE(8)
-                                ok = mbar_wait(bar_sfree, blk & 1, abort_flag);
-                                if (!ok) break;
-                                PROF(3)
-                                TRACE(5)
-                                tc_fence_after();
-                                ok = do_s(kbase + (j + 1 - lo));
-                                if (!ok) break;
-                            }
-                            // dQ += dS(j) K_j
-                            PROF(7)
-                            ok = mbar_wait(bar_dsready, blk & 1, abort_flag);
-                            if (!ok) break;
-                            PROF(4)
-                            TRACE(6)
-                            tc_fence_after();
-                            const uint32_t kidx = kbase + (j - lo);
-                            {
-                                const uint64_t ka = sdesc_advance(mdesc0, L::kKOff + (kidx % L::kKStages) * L::kTileBytes);
-    #pragma unroll
-                                for (int kk = 0; kk < 8; ++kk)  // 16 keys per step; group c left dS of its keys at columns CW c ..
-                                    mma_ts(tmem_base + kColDQ,
-                                           tmem_base + kColDP + (kk / (kDqCW / 16)) * kDqCW + (kk % (kDqCW / 16)) * 8,
-                                           sdesc_advance(ka, kk * 2048), idesc_dq, (j > lo || kk > 0) ? 1u : 0u);
-                                tc_commit(&bar_kempty[kidx % L::kKStages]);
-                            }
-                            TRACE(7)
-                            if (j + 1 <= hi) ok = do_dp();  // dP(j+1) over dS(j), after dQ(j) in pipe order
-                            TRACE(15)
-                            TRACE(16)
-                        }
-                        if (!ok) break;
-                        kcnt = kbase + (hi - lo + 1);
-                        tc_commit(bar_dqfull);
+                        TRACE(24)
+                        tc_fence_after();
+                        ok = do_dp();
+                        TRACE(25)
                     }
                 }
+                kcnt = kbase + (hi - lo + 1);
+                ++ucnt;
+                u = nx;
             }
             PROF_FLUSH(true, 512 * 24 + 8)
         }
         __syncwarp();
     } else {
         // ---------------- compute groups ----------------
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kDqRegsCompute));
         constexpr int CW = kDqCW;
         const int c = warp >> 2;  // which CW key columns of each query row this group owns
         // staging duty: even groups copy Q, odd groups dO; group pair c >> 1 takes that 64-column half
@@ -302,133 +383,160 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t t_s = tmem_base + lane_addr + kColS + CW * c;
         const uint32_t t_dp = tmem_base + lane_addr + kColDP + CW * c;
-        uint32_t bcnt = 0, blk = 0;
+        uint32_t ucnt = 0, blk = 0;
         bool ok = true;
         PROF_DECL
         TRACE_DECL(1 + warp, cta == 0 && lane == 0)
-        for (int idx = tile_begin; idx < tile_end && ok; ++idx) {
-            const int t = p.cta_tiles[idx];
-            for (int sub = 0; sub < 2 && ok; ++sub) {
-                const int64_t q0 = (int64_t)(t / p.H) * (2 * kBlk) + sub * kBlk;
-                if (q0 >= p.T) continue;
-                const int lo = p.tok_start[q0] / kBlk, hi = (int)(q0 / kBlk);
-                const int64_t row = q0 + r;
-                const bool row_ok = row < p.T;
-                const int kstart = row_ok ? p.tok_start[row] : 0;
-                const int64_t last_row = (q0 + kBlk <= p.T ? q0 + kBlk : p.T) - 1;
-                const int max_kstart = p.tok_start[last_row];
-                for (int hh = 0; hh < heads_per_shard && ok; ++hh) {
-                    const int h = (t % p.H) * heads_per_shard + hh;
-                    const float lse2 = p.lse2[(size_t)h * p.Tpad + row];  // padded rows hold zeros
-                    const float dsum = p.dvec[(size_t)h * p.Tpad + row];
-                    // ---- stage this group's operand (Q or dO) row from shared memory into TMEM ----
-                    // The MMAs that read the previous unit's copy have completed: their s_full / dp_full
-                    // completions were waited for above in program order.
-                    ok = mbar_wait(st_op == 0 ? bar_qfull : bar_dofull, bcnt & 1, abort_flag);
-                    if (!ok) break;
-                    {
-                        if (st_half < D / 64) {
-                            const uint8_t* src = smem + (st_op == 0 ? L::kQOff : L::kDoOff) + st_half * L::kHalfBytes + r * 128;
-                            const uint32_t t_dst = tmem_base + lane_addr + (st_op == 0 ? kColQ : kColDO) + 32 * st_half;
-                            uint32_t w[32];
+        // Copies this thread's row of Q or dO (its group's duty) of the unit whose tile has landed into TMEM.
+        // The caller has seen every MMA that read the previous copy complete (s_full for Q, dp_full for dO).
+        auto stage = [&](uint32_t parity) -> bool {
+            if (!mbar_wait(st_op == 0 ? bar_qfull : bar_dofull, parity, abort_flag)) return false;
+            if (st_half < D / 64) {
+                const uint8_t* src = smem + (st_op == 0 ? L::kQOff : L::kDoOff) + st_half * L::kHalfBytes + r * 128;
+                const uint32_t t_dst = tmem_base + lane_addr + (st_op == 0 ? kColQ : kColDO) + 32 * st_half;
+                uint32_t w[32];
 #pragma unroll
-                            for (int ch = 0; ch < 8; ++ch) {
-                                const uint4 v = *reinterpret_cast<const uint4*>(src + ((ch ^ (r & 7)) << 4));
-                                w[4 * ch] = v.x; w[4 * ch + 1] = v.y; w[4 * ch + 2] = v.z; w[4 * ch + 3] = v.w;
-                            }
-                            tmem_st32(t_dst, w);
-                            tmem_st_wait();
-                        }
-                        mbar_arrive(st_op == 0 ? bar_qempty : bar_doempty);  // the smem tile may be reloaded
-                        tc_fence_before();
-                        mbar_arrive(bar_qtready);
+                for (int ch = 0; ch < 8; ++ch) {
+                    const uint4 v = *reinterpret_cast<const uint4*>(src + ((ch ^ (r & 7)) << 4));
+                    w[4 * ch] = v.x; w[4 * ch + 1] = v.y; w[4 * ch + 2] = v.z; w[4 * ch + 3] = v.w;
+                }
+                tmem_st32(t_dst, w);
+                tmem_st_wait();
+            }
+            mbar_arrive(st_op == 0 ? bar_qempty : bar_doempty);  // the smem tile may be reloaded
+            tc_fence_before();
+            mbar_arrive(st_op == 0 ? bar_qtready : bar_dotready);
+            return true;
+        };
+        // Per-row values of a unit, fetched one unit ahead so the loads are off the path between units.
+        struct RowCtx {
+            float lse2, dsum;
+            int kstart, max_kstart;
+            bool row_ok;
+        };
+        auto load_ctx = [&](const DqUnit& un) {
+            RowCtx x;
+            const int64_t row = un.q0 + r;
+            x.row_ok = row < p.T;
+            x.kstart = x.row_ok ? p.tok_start[row] : 0;
+            const int64_t last_row = (un.q0 + kBlk <= p.T ? un.q0 + kBlk : p.T) - 1;
+            x.max_kstart = p.tok_start[last_row];
+            x.lse2 = p.lse2[(size_t)un.h * p.Tpad + row];  // padded rows hold zeros
+            x.dsum = p.dvec[(size_t)un.h * p.Tpad + row];
+            return x;
+        };
+        DqUnitIter units(p, tile_begin, tile_end, heads_per_shard);
+        DqUnit u = units.next();
+        RowCtx cx{};
+        if (u.valid) {
+            cx = load_ctx(u);
+            ok = stage(0);
+        }
+        while (u.valid && ok) {
+            const DqUnit nx = units.next();
+            RowCtx cx_next{};
+            if (nx.valid) cx_next = load_ctx(nx);
+            const int lo = u.lo, hi = u.hi, h = u.h;
+            const int64_t row = u.q0 + r;
+            const bool row_ok = cx.row_ok;
+            const int kstart = cx.kstart, max_kstart = cx.max_kstart;
+            const float lse2 = cx.lse2, dsum = cx.dsum;
+            for (int j = lo; j <= hi && ok; ++j, ++blk) {
+                const int k0 = j * kBlk;
+                const bool need_mask = (j == hi) || (k0 < max_kstart) || !row_ok;
+                const int c_lo = (row_ok ? kstart - k0 : kBlk) - CW * c;    // first visible column of this group's range
+                const int c_hi = (row_ok ? (int)(row - k0) : -1) - CW * c;  // last visible column
+                // ---- P = exp2(S c - LSE) ----
+                PROF(4)
+                ok = mbar_wait(bar_sfull, blk & 1, abort_flag);
+                if (!ok) break;
+                PROF(0)
+                TRACE(10)
+                tc_fence_after();
+                uint32_t sv[CW];
+#pragma unroll
+                for (int i = 0; i < CW; i += 32) tmem_ld32(t_s + i, sv + i);
+                tmem_ld_wait();
+                tc_fence_before();
+                mbar_arrive(bar_sfree);  // S(j+1) may overwrite the columns
+                TRACE(14)
+                float pf[CW];
+#pragma unroll
+                for (int i = 0; i < CW; i += 2) {
+                    pf[i] = ex2_sel(fmaf(__uint_as_float(sv[i]), p.scale_log2, -lse2), i);
+                    pf[i + 1] = ex2_sel(fmaf(__uint_as_float(sv[i + 1]), p.scale_log2, -lse2), i + 1);
+                }
+                if (need_mask) {
+#pragma unroll
+                    for (int i = 0; i < CW; ++i)
+                        if (i < c_lo || i > c_hi) pf[i] = 0.f;
+                }
+                // ---- dS = P o (dP - D), packed over this half's own dP columns ----
+                PROF(1)
+                TRACE(11)
+                ok = mbar_wait(bar_dpfull, blk & 1, abort_flag);
+                if (!ok) break;
+                PROF(2)
+                TRACE(12)
+                tc_fence_after();
+                uint32_t dpv[CW];
+#pragma unroll
+                for (int i = 0; i < CW; i += 32) tmem_ld32(t_dp + i, dpv + i);
+                tmem_ld_wait();
+                {
+                    uint32_t pk[CW / 2];
+#pragma unroll
+                    for (int i = 0; i < CW; i += 2)
+                        pk[i >> 1] = pack_bf16x2(pf[i] * (__uint_as_float(dpv[i]) - dsum),
+                                                 pf[i + 1] * (__uint_as_float(dpv[i + 1]) - dsum));
+                    if constexpr (CW == 64) tmem_st32(t_dp, pk); else tmem_st16(t_dp, pk);
+                }
+                tmem_st_wait();
+                tc_fence_before();
+                mbar_arrive(bar_dsready);
+                // Last block of the unit: every S and dP MMA that read this unit's Q / dO copy has completed, so
+                // the next unit's row goes into TMEM now, while the tensor pipe runs the last dQ.
+                if (j == hi && nx.valid) {
+                    TRACE(26)
+                    ok = stage((ucnt + 1) & 1);
+                    TRACE(27)
+                }
+                PROF(3)
+                TRACE(13)
+            }
+            if (!ok) break;
+            // ---- epilogue: dQ * scale to global ----
+            ok = mbar_wait(bar_dqfull, ucnt & 1, abort_flag);
+            if (!ok) break;
+            TRACE(28)
+            tc_fence_after();
+            constexpr int kCols = D / kDqGroups;
+            constexpr int kChunk = kCols < 32 ? kCols : 32;
+            const uint32_t t_dq = tmem_base + lane_addr + kColDQ + c * kCols;
+            __nv_bfloat16* gdst = p.dq + ((size_t)row * p.hq + h) * D + c * kCols;
+#pragma unroll
+            for (int cc = 0; cc < kCols; cc += kChunk) {
+                uint32_t v[kChunk];
+                if constexpr (kChunk == 32) tmem_ld32(t_dq + cc, v); else tmem_ld16(t_dq + cc, v);
+                tmem_ld_wait();
+                if (row_ok) {
+#pragma unroll
+                    for (int i = 0; i < kChunk; i += 8) {
+                        uint4 w;
+                        w.x = pack_bf16x2(__uint_as_float(v[i]) * p.scale, __uint_as_float(v[i + 1]) * p.scale);
+                        w.y = pack_bf16x2(__uint_as_float(v[i + 2]) * p.scale, __uint_as_float(v[i + 3]) * p.scale);
+                        w.z = pack_bf16x2(__uint_as_float(v[i + 4]) * p.scale, __uint_as_float(v[i + 5]) * p.scale);
+                        w.w = pack_bf16x2(__uint_as_float(v[i + 6]) * p.scale, __uint_as_float(v[i + 7]) * p.scale);
+                        *reinterpret_cast<uint4*>(gdst + cc + i) = w;
                     }
-                    ++bcnt;
-                    for (int j = lo; j <= hi && ok; ++j, ++blk) {
-                        const int k0 = j * kBlk;
-                        const bool need_mask = (j == hi) || (k0 < max_kstart) || !row_ok;
-                        const int c_lo = (row_ok ? kstart - k0 : kBlk) - CW * c;    // first visible column of this group's range
-                        const int c_hi = (row_ok ? (int)(row - k0) : -1) - CW * c;  // last visible column
-                        // ---- P = exp2(S c - LSE) ----
-                        PROF(4)
-                        ok = mbar_wait(bar_sfull, blk & 1, abort_flag);
-                        if (!ok) break;
-                        PROF(0)
-                        TRACE(10)
-                        tc_fence_after();
-                        uint32_t sv[CW];
-#pragma unroll
-                        for (int i = 0; i < CW; i += 32) tmem_ld32(t_s + i, sv + i);
-                        tmem_ld_wait();
-                        tc_fence_before();
-                        mbar_arrive(bar_sfree);  // S(j+1) may overwrite the columns
-                        TRACE(14)
-                        float pf[CW];
-#pragma unroll
-                        for (int i = 0; i < CW; i += 2) {
-                            pf[i] = ex2_sel(fmaf(__uint_as_float(sv[i]), p.scale_log2, -lse2), i);
-                            pf[i + 1] = ex2_sel(fmaf(__uint_as_float(sv[i + 1]), p.scale_log2, -lse2), i + 1);
-                        }
-                        if (need_mask) {
-#pragma unroll
-                            for (int i = 0; i < CW; ++i)
-                                if (i < c_lo || i > c_hi) pf[i] = 0.f;
-                        }
-                        // ---- dS = P o (dP - D), packed over this half's own dP columns ----
-                        PROF(1)
-                        TRACE(11)
-                        ok = mbar_wait(bar_dpfull, blk & 1, abort_flag);
-                        if (!ok) break;
-                        PROF(2)
-                        TRACE(12)
-                        tc_fence_after();
-                        uint32_t dpv[CW];
-#pragma unroll
-                        for (int i = 0; i < CW; i += 32) tmem_ld32(t_dp + i, dpv + i);
-                        tmem_ld_wait();
-                        {
-                            uint32_t pk[CW / 2];
-#pragma unroll
-                            for (int i = 0; i < CW; i += 2)
-                                pk[i >> 1] = pack_bf16x2(pf[i] * (__uint_as_float(dpv[i]) - dsum),
-                                                         pf[i + 1] * (__uint_as_float(dpv[i + 1]) - dsum));
-                            if constexpr (CW == 64) tmem_st32(t_dp, pk); else tmem_st16(t_dp, pk);
-                        }
-                        tmem_st_wait();
-                        tc_fence_before();
-                        mbar_arrive(bar_dsready);
-                        PROF(3)
-                        TRACE(13)
-                    }
-                    if (!ok) break;
-                    // ---- epilogue: dQ * scale to global ----
-                    ok = mbar_wait(bar_dqfull, (bcnt - 1) & 1, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after();
-                    constexpr int kCols = D / kDqGroups;
-                    constexpr int kChunk = kCols < 32 ? kCols : 32;
-                    const uint32_t t_dq = tmem_base + lane_addr + kColDQ + c * kCols;
-                    __nv_bfloat16* gdst = p.dq + ((size_t)row * p.hq + h) * D + c * kCols;
-#pragma unroll
-                    for (int cc = 0; cc < kCols; cc += kChunk) {
-                        uint32_t v[kChunk];
-                        if constexpr (kChunk == 32) tmem_ld32(t_dq + cc, v); else tmem_ld16(t_dq + cc, v);
-                        tmem_ld_wait();
-                        if (row_ok) {
-#pragma unroll
-                            for (int i = 0; i < kChunk; i += 8) {
-                                uint4 w;
-                                w.x = pack_bf16x2(__uint_as_float(v[i]) * p.scale, __uint_as_float(v[i + 1]) * p.scale);
-                                w.y = pack_bf16x2(__uint_as_float(v[i + 2]) * p.scale, __uint_as_float(v[i + 3]) * p.scale);
-                                w.z = pack_bf16x2(__uint_as_float(v[i + 4]) * p.scale, __uint_as_float(v[i + 5]) * p.scale);
-                                w.w = pack_bf16x2(__uint_as_float(v[i + 6]) * p.scale, __uint_as_float(v[i + 7]) * p.scale);
-                                *reinterpret_cast<uint4*>(gdst + cc + i) = w;
-                            }
-                        }
-                    }
-                    tc_fence_before();  // the next dQ MMA follows this group's next ds_ready arrival
                 }
             }
+            tc_fence_before();
+            mbar_arrive(bar_dqempty);  // the next unit's first dQ MMA may overwrite the accumulator
+            TRACE(29)
+            ++ucnt;
+            u = nx;
+            cx = cx_next;
         }
         PROF_FLUSH(threadIdx.x == 0, 512 * 24)
     }

@@ -513,6 +513,7 @@ static int launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtens
     if (!configured) {
         if (cudaFuncSetAttribute(k_attn_fwd<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kAlloc) != cudaSuccess)
             return LIBRA_ERR_CUDA;
+        if (!regs_pool_ok(k_attn_fwd<D>, 256, LIBRA_FWD_REG_INC, 128, LIBRA_FWD_REG_DEC)) return LIBRA_ERR_UNSUPPORTED;
         configured = true;
     }
     k_attn_fwd<D><<<W, kFwdThreads, L::kAlloc, s>>>(tq, tk, tv, prm);

@@ -59,3 +59,16 @@ int make_thd_map(CUtensorMap* m, const void* base, int64_t T, int H, int d, int 
 // fp32 matrix [rows, cols] (cols contiguous); box = box_cols x box_rows, 128-byte swizzle.
 int make_f32_2d_map(CUtensorMap* m, const void* base, int64_t rows, int64_t cols, int box_cols, int box_rows);
 }  // namespace libra
+
+// setmaxnreg moves registers inside the pool the CTA got at launch (registers per thread as compiled x
+// threads): what the shrinking warps release must cover what the growing warps ask for, or the last
+// warpgroup to grow waits for ever.  Checked on the host against the compiled register count before the
+// first launch, so that a build with other flags fails with an error instead.
+template <typename Kernel>
+static inline bool regs_pool_ok(Kernel k, int threads_grow, int regs_grow, int threads_shrink, int regs_shrink) {
+    cudaFuncAttributes a;
+    if (cudaFuncGetAttributes(&a, k) != cudaSuccess) return false;
+    const long long released = (long long)(a.numRegs - regs_shrink) * threads_shrink;
+    const long long wanted = (long long)(regs_grow - a.numRegs) * threads_grow;
+    return a.numRegs >= regs_shrink && wanted <= released;
+}

@@ -53,6 +53,29 @@ __global__ void k_block_weights(const int32_t* __restrict__ tok_start, const int
     weight_blk[b] = w;
 }
 
+// Block-count weight (LIBRA_WEIGHT_BLOCKS): the token axis is cut into chunks at multiples of g.  For a
+// chunk of query rows [r0, r1] the visible keys span the chunks from the one holding the first key of r0's
+// sample to the one holding r1 (row r0 sees a key in every chunk of that range, later rows see no chunk
+// outside it); for a chunk of keys [c0, c1] the attending queries span the chunks from the one holding c0
+// to the one holding the last token of c1's sample.
+__global__ void k_block_weights_blocks(const int32_t* __restrict__ tok_start, const int32_t* __restrict__ tok_end,
+                                       int64_t T, int tile, int64_t NB, int key_major, int g, int unit_cost,
+                                       int64_t* __restrict__ weight_blk) {
+    const int64_t b = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (b >= NB) return;
+    const int64_t t0 = b * tile;
+    const int64_t t1 = (t0 + tile < T) ? t0 + tile : T;
+    int64_t w = 0;
+    for (int64_t c = t0 / g; c * g < t1; ++c) {
+        const int64_t first = c * g > t0 ? c * g : t0;
+        const int64_t last = ((c + 1) * g < t1 ? (c + 1) * g : t1) - 1;
+        const int64_t n = key_major ? ((int64_t)tok_end[last] - 1) / g - first / g + 1
+                                    : last / g - (int64_t)tok_start[first] / g + 1;
+        w += 8 * n + unit_cost;
+    }
+    weight_blk[b] = w;
+}
+
 // Order of Algorithm 2: decreasing weight, then increasing id.  All H shards of a block weigh
 // the same and their ids b*H+h are consecutive, so ordering the blocks orders the tiles.
 // rank(b) = number of blocks that precede b; one thread per block, O(NB) each.
@@ -193,7 +216,7 @@ static void free_dir(PlanDir& d) {
     d = PlanDir();
 }
 
-static int build_dir(libra_plan* p, PlanDir& d, int key_major) {
+static int build_dir(libra_plan* p, PlanDir& d, int key_major, const libra_plan_opts& o) {
     const int64_t T = p->T;
     d.NB = (T + d.tile - 1) / d.tile;
     if (d.NB * (int64_t)d.H >= (int64_t)INT32_MAX) return LIBRA_ERR_OVERFLOW;
@@ -216,8 +239,14 @@ static int build_dir(libra_plan* p, PlanDir& d, int key_major) {
     cudaStream_t s = p->stream;
     cudaMemsetAsync(d.d_busy, 0, sizeof(uint64_t) * 2 * d.W, s);
     cudaMemsetAsync(d.d_busy2, 0, sizeof(uint64_t) * 2 * d.W, s);
-    k_block_weights<<<grid_for(d.NB, 128), 128, 0, s>>>(p->d_tok_start, p->d_tok_end, T, d.tile, d.NB, key_major,
-                                                        d.d_weight_blk);
+    if (o.weight_model == LIBRA_WEIGHT_BLOCKS)
+        k_block_weights_blocks<<<grid_for(d.NB, 128), 128, 0, s>>>(p->d_tok_start, p->d_tok_end, T, d.tile, d.NB,
+                                                                   key_major, o.cost_block ? o.cost_block : 128,
+                                                                   key_major ? o.unit_cost_kv : o.unit_cost_q,
+                                                                   d.d_weight_blk);
+    else
+        k_block_weights<<<grid_for(d.NB, 128), 128, 0, s>>>(p->d_tok_start, p->d_tok_end, T, d.tile, d.NB, key_major,
+                                                            d.d_weight_blk);
     k_rank_blocks<<<grid_for(d.NB, 256), 256, 0, s>>>(d.d_weight_blk, d.NB, d.d_blk_order);
     if (d.W <= 160)
         k_place<5><<<1, 32, 0, s>>>(d.d_weight_blk, d.d_blk_order, d.NT, d.H, d.W, d.d_cta_of_tile, d.d_pos,
@@ -244,10 +273,12 @@ extern "C" int libra_plan_tiles(const int32_t* cu_seqlens_dev, int n_samples, in
                                 const libra_plan_opts* opts, void* stream, libra_plan_t** plan_out) {
     if (!cu_seqlens_dev || !plan_out || n_samples <= 0 || n_heads <= 0 || tile_q <= 0) return LIBRA_ERR_INVALID_ARG;
     *plan_out = nullptr;
-    libra_plan_opts o = {0, 0, 0, 0, 0};
+    libra_plan_opts o = {0, 0, 0, 0, 0, 0, 0, 0, 0};
     if (opts) o = *opts;
     if (o.n_workers < 0 || o.tile_kv < 0 || o.n_heads_kv < 0 || o.total_tokens < 0) return LIBRA_ERR_INVALID_ARG;
     if (o.directions & ~(LIBRA_DIR_Q | LIBRA_DIR_KV)) return LIBRA_ERR_INVALID_ARG;
+    if (o.weight_model != LIBRA_WEIGHT_PAIRS && o.weight_model != LIBRA_WEIGHT_BLOCKS) return LIBRA_ERR_INVALID_ARG;
+    if (o.cost_block < 0 || o.unit_cost_q < 0 || o.unit_cost_kv < 0) return LIBRA_ERR_INVALID_ARG;
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return LIBRA_ERR_NO_DEVICE;
     int sms = 0;
@@ -282,12 +313,12 @@ extern "C" int libra_plan_tiles(const int32_t* cu_seqlens_dev, int n_samples, in
         if (dirs & LIBRA_DIR_Q) {
             PlanDir& d = p->dir[0];
             d.tile = tile_q; d.H = n_heads; d.W = W;
-            rc = build_dir(p, d, 0);
+            rc = build_dir(p, d, 0, o);
         }
         if (rc == LIBRA_OK && (dirs & LIBRA_DIR_KV)) {
             PlanDir& d = p->dir[1];
             d.tile = o.tile_kv ? o.tile_kv : 128; d.H = o.n_heads_kv ? o.n_heads_kv : n_heads; d.W = W;
-            rc = build_dir(p, d, 1);
+            rc = build_dir(p, d, 1, o);
         }
     }
     if (rc != LIBRA_OK) {

@@ -169,3 +169,61 @@ def test_zero_length_samples_and_ragged_tail():
         assert a[key].tolist() == b[key].tolist()
     assert a["n_blocks"] == 5
     assert a["weight"].reshape(-1, 2)[-1, 0] == 1 + 2 + 3  # tokens 16..18 of the last sample
+
+
+# ---- block-count weight (a time proxy, not in the paper) -------------------------------------------
+
+def _brute_block_weights(lengths, tile, direction, g, unit_cost):
+    """Every visible (q, k) pair marks the cell (q // g, k // g); a tile's weight counts, per chunk piece
+    it holds, the marked cells of that piece's rows (query-major) or columns (key-major)."""
+    T = sum(lengths)
+    sid = np.repeat(np.arange(len(lengths)), lengths)
+    cells = {}  # piece -> set of chunks on the other axis
+    for q in range(T):
+        for k in range(q + 1):
+            if sid[q] != sid[k]:
+                continue
+            own, other = (q, k) if direction == 0 else (k, q)
+            cells.setdefault((own // tile, own // g), set()).add(other // g)
+    nb = -(-T // tile)
+    w = [0] * nb
+    for (b, _chunk), others in cells.items():
+        w[b] += 8 * len(others) + unit_cost
+    return w
+
+
+@pytest.mark.parametrize("seed", range(8))
+@pytest.mark.parametrize("direction", [0, 1])
+def test_block_weights_brute_force(seed, direction):
+    rng = np.random.default_rng(100 + seed)
+    total = int(rng.integers(20, 260))
+    lengths = [x for x in pools.random_layout(rng, total, int(rng.integers(1, 90)))]
+    g = int(rng.choice([2, 4, 8, 16]))
+    tile = int(rng.choice([g, 2 * g, 3 * g, 5, 7, 1]))   # aligned, and tiles that cut chunks into pieces
+    unit = int(rng.integers(0, 20))
+    H = int(rng.integers(1, 4))
+    p = oracle.plan(pools.cu_seqlens(lengths), H, tile, 5, direction, weight_model=1, cost_block=g, unit_cost=unit)
+    want = _brute_block_weights(lengths, tile, direction, g, unit)
+    assert p["weight"].reshape(-1, H).tolist() == [[w] * H for w in want]
+
+
+def test_block_weights_single_sample_closed_form():
+    # one sample of 10 chunks, tile = 2 chunks: row chunk i sees chunks 0..i, key chunk i is seen by chunks i..9
+    g, n = 16, 10
+    pq = oracle.plan(pools.cu_seqlens([g * n]), 1, 2 * g, 3, 0, weight_model=1, cost_block=g, unit_cost=5)
+    pk = oracle.plan(pools.cu_seqlens([g * n]), 1, 2 * g, 3, 1, weight_model=1, cost_block=g, unit_cost=5)
+    assert pq["weight"].tolist() == [8 * ((2 * b + 1) + (2 * b + 2)) + 10 for b in range(5)]
+    assert pk["weight"].tolist() == [8 * ((n - 2 * b) + (n - 2 * b - 1)) + 10 for b in range(5)]
+    assert pq["weight"].sum() == pk["weight"].sum()   # both count the same lower-triangular cells
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_block_model_placement_vs_heap_simulation(seed):
+    rng = np.random.default_rng(200 + seed)
+    lengths = pools.random_layout(rng, int(rng.integers(500, 4000)), int(rng.integers(1, 900)))
+    H, W = int(rng.integers(1, 5)), int(rng.integers(2, 40))
+    p = oracle.plan(pools.cu_seqlens(lengths), H, 256, W, 0, weight_model=1, cost_block=128, unit_cost=12)
+    order, owner, _lists, loads = _heap_lpt(p["weight"], W)
+    assert p["order"].tolist() == order
+    assert p["cta_of_tile"].tolist() == owner
+    assert p["loads"].tolist() == loads

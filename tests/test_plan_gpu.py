@@ -44,6 +44,45 @@ def test_benchmark_configs(idx, skew):
     _compare(cu, spec.hq, 256, 148, tile_kv=128, H_kv=spec.hkv)
 
 
+def _compare_blocks(cu_np, H, tile, W, tile_kv, H_kv, g, uq, ukv):
+    """Block-count weight model: device plan == oracle plan, bit for bit."""
+    from paper_2607_23250_b200 import binding as lb
+    cu = torch.from_numpy(cu_np).cuda()
+    plan = lb.libra_plan_tiles(cu, H, tile, n_workers=W, tile_kv=tile_kv, n_heads_kv=H_kv,
+                               weight_model=lb.LIBRA_WEIGHT_BLOCKS, cost_block=g, unit_cost_q=uq, unit_cost_kv=ukv)
+    assert plan.status() == 0
+    for direction, d_or, t, h, u in ((lb.LIBRA_DIR_Q, 0, tile, H, uq), (lb.LIBRA_DIR_KV, 1, tile_kv, H_kv, ukv)):
+        got = plan.export(direction)
+        want = oracle.plan(cu_np, h, t, W, d_or, weight_model=1, cost_block=g or 128, unit_cost=u)
+        for k in KEYS:
+            assert np.array_equal(got[k], want[k]), (direction, k)
+    plan.destroy()
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_block_model_random_layouts(seed):
+    rng = np.random.default_rng(300 + seed)
+    lengths = pools.random_layout(rng, int(rng.integers(10, 6000)), int(rng.integers(1, 700)))
+    _compare_blocks(pools.cu_seqlens(lengths), int(rng.integers(1, 9)), int(rng.choice([3, 16, 100, 128, 256])),
+                    int(rng.integers(1, 400)), int(rng.choice([7, 64, 128])), int(rng.integers(1, 5)),
+                    int(rng.choice([0, 4, 32, 128])), int(rng.integers(0, 30)), int(rng.integers(0, 30)))
+
+
+@pytest.mark.parametrize("idx,skew", [(1, 0), (2, 0), (3, 0), (5, 0.5)])
+def test_block_model_benchmark_configs(idx, skew):
+    spec = pools.config(idx, skew)
+    cu = pools.cu_seqlens(pools.pool_lengths(spec))
+    _compare_blocks(cu, spec.hkv, 256, 148, 128, spec.hkv, 0, 12, 6)
+
+
+def test_block_model_rejects_bad_options():
+    from paper_2607_23250_b200 import binding as lb
+    cu = torch.tensor([0, 9], dtype=torch.int32).cuda()
+    for kw in (dict(weight_model=2), dict(weight_model=1, cost_block=-1), dict(weight_model=1, unit_cost_q=-3)):
+        with pytest.raises(Exception):
+            lb.libra_plan_tiles(cu, 1, 4, n_workers=2, **kw)
+
+
 def test_edge_cases():
     _compare(np.array([0, 1], dtype=np.int32), 1, 256, 148)                      # one token
     _compare(np.array([0, 0, 3, 3, 3, 700, 700], dtype=np.int32), 2, 256, 5)     # empty samples, ragged tail
