@@ -170,7 +170,10 @@ def run_ours(args):
     t = pools.make_tensors(T, hq, hkv, d, seed=rank, device=f"cuda:{local}")
     q, k, v, dout = t["q"], t["k"], t["v"], t["dout"]
     cu = torch.from_numpy(cu_np).to(dev)
-    plan = lb.libra_plan_tiles(cu, hq, 256, tile_kv=128, n_heads_kv=hkv, total_tokens=T)
+    blocks = args.weight_model == "blocks"
+    plan = lb.libra_plan_tiles(cu, hq, 256, tile_kv=128, n_heads_kv=hkv, total_tokens=T,
+                               weight_model=lb.LIBRA_WEIGHT_BLOCKS if blocks else lb.LIBRA_WEIGHT_PAIRS,
+                               unit_cost_q=12 if blocks else 0, unit_cost_kv=6 if blocks else 0)
     assert plan.status() == 0
     plan.set_timing(True)
     out = torch.empty_like(q)
@@ -285,6 +288,7 @@ def finish(args, rank, world, spec, lengths, plan, value, ms_per_step, kern, bus
                                    f"{len(lengths)} samples (log-normal median 644, sigma 1.6), Hq {hq} / Hkv {hkv} / d {d}, "
                                    f"causal per sample, fwd+bwd; plan built once and reused",
                        "tile_q": 256, "tile_kv": 128, "n_workers": plan.info()["n_workers"],
+                       "tile_weight": "blocks (time proxy)" if blocks else "causal pairs (Eq. 6)",
                        "l2": "inputs larger than L2 (Q alone is %.2f GB)" % (q.numel() * 2 / 1e9),
                        "per_rank_pool": "seed = rank"},
             "pct_of_bf16_peak": {"burst_measured": round(100 * value / world / peaks["burst"], 2),
@@ -354,6 +358,8 @@ def main():
     ap.add_argument("--config", type=int, default=2)
     ap.add_argument("--skew", type=float, default=0.0)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--weight-model", default="pairs", choices=["pairs", "blocks"],
+                    help="tile weight of the plan: the paper's pair count, or the executed-block count")
     ap.add_argument("--seqs", type=int, default=0, help="override the number of packed sequences (profiling runs)")
     ap.add_argument("--skip-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
     ap.add_argument("--skip-cpu", action="store_true", help="skip the CPU oracle leg (profiling runs)")
