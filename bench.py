@@ -288,7 +288,7 @@ def finish(args, rank, world, spec, lengths, plan, value, ms_per_step, kern, bus
                                    f"{len(lengths)} samples (log-normal median 644, sigma 1.6), Hq {hq} / Hkv {hkv} / d {d}, "
                                    f"causal per sample, fwd+bwd; plan built once and reused",
                        "tile_q": 256, "tile_kv": 128, "n_workers": plan.info()["n_workers"],
-                       "tile_weight": "blocks (time proxy)" if blocks else "causal pairs (Eq. 6)",
+                       "tile_weight": "blocks (time proxy)" if args.weight_model == "blocks" else "causal pairs (Eq. 6)",
                        "l2": "inputs larger than L2 (Q alone is %.2f GB)" % (q.numel() * 2 / 1e9),
                        "per_rank_pool": "seed = rank"},
             "pct_of_bf16_peak": {"burst_measured": round(100 * value / world / peaks["burst"], 2),
