@@ -198,6 +198,28 @@ int libra_attn_pool_bwd_noalloc(const void* q_dev, const void* k_dev, const void
                                 void* dq_dev, void* dk_dev, void* dv_dev,
                                 const libra_dims* dims, void* stream);
 
+/* ---- Variance-Reduced Sequence Placement (Section 4.2, Algorithm 1) ----------------------
+ * Groups the D packed sequences of one optimizer-step window into K = D / P pools of exactly P
+ * sequences with even summed attention work.  The paper runs it on a CPU core in the data path;
+ * these two calls run it in device kernels on `stream` (no allocation, no synchronisation).
+ *
+ * libra_vrsp_work: work_dev[i] = F_i = sum over the raw samples j of packed sequence i of
+ *   len_ij^2 (Eq. 4).  sample_offsets_dev: int32[n_samples_total + 1], the sample start offsets of
+ *   all sequences laid end to end (non-decreasing; only differences are used);
+ *   seq_first_sample_dev: int32[D + 1], index of each sequence's first sample.
+ * libra_vrsp_place: sequences in the order (F descending, index ascending) go one by one to the
+ *   pool with the smallest load among those holding fewer than P sequences (lowest pool index on
+ *   ties).  Outputs (device): order_dev int32[D], the reordered list S' as input indices, pools
+ *   laid end to end in pool order, a pool's sequences in the order they were appended (pool k of
+ *   the window is GA index k / (DP/P), pool k % (DP/P) of that index: GA-major, pool-minor);
+ *   pool_of_seq_dev int32[D]; pool_load_dev int64[K].  scratch_dev: int32[D], overwritten.
+ * Errors: INVALID_ARG (null, D <= 0, P <= 0, P does not divide D), UNSUPPORTED (K > 1024 or
+ * D > 2^20), CUDA. */
+int libra_vrsp_work(const int32_t* sample_offsets_dev, const int32_t* seq_first_sample_dev, int n_sequences,
+                    int64_t* work_dev, void* stream);
+int libra_vrsp_place(const int64_t* work_dev, int n_sequences, int pool_size, int32_t* order_dev,
+                     int32_t* pool_of_seq_dev, int64_t* pool_load_dev, int32_t* scratch_dev, void* stream);
+
 /* ---- instrumentation -------------------------------------------------------------------
  * Per-CTA busy time of the most recent launch of kernel `which` (LIBRA_KERNEL_*) that used this
  * plan: nanoseconds between the CTA starting and finishing its tile list, read with the GPU's

@@ -166,3 +166,24 @@ def plan(cu, n_heads, tile, n_workers, direction=0, weight_model=0, cost_block=1
                                       ctypes.c_int(unit_cost), *outs), "oracle_plan_blocks")
     res["n_blocks"] = int(nb)
     return res
+
+
+def vrsp_work(sample_offsets, seq_first_sample):
+    """F_i = sum of squared raw-sample lengths of packed sequence i (Eq. 4)."""
+    so = _arr(sample_offsets, np.int32)
+    fs = _arr(seq_first_sample, np.int32)
+    D = len(fs) - 1
+    out = np.empty(D, np.int64)
+    _check(_load().oracle_vrsp_work(_p(so), _p(fs), ctypes.c_int(D), _p(out)), "oracle_vrsp_work")
+    return out
+
+
+def vrsp_place(work, pool_size):
+    """Algorithm 1 -> dict(order, pool_of_seq, pool_load)."""
+    w = _arr(work, np.int64)
+    D = len(w)
+    res = dict(order=np.empty(D, np.int32), pool_of_seq=np.empty(D, np.int32),
+               pool_load=np.empty(max(D // pool_size, 1), np.int64))
+    _check(_load().oracle_vrsp_place(_p(w), ctypes.c_int(D), ctypes.c_int(pool_size), _p(res["order"]),
+                                     _p(res["pool_of_seq"]), _p(res["pool_load"])), "oracle_vrsp_place")
+    return res

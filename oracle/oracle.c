@@ -74,6 +74,7 @@ static int cmp_tiles(const void* a, const void* b) {
 /* Steps 3-5, common to both weight models: order, place, list. */
 static int place_tiles(int64_t NT, int W, const int64_t* weight, int32_t* order, int32_t* cta_of_tile,
                        int32_t* cta_offsets, int32_t* cta_tiles, int64_t* loads) {
+    if (W <= 0 || NT < 0) return -1;
     /* step 3 */
     tile_key* keys = (tile_key*)malloc(sizeof(tile_key) * (size_t)NT);
     if (!keys) return -2;
@@ -190,4 +191,82 @@ int oracle_plan_blocks(const int32_t* cu, int n, int H, int tile, int W, int dir
         for (int h = 0; h < H; ++h) weight[b * H + h] = w;
     }
     return place_tiles(NT, W, weight, order, cta_of_tile, cta_offsets, cta_tiles, loads);
+}
+
+/* ------------------------------------------------------------------------------------
+ * Variance-Reduced Sequence Placement (Section 4.2, Algorithm 1), in the algorithm's order:
+ *   work      F_i = sum_j len_ij^2 over the raw samples of packed sequence i      (Eq. 4)
+ *   pools     K = D / P, all empty
+ *   order     sequences by decreasing F, then increasing index
+ *   heap      min-heap of (load_k, k) over the pools that are not full
+ *   loop      pop the minimum, append the sequence to that pool, add F to its load, push the
+ *             pool back if it still holds fewer than P sequences
+ *   output    the pools laid end to end in pool order (GA-major, pool-minor numbering of pools)
+ * The heap is a plain array-based binary heap ordered lexicographically on (load, k).
+ * ------------------------------------------------------------------------------------ */
+int oracle_vrsp_work(const int32_t* sample_offsets, const int32_t* seq_first_sample, int D, int64_t* work) {
+    if (!sample_offsets || !seq_first_sample || !work || D <= 0) return -1;
+    for (int i = 0; i < D; ++i) {
+        int64_t f = 0;
+        for (int j = seq_first_sample[i]; j < seq_first_sample[i + 1]; ++j) {
+            const int64_t len = (int64_t)sample_offsets[j + 1] - sample_offsets[j];
+            f += len * len;
+        }
+        work[i] = f;
+    }
+    return 0;
+}
+
+typedef struct { int64_t load; int32_t k; } pool_key;
+
+static int pool_less(pool_key a, pool_key b) { return a.load < b.load || (a.load == b.load && a.k < b.k); }
+
+static void heap_push(pool_key* h, int* n, pool_key x) {
+    int i = (*n)++;
+    h[i] = x;
+    while (i > 0 && pool_less(h[i], h[(i - 1) / 2])) {
+        pool_key t = h[i]; h[i] = h[(i - 1) / 2]; h[(i - 1) / 2] = t;
+        i = (i - 1) / 2;
+    }
+}
+
+static pool_key heap_pop(pool_key* h, int* n) {
+    pool_key top = h[0];
+    h[0] = h[--(*n)];
+    int i = 0;
+    for (;;) {
+        int l = 2 * i + 1, r = l + 1, m = i;
+        if (l < *n && pool_less(h[l], h[m])) m = l;
+        if (r < *n && pool_less(h[r], h[m])) m = r;
+        if (m == i) break;
+        pool_key t = h[i]; h[i] = h[m]; h[m] = t;
+        i = m;
+    }
+    return top;
+}
+
+int oracle_vrsp_place(const int64_t* work, int D, int P, int32_t* order /*[D]*/, int32_t* pool_of_seq /*[D]*/,
+                      int64_t* pool_load /*[D/P]*/) {
+    if (!work || !order || !pool_of_seq || !pool_load || D <= 0 || P <= 0 || D % P != 0) return -1;
+    const int K = D / P;
+    tile_key* keys = (tile_key*)malloc(sizeof(tile_key) * (size_t)D);
+    pool_key* heap = (pool_key*)malloc(sizeof(pool_key) * (size_t)K);
+    int32_t* fill = (int32_t*)calloc((size_t)K, sizeof(int32_t));
+    if (!keys || !heap || !fill) { free(keys); free(heap); free(fill); return -2; }
+    for (int i = 0; i < D; ++i) { keys[i].w = work[i]; keys[i].id = i; }
+    qsort(keys, (size_t)D, sizeof(tile_key), cmp_tiles);  /* decreasing F, then increasing index */
+    int n = 0;
+    for (int k = 0; k < K; ++k) { pool_load[k] = 0; pool_key x = {0, k}; heap_push(heap, &n, x); }
+    for (int x = 0; x < D; ++x) {
+        const int32_t i = keys[x].id;
+        pool_key top = heap_pop(heap, &n);
+        const int k = top.k;
+        order[(int64_t)k * P + fill[k]] = i;
+        fill[k] += 1;
+        pool_of_seq[i] = k;
+        pool_load[k] += work[i];
+        if (fill[k] < P) { pool_key back = {pool_load[k], k}; heap_push(heap, &n, back); }
+    }
+    free(keys); free(heap); free(fill);
+    return 0;
 }

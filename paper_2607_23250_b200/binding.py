@@ -204,3 +204,28 @@ def libra_attn_pool_bwd_noalloc(q, k, v, out, lse, dout, plan: Plan, dq, dk, dv,
                                             _ptr(plan.cu_seqlens), plan._h, _ptr(dq), _ptr(dk), _ptr(dv),
                                             ctypes.byref(dims), _stream(stream)), "libra_attn_pool_bwd_noalloc")
     return dq, dk, dv
+
+
+def libra_vrsp_work(sample_offsets: torch.Tensor, seq_first_sample: torch.Tensor, stream=None) -> torch.Tensor:
+    """F_i = sum of squared raw-sample lengths of packed sequence i (int64, on the device)."""
+    for t in (sample_offsets, seq_first_sample):
+        assert t.is_cuda and t.dtype == torch.int32 and t.is_contiguous()
+    D = seq_first_sample.numel() - 1
+    work = torch.empty(D, dtype=torch.int64, device=sample_offsets.device)
+    _check(_lib.libra_vrsp_work(_ptr(sample_offsets), _ptr(seq_first_sample), ctypes.c_int(D), _ptr(work),
+                                _stream(stream)), "libra_vrsp_work")
+    return work
+
+
+def libra_vrsp_place(work: torch.Tensor, pool_size: int, stream=None):
+    """Algorithm 1 on the device -> dict(order, pool_of_seq, pool_load) of device tensors."""
+    assert work.is_cuda and work.dtype == torch.int64 and work.is_contiguous()
+    D = work.numel()
+    dev = work.device
+    order = torch.empty(D, dtype=torch.int32, device=dev)
+    pool_of_seq = torch.empty(D, dtype=torch.int32, device=dev)
+    pool_load = torch.empty(max(D // max(pool_size, 1), 1), dtype=torch.int64, device=dev)
+    scratch = torch.empty(D, dtype=torch.int32, device=dev)
+    _check(_lib.libra_vrsp_place(_ptr(work), ctypes.c_int(D), ctypes.c_int(pool_size), _ptr(order), _ptr(pool_of_seq),
+                                 _ptr(pool_load), _ptr(scratch), _stream(stream)), "libra_vrsp_place")
+    return dict(order=order, pool_of_seq=pool_of_seq, pool_load=pool_load)
