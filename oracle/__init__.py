@@ -187,3 +187,53 @@ def vrsp_place(work, pool_size):
     _check(_load().oracle_vrsp_place(_p(w), ctypes.c_int(D), ctypes.c_int(pool_size), _p(res["order"]),
                                      _p(res["pool_of_seq"]), _p(res["pool_load"])), "oracle_vrsp_place")
     return res
+
+
+def tap_place(f, q_home, v_qo, kv_off, kv_grp, v_g, resident, n_workers, tau_num=3, tau_den=100):
+    """Algorithm 2 on explicit tile / KV-group tables -> dict(sigma, loads, C, comm_total)."""
+    f = _arr(f, np.int64); q_home = _arr(q_home, np.int32); v_qo = _arr(v_qo, np.int64)
+    kv_off = _arr(kv_off, np.int32); kv_grp = _arr(kv_grp if len(kv_grp) else [0], np.int32)
+    v_g = _arr(v_g if len(v_g) else [0], np.int64); resident = _arr(resident if len(resident) else [-1], np.int32)
+    NT, NG, W = len(f), len(v_g), n_workers
+    res = dict(sigma=np.empty(NT, np.int32), loads=np.empty(W, np.int64), C=np.empty((W, NG), np.uint8))
+    total = ctypes.c_int64(0)
+    _check(_load().oracle_tap_place(ctypes.c_int64(NT), ctypes.c_int(W), ctypes.c_int64(NG), _p(f), _p(q_home), _p(v_qo),
+                                    _p(kv_off), _p(kv_grp), _p(v_g), _p(resident), ctypes.c_int(tau_num),
+                                    ctypes.c_int(tau_den), _p(res["sigma"]), _p(res["loads"]), _p(res["C"]),
+                                    ctypes.byref(total)), "oracle_tap_place")
+    res["comm_total"] = int(total.value)
+    return res
+
+
+def tap_layout(cu, seq_off, cp, block, n_shards, hq, hkv, d):
+    """Tile and KV-group tables of a pool for Algorithm 2 (see oracle_tap_layout)."""
+    cu = _arr(cu, np.int32); so = _arr(seq_off, np.int32)
+    n, P = len(cu) - 1, len(so) - 1
+    lib = _load()
+    lib.oracle_tap_num_tiles.restype = ctypes.c_int64
+    NT = int(lib.oracle_tap_num_tiles(_p(so), ctypes.c_int(P), ctypes.c_int(block), ctypes.c_int(n_shards)))
+    res = dict(f=np.empty(NT, np.int64), q_home=np.empty(NT, np.int32), v_qo=np.empty(NT, np.int64),
+               kv_off=np.empty(NT + 1, np.int32), kv_grp=np.empty(NT + n * n_shards + 1, np.int32),
+               v_g=np.empty(n * n_shards, np.int64), resident=np.empty(n * n_shards, np.int32))
+    _check(lib.oracle_tap_layout(_p(cu), ctypes.c_int(n), _p(so), ctypes.c_int(P), ctypes.c_int(cp), ctypes.c_int(block),
+                                 ctypes.c_int(n_shards), ctypes.c_int(hq), ctypes.c_int(hkv), ctypes.c_int(d),
+                                 _p(res["f"]), _p(res["q_home"]), _p(res["v_qo"]), _p(res["kv_off"]), _p(res["kv_grp"]),
+                                 _p(res["v_g"]), _p(res["resident"])), "oracle_tap_layout")
+    res["kv_grp"] = res["kv_grp"][:res["kv_off"][-1]].copy()
+    res["n_workers"] = P * cp
+    return res
+
+
+def tap_exchange(cu, seq_off, cp, n_shards, hkv, d, sigma, q_home, v_qo, C, resident):
+    """Forward and backward send-byte matrices [src, dst] implied by an assignment."""
+    cu = _arr(cu, np.int32); so = _arr(seq_off, np.int32)
+    n, P = len(cu) - 1, len(so) - 1
+    W = P * cp
+    sigma = _arr(sigma, np.int32); q_home = _arr(q_home, np.int32); v_qo = _arr(v_qo, np.int64)
+    C = np.ascontiguousarray(C, dtype=np.uint8); resident = _arr(resident, np.int32)
+    fwd = np.empty((W, W), np.int64); bwd = np.empty((W, W), np.int64)
+    _check(_load().oracle_tap_exchange(_p(cu), ctypes.c_int(n), _p(so), ctypes.c_int(P), ctypes.c_int(cp),
+                                       ctypes.c_int(n_shards), ctypes.c_int(hkv), ctypes.c_int(d),
+                                       ctypes.c_int64(len(sigma)), _p(sigma), _p(q_home), _p(v_qo), _p(C), _p(resident),
+                                       _p(fwd), _p(bwd)), "oracle_tap_exchange")
+    return fwd, bwd

@@ -270,3 +270,180 @@ int oracle_vrsp_place(const int64_t* work, int D, int P, int32_t* order /*[D]*/,
     free(keys); free(heap); free(fill);
     return 0;
 }
+
+/* ------------------------------------------------------------------------------------
+ * Communication-aware SH-Tile placement (Section 4.3.2, Algorithm 2, Eq. 8) in the
+ * algorithm's order and notation.
+ *   tiles t with estimated work f_t, Q-home q(t), Q + output volume V_Q(t) + V_O(t) and the set
+ *   K(t) of KV groups they reference (CSR lists); KV groups g with volume V_g; workers r with load
+ *   L_r and the set C_r of KV groups already selected for them.
+ *   C       = (1 + tau) * sum(f) / |W|.  tau = tau_num / tau_den, and "L_r + f_t <= C" is tested in
+ *             integers as  tau_den * |W| * (L_r + f_t) <= (tau_den + tau_num) * sum(f).
+ *   order   = tiles by decreasing f, then tile id.
+ *   Delta_comm(t, r) = sum of V_g over g in K(t) \ C_r, plus V_Q(t) + V_O(t) if r != q(t).
+ *   F       = workers with L_r + f_t <= C; if F is not empty the tile goes to
+ *             argmin over F of (Delta_comm, L_r, r), else to argmin over W of (L_r, Delta_comm, r).
+ *   then    L_r* += f_t and C_r* gains K(t).
+ * C_r starts as the groups worker r already holds in full (resident[g] == r): the paper charges no
+ * transfer for resident groups (Section 4.3.3) and does not say how C_r is initialised.
+ * Outputs: sigma, L, the final C (W x NG bytes, 1 = selected or resident) and the summed
+ * Delta_comm of the choices taken.
+ * ------------------------------------------------------------------------------------ */
+int oracle_tap_place(int64_t NT, int W, int64_t NG, const int64_t* f, const int32_t* q_home, const int64_t* v_qo,
+                     const int32_t* kv_off, const int32_t* kv_grp, const int64_t* v_g, const int32_t* resident,
+                     int tau_num, int tau_den, int32_t* sigma, int64_t* L, uint8_t* C, int64_t* comm_total) {
+    if (NT < 0 || W <= 0 || NG < 0 || tau_num < 0 || tau_den <= 0) return -1;
+    int64_t sum_f = 0;
+    for (int64_t t = 0; t < NT; ++t) { if (f[t] < 0) return -1; sum_f += f[t]; }
+    if (sum_f > (INT64_MAX / ((int64_t)(tau_den + tau_num) * 2)) / W) return -3;  /* the integer test would overflow */
+    tile_key* keys = (tile_key*)malloc(sizeof(tile_key) * (size_t)(NT ? NT : 1));
+    if (!keys) return -2;
+    for (int64_t t = 0; t < NT; ++t) { keys[t].w = f[t]; keys[t].id = (int32_t)t; }
+    qsort(keys, (size_t)NT, sizeof(tile_key), cmp_tiles);
+    for (int r = 0; r < W; ++r) L[r] = 0;
+    for (int r = 0; r < W; ++r)
+        for (int64_t g = 0; g < NG; ++g) C[(int64_t)r * NG + g] = resident[g] == r ? 1 : 0;
+    *comm_total = 0;
+    for (int64_t x = 0; x < NT; ++x) {
+        const int32_t t = keys[x].id;
+        int best = -1;
+        int64_t best_d = 0;
+        int have_feasible = 0;
+        for (int pass = 0; pass < 2 && best < 0; ++pass) {   /* pass 0: over F; pass 1: over W when F is empty */
+            for (int r = 0; r < W; ++r) {
+                const int feasible = (int64_t)tau_den * W * (L[r] + f[t]) <= (int64_t)(tau_den + tau_num) * sum_f;
+                if (pass == 0 && !feasible) continue;
+                int64_t delta = r != q_home[t] ? v_qo[t] : 0;
+                for (int32_t e = kv_off[t]; e < kv_off[t + 1]; ++e)
+                    if (!C[(int64_t)r * NG + kv_grp[e]]) delta += v_g[kv_grp[e]];
+                int better;
+                if (best < 0) better = 1;
+                else if (pass == 0) better = delta < best_d || (delta == best_d && L[r] < L[best]);
+                else better = L[r] < L[best] || (L[r] == L[best] && delta < best_d);
+                if (better) { best = r; best_d = delta; }   /* equal keys keep the lower r */
+            }
+            if (pass == 0 && best >= 0) have_feasible = 1;
+        }
+        (void)have_feasible;
+        sigma[t] = best;
+        L[best] += f[t];
+        for (int32_t e = kv_off[t]; e < kv_off[t + 1]; ++e) C[(int64_t)best * NG + kv_grp[e]] = 1;
+        *comm_total += best_d;
+    }
+    free(keys);
+    return 0;
+}
+
+/* ------------------------------------------------------------------------------------
+ * Tables of a sequence pool for Algorithm 2 (Sections 4.1, 4.3.1) and the exchange volumes that an
+ * assignment implies (Section 4.3.3).
+ *
+ * The pool holds P packed sequences; sequence s occupies tokens [seq_off[s], seq_off[s+1]) of the
+ * pool's sample list cu[0..n] and belongs to the CP workers s*CP .. s*CP+CP-1.  The paper leaves the
+ * split of a sequence over its CP group open; here worker c of the group holds the c-th run of
+ * ceil(L_s / CP) consecutive tokens.
+ *   blocks   every sequence is cut at multiples of B from its own start; tile id = block * H + h
+ *            with blocks numbered sequence by sequence                                    (Eq. 5)
+ *   f        causal pairs of the block, Eq. 6 without the common factor
+ *   q(t)     the worker that holds the block's first token
+ *   V_Q = V_O = tokens * (hq / H) * d * 2 bytes (bf16)
+ *   K(t)     the samples with a token in the block, on head shard h; group id g = j * H + h (Eq. 7)
+ *   V_g      K and V of the whole sample on the shard: 2 * len_j * kv_heads_per_shard * d * 2 bytes,
+ *            kv_heads_per_shard = hkv / H if H <= hkv, else 1 (shards share a replicated kv head)
+ *   resident the worker that holds every token of sample j, or -1
+ * ------------------------------------------------------------------------------------ */
+static int tap_owner(const int32_t* seq_off, int s, int CP, int64_t tok) {
+    const int64_t len = seq_off[s + 1] - seq_off[s];
+    const int64_t run = (len + CP - 1) / CP;
+    return s * CP + (int)((tok - seq_off[s]) / (run > 0 ? run : 1));
+}
+
+int64_t oracle_tap_num_tiles(const int32_t* seq_off, int P, int B, int H) {
+    int64_t nb = 0;
+    for (int s = 0; s < P; ++s) nb += ((int64_t)seq_off[s + 1] - seq_off[s] + B - 1) / B;
+    return nb * H;
+}
+
+int oracle_tap_layout(const int32_t* cu, int n, const int32_t* seq_off, int P, int CP, int B, int H, int hq, int hkv,
+                      int d, int64_t* f, int32_t* q_home, int64_t* v_qo, int32_t* kv_off, int32_t* kv_grp /*[<= NB + n] * H*/,
+                      int64_t* v_g /*[n*H]*/, int32_t* resident /*[n*H]*/) {
+    if (!cu || !seq_off || n <= 0 || P <= 0 || CP <= 0 || B <= 0 || H <= 0 || hq % H != 0) return -1;
+    if (!((H <= hkv && hkv % H == 0) || (H > hkv && H % hkv == 0))) return -1;
+    const int kvps = H <= hkv ? hkv / H : 1;
+    for (int j = 0; j < n; ++j) {
+        const int64_t a = cu[j], e = cu[j + 1];
+        int s = 0;
+        while (s + 1 < P && seq_off[s + 1] <= a && !(a == e && seq_off[s + 1] > a)) ++s;  /* sequence of the sample */
+        int res = -1;
+        if (e > a) {
+            const int first = tap_owner(seq_off, s, CP, a), last = tap_owner(seq_off, s, CP, e - 1);
+            res = first == last ? first : -1;
+        }
+        for (int h = 0; h < H; ++h) {
+            v_g[(int64_t)j * H + h] = 2 * (e - a) * kvps * d * 2;
+            resident[(int64_t)j * H + h] = res;
+        }
+    }
+    int64_t blk = 0;
+    int32_t refs = 0;
+    for (int s = 0; s < P; ++s) {
+        for (int64_t q0 = seq_off[s]; q0 < seq_off[s + 1]; q0 += B, ++blk) {
+            const int64_t q1 = q0 + B < seq_off[s + 1] ? q0 + B : seq_off[s + 1];
+            int64_t w = 0;
+            for (int j = 0; j < n; ++j) {
+                const int64_t lo = q0 > cu[j] ? q0 : cu[j], hi = q1 < cu[j + 1] ? q1 : cu[j + 1];
+                for (int64_t g = lo; g < hi; ++g) w += g - cu[j] + 1;
+            }
+            for (int h = 0; h < H; ++h) {
+                const int64_t t = blk * H + h;
+                f[t] = w;
+                q_home[t] = tap_owner(seq_off, s, CP, q0);
+                v_qo[t] = 2 * ((q1 - q0) * (hq / H) * d * 2);
+                kv_off[t] = refs;
+                for (int j = 0; j < n; ++j) {
+                    const int64_t lo = q0 > cu[j] ? q0 : cu[j], hi = q1 < cu[j + 1] ? q1 : cu[j + 1];
+                    if (lo < hi) kv_grp[refs++] = j * H + h;
+                }
+            }
+        }
+    }
+    kv_off[blk * H] = refs;
+    return 0;
+}
+
+/* Bytes every worker sends to every other in the forward pass under assignment sigma with final
+ * residency C (from oracle_tap_place): a KV group selected for destination r and not resident there
+ * is fetched once per destination, each token run from the worker that holds it (runs already at r
+ * do not move); a tile away from its Q-home has its Q sent there and its output sent back.  The
+ * backward pass moves dO along the Q path, dQ along the output path and dK/dV back along the KV
+ * paths, so its matrix is the forward's KV part transposed plus the same Q / output part. */
+int oracle_tap_exchange(const int32_t* cu, int n, const int32_t* seq_off, int P, int CP, int H, int hkv, int d,
+                        int64_t NT, const int32_t* sigma, const int32_t* q_home, const int64_t* v_qo,
+                        const uint8_t* C, const int32_t* resident, int64_t* fwd /*[W*W] src-major*/, int64_t* bwd) {
+    const int W = P * CP;
+    const int kvps = H <= hkv ? hkv / H : 1;
+    for (int64_t i = 0; i < (int64_t)W * W; ++i) fwd[i] = bwd[i] = 0;
+    for (int r = 0; r < W; ++r)
+        for (int j = 0; j < n; ++j)
+            for (int h = 0; h < H; ++h) {
+                const int64_t g = (int64_t)j * H + h;
+                if (!C[(int64_t)r * n * H + g] || resident[g] == r) continue;
+                int s = 0;
+                while (s + 1 < P && seq_off[s + 1] <= cu[j]) ++s;
+                for (int64_t tok = cu[j]; tok < cu[j + 1]; ++tok) {
+                    const int w = tap_owner(seq_off, s, CP, tok);
+                    if (w == r) continue;
+                    fwd[(int64_t)w * W + r] += 2 * (int64_t)kvps * d * 2;
+                    bwd[(int64_t)r * W + w] += 2 * (int64_t)kvps * d * 2;
+                }
+            }
+    for (int64_t t = 0; t < NT; ++t) {
+        const int q = q_home[t], r = sigma[t];
+        if (q == r) continue;
+        fwd[(int64_t)q * W + r] += v_qo[t] / 2;   /* Q out */
+        fwd[(int64_t)r * W + q] += v_qo[t] / 2;   /* output back */
+        bwd[(int64_t)q * W + r] += v_qo[t] / 2;   /* dO along the Q path */
+        bwd[(int64_t)r * W + q] += v_qo[t] / 2;   /* dQ along the output path */
+    }
+    return 0;
+}
