@@ -220,6 +220,49 @@ int libra_vrsp_work(const int32_t* sample_offsets_dev, const int32_t* seq_first_
 int libra_vrsp_place(const int64_t* work_dev, int n_sequences, int pool_size, int32_t* order_dev,
                      int32_t* pool_of_seq_dev, int64_t* pool_load_dev, int32_t* scratch_dev, void* stream);
 
+/* ---- Tiled Attention Pooling across workers (Section 4.3: Eq. 5-8, Algorithm 2, exchange plan) ----
+ * Plans one sequence pool: P packed sequences, each held by its own group of CP workers, W = P * CP
+ * workers in all.  Everything runs in device kernels on `stream`; the paper runs it on CPU cores.
+ * This is the planning half only: the transfers it describes and the head-chunk pipeline that
+ * overlaps them with attention need more than one GPU and are not part of this library.
+ *
+ * Layout (a reading; the paper does not fix how a sequence is split over its CP group): sequence s
+ * is tokens [seq_offsets[s], seq_offsets[s+1]) of the pool's sample list (a sequence boundary is
+ * a sample boundary); worker s*CP + c holds the c-th run of ceil(L_s / CP) consecutive tokens.
+ *   tiles   : every sequence is cut at multiples of `block` tokens from its own start; blocks are
+ *             numbered sequence by sequence; tile id = block * n_shards + h            (Eq. 5)
+ *   f       : causal pairs of the block                                               (Eq. 6)
+ *   q(t)    : the worker holding the block's first token;
+ *             V_Q = V_O = tokens * (hq / n_shards) * head_dim * 2 bytes
+ *   K(t)    : the samples with a token in the block, on shard h                         (Eq. 7)
+ *   V_g     : 2 * len * kv_heads_per_shard * head_dim * 2 bytes, kv_heads_per_shard = hkv / n_shards,
+ *             or 1 when n_shards > hkv (shards then share a replicated kv head)
+ *   C_r     : starts as the groups worker r holds in full (resident groups need no transfer)
+ *   placement: Algorithm 2 with tau = tau_num / tau_den; "L_r + f <= C" is evaluated exactly as
+ *             tau_den * W * (L_r + f) <= (tau_den + tau_num) * sum(f)
+ * Outputs (device): sigma_dev int32[NT] destination worker of every tile; loads_dev int64[W];
+ * fwd_bytes_dev / bwd_bytes_dev int64[W * W], bytes worker src sends to worker dst ([src * W + dst]) in
+ * the forward / backward pass: each KV group selected for a destination and not resident there is
+ * fetched once per destination, run by run from the workers that hold it (runs already there do
+ * not move), a tile away from its Q-home has Q sent out and the output sent back; backward: dO along
+ * the Q path, dQ along the output path, dK/dV back along the KV paths.  comm_total_dev int64[1]: the
+ * summed Delta_comm (Eq. 8) of the choices taken.  status_dev int[1]: 0 or LIBRA_ERR_OVERFLOW.
+ * seq_offsets_host is a HOST array of n_sequences + 1 entries (read before the call returns).
+ * Scratch comes from the stream-ordered allocator and is released on `stream`.
+ * Errors: INVALID_ARG, UNSUPPORTED (W > 1024, more than 65536 blocks), CUDA. */
+typedef struct {
+    int cp;                 /* workers per packed sequence */
+    int block;              /* B, tokens per block */
+    int n_shards;           /* H head shards; divides hq; divides or is a multiple of hkv */
+    int hq, hkv, head_dim;
+    int tau_num, tau_den;   /* soft cap slack, the paper uses 3 / 100 */
+} libra_tap_opts;
+int64_t libra_tap_num_tiles(const int32_t* seq_offsets_host, int n_sequences, int block, int n_shards);
+int libra_tap_plan(const int32_t* cu_seqlens_dev, int n_samples, const int32_t* seq_offsets_host,
+                   int n_sequences, const libra_tap_opts* opts, int32_t* sigma_dev, int64_t* loads_dev,
+                   int64_t* fwd_bytes_dev, int64_t* bwd_bytes_dev, int64_t* comm_total_dev,
+                   int* status_dev, void* stream);
+
 /* ---- instrumentation -------------------------------------------------------------------
  * Per-CTA busy time of the most recent launch of kernel `which` (LIBRA_KERNEL_*) that used this
  * plan: nanoseconds between the CTA starting and finishing its tile list, read with the GPU's

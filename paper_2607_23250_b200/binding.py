@@ -229,3 +229,35 @@ def libra_vrsp_place(work: torch.Tensor, pool_size: int, stream=None):
     _check(_lib.libra_vrsp_place(_ptr(work), ctypes.c_int(D), ctypes.c_int(pool_size), _ptr(order), _ptr(pool_of_seq),
                                  _ptr(pool_load), _ptr(scratch), _stream(stream)), "libra_vrsp_place")
     return dict(order=order, pool_of_seq=pool_of_seq, pool_load=pool_load)
+
+
+class TapOpts(ctypes.Structure):
+    _fields_ = [("cp", ctypes.c_int), ("block", ctypes.c_int), ("n_shards", ctypes.c_int), ("hq", ctypes.c_int),
+                ("hkv", ctypes.c_int), ("head_dim", ctypes.c_int), ("tau_num", ctypes.c_int), ("tau_den", ctypes.c_int)]
+
+
+_lib.libra_tap_num_tiles.restype = ctypes.c_int64
+
+
+def libra_tap_plan(cu_seqlens: torch.Tensor, seq_offsets, cp: int, block: int, n_shards: int, hq: int, hkv: int,
+                   head_dim: int, tau_num: int = 3, tau_den: int = 100, stream=None):
+    """Tiles, Algorithm 2 and the exchange volumes of one pool -> dict of device tensors
+    (sigma, loads, fwd_bytes [W, W], bwd_bytes [W, W], comm_total, status)."""
+    assert cu_seqlens.is_cuda and cu_seqlens.dtype == torch.int32 and cu_seqlens.is_contiguous()
+    so = (ctypes.c_int32 * len(seq_offsets))(*[int(x) for x in seq_offsets])
+    P = len(seq_offsets) - 1
+    W = P * cp
+    NT = int(_lib.libra_tap_num_tiles(so, ctypes.c_int(P), ctypes.c_int(block), ctypes.c_int(n_shards)))
+    if NT <= 0:
+        raise RuntimeError("libra_tap_num_tiles: bad arguments")
+    dev = cu_seqlens.device
+    out = dict(sigma=torch.empty(NT, dtype=torch.int32, device=dev), loads=torch.empty(W, dtype=torch.int64, device=dev),
+               fwd_bytes=torch.empty((W, W), dtype=torch.int64, device=dev),
+               bwd_bytes=torch.empty((W, W), dtype=torch.int64, device=dev),
+               comm_total=torch.empty(1, dtype=torch.int64, device=dev), status=torch.empty(1, dtype=torch.int32, device=dev))
+    opts = TapOpts(cp, block, n_shards, hq, hkv, head_dim, tau_num, tau_den)
+    _check(_lib.libra_tap_plan(_ptr(cu_seqlens), ctypes.c_int(cu_seqlens.numel() - 1), so, ctypes.c_int(P),
+                               ctypes.byref(opts), _ptr(out["sigma"]), _ptr(out["loads"]), _ptr(out["fwd_bytes"]),
+                               _ptr(out["bwd_bytes"]), _ptr(out["comm_total"]), _ptr(out["status"]), _stream(stream)),
+           "libra_tap_plan")
+    return out
