@@ -533,6 +533,7 @@ static int set_smem(Kernel k, int bytes) {
 
 template <int D>
 static int launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tdo,
+                      const CUtensorMap& tdq,
                       const DkvParams& pa, int Wa, const DqParams& pb, int Wb, libra_plan_t* mp, cudaStream_t s) {
     static bool configured = false;
     if (!configured) {
@@ -544,7 +545,7 @@ static int launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtens
     if (mp->timing) cudaEventRecord(mp->ev[1][0], s);
     k_attn_bwd_dkdv<D><<<Wa, kBwdThreads, DkvSmem<D>::kBytes, s>>>(tq, tk, tv, tdo, pa);
     if (mp->timing) { cudaEventRecord(mp->ev[1][1], s); mp->ev_valid[1] = 1; cudaEventRecord(mp->ev[2][0], s); }
-    k_attn_bwd_dq<D><<<Wb, kDqThreads, DqSmem<D>::kBytes, s>>>(tq, tk, tv, tdo, pb);
+    k_attn_bwd_dq<D><<<Wb, kDqThreads, DqSmem<D>::kBytes, s>>>(tq, tk, tv, tdo, tdq, pb);
     if (mp->timing) { cudaEventRecord(mp->ev[2][1], s); mp->ev_valid[2] = 1; }
     count_launch(2);
     return cudaGetLastError() == cudaSuccess ? LIBRA_OK : LIBRA_ERR_CUDA;
@@ -599,11 +600,12 @@ extern "C" int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const v
     float* lse2 = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(workspace_dev) + ws.stat_bytes);
     cudaStream_t s = (cudaStream_t)stream;
 
-    CUtensorMap tq, tk, tv, tdo;
+    CUtensorMap tq, tk, tv, tdo, tdq;
     int rc = make_thd_map(&tq, q_dev, T, dims->hq, D, kBlk);
     if (rc == LIBRA_OK) rc = make_thd_map(&tk, k_dev, T, dims->hkv, D, kBlk);
     if (rc == LIBRA_OK) rc = make_thd_map(&tv, v_dev, T, dims->hkv, D, kBlk);
     if (rc == LIBRA_OK) rc = make_thd_map(&tdo, dout_dev, T, dims->hq, D, kBlk);
+    if (rc == LIBRA_OK) rc = make_thd_map(&tdq, dq_dev, T, dims->hq, D, kBlk);
     if (rc != LIBRA_OK) return rc;
 
     {
@@ -651,6 +653,6 @@ extern "C" int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const v
     pb.status = plan->d_status + 2;
     pb.busy = dq_dir.d_busy2;
     libra_plan_t* mp = const_cast<libra_plan_t*>(plan);
-    return D == 128 ? launch_bwd<128>(tq, tk, tv, tdo, pa, dkv_dir.W, pb, dq_dir.W, mp, s)
-                    : launch_bwd<64>(tq, tk, tv, tdo, pa, dkv_dir.W, pb, dq_dir.W, mp, s);
+    return D == 128 ? launch_bwd<128>(tq, tk, tv, tdo, tdq, pa, dkv_dir.W, pb, dq_dir.W, mp, s)
+                    : launch_bwd<64>(tq, tk, tv, tdo, tdq, pa, dkv_dir.W, pb, dq_dir.W, mp, s);
 }

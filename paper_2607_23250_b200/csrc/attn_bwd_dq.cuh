@@ -27,7 +27,7 @@ constexpr int kDqCW = 128 / kDqGroups;            // S / dP columns per compute 
 // registers to the compute groups with setmaxnreg.
 constexpr int kDqThreads = (4 * kDqGroups + 4) * 32;
 constexpr int kDqRegsCompute = 104, kDqRegsOther = 40;  // from 96 at launch: 4 x 128 x 8 asked, 128 x 56 released
-constexpr int kDqTmaWarp = 4 * kDqGroups, kDqMmaWarp = 4 * kDqGroups + 1;
+constexpr int kDqTmaWarp = 4 * kDqGroups, kDqMmaWarp = 4 * kDqGroups + 1, kDqStoreWarp = 4 * kDqGroups + 2;
 
 template <int D>
 struct DqSmem {
@@ -41,8 +41,8 @@ struct DqSmem {
     static constexpr int kVOff = kKOff + kKStages * kTileBytes;
     static constexpr int kBarOff = kVOff + kVStages * kTileBytes;
     // q_full, q_empty, do_full, do_empty, k_full[3], k_empty[3], v_full[2], v_empty[2], qt_ready,
-    // s_full, s_free, dp_full, ds_ready, dq_full, dot_ready, dq_empty
-    static constexpr int kNumBars = 22;
+    // s_full, s_free, dp_full, ds_ready, dq_full, dot_ready, dq_empty, dq_staged
+    static constexpr int kNumBars = 23;
     static constexpr int kMiscOff = kBarOff + kNumBars * 8;
     static constexpr int kBytes = kMiscOff + 16;
     static_assert(kBytes <= kSmemMax, "exceeds the shared memory of an sm_100 CTA");
@@ -101,7 +101,8 @@ struct DqUnitIter {
 template <int D>
 __global__ void __launch_bounds__(kDqThreads, 1)
 k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-              const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do, const DqParams p) {
+              const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
+              const __grid_constant__ CUtensorMap tm_dq, const DqParams p) {
     using L = DqSmem<D>;
     extern __shared__ __align__(1024) uint8_t smem[];
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBarOff);
@@ -121,6 +122,7 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     uint64_t* bar_dqfull = bars + 19;
     uint64_t* bar_dotready = bars + 20;
     uint64_t* bar_dqempty = bars + 21;
+    uint64_t* bar_dqstaged = bars + 22;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::kMiscOff);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kMiscOff + 4);
 
@@ -134,7 +136,7 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     }
     if (threadIdx.x == 0) {
         mbar_init(bar_qfull, 1);
-        mbar_init(bar_qempty, 64 * kDqGroups);   // the groups that stage Q
+        mbar_init(bar_qempty, 1);                // the thread that stores dQ through the Q tile
         mbar_init(bar_dofull, 1);
         mbar_init(bar_doempty, 64 * kDqGroups);  // the groups that stage dO
         for (int s = 0; s < L::kKStages; ++s) { mbar_init(&bar_kfull[s], 1); mbar_init(&bar_kempty[s], 1); }
@@ -142,6 +144,7 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         mbar_init(bar_qtready, 64 * kDqGroups);   // the groups that stage Q
         mbar_init(bar_dotready, 64 * kDqGroups);  // the groups that stage dO
         mbar_init(bar_dqempty, 128 * kDqGroups);
+        mbar_init(bar_dqstaged, 128 * kDqGroups);
         mbar_init(bar_sfull, 1);
         mbar_init(bar_sfree, 128 * kDqGroups);
         mbar_init(bar_dpfull, 1);
@@ -160,6 +163,7 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         prefetch_tmap(&tm_k);
         prefetch_tmap(&tm_v);
         prefetch_tmap(&tm_do);
+        prefetch_tmap(&tm_dq);
     }
     tc_fence_before();
     __syncthreads();
@@ -175,8 +179,40 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
 
     // All roles walk the same sequence of sub-blocks: (tile, sub-block of 128 rows, head of the shard).
     // A sub-block past the end of the pool is skipped by every role.
-    if (warp > kDqMmaWarp) {
+    if (warp > kDqStoreWarp) {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kDqRegsOther));
+    } else if (warp == kDqStoreWarp) {
+        // ---------------- dQ store ----------------
+        // The compute groups leave a unit's dQ tile (bf16, the swizzled layout of the tensor map) in the Q tile
+        // of shared memory, which is idle between the copy of the next unit's Q into TMEM and the load of the
+        // one after; one thread writes it out with bulk tensor stores.  Rows stored straight from registers
+        // (one row per thread, rows 2*hq*D bytes apart) touch 32 cache lines per instruction and took ~3000
+        // cycles per unit.
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kDqRegsOther));
+        if (elect_one()) {
+            DqUnitIter units(p, tile_begin, tile_end, heads_per_shard);
+            DqUnit u = units.next();
+            uint32_t cnt = 0;
+            bool ok = true;
+            if (u.valid) {  // first unit: its Q rows have been copied to TMEM, the tile may be reloaded
+                ok = mbar_wait(bar_dqstaged, 0, abort_flag);
+                cnt = 1;
+                if (ok) mbar_arrive(bar_qempty);
+            }
+            while (u.valid && ok) {
+                ok = mbar_wait(bar_dqstaged, cnt & 1, abort_flag);
+                ++cnt;
+                if (!ok) break;
+                for (int half = 0; half < D / 64; ++half)
+                    tma_store_3d(&tm_dq, smem + L::kQOff + half * L::kHalfBytes, half * 64, u.h, (int)u.q0);
+                tma_store_commit();
+                tma_store_wait_read();
+                mbar_arrive(bar_qempty);
+                u = units.next();
+            }
+            asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");  // all of this thread's stores have landed
+        }
+        __syncwarp();
     } else if (warp == kDqTmaWarp) {
         // ---------------- TMA producer ----------------
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kDqRegsOther));
@@ -194,23 +230,26 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             };
             DqUnitIter units(p, tile_begin, tile_end, heads_per_shard);
             DqUnit u = units.next();
+            // Q and dO of unit `un`, whose tiles go through phase `cnt` of their barriers.  The shared-memory
+            // copies are free again as soon as the compute groups have moved the previous unit's rows into
+            // TMEM, which happens at the end of the unit before it: the next unit's Q and dO (first touches,
+            // DRAM latency) can therefore be requested a whole unit ahead.
+            auto load_q_do = [&](const DqUnit& un, uint32_t cnt) -> bool {
+                if (!mbar_wait(bar_qempty, (cnt & 1) ^ 1, abort_flag)) return false;
+                mbar_arrive_expect_tx(bar_qfull, L::kTileBytes);
+                for (int half = 0; half < D / 64; ++half)
+                    tma_load_3d(smem + L::kQOff + half * L::kHalfBytes, &tm_q, bar_qfull, half * 64, un.h, (int)un.q0);
+                if (!mbar_wait(bar_doempty, (cnt & 1) ^ 1, abort_flag)) return false;
+                mbar_arrive_expect_tx(bar_dofull, L::kTileBytes);
+                for (int half = 0; half < D / 64; ++half)
+                    tma_load_3d(smem + L::kDoOff + half * L::kHalfBytes, &tm_do, bar_dofull, half * 64, un.h, (int)un.q0);
+                return true;
+            };
+            if (u.valid) ok = load_q_do(u, 0);
             while (u.valid && ok) {
                 const DqUnit nx = units.next();
                 const int h = u.h, kvh = h / G, lo = u.lo, hi = u.hi;
-                ok = mbar_wait(bar_qempty, (ucnt & 1) ^ 1, abort_flag);
-                if (!ok) break;
-                {
-                    mbar_arrive_expect_tx(bar_qfull, L::kTileBytes);
-                    for (int half = 0; half < D / 64; ++half)
-                        tma_load_3d(smem + L::kQOff + half * L::kHalfBytes, &tm_q, bar_qfull, half * 64, h, (int)u.q0);
-                }
-                ok = mbar_wait(bar_doempty, (ucnt & 1) ^ 1, abort_flag);
-                if (!ok) break;
-                {
-                    mbar_arrive_expect_tx(bar_dofull, L::kTileBytes);
-                    for (int half = 0; half < D / 64; ++half)
-                        tma_load_3d(smem + L::kDoOff + half * L::kHalfBytes, &tm_do, bar_dofull, half * 64, h, (int)u.q0);
-                }
+                const int j_q = lo + 1 < hi ? lo + 1 : hi;  // after this block's K/V the next unit's Q / dO are requested
                 ++ucnt;
                 const int j_next = hi - kAhead > lo ? hi - kAhead : lo;  // where the next unit's first tiles are requested
                 for (int j = lo; j <= hi && ok; ++j) {
@@ -244,6 +283,12 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                                         &bar_vfull[vs], half * 64, kvh, j * kBlk);
                     }
                     ++vcnt;
+                    if (j == j_q && nx.valid) {
+                        ok = load_q_do(nx, ucnt);
+                        if (!ok) break;
+                        if (kAhead == 0)   // pull the next unit's first K / V blocks into L2 meanwhile
+                            for (int jj = nx.lo; jj <= nx.hi && jj < nx.lo + 2; ++jj) prefetch_kv(nx.h / G, jj);
+                    }
                 }
                 u = nx;
             }
@@ -403,7 +448,7 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 tmem_st32(t_dst, w);
                 tmem_st_wait();
             }
-            mbar_arrive(st_op == 0 ? bar_qempty : bar_doempty);  // the smem tile may be reloaded
+            if (st_op == 1) mbar_arrive(bar_doempty);  // the dO tile may be reloaded (the Q tile: see the dQ store)
             tc_fence_before();
             mbar_arrive(st_op == 0 ? bar_qtready : bar_dotready);
             return true;
@@ -431,12 +476,13 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         if (u.valid) {
             cx = load_ctx(u);
             ok = stage(0);
+            mbar_arrive(bar_dqstaged);   // phase 0: the store thread frees the Q tile once every row has been read
         }
         while (u.valid && ok) {
             const DqUnit nx = units.next();
             RowCtx cx_next{};
             if (nx.valid) cx_next = load_ctx(nx);
-            const int lo = u.lo, hi = u.hi, h = u.h;
+            const int lo = u.lo, hi = u.hi;
             const int64_t row = u.q0 + r;
             const bool row_ok = cx.row_ok;
             const int kstart = cx.kstart, max_kstart = cx.max_kstart;
@@ -510,27 +556,30 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             if (!ok) break;
             TRACE(28)
             tc_fence_after();
-            constexpr int kCols = D / kDqGroups;
-            constexpr int kChunk = kCols < 32 ? kCols : 32;
+            constexpr int kCols = D / kDqGroups;   // this group's dQ columns: kCols * 2 bytes of every row
             const uint32_t t_dq = tmem_base + lane_addr + kColDQ + c * kCols;
-            __nv_bfloat16* gdst = p.dq + ((size_t)row * p.hq + h) * D + c * kCols;
+            uint32_t v[kCols];
+            if constexpr (kCols == 32) tmem_ld32(t_dq, v); else tmem_ld16(t_dq, v);
+            tmem_ld_wait();
+            TRACE(30)
+            // The Q tile still holds the next unit's Q until every row of it has been copied to TMEM.
+            if (nx.valid) ok = mbar_wait(bar_qtready, (ucnt + 1) & 1, abort_flag);
+            if (!ok) break;
+            {
+                uint8_t* dst = smem + L::kQOff + ((c * kCols) / 64) * L::kHalfBytes + r * 128;
+                const int chunk0 = ((c * kCols) % 64) / 8;  // first 16-byte chunk of this group's columns
 #pragma unroll
-            for (int cc = 0; cc < kCols; cc += kChunk) {
-                uint32_t v[kChunk];
-                if constexpr (kChunk == 32) tmem_ld32(t_dq + cc, v); else tmem_ld16(t_dq + cc, v);
-                tmem_ld_wait();
-                if (row_ok) {
-#pragma unroll
-                    for (int i = 0; i < kChunk; i += 8) {
-                        uint4 w;
-                        w.x = pack_bf16x2(__uint_as_float(v[i]) * p.scale, __uint_as_float(v[i + 1]) * p.scale);
-                        w.y = pack_bf16x2(__uint_as_float(v[i + 2]) * p.scale, __uint_as_float(v[i + 3]) * p.scale);
-                        w.z = pack_bf16x2(__uint_as_float(v[i + 4]) * p.scale, __uint_as_float(v[i + 5]) * p.scale);
-                        w.w = pack_bf16x2(__uint_as_float(v[i + 6]) * p.scale, __uint_as_float(v[i + 7]) * p.scale);
-                        *reinterpret_cast<uint4*>(gdst + cc + i) = w;
-                    }
+                for (int i = 0; i < kCols; i += 8) {
+                    uint4 w;
+                    w.x = pack_bf16x2(__uint_as_float(v[i]) * p.scale, __uint_as_float(v[i + 1]) * p.scale);
+                    w.y = pack_bf16x2(__uint_as_float(v[i + 2]) * p.scale, __uint_as_float(v[i + 3]) * p.scale);
+                    w.z = pack_bf16x2(__uint_as_float(v[i + 4]) * p.scale, __uint_as_float(v[i + 5]) * p.scale);
+                    w.w = pack_bf16x2(__uint_as_float(v[i + 6]) * p.scale, __uint_as_float(v[i + 7]) * p.scale);
+                    *reinterpret_cast<uint4*>(dst + (((chunk0 + i / 8) ^ (r & 7)) << 4)) = w;
                 }
             }
+            fence_proxy_async_smem();     // the bulk store reads these writes through the async proxy
+            mbar_arrive(bar_dqstaged);
             tc_fence_before();
             mbar_arrive(bar_dqempty);  // the next unit's first dQ MMA may overwrite the accumulator
             TRACE(29)
