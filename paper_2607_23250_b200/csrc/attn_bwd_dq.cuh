@@ -72,13 +72,15 @@ struct DqUnit {
 struct DqUnitIter {
     const DqParams& p;
     int idx, end, sub, hh, hps;
+    int t;  // cta_tiles[idx], fetched when idx moves so that the load has a unit's time to land
     __device__ DqUnitIter(const DqParams& p_, int begin, int end_, int heads_per_shard)
-        : p(p_), idx(begin), end(end_), sub(0), hh(0), hps(heads_per_shard) {}
+        : p(p_), idx(begin), end(end_), sub(0), hh(0), hps(heads_per_shard) {
+        t = idx < end ? p.cta_tiles[idx] : 0;
+    }
     __device__ DqUnit next() {
         DqUnit u;
         u.valid = false;
         while (idx < end) {
-            const int t = p.cta_tiles[idx];
             const int64_t q0 = (int64_t)(t / p.H) * (2 * kBlk) + sub * kBlk;
             const bool live = q0 < p.T;
             if (live) {
@@ -90,7 +92,11 @@ struct DqUnitIter {
             }
             if (!live || ++hh == hps) {
                 hh = 0;
-                if (++sub == 2) { sub = 0; ++idx; }
+                if (++sub == 2) {
+                    sub = 0;
+                    ++idx;
+                    t = idx < end ? p.cta_tiles[idx] : 0;
+                }
             }
             if (live) return u;
         }
