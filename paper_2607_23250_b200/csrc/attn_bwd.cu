@@ -23,7 +23,16 @@
 
 namespace libra {
 
-constexpr int kBwdThreads = 320;
+#ifndef LIBRA_DKV_GROUPS
+#define LIBRA_DKV_GROUPS 2
+#endif
+constexpr int kDkvGroups = LIBRA_DKV_GROUPS;            // compute warpgroups: each owns 128 / kDkvGroups query columns
+constexpr int kDkvCW = 128 / kDkvGroups;                // S^T / dP^T columns per compute thread
+constexpr int kDkvTmaWarp = 4 * kDkvGroups, kDkvMmaWarp = 4 * kDkvGroups + 1;
+// two groups: 10 warps at 168 registers; four groups: the producer / MMA warps get a warpgroup of their own
+// (two of its warps idle) and hand registers to the compute groups, as in the dQ kernel
+constexpr int kBwdThreads = kDkvGroups == 2 ? 320 : (4 * kDkvGroups + 4) * 32;
+constexpr int kDkvRegsCompute = 104, kDkvRegsOther = 40;
 constexpr int kBlk = 128;
 constexpr int kSmemMax = 232448;  // 227 KB per CTA on sm_100
 
@@ -137,20 +146,20 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             mbar_init(&bar_doempty[s], 1);
         }
         mbar_init(bar_sfull, 1);
-        mbar_init(bar_pready, 256);
+        mbar_init(bar_pready, 128 * kDkvGroups);
         mbar_init(bar_dpfull, 1);
-        mbar_init(bar_dsready, 256);
+        mbar_init(bar_dsready, 128 * kDkvGroups);
         mbar_init(bar_dkvfull, 1);
-        mbar_init(bar_dkvempty, 256);
+        mbar_init(bar_dkvempty, 128 * kDkvGroups);
         *abort_flag = 0;
         fence_mbar_init();
         p.busy[2 * cta] = globaltimer_ns();
     }
-    if (warp == 9) {
+    if (warp == kDkvMmaWarp) {
         tmem_alloc(tmem_slot, 512);
         tmem_relinquish();
     }
-    if (warp == 8 && lane == 0) {
+    if (warp == kDkvTmaWarp && lane == 0) {
         prefetch_tmap(&tm_q);
         prefetch_tmap(&tm_k);
         prefetch_tmap(&tm_v);
@@ -166,8 +175,11 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     const int unit_end = p.cta_offsets[cta + 1];
     const int G = p.hq / p.hkv;
 
-    if (warp == 8) {
+    if (warp > kDkvMmaWarp) {
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kDkvRegsOther));  // only with four groups
+    } else if (warp == kDkvTmaWarp) {
         // ---------------- TMA producer ----------------
+        if constexpr (kDkvGroups > 2) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kDkvRegsOther));
         if (elect_one()) {  // one elected thread runs the whole role
             uint32_t ucnt = 0, it_all = 0;
             bool ok = true;
@@ -215,8 +227,9 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             }
         }
         __syncwarp();
-    } else if (warp == 9) {
+    } else if (warp == kDkvMmaWarp) {
         // ---------------- MMA issuer ----------------
+        if constexpr (kDkvGroups > 2) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kDkvRegsOther));
         if (elect_one()) {  // one elected thread runs the whole role
             constexpr uint32_t idesc_s = make_idesc(128, 128, 0, 0);  // S^T, dP^T: both operands K-major
             constexpr uint32_t idesc_acc = make_idesc(128, D, 0, 1);  // dV, dK: A from TMEM, B MN-major
@@ -242,7 +255,8 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const uint64_t db = sdesc_advance(mdesc0, b_off);
     #pragma unroll
                 for (int kk = 0; kk < 8; ++kk)  // 16 queries per step
-                    mma_ts(tmem_base + d_col, tmem_base + a_col + (kk / 4) * 64 + (kk % 4) * 8, sdesc_advance(db, kk * 2048),
+                    mma_ts(tmem_base + d_col, tmem_base + a_col + (kk / (kDkvCW / 16)) * kDkvCW + (kk % (kDkvCW / 16)) * 8,
+                           sdesc_advance(db, kk * 2048),
                            idesc_acc, (accumulate || kk > 0) ? 1u : 0u);
             };
             for (int idx = unit_begin; idx < unit_end && ok; ++idx) {
@@ -336,11 +350,13 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         __syncwarp();
     } else {
         // ---------------- compute groups ----------------
-        const int c = warp >> 2;  // query-column half of each key row
+        if constexpr (kDkvGroups > 2) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kDkvRegsCompute));
+        constexpr int CW = kDkvCW;
+        const int c = warp >> 2;  // which CW query columns of each key row this group owns
         const int r = (warp & 3) * 32 + lane;
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t t_s = tmem_base + lane_addr + kColS + 64 * c;
-        const uint32_t t_dp = tmem_base + lane_addr + kColDP + 64 * c;
+        const uint32_t t_s = tmem_base + lane_addr + kColS + CW * c;
+        const uint32_t t_dp = tmem_base + lane_addr + kColDP + CW * c;
         uint32_t ucnt = 0, it_all = 0;
         bool ok = true;
         PROF_DECL
@@ -362,23 +378,23 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             for (int it = 0; it < n_it && ok; ++it, ++it_all) {
                 const int qb = (i_lo + it % nblk) * kBlk;
                 const uint32_t st = it_all & 1, par = (it_all >> 1) & 1;
-                const float* lse2 = reinterpret_cast<const float*>(smem + L::kStatOff + st * 1024) + 64 * c;
+                const float* lse2 = reinterpret_cast<const float*>(smem + L::kStatOff + st * 1024) + CW * c;
                 const float* dvec = lse2 + 128;
                 const bool need_mask = (qb == k0) || (qb + kBlk - 1 >= min_kend) || partial;
-                const int j_lo = (int)(key - qb) - 64 * c;  // first visible column of this half
-                const int j_hi = kend - 1 - qb - 64 * c;    // last visible column
+                const int j_lo = (int)(key - qb) - CW * c;  // first visible column of this group's range
+                const int j_hi = kend - 1 - qb - CW * c;    // last visible column
                 // ---- exp phase: P^T = exp2(S^T * c - LSE) ----
                 ok = mbar_wait(&bar_qfull[st], par, abort_flag) && mbar_wait(bar_sfull, it_all & 1, abort_flag);
                 if (!ok) break;
                 PROF(0)
                 tc_fence_after();
-                uint32_t sv[64];
-                tmem_ld32(t_s, sv);
-                tmem_ld32(t_s + 32, sv + 32);
-                tmem_ld_wait();
-                float pf[64];
+                uint32_t sv[CW];
 #pragma unroll
-                for (int j = 0; j < 64; j += 4) {
+                for (int j = 0; j < CW; j += 32) tmem_ld32(t_s + j, sv + j);
+                tmem_ld_wait();
+                float pf[CW];
+#pragma unroll
+                for (int j = 0; j < CW; j += 4) {
                     const float4 l4 = *reinterpret_cast<const float4*>(lse2 + j);
                     pf[j] = ex2_sel(fmaf(__uint_as_float(sv[j]), p.scale_log2, -l4.x), j);
                     pf[j + 1] = ex2_sel(fmaf(__uint_as_float(sv[j + 1]), p.scale_log2, -l4.y), j + 1);
@@ -387,14 +403,15 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 }
                 if (need_mask) {
 #pragma unroll
-                    for (int j = 0; j < 64; ++j)
+                    for (int j = 0; j < CW; ++j)
                         if (j < j_lo || j > j_hi) pf[j] = 0.f;
                 }
                 {
-                    uint32_t pk[32];
+                    uint32_t pk[CW / 2];
 #pragma unroll
-                    for (int j = 0; j < 64; j += 2) pk[j >> 1] = pack_bf16x2(pf[j], pf[j + 1]);
-                    tmem_st32(t_s, pk);  // packed P^T of this half sits in the first 32 columns of its own S^T half
+                    for (int j = 0; j < CW; j += 2) pk[j >> 1] = pack_bf16x2(pf[j], pf[j + 1]);
+                    // packed P^T of this group sits in the first CW / 2 columns of its own S^T range
+                    if constexpr (CW == 64) tmem_st32(t_s, pk); else tmem_st16(t_s, pk);
                 }
                 tmem_st_wait();
                 tc_fence_before();
@@ -405,21 +422,21 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 if (!ok) break;
                 PROF(2)
                 tc_fence_after();
-                uint32_t dpv[64];
-                tmem_ld32(t_dp, dpv);
-                tmem_ld32(t_dp + 32, dpv + 32);
+                uint32_t dpv[CW];
+#pragma unroll
+                for (int j = 0; j < CW; j += 32) tmem_ld32(t_dp + j, dpv + j);
                 tmem_ld_wait();
                 {
-                    uint32_t pk[32];
+                    uint32_t pk[CW / 2];
 #pragma unroll
-                    for (int j = 0; j < 64; j += 4) {
+                    for (int j = 0; j < CW; j += 4) {
                         const float4 d4 = *reinterpret_cast<const float4*>(dvec + j);
                         pk[j >> 1] = pack_bf16x2(pf[j] * (__uint_as_float(dpv[j]) - d4.x),
                                                  pf[j + 1] * (__uint_as_float(dpv[j + 1]) - d4.y));
                         pk[(j >> 1) + 1] = pack_bf16x2(pf[j + 2] * (__uint_as_float(dpv[j + 2]) - d4.z),
                                                        pf[j + 3] * (__uint_as_float(dpv[j + 3]) - d4.w));
                     }
-                    tmem_st32(t_dp, pk);
+                    if constexpr (CW == 64) tmem_st32(t_dp, pk); else tmem_st16(t_dp, pk);
                 }
                 tmem_st_wait();
                 tc_fence_before();
@@ -431,7 +448,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             ok = mbar_wait(bar_dkvfull, ucnt & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            constexpr int kCols = D / 2;  // columns of dK and dV this group stores
+            constexpr int kCols = D / kDkvGroups;  // columns of dK and dV this group stores
             const uint32_t t_dk = tmem_base + lane_addr + kColDK + c * kCols;
             const uint32_t t_dv = tmem_base + lane_addr + kColDV + c * kCols;
             const size_t gofs = ((size_t)key * p.hkv + kvh) * D + c * kCols;
@@ -440,13 +457,16 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const float mul = which == 0 ? p.scale : 1.0f;
                 __nv_bfloat16* gdst = (which == 0 ? p.dk : p.dv) + gofs;
 #pragma unroll
-                for (int cc = 0; cc < kCols; cc += 32) {
-                    uint32_t v[32];
-                    tmem_ld32((which == 0 ? t_dk : t_dv) + cc, v);
+                constexpr int kChunk = kCols < 32 ? kCols : 32;
+#pragma unroll
+                for (int cc = 0; cc < kCols; cc += kChunk) {
+                    uint32_t v[kChunk];
+                    if constexpr (kChunk == 32) tmem_ld32((which == 0 ? t_dk : t_dv) + cc, v);
+                    else tmem_ld16((which == 0 ? t_dk : t_dv) + cc, v);
                     tmem_ld_wait();
                     if (key_ok) {
 #pragma unroll
-                        for (int i = 0; i < 32; i += 8) {
+                        for (int i = 0; i < kChunk; i += 8) {
                             uint4 w;
                             w.x = pack_bf16x2(__uint_as_float(v[i]) * mul, __uint_as_float(v[i + 1]) * mul);
                             w.y = pack_bf16x2(__uint_as_float(v[i + 2]) * mul, __uint_as_float(v[i + 3]) * mul);
@@ -468,7 +488,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     // ---------------- teardown ----------------
     tc_fence_before();
     __syncthreads();
-    if (warp == 9) tmem_dealloc(tmem_base, 512);
+    if (warp == kDkvMmaWarp) tmem_dealloc(tmem_base, 512);
     if (threadIdx.x == 0) {
         if (*abort_flag) atomicExch(p.status, LIBRA_ERR_TIMEOUT);
         p.busy[2 * cta + 1] = globaltimer_ns();
@@ -539,6 +559,8 @@ static int launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtens
     if (!configured) {
         if (set_smem(k_attn_bwd_dkdv<D>, DkvSmem<D>::kBytes) != LIBRA_OK) return LIBRA_ERR_CUDA;
         if (set_smem(k_attn_bwd_dq<D>, DqSmem<D>::kBytes) != LIBRA_OK) return LIBRA_ERR_CUDA;
+        if (kDkvGroups > 2 && !regs_pool_ok(k_attn_bwd_dkdv<D>, 128 * kDkvGroups, kDkvRegsCompute, 128, kDkvRegsOther))
+            return LIBRA_ERR_UNSUPPORTED;
         if (!regs_pool_ok(k_attn_bwd_dq<D>, 128 * kDqGroups, kDqRegsCompute, 128, kDqRegsOther)) return LIBRA_ERR_UNSUPPORTED;
         configured = true;
     }
