@@ -12,14 +12,14 @@ pytestmark = pytest.mark.gpu
 TOL_G = 5e-2   # max-abs error relative to max magnitude (the benchmark's stated bound for dQ/dK/dV)
 
 
-def _run(lengths, hq, hkv, d, seed=0, W=0, qscale=1.0):
+def _run(lengths, hq, hkv, d, seed=0, W=0, qscale=1.0, H=0):
     from paper_2607_23250_b200 import binding as lb
     cu_np = pools.cu_seqlens(lengths)
     T = int(cu_np[-1])
     t = pools.make_tensors(T, hq, hkv, d, seed=seed, scale=qscale)
     q, k, v, dout = (t[n].cuda() for n in ("q", "k", "v", "dout"))
     cu = torch.from_numpy(cu_np).cuda()
-    plan = lb.libra_plan_tiles(cu, hq, 256, n_workers=W, tile_kv=128, n_heads_kv=hkv)
+    plan = lb.libra_plan_tiles(cu, H or hq, 256, n_workers=W, tile_kv=128, n_heads_kv=hkv)
     out, lse = lb.libra_attn_pool_fwd(q, k, v, plan)
     dq, dk, dv = lb.libra_attn_pool_bwd(q, k, v, out, lse, dout, plan)
     torch.cuda.synchronize()
@@ -61,6 +61,16 @@ def test_random_small_pools(seed):
     hq = hkv * int(rng.choice([1, 2, 4]))
     d = int(rng.choice([64, 128]))
     got, ref, cu = _run(lengths, hq, hkv, d, seed=seed, W=int(rng.choice([0, 3, 37])))
+    _check(got, ref, cu)
+
+
+@pytest.mark.parametrize("H,d,T", [(2, 128, 256 * 3 + 100), (1, 64, 256 * 2 + 129), (4, 128, 700), (1, 128, 128)])
+def test_head_shards_wider_than_one_head(H, d, T):
+    """Query-major tiles that carry several heads (units of one tile follow each other head by head), with a last
+    tile whose second 128-row half is partly or wholly past the end of the pool."""
+    rng = np.random.default_rng(T + H)
+    lengths = pools.random_layout(rng, T, 400)
+    got, ref, cu = _run(lengths, 4, 2, d, seed=11, H=H, W=int(rng.choice([0, 2, 5])))
     _check(got, ref, cu)
 
 
