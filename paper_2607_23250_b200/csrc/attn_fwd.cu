@@ -237,9 +237,11 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             const int lo = r[0].lo, hi = act1 ? r[1].hi : r[0].hi;
             for (int hh = 0; hh < heads_per_shard && ok; ++hh) {
                 PROF(7)
+                TRACE(21)
                 ok = warp_wait(bar_qfull, qcnt & 1, abort_flag);
                 if (!ok) break;
                 PROF(0)
+                TRACE(22)
                 ++qcnt;
                 // prologue: S(lo)
                 uint32_t st = ring % L::kStages;
@@ -252,6 +254,7 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                     tc_commit(&bar_empty[st]);
                     if (lo == hi) tc_commit(bar_qempty);  // no later MMA of this tile reads Q
                 }
+                TRACE(23)
                 ++ring;
                 for (int j = lo; j <= hi && ok; ++j) {
                     TRACE(20)
@@ -306,6 +309,7 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         uint32_t scnt = 0, ocnt = 0;
         bool ok = true;
         PROF_DECL
+        TRACE_DECL(1 + g, cta == 0 && (warp & 3) == 0 && lane == 0)
         for (int idx = tile_begin; idx < tile_end && ok; ++idx) {
             const int t = p.cta_tiles[idx];
             const int64_t qs = (int64_t)(t / p.H) * (2 * kBM) + g * kBM;
@@ -416,9 +420,11 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 }
                 if (!ok) break;
                 // epilogue: wait for the last PV, normalise, store
+                TRACE(24)
                 ok = mbar_wait(&bar_odone[g], (ocnt - 1) & 1, abort_flag);
                 if (!ok) break;
                 PROF(2)
+                TRACE(25)
                 tc_fence_after();
                 const float inv_l = (l_sum > 0.f) ? 1.0f / l_sum : 0.f;
                 __nv_bfloat16* orow_ptr = p.out + ((size_t)row * p.hq + h) * D;
@@ -444,6 +450,7 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 // the next PV into this slot's O may only start after these reads: it is issued
                 // after this group's next p_ready arrival, which follows in program order
                 tc_fence_before();
+                TRACE(26)
             }
         }
         PROF_FLUSH(threadIdx.x == 0, 0)
