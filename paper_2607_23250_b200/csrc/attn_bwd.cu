@@ -301,8 +301,10 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     #endif
                     tc_fence_after();
                     {
+                        TRACE(10)
                         issue_acc(kColDV, kColS, L::kDoOff + st * L::kTileBytes, it > 0);
                         tc_commit(&bar_doempty[st]);
+                        TRACE(11)
                     }
                     // S(it+1)
                     if (more) {
@@ -313,6 +315,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         {
                             issue_kmajor(kColS, L::kKOff, L::kQOff + (nx & 1) * L::kTileBytes);
                             tc_commit(bar_sfull);
+                            TRACE(12)
                         }
                     }
                     // dK(it) += dS^T Q
@@ -324,8 +327,10 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     PROF(2)
                     tc_fence_after();
                     {
+                        TRACE(13)
                         issue_acc(kColDK, kColDP, L::kQOff + st * L::kTileBytes, it > 0);
                         tc_commit(&bar_qempty[st]);
+                        TRACE(14)
                     }
                     // dP(it+1)
                     if (more) {
@@ -336,6 +341,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         {
                             issue_kmajor(kColDP, L::kVOff, L::kDoOff + (nx & 1) * L::kTileBytes);
                             tc_commit(bar_dpfull);
+                            TRACE(15)
                         }
                     }
                 }
@@ -360,6 +366,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         uint32_t ucnt = 0, it_all = 0;
         bool ok = true;
         PROF_DECL
+        TRACE_DECL(1 + warp, cta == 0 && lane == 0)
 #if defined(LIBRA_DBG_FREE_MMA) && !defined(LIBRA_DBG_FREE_MMA_COMPUTE_ON)
         ok = false;
 #endif
@@ -387,6 +394,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 ok = mbar_wait(&bar_qfull[st], par, abort_flag) && mbar_wait(bar_sfull, it_all & 1, abort_flag);
                 if (!ok) break;
                 PROF(0)
+                TRACE(2)
                 tc_fence_after();
                 uint32_t sv[CW];
 #pragma unroll
@@ -417,10 +425,12 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 tc_fence_before();
                 mbar_arrive(bar_pready);
                 PROF(1)
+                TRACE(3)
                 // ---- dS phase: dS^T = P^T o (dP^T - D), packed over this half's own dP^T columns ----
                 ok = mbar_wait(bar_dpfull, it_all & 1, abort_flag);
                 if (!ok) break;
                 PROF(2)
+                TRACE(4)
                 tc_fence_after();
                 uint32_t dpv[CW];
 #pragma unroll
@@ -442,6 +452,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 tc_fence_before();
                 mbar_arrive(bar_dsready);
                 PROF(3)
+                TRACE(5)
             }
             if (!ok) break;
             // ---- unit epilogue: dK * scale and dV to global ----

@@ -18,6 +18,9 @@
 
 namespace libra {
 
+#ifndef LIBRA_TRACE_DQ
+#define LIBRA_TRACE_DQ 1   // trace builds: 0 leaves the trace buffer to the dK/dV kernel
+#endif
 #ifndef LIBRA_DQ_PREFETCH
 #define LIBRA_DQ_PREFETCH 0
 #endif
@@ -312,7 +315,7 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             uint32_t kcnt = 0, vcnt = 0, blk = 0;
             bool ok = true;
             PROF_DECL
-            TRACE_DECL(0, cta == 0)
+            TRACE_DECL(0, cta == 0 && LIBRA_TRACE_DQ)
             // C[tmem d_col] = A[tmem a_col, bf16 packed over the head dimension] * B(K-major tile at b_off)^T
             auto issue_qk = [&](uint32_t d_col, uint32_t a_col, uint32_t b_off) {
                 const uint64_t db = sdesc_advance(kdesc0, b_off);
@@ -437,7 +440,7 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         uint32_t ucnt = 0, blk = 0;
         bool ok = true;
         PROF_DECL
-        TRACE_DECL(1 + warp, cta == 0 && lane == 0)
+        TRACE_DECL(1 + warp, cta == 0 && lane == 0 && LIBRA_TRACE_DQ)
         // Copies this thread's row of Q or dO (its group's duty) of the unit whose tile has landed into TMEM.
         // The caller has seen every MMA that read the previous copy complete (s_full for Q, dp_full for dO).
         auto stage = [&](uint32_t parity) -> bool {
