@@ -171,9 +171,20 @@ def run_ours(args):
     q, k, v, dout = t["q"], t["k"], t["v"], t["dout"]
     cu = torch.from_numpy(cu_np).to(dev)
     blocks = args.weight_model == "blocks"
-    plan = lb.libra_plan_tiles(cu, hq, 256, tile_kv=128, n_heads_kv=hkv, total_tokens=T,
-                               weight_model=lb.LIBRA_WEIGHT_BLOCKS if blocks else lb.LIBRA_WEIGHT_PAIRS,
-                               unit_cost_q=12 if blocks else 0, unit_cost_kv=6 if blocks else 0)
+
+    def make_plan():
+        return lb.libra_plan_tiles(cu, hq, 256, tile_kv=128, n_heads_kv=hkv, total_tokens=T,
+                                   weight_model=lb.LIBRA_WEIGHT_BLOCKS if blocks else lb.LIBRA_WEIGHT_PAIRS,
+                                   unit_cost_q=12 if blocks else 0, unit_cost_kv=6 if blocks else 0)
+
+    make_plan().destroy()                     # first call pays for the module load
+    torch.cuda.synchronize()
+    pe0, pe1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    pe0.record()
+    plan = make_plan()                        # built once, outside the timed steps (the paper reuses it across layers)
+    pe1.record()
+    torch.cuda.synchronize()
+    plan_ms = pe0.elapsed_time(pe1)
     assert plan.status() == 0
     plan.set_timing(True)
     out = torch.empty_like(q)
@@ -232,7 +243,7 @@ def run_ours(args):
         e2e = run_e2e(args, step_on, barrier, dict(q=q, k=k, v=v, dout=dout),
                       dict(out=out, lse=lse, dq=dq, dk=dk, dv=dv), world, dev, ff + fb)
     finish(args, rank, world, spec, lengths, plan, value, ms_per_step, (kern_f, kern_b, kern_q),
-           (busy_f, busy_b, busy_q), clocks, launches, e2e, ff, fb, q)
+           (busy_f, busy_b, busy_q), clocks, launches, e2e, ff, fb, q, plan_ms)
     plan.destroy()
     if world > 1:
         dist.destroy_process_group()
@@ -298,7 +309,8 @@ def run_e2e(args, step_on, barrier, dev_in, dev_out, world, dev, flops):
             "d2h_bytes_per_step": d2h, "ms_per_step": round(e2e_ms, 3)}
 
 
-def finish(args, rank, world, spec, lengths, plan, value, ms_per_step, kern, busy, clocks, launches, e2e, ff, fb, q):
+def finish(args, rank, world, spec, lengths, plan, value, ms_per_step, kern, busy, clocks, launches, e2e, ff, fb, q,
+           plan_ms=None):
     kern_f, kern_b, kern_q = kern
     busy_f, busy_b, busy_q = busy
     from paper_2607_23250_b200 import binding as lb  # noqa: F401
@@ -338,6 +350,7 @@ def finish(args, rank, world, spec, lengths, plan, value, ms_per_step, kern, bus
             "clocks": clocks,
             "e2e": e2e,
             "gpu_launches": int(launches),
+            "plan_ms": None if plan_ms is None else round(plan_ms, 3),
             "roofline": {"bound": "tensor", "kernel": "k_attn_bwd_dkdv", "achieved": round(ach, 1),
                          "peak": peaks["sustained"], "unit": "TFLOP/s", "frac": round(ach / peaks["sustained"], 4),
                          "peak_kind": f"bf16 sustained, {peaks['source']}", "traffic": traffic,
