@@ -111,7 +111,8 @@ typedef struct {
  * With opts->weight_model = LIBRA_WEIGHT_BLOCKS the weight is the block count described at
  * LIBRA_WEIGHT_BLOCKS above; everything else is unchanged.
  * Errors: INVALID_ARG (null, n_samples <= 0, n_heads <= 0, tile_q <= 0, a negative option,
- * an unknown weight model), OVERFLOW
+ * an unknown weight model), OVERFLOW (n_heads * T^2 >= 9e15, the bound under which loads fit the
+ * placement's packed keys; or
  * (NB * H >= 2^31), CUDA; a malformed cu_seqlens is detected on the device and reported
  * by libra_plan_status as BAD_SEQLENS.
  */

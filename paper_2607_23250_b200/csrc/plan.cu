@@ -99,9 +99,10 @@ __global__ void k_rank_blocks(const int64_t* __restrict__ weight_blk, int64_t NB
 }
 
 // Sequential placement by one warp.  Worker r's load lives in lane r % 32, register r / 32.
-// Per tile: every lane finds its lightest worker, a shuffle tree finds the warp's
+// Per tile: every lane finds its lightest worker, two warp reductions find the warp's
 // (load, index) minimum, the owning lane adds the weight.  Ties go to the lowest index
-// because the comparison is lexicographic on (load, index).
+// because the comparison is lexicographic on (load, index).  Loads stay below 2^53 (checked on the
+// host from the weight total), so load * 1024 + index fits 64 bits.
 template <int PER>
 __global__ void __launch_bounds__(32) k_place(const int64_t* __restrict__ weight_blk,
                                               const int32_t* __restrict__ blk_order, int64_t NT, int H, int W,
@@ -129,18 +130,18 @@ __global__ void __launch_bounds__(32) k_place(const int64_t* __restrict__ weight
         for (int i = 0; i < lim; ++i) {
             const int64_t w = __shfl_sync(0xffffffffu, w_l, i);
             const int32_t t = __shfl_sync(0xffffffffu, t_l, i);
-            int64_t best = load[0];
-            int32_t bidx = lane;
+            // (load, worker) packed into one 64-bit key, compared lexicographically by two hardware warp
+            // reductions (high word, then low word among the lanes that tie on it) instead of a shuffle tree
+            uint64_t key = ~0ull;
 #pragma unroll
-            for (int k = 1; k < PER; ++k) {
-                if (load[k] < best) { best = load[k]; bidx = lane + 32 * k; }
+            for (int k = 0; k < PER; ++k) {
+                const uint64_t kk = load[k] == INT64_MAX ? ~0ull : (((uint64_t)load[k] << 10) | (uint32_t)(lane + 32 * k));
+                key = kk < key ? kk : key;
             }
-#pragma unroll
-            for (int off = 16; off > 0; off >>= 1) {
-                const int64_t ob = __shfl_xor_sync(0xffffffffu, best, off);
-                const int32_t oi = __shfl_xor_sync(0xffffffffu, bidx, off);
-                if (ob < best || (ob == best && oi < bidx)) { best = ob; bidx = oi; }
-            }
+            const uint32_t hi = (uint32_t)(key >> 32), lo = (uint32_t)key;
+            const uint32_t mhi = __reduce_min_sync(0xffffffffu, hi);
+            const uint32_t mlo = __reduce_min_sync(0xffffffffu, hi == mhi ? lo : 0xffffffffu);
+            const int32_t bidx = (int32_t)(mlo & 1023u);
             int32_t my_pos = 0;
             if ((bidx & 31) == lane) {
 #pragma unroll
@@ -220,6 +221,8 @@ static int build_dir(libra_plan* p, PlanDir& d, int key_major, const libra_plan_
     const int64_t T = p->T;
     d.NB = (T + d.tile - 1) / d.tile;
     if (d.NB * (int64_t)d.H >= (int64_t)INT32_MAX) return LIBRA_ERR_OVERFLOW;
+    // a worker's load is at most the weight total <= H * T^2 / 2 + ...; the placement packs load * 1024 + index
+    if ((long double)d.H * (long double)T * (long double)T >= 9.0e15L) return LIBRA_ERR_OVERFLOW;
     if (d.NB > 65536) return LIBRA_ERR_UNSUPPORTED;  // the rank sort is quadratic in blocks
     if (d.W > 1024) return LIBRA_ERR_UNSUPPORTED;
     d.NT = d.NB * d.H;
