@@ -109,13 +109,18 @@ __global__ void __launch_bounds__(32) k_place(const int64_t* __restrict__ weight
                                               int32_t* __restrict__ cta_of_tile, int32_t* __restrict__ pos,
                                               int32_t* __restrict__ cta_offsets, int64_t* __restrict__ loads) {
     const int lane = threadIdx.x;
-    int64_t load[PER];
+    // key[k] = load * 1024 + worker index of worker lane + 32 k (all ones: no such worker); the lane's
+    // lightest worker is kept up to date, so a placement only recomputes it in the lane that changed
+    uint64_t key[PER];
     int32_t cnt[PER];
 #pragma unroll
     for (int i = 0; i < PER; ++i) {
-        load[i] = (lane + 32 * i < W) ? 0 : INT64_MAX;
+        key[i] = (lane + 32 * i < W) ? (uint64_t)(lane + 32 * i) : ~0ull;
         cnt[i] = 0;
     }
+    uint64_t best = key[0];
+#pragma unroll
+    for (int k = 1; k < PER; ++k) best = key[k] < best ? key[k] : best;
     for (int64_t x0 = 0; x0 < NT; x0 += 32) {
         // each lane fetches one upcoming tile, then they are broadcast one by one
         const int64_t xl = x0 + lane;
@@ -130,24 +135,21 @@ __global__ void __launch_bounds__(32) k_place(const int64_t* __restrict__ weight
         for (int i = 0; i < lim; ++i) {
             const int64_t w = __shfl_sync(0xffffffffu, w_l, i);
             const int32_t t = __shfl_sync(0xffffffffu, t_l, i);
-            // (load, worker) packed into one 64-bit key, compared lexicographically by two hardware warp
-            // reductions (high word, then low word among the lanes that tie on it) instead of a shuffle tree
-            uint64_t key = ~0ull;
-#pragma unroll
-            for (int k = 0; k < PER; ++k) {
-                const uint64_t kk = load[k] == INT64_MAX ? ~0ull : (((uint64_t)load[k] << 10) | (uint32_t)(lane + 32 * k));
-                key = kk < key ? kk : key;
-            }
-            const uint32_t hi = (uint32_t)(key >> 32), lo = (uint32_t)key;
+            // lexicographic (load, worker) minimum over the warp: two hardware reductions, high word first,
+            // then the low word among the lanes that tie on it
+            const uint32_t hi = (uint32_t)(best >> 32), lo = (uint32_t)best;
             const uint32_t mhi = __reduce_min_sync(0xffffffffu, hi);
             const uint32_t mlo = __reduce_min_sync(0xffffffffu, hi == mhi ? lo : 0xffffffffu);
             const int32_t bidx = (int32_t)(mlo & 1023u);
-            int32_t my_pos = 0;
             if ((bidx & 31) == lane) {
+                int32_t my_pos = 0;
 #pragma unroll
                 for (int k = 0; k < PER; ++k) {
-                    if (k == (bidx >> 5)) { load[k] += w; my_pos = cnt[k]++; }
+                    if (k == (bidx >> 5)) { key[k] += (uint64_t)w << 10; my_pos = cnt[k]++; }
                 }
+                best = key[0];
+#pragma unroll
+                for (int k = 1; k < PER; ++k) best = key[k] < best ? key[k] : best;
                 cta_of_tile[t] = bidx;
                 pos[t] = my_pos;
             }
@@ -156,7 +158,7 @@ __global__ void __launch_bounds__(32) k_place(const int64_t* __restrict__ weight
 #pragma unroll
     for (int i = 0; i < PER; ++i) {
         const int r = lane + 32 * i;
-        if (r < W) { loads[r] = load[i]; cta_offsets[r + 1] = cnt[i]; }
+        if (r < W) { loads[r] = (int64_t)(key[i] >> 10); cta_offsets[r + 1] = cnt[i]; }
     }
     __syncwarp();
     if (lane == 0) {  // counts -> offsets
