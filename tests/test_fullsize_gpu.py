@@ -1,4 +1,5 @@
-"""Full-size parity: the Qwen3-8B-shaped pool in the launch configuration the benchmark times.
+"""Full-size parity: the Qwen3-8B-shaped pool in the launch configuration the benchmark times, plus the 30B-shaped
+pool with Pareto-tailed samples and the fully skewed pool of 65536-token samples.
 
 The whole oracle would take minutes here, so outputs are sampled: rows of O / LSE / dQ and
 columns of dK / dV are recomputed one by one by the CPU oracle on the (sample, kv-head group)
@@ -23,10 +24,10 @@ def _rel(got, want, floor=1e-3):
     return float(np.abs(np.asarray(got, np.float64) - want).max() / max(np.abs(want).max(), floor))
 
 
-@pytest.fixture(scope="module")
-def run():
+@pytest.fixture(scope="module", params=[(2, 0.0), (3, 0.0), (5, 1.0)], ids=["config2", "config3", "config5_skew1"])
+def run(request):
     from paper_2607_23250_b200 import binding as lb
-    spec = pools.config(2)
+    spec = pools.config(*request.param)
     lengths = pools.pool_lengths(spec)
     cu_np = pools.cu_seqlens(lengths)
     T, hq, hkv, d = spec.total_tokens, spec.hq, spec.hkv, spec.head_dim
@@ -42,6 +43,8 @@ def run():
     res = dict(spec=spec, lengths=lengths, cu=cu_np, t=t, out=out, lse=lse, dq=dq, dk=dk, dv=dv, plan=plan, lb=lb)
     yield res
     plan.destroy()
+    del res
+    torch.cuda.empty_cache()
 
 
 def _sub(run, j, kvh):
@@ -97,7 +100,9 @@ def test_short_samples_full_gradient(run):
     rng = np.random.default_rng(1)
     lengths = np.asarray(run["lengths"])
     small = [j for j in range(len(lengths)) if 2 <= lengths[j] <= 1500]
-    for j in rng.choice(small, 4, replace=False):
+    if not small:
+        pytest.skip("the pool has no short samples")
+    for j in rng.choice(small, min(4, len(small)), replace=False):
         kvh = int(rng.integers(0, run["spec"].hkv))
         s = _sub(run, int(j), kvh)
         cu = [0, s["n"]]
