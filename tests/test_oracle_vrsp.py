@@ -107,3 +107,20 @@ def test_beats_production_order_on_long_tailed_windows(P):
         assert r_vrsp <= r_prod
         ratios.append((r_vrsp - 1) / max(r_prod - 1, 1e-12))
     assert np.mean(ratios) < 0.5
+
+
+def test_production_order_follows_the_concentration_estimate():
+    """Section 3.2, Eq. 3: under random grouping E[R] - 1 is about CV / sqrt(P) * sqrt(2 ln(D / P)).  On synthetic
+    windows (D = 128) production-order grouping must follow that estimate within a factor of two for P = 4..16,
+    and VRSP must sit an order of magnitude below it from P = 8 on."""
+    import math
+    D = 128
+    works = [_window(1000 + seed, D) for seed in range(10)]
+    for P in (4, 8, 16):
+        K = D // P
+        prod = np.mean([w.reshape(K, P).sum(1).max() / (w.sum() / K) - 1 for w in works])
+        est = np.mean([w.std() / w.mean() / math.sqrt(P) * math.sqrt(2 * math.log(K)) for w in works])
+        vrsp = np.mean([oracle.vrsp_place(w, P)["pool_load"].max() / (w.sum() / K) - 1 for w in works])
+        assert 0.5 * est <= prod <= 2.0 * est, (P, prod, est)
+        if P >= 8:
+            assert vrsp <= 0.1 * prod, (P, vrsp, prod)
