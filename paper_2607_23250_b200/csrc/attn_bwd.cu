@@ -514,34 +514,50 @@ namespace libra {
 
 // ---- prep kernel ------------------------------------------------------------------------------
 
-// One warp per (token, head): D = <dO, O>; LSE to log2 units; rows in [T, Tpad) get zeros.
+// D = <dO, O> per (token, head) and LSE in log2 units; rows in [T, Tpad) get zeros.
+// One warp per (head, 32 consecutive tokens): a row is read by the whole warp (one contiguous 2 D bytes), lane i
+// keeps the sum of row i, so the two statistics leave as one coalesced 128-byte store each.  Rows are taken
+// four at a time to keep several loads in flight.
 template <int D>
 __global__ void k_bwd_prep(const __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __restrict__ dout,
                            const float* __restrict__ lse, int64_t T, int64_t Tpad, int hq, float* __restrict__ dvec,
                            float* __restrict__ lse2) {
     const int64_t w = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
-    if (w >= Tpad * hq) return;
-    const int64_t t = w / hq;
-    const int h = (int)(w % hq);
-    float acc = 0.f;
-    if (t < T) {
-        constexpr int kPer = D / 32;  // 2 or 4 elements per lane
-        const __nv_bfloat16* o = out + ((size_t)t * hq + h) * D + lane * kPer;
-        const __nv_bfloat16* g = dout + ((size_t)t * hq + h) * D + lane * kPer;
+    const int64_t groups = Tpad / 32;  // Tpad is a multiple of 128
+    if (w >= groups * hq) return;
+    const int h = (int)(w / groups);
+    const int64_t t0 = (w % groups) * 32;
+    constexpr int kPer = D / 32;  // 2 or 4 elements per lane
+    float mine = 0.f;
+#pragma unroll 2
+    for (int i0 = 0; i0 < 32; i0 += 4) {
+        float acc[4];
 #pragma unroll
-        for (int i = 0; i < kPer; i += 2) {
-            const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(o + i));
-            const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(g + i));
-            acc += a.x * b.x + a.y * b.y;
+        for (int u = 0; u < 4; ++u) {
+            const int64_t t = t0 + i0 + u;
+            acc[u] = 0.f;
+            if (t < T) {
+                const __nv_bfloat16* o = out + ((size_t)t * hq + h) * D + lane * kPer;
+                const __nv_bfloat16* g = dout + ((size_t)t * hq + h) * D + lane * kPer;
+#pragma unroll
+                for (int i = 0; i < kPer; i += 2) {
+                    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(o + i));
+                    const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(g + i));
+                    acc[u] += a.x * b.x + a.y * b.y;
+                }
+            }
         }
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+        for (int u = 0; u < 4; ++u) {
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) acc[u] += __shfl_xor_sync(0xffffffffu, acc[u], off);
+            if (lane == i0 + u) mine = acc[u];
+        }
     }
-    if (lane == 0) {
-        dvec[(size_t)h * Tpad + t] = acc;
-        lse2[(size_t)h * Tpad + t] = t < T ? lse[(size_t)h * T + t] * 1.4426950408889634f : 0.f;
-    }
+    const int64_t t = t0 + lane;
+    dvec[(size_t)h * Tpad + t] = mine;
+    lse2[(size_t)h * Tpad + t] = t < T ? lse[(size_t)h * T + t] * 1.4426950408889634f : 0.f;
 }
 
 struct BwdWorkspace {
@@ -642,7 +658,7 @@ extern "C" int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const v
     if (rc != LIBRA_OK) return rc;
 
     {
-        const int64_t warps = ws.Tpad * dims->hq;
+        const int64_t warps = ws.Tpad / 32 * dims->hq;
         const unsigned grid = (unsigned)((warps * 32 + 255) / 256);
         if (D == 128)
             k_bwd_prep<128><<<grid, 256, 0, s>>>((const __nv_bfloat16*)out_dev, (const __nv_bfloat16*)dout_dev, lse_dev,
