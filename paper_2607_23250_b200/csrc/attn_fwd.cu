@@ -281,9 +281,11 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                             ++pcnt[g];
                             tc_fence_after();
                             if (leader) issue_pv(g, st_v, j != r[g].lo);
+                            TRACE(10 + g)
                         }
                         if (j + 1 <= hi && j + 1 >= r[g].lo && j + 1 <= r[g].hi) {
                             if (leader) issue_s(g, st_k);
+                            TRACE(12 + g)
                         }
                     }
                     if (!ok) break;
@@ -328,6 +330,7 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                     PROF(3)
                     ok = mbar_wait(&bar_sfull[g], scnt & 1, abort_flag);
                     if (!ok) break;
+                    TRACE(2)
                     PROF(0)
                     ++scnt;
                     tc_fence_after();
@@ -415,6 +418,7 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                     tmem_st_wait();
                     tc_fence_before();
                     mbar_arrive(&bar_pready[g]);
+                    TRACE(3)
                     PROF(1)
                     ++ocnt;
                 }
