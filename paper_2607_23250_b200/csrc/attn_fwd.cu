@@ -37,8 +37,8 @@ struct FwdSmem {
     static constexpr int kQOff = 0;
     static constexpr int kRingOff = 2 * kTileBytes;
     static constexpr int kBarOff = kRingOff + kStages * kTileBytes;
-    // barriers: full[kStages], empty[kStages], q_full, q_empty, s_full[2], p_ready[2], o_done[2]
-    static constexpr int kNumBars = 2 * kStages + 8;
+    // barriers: full[kStages], empty[kStages], q_full, q_empty, s_full[2], p_ready[2], o_done[2], p_half[2]
+    static constexpr int kNumBars = 2 * kStages + 10;
     static constexpr int kMiscOff = kBarOff + kNumBars * 8;
     static constexpr int kBytes = kMiscOff + 16;
     static constexpr int kAlloc = kBytes + 1024;  // slack to align the base to 1024 B
@@ -109,6 +109,7 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     uint64_t* bar_sfull = bar_qfull + 2;   // [2]
     uint64_t* bar_pready = bar_qfull + 4;  // [2]
     uint64_t* bar_odone = bar_qfull + 6;   // [2]
+    uint64_t* bar_phalf = bar_qfull + 8;   // [2] P of the first 64 keys is in TMEM
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::kMiscOff);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kMiscOff + 4);
 
@@ -124,6 +125,7 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             mbar_init(&bar_sfull[g], 1);
             mbar_init(&bar_pready[g], kBM);
             mbar_init(&bar_odone[g], 1);
+            mbar_init(&bar_phalf[g], kBM);
         }
         *abort_flag = 0;
         fence_mbar_init();
@@ -220,14 +222,15 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             }
             tc_commit(&bar_sfull[g]);
         };
-        auto issue_pv = [&](int g, uint32_t stage, bool accumulate) {
+        // O[g] (+)= P[g] V over the key steps [kk0, kk1) of 16 keys; the softmax group hands P over in two halves
+        auto issue_pv = [&](int g, uint32_t stage, bool accumulate, int kk0, int kk1) {
             const uint64_t va = sdesc_advance(desc_v, stage * L::kTileBytes);
 #pragma unroll
-            for (int kk = 0; kk < kBN / 16; ++kk) {
+            for (int kk = kk0; kk < kk1; ++kk) {
                 mma_ts(tmem_base + 2 * kBN + g * D, tmem_base + g * kBN + kk * 8, sdesc_advance(va, kk * 2048), idesc_pv,
                        (accumulate || kk > 0) ? 1u : 0u);
             }
-            tc_commit(&bar_odone[g]);
+            if (kk1 == kBN / 16) tc_commit(&bar_odone[g]);
         };
         for (int idx = tile_begin; idx < tile_end && ok; ++idx) {
             const int t = p.cta_tiles[idx];
@@ -275,12 +278,16 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                     for (int g = 0; g < 2 && ok; ++g) {
                         if (j >= r[g].lo && j <= r[g].hi) {
                             PROF(7)
-                            ok = warp_wait(&bar_pready[g], pcnt[g] & 1, abort_flag);
+                            ok = warp_wait(&bar_phalf[g], pcnt[g] & 1, abort_flag);   // P of keys 0..63
+                            if (!ok) break;
+                            tc_fence_after();
+                            if (leader) issue_pv(g, st_v, j != r[g].lo, 0, kBN / 32);
+                            ok = warp_wait(&bar_pready[g], pcnt[g] & 1, abort_flag);  // the rest, while those MMAs run
                             if (!ok) break;
                             PROF(3 + g)
                             ++pcnt[g];
                             tc_fence_after();
-                            if (leader) issue_pv(g, st_v, j != r[g].lo);
+                            if (leader) issue_pv(g, st_v, j != r[g].lo, kBN / 32, kBN / 16);
                             TRACE(10 + g)
                         }
                         if (j + 1 <= hi && j + 1 >= r[g].lo && j + 1 <= r[g].hi) {
@@ -408,6 +415,11 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                             pk[i >> 1] = pack_bf16x2(p0, p1);
                         }
                         tmem_st16(t_s + (c >> 1), pk);
+                        if (c == kBN / 2 - 32) {  // P of the first 64 keys is complete: its PV steps can start
+                            tmem_st_wait();
+                            tc_fence_before();
+                            mbar_arrive(&bar_phalf[g]);
+                        }
                     }
                     {
                         float a, b;
