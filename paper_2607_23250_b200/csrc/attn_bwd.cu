@@ -77,8 +77,8 @@ struct DkvSmem {
     static constexpr int kStatOff = 6 * kTileBytes;  // per Q stage: lse2[128], dvec[128]
     static constexpr int kBarOff = kStatOff + 2 * 1024;
     // kv_full, kv_empty, q_full[2], q_empty[2], do_full[2], do_empty[2], s_full, p_ready, dp_full,
-    // ds_ready, dkv_full, dkv_empty
-    static constexpr int kNumBars = 16;
+    // ds_ready, dkv_full, dkv_empty, p_half
+    static constexpr int kNumBars = 17;
     static constexpr int kMiscOff = kBarOff + kNumBars * 8;
     static constexpr int kBytes = kMiscOff + 16;
     static_assert(kBytes <= kSmemMax, "exceeds the shared memory of an sm_100 CTA");
@@ -125,6 +125,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     uint64_t* bar_dsready = bars + 13;
     uint64_t* bar_dkvfull = bars + 14;
     uint64_t* bar_dkvempty = bars + 15;
+    uint64_t* bar_phalf = bars + 16;   // the first half of every group's P^T columns is in TMEM
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::kMiscOff);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kMiscOff + 4);
 
@@ -151,6 +152,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         mbar_init(bar_dsready, 128 * kDkvGroups);
         mbar_init(bar_dkvfull, 1);
         mbar_init(bar_dkvempty, 128 * kDkvGroups);
+        mbar_init(bar_phalf, 128 * kDkvGroups);
         *abort_flag = 0;
         fence_mbar_init();
         p.busy[2 * cta] = globaltimer_ns();
@@ -250,14 +252,19 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     mma_ss(tmem_base + d_col, sdesc_advance(da, off), sdesc_advance(db, off), idesc_s, kk > 0);
                 }
             };
-            // C[tmem] (+)= A(TMEM, bf16 packed: queries 64c.. at columns a_col + 64c ..) * B(MN-major tile)
-            auto issue_acc = [&](uint32_t d_col, uint32_t a_col, uint32_t b_off, bool accumulate) {
+            // C[tmem] (+)= A(TMEM, bf16 packed: group c's queries at columns a_col + CW c ..) * B(MN-major tile).
+            // `half` 0 / 1 issues the key steps that read the first / second half of every group's columns
+            // (the compute groups hand P^T over in two halves), 2 issues all of them.
+            auto issue_acc = [&](uint32_t d_col, uint32_t a_col, uint32_t b_off, bool accumulate, int half) {
                 const uint64_t db = sdesc_advance(mdesc0, b_off);
-    #pragma unroll
-                for (int kk = 0; kk < 8; ++kk)  // 16 queries per step
-                    mma_ts(tmem_base + d_col, tmem_base + a_col + (kk / (kDkvCW / 16)) * kDkvCW + (kk % (kDkvCW / 16)) * 8,
-                           sdesc_advance(db, kk * 2048),
-                           idesc_acc, (accumulate || kk > 0) ? 1u : 0u);
+                constexpr int kPerGroup = kDkvCW / 16;  // key steps of 16 queries per group
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    const int within = kk % kPerGroup;
+                    if (half != 2 && (within >= kPerGroup / 2) != (half == 1)) continue;
+                    mma_ts(tmem_base + d_col, tmem_base + a_col + (kk / kPerGroup) * kDkvCW + within * 8,
+                           sdesc_advance(db, kk * 2048), idesc_acc, (accumulate || kk > 0) ? 1u : 0u);
+                }
             };
             for (int idx = unit_begin; idx < unit_end && ok; ++idx) {
                 const int t = p.cta_tiles[idx];
@@ -288,21 +295,19 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     const bool more = it + 1 < n_it;
                     // dV(it) += P^T dO
                     PROF(7)
-    #ifndef LIBRA_DBG_FREE_MMA
-                    ok = mbar_wait(bar_pready, it_all & 1, abort_flag);
-                    if (!ok) break;
-    #endif
-                    PROF(0)
-    #ifndef LIBRA_DBG_FREE_MMA
-                    if (it == 0 && ucnt > 0) {  // previous unit's dK/dV must have been read out
+                    ok = mbar_wait(bar_phalf, it_all & 1, abort_flag);   // first half of P^T
+                    if (ok && it == 0 && ucnt > 0)                        // previous unit's dK/dV must have been read out
                         ok = mbar_wait(bar_dkvempty, (ucnt - 1) & 1, abort_flag);
-                        if (!ok) break;
-                    }
-    #endif
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_acc(kColDV, kColS, L::kDoOff + st * L::kTileBytes, it > 0, 0);
+                    ok = mbar_wait(bar_pready, it_all & 1, abort_flag);  // second half, while those MMAs run
+                    if (!ok) break;
+                    PROF(0)
                     tc_fence_after();
                     {
                         TRACE(10)
-                        issue_acc(kColDV, kColS, L::kDoOff + st * L::kTileBytes, it > 0);
+                        issue_acc(kColDV, kColS, L::kDoOff + st * L::kTileBytes, it > 0, 1);
                         tc_commit(&bar_doempty[st]);
                         TRACE(11)
                     }
@@ -328,7 +333,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     tc_fence_after();
                     {
                         TRACE(13)
-                        issue_acc(kColDK, kColDP, L::kQOff + st * L::kTileBytes, it > 0);
+                        issue_acc(kColDK, kColDP, L::kQOff + st * L::kTileBytes, it > 0, 2);
                         tc_commit(&bar_qempty[st]);
                         TRACE(14)
                     }
@@ -401,25 +406,36 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 for (int j = 0; j < CW; j += 32) tmem_ld32(t_s + j, sv + j);
                 tmem_ld_wait();
                 float pf[CW];
+                // two halves: the dV key steps over the first half of this group's queries start while the second
+                // half's exponentials are computed (S(it+1) has to wait for all of dV(it), which overwrites nothing
+                // but reads P^T from the columns S(it+1) goes to)
 #pragma unroll
-                for (int j = 0; j < CW; j += 4) {
-                    const float4 l4 = *reinterpret_cast<const float4*>(lse2 + j);
-                    pf[j] = ex2_sel(fmaf(__uint_as_float(sv[j]), p.scale_log2, -l4.x), j);
-                    pf[j + 1] = ex2_sel(fmaf(__uint_as_float(sv[j + 1]), p.scale_log2, -l4.y), j + 1);
-                    pf[j + 2] = ex2_sel(fmaf(__uint_as_float(sv[j + 2]), p.scale_log2, -l4.z), j + 2);
-                    pf[j + 3] = ex2_sel(fmaf(__uint_as_float(sv[j + 3]), p.scale_log2, -l4.w), j + 3);
-                }
-                if (need_mask) {
+                for (int half = 0; half < 2; ++half) {
+                    constexpr int HW = CW / 2;
+                    const int b0 = half * HW;
 #pragma unroll
-                    for (int j = 0; j < CW; ++j)
-                        if (j < j_lo || j > j_hi) pf[j] = 0.f;
-                }
-                {
-                    uint32_t pk[CW / 2];
+                    for (int j = b0; j < b0 + HW; j += 4) {
+                        const float4 l4 = *reinterpret_cast<const float4*>(lse2 + j);
+                        pf[j] = ex2_sel(fmaf(__uint_as_float(sv[j]), p.scale_log2, -l4.x), j);
+                        pf[j + 1] = ex2_sel(fmaf(__uint_as_float(sv[j + 1]), p.scale_log2, -l4.y), j + 1);
+                        pf[j + 2] = ex2_sel(fmaf(__uint_as_float(sv[j + 2]), p.scale_log2, -l4.z), j + 2);
+                        pf[j + 3] = ex2_sel(fmaf(__uint_as_float(sv[j + 3]), p.scale_log2, -l4.w), j + 3);
+                    }
+                    if (need_mask) {
 #pragma unroll
-                    for (int j = 0; j < CW; j += 2) pk[j >> 1] = pack_bf16x2(pf[j], pf[j + 1]);
+                        for (int j = b0; j < b0 + HW; ++j)
+                            if (j < j_lo || j > j_hi) pf[j] = 0.f;
+                    }
+                    uint32_t pk[HW / 2];
+#pragma unroll
+                    for (int j = 0; j < HW; j += 2) pk[j >> 1] = pack_bf16x2(pf[b0 + j], pf[b0 + j + 1]);
                     // packed P^T of this group sits in the first CW / 2 columns of its own S^T range
-                    if constexpr (CW == 64) tmem_st32(t_s, pk); else tmem_st16(t_s, pk);
+                    if constexpr (HW == 32) tmem_st16(t_s + b0 / 2, pk); else tmem_st8(t_s + b0 / 2, pk);
+                    if (half == 0) {
+                        tmem_st_wait();
+                        tc_fence_before();
+                        mbar_arrive(bar_phalf);
+                    }
                 }
                 tmem_st_wait();
                 tc_fence_before();
@@ -467,7 +483,6 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             for (int which = 0; which < 2; ++which) {
                 const float mul = which == 0 ? p.scale : 1.0f;
                 __nv_bfloat16* gdst = (which == 0 ? p.dk : p.dv) + gofs;
-#pragma unroll
                 constexpr int kChunk = kCols < 32 ? kCols : 32;
 #pragma unroll
                 for (int cc = 0; cc < kCols; cc += kChunk) {
