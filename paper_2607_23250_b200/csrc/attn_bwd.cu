@@ -246,7 +246,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             // C[tmem] = A(K-major tile) * B(K-major tile)^T over the head dimension; offsets from smem base
             auto issue_kmajor = [&](uint32_t d_col, uint32_t a_off, uint32_t b_off) {
                 const uint64_t da = sdesc_advance(kdesc0, a_off), db = sdesc_advance(kdesc0, b_off);
-    #pragma unroll
+#pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
                     const uint32_t off = (kk / 4) * L::kHalfBytes + (kk % 4) * 32;
                     mma_ss(tmem_base + d_col, sdesc_advance(da, off), sdesc_advance(db, off), idesc_s, kk > 0);
@@ -325,10 +325,8 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     }
                     // dK(it) += dS^T Q
                     PROF(7)
-    #ifndef LIBRA_DBG_FREE_MMA
                     ok = mbar_wait(bar_dsready, it_all & 1, abort_flag);
                     if (!ok) break;
-    #endif
                     PROF(2)
                     tc_fence_after();
                     {
@@ -372,9 +370,6 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         bool ok = true;
         PROF_DECL
         TRACE_DECL(1 + warp, cta == 0 && lane == 0)
-#if defined(LIBRA_DBG_FREE_MMA) && !defined(LIBRA_DBG_FREE_MMA_COMPUTE_ON)
-        ok = false;
-#endif
         for (int idx = unit_begin; idx < unit_end && ok; ++idx) {
             const int t = p.cta_tiles[idx];
             const int kvh = t % p.hkv;

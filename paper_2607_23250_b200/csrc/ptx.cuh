@@ -37,11 +37,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-#ifdef LIBRA_DBG_TEST_WAIT
-        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-#else
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-#endif
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
         : "r"(smem_u32(bar)), "r"(parity)
@@ -243,15 +239,10 @@ __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.
 
 // ---- small math ---------------------------------------------------------------------------
 __device__ __forceinline__ float ex2_approx(float x) {
-#ifdef LIBRA_DBG_NO_EX2
-    return x * 0.001f;
-#else
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
-#endif
 }
-__device__ __forceinline__ float ex2_approx(float x);
 // 2^x without the special-function unit (the MUFU pipe does 16 exp2 per clock per SM, the FMA
 // pipes 128 flops): round x to the nearest integer n with the magic-number trick, evaluate 2^f on
 // f = x - n in [-0.5, 0.5] with a cubic (relative error < 1e-4, far below bf16 resolution),
