@@ -4,18 +4,20 @@
 // rows; (2) the dK/dV kernel over key-major tiles; (3) the dQ kernel over query-major tiles.
 // Splitting dQ off costs two extra GEMMs per block pair (S and dP are recomputed) but needs no
 // cross-CTA reduction at all: no fp32 dQ accumulator, no atomics, no shared-memory staging, and
-// the result is deterministic.  Both kernels are persistent and warp-specialised (320 threads:
-// warps 0-3 / 4-7 compute groups, warp 8 TMA, warp 9 MMA) and keep their accumulators in TMEM.
+// the result is deterministic.  Both kernels are persistent and warp-specialised (compute warpgroups,
+// one TMA thread, one MMA-issuing thread; the dQ kernel also has a store thread) and keep their
+// accumulators in TMEM.
 //
 // dK/dV kernel: a unit is 128 keys x one kv head; K and V stay in shared memory, dK and dV in
 // TMEM, while the CTA streams every (query head of the group, 128-row query block) that sees the
 // keys.  Keys sit in TMEM lanes:
 //   S^T  = K Q^T   (SS)   P^T  = exp2(S^T c - LSE)   -> bf16 over S^T     dV += P^T dO   (A in TMEM)
 //   dP^T = V dO^T  (SS)   dS^T = P^T o (dP^T - D)    -> bf16 over dP^T    dK += dS^T Q   (A in TMEM)
-// dQ kernel: a unit is 128 query rows x one head; Q and dO stay in shared memory, dQ in TMEM, the
-// CTA streams the key blocks the rows see (as the forward does).  Queries sit in TMEM lanes:
-//   S  = Q K^T (SS, double-buffered)   dP = dO V^T (SS)   dS = P o (dP - D) -> bf16 over S
-//   dQ += dS K (A in TMEM)
+// P^T is handed to the dV MMA in two halves, so half of dV(it) runs under the second half's exponentials.
+// dQ kernel (attn_bwd_dq.cuh): a unit is 128 query rows x one head; Q and dO are copied once per unit from
+// shared memory into TMEM, dQ accumulates in TMEM, the CTA streams the key blocks the rows see (as the
+// forward does).  Queries sit in TMEM lanes:
+//   S  = Q K^T   dP = dO V^T   dS = P o (dP - D) -> bf16 over dP   dQ += dS K     (every A operand in TMEM)
 #include <math.h>
 
 #include "common.h"

@@ -7,11 +7,13 @@
 // pool's token axis, so the diagonal block of a sub-tile is aligned with it and every other
 // visible block is either dense or needs the per-row sample-start mask.
 //
-// Roles (320 threads): warps 0-3 and 4-7 are the softmax groups of slot 0 and 1 (one row per
+// Roles (384 threads): warps 0-3 and 4-7 are the softmax groups of slot 0 and 1 (one row per
 // thread, S read from TMEM, P written back to TMEM as bf16 over S), warp 8 issues TMA loads,
-// warp 9 issues tcgen05.mma.  TMEM: S0 | S1 | O0 | O1, 128 fp32 columns each.
+// warp 9 issues tcgen05.mma, warps 10-11 only hand their registers to the softmax groups.
+// TMEM: S0 | S1 | O0 | O1, 128 fp32 columns each.
 // Pipeline per key block j:   PV0(j) S0(j+1) PV1(j) S1(j+1)   on the tensor pipe, while the
-// softmax group of one slot works during the other slot's MMAs.
+// softmax group of one slot works during the other slot's MMAs.  P is handed over in two halves
+// (keys 0-63, then 64-127), so the first four key steps of PV run under the second half's exponentials.
 #include <math.h>
 
 #include "common.h"
