@@ -238,12 +238,39 @@ def run_ours(args):
     ms_per_step, work = sharding.aggregate(total_ms / args.steps, float(ff + fb), device=dev)
     value = work / (ms_per_step * 1e-3) / 1e12
 
+    # ---- the same steps under the plan's other tile weight (context for the busy-time spread, not the headline)
+    alt = None
+    if world == 1 and not args.skip_e2e:
+        other = not blocks
+        plan2 = lb.libra_plan_tiles(cu, hq, 256, tile_kv=128, n_heads_kv=hkv, total_tokens=T,
+                                    weight_model=lb.LIBRA_WEIGHT_BLOCKS if other else lb.LIBRA_WEIGHT_PAIRS,
+                                    unit_cost_q=12 if other else 0, unit_cost_kv=6 if other else 0)
+
+        def step2():
+            lb.libra_attn_pool_fwd(q, k, v, plan2, out=out, lse=lse)
+            lb.libra_attn_pool_bwd(q, k, v, out, lse, dout, plan2, dq=dq, dk=dk, dv=dv, workspace=ws)
+
+        for _ in range(3):
+            step2()
+        barrier()
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record()
+        for _ in range(args.steps):
+            step2()
+        a1.record()
+        barrier()
+        spread = [plan2.busy_times(kk).astype(np.float64) for kk in (lb.KERNEL_FWD, lb.KERNEL_BWD_DKDV, lb.KERNEL_BWD_DQ)]
+        alt = {"tile_weight": "blocks (time proxy)" if other else "causal pairs (Eq. 6)",
+               "value": round((ff + fb) / (a0.elapsed_time(a1) / args.steps * 1e-3) / 1e12, 2), "unit": "TFLOP/s",
+               "busy_max_over_mean": {n: round(float(b.max() / b.mean()), 4) for n, b in zip(("fwd", "bwd_dkdv", "bwd_dq"), spread)}}
+        plan2.destroy()
+
     e2e = None
     if not args.skip_e2e:
         e2e = run_e2e(args, step_on, barrier, dict(q=q, k=k, v=v, dout=dout),
                       dict(out=out, lse=lse, dq=dq, dk=dk, dv=dv), world, dev, ff + fb)
     finish(args, rank, world, spec, lengths, plan, value, ms_per_step, (kern_f, kern_b, kern_q),
-           (busy_f, busy_b, busy_q), clocks, launches, e2e, ff, fb, q, plan_ms)
+           (busy_f, busy_b, busy_q), clocks, launches, e2e, ff, fb, q, plan_ms, alt)
     plan.destroy()
     if world > 1:
         dist.destroy_process_group()
@@ -310,7 +337,7 @@ def run_e2e(args, step_on, barrier, dev_in, dev_out, world, dev, flops):
 
 
 def finish(args, rank, world, spec, lengths, plan, value, ms_per_step, kern, busy, clocks, launches, e2e, ff, fb, q,
-           plan_ms=None):
+           plan_ms=None, alt=None):
     kern_f, kern_b, kern_q = kern
     busy_f, busy_b, busy_q = busy
     from paper_2607_23250_b200 import binding as lb  # noqa: F401
@@ -351,6 +378,7 @@ def finish(args, rank, world, spec, lengths, plan, value, ms_per_step, kern, bus
             "e2e": e2e,
             "gpu_launches": int(launches),
             "plan_ms": None if plan_ms is None else round(plan_ms, 3),
+            "other_tile_weight": alt,
             "roofline": {"bound": "tensor", "kernel": "k_attn_bwd_dkdv", "achieved": round(ach, 1),
                          "peak": peaks["sustained"], "unit": "TFLOP/s", "frac": round(ach / peaks["sustained"], 4),
                          "peak_kind": f"bf16 sustained, {peaks['source']}", "traffic": traffic,
