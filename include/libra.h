@@ -37,7 +37,7 @@ extern "C" {
 #define LIBRA_ERR_PLAN_MISMATCH (-3)  /* plan was built for another T / head count / direction      */
 #define LIBRA_ERR_CUDA          (-4)  /* a CUDA runtime or driver call failed                        */
 #define LIBRA_ERR_OVERFLOW      (-5)  /* tile ids or loads would not fit their integer types         */
-#define LIBRA_ERR_TIMEOUT       (-6)  /* a bounded device-side wait gave up (reported by libra_status)*/
+#define LIBRA_ERR_TIMEOUT       (-6)  /* a bounded device-side wait gave up (see libra_busy_times)   */
 #define LIBRA_ERR_BAD_SEQLENS   (-7)  /* cu_seqlens failed the device-side check                      */
 #define LIBRA_ERR_NO_DEVICE     (-8)  /* no CUDA device / not an sm_100 device                        */
 #define LIBRA_ERR_SCRATCH_TOO_SMALL (-9) /* problem needs more than the library's built-in scratch    */
@@ -112,9 +112,10 @@ typedef struct {
  * LIBRA_WEIGHT_BLOCKS above; everything else is unchanged.
  * Errors: INVALID_ARG (null, n_samples <= 0, n_heads <= 0, tile_q <= 0, a negative option,
  * an unknown weight model), OVERFLOW (n_heads * T^2 >= 9e15, the bound under which loads fit the
- * placement's packed keys; or
- * (NB * H >= 2^31), CUDA; a malformed cu_seqlens is detected on the device and reported
- * by libra_plan_status as BAD_SEQLENS.
+ * placement's packed keys, or NB * H >= 2^31), CUDA.  A malformed cu_seqlens is detected on the
+ * device and reported by libra_plan_status as BAD_SEQLENS; the per-token sample bounds of such a
+ * plan are clamped into [0, T], and the attention kernels given it do no work: they leave their
+ * outputs untouched and report BAD_SEQLENS through libra_busy_times.
  */
 int libra_plan_tiles(const int32_t* cu_seqlens_dev, int n_samples, int n_heads, int tile_q,
                      const libra_plan_opts* opts /* nullable */, void* stream,
@@ -250,7 +251,10 @@ int libra_vrsp_place(const int64_t* work_dev, int n_sequences, int pool_size, in
  * summed Delta_comm (Eq. 8) of the choices taken.  status_dev int[1]: 0 or LIBRA_ERR_OVERFLOW.
  * seq_offsets_host is a HOST array of n_sequences + 1 entries (read before the call returns).
  * Scratch comes from the stream-ordered allocator and is released on `stream`.
- * Errors: INVALID_ARG, UNSUPPORTED (W > 1024, more than 65536 blocks), CUDA. */
+ * When status_dev reports OVERFLOW (the integer soft-cap test could exceed 64 bits) sigma_dev holds
+ * every tile's Q-home and the byte matrices are zero.
+ * Errors: INVALID_ARG, UNSUPPORTED (W > 1024, more than 65536 blocks), OVERFLOW (the pool's work total
+ * n_shards * T (T + 1) / 2 does not fit 64 bits), CUDA. */
 typedef struct {
     int cp;                 /* workers per packed sequence */
     int block;              /* B, tokens per block */
@@ -268,8 +272,17 @@ int libra_tap_plan(const int32_t* cu_seqlens_dev, int n_samples, const int32_t* 
  * Per-CTA busy time of the most recent launch of kernel `which` (LIBRA_KERNEL_*) that used this
  * plan: nanoseconds between the CTA starting and finishing its tile list, read with the GPU's
  * global timer.  Copies n_workers values to ns_host and synchronises the device.  Returns the
- * kernel status (LIBRA_ERR_TIMEOUT if a bounded wait gave up). */
+ * status of the most recent forward (LIBRA_KERNEL_FWD) or backward (the other two) launch:
+ * LIBRA_OK, LIBRA_ERR_TIMEOUT if a bounded wait gave up, LIBRA_ERR_BAD_SEQLENS if the plan's
+ * cu_seqlens was malformed and the kernels therefore did no work. */
 int libra_busy_times(const libra_plan_t* plan, int which, uint64_t* ns_host);
+
+/* Budget of one device-side wait of the attention kernels launched with this plan, in nanoseconds
+ * (0 restores the default of 2 s, the maximum is 4 s).  Every wait on a barrier inside the kernels
+ * is bounded: a wait that outlives the budget makes its CTA stop issuing work, let the copies and
+ * MMAs it has in flight finish, free its tensor memory and return, and the launch reports
+ * LIBRA_ERR_TIMEOUT through libra_busy_times.  A healthy run never comes near the default. */
+int libra_plan_set_wait_limit_ns(libra_plan_t* plan, uint64_t ns);
 
 /* Kernel timing: when enabled, every forward / backward call records CUDA events on its
  * stream around each persistent kernel (not around the row-statistics launch).

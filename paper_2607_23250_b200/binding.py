@@ -29,7 +29,7 @@ ERR_SCRATCH_TOO_SMALL = -9
 EXPORTS = ["libra_plan_tiles", "libra_plan_info", "libra_plan_status", "libra_plan_export",
            "libra_plan_destroy", "libra_attn_pool_fwd", "libra_attn_pool_bwd_workspace_bytes",
            "libra_attn_pool_bwd", "libra_attn_pool_bwd_noalloc_max_bytes", "libra_attn_pool_bwd_noalloc",
-           "libra_busy_times", "libra_plan_set_timing", "libra_kernel_time_ms", "libra_launch_count",
+           "libra_busy_times", "libra_plan_set_wait_limit_ns", "libra_plan_set_timing", "libra_kernel_time_ms", "libra_launch_count",
            "libra_strerror"]
 
 
@@ -113,6 +113,9 @@ class Plan:
         out = np.zeros(w, np.uint64)
         _check(_lib.libra_busy_times(self._h, which, _np(out)), "libra_busy_times")
         return out
+
+    def set_wait_limit_ns(self, ns: int):
+        _check(_lib.libra_plan_set_wait_limit_ns(self._h, ctypes.c_uint64(ns)), "libra_plan_set_wait_limit_ns")
 
     def set_timing(self, enabled=True):
         _check(_lib.libra_plan_set_timing(self._h, 1 if enabled else 0), "libra_plan_set_timing")

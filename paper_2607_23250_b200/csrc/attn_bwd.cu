@@ -98,6 +98,8 @@ struct DkvParams {
     int hq, hkv;
     float scale, scale_log2;
     int* status;
+    const int* plan_status;  // the planner's verdict on cu_seqlens: non-zero = do not run
+    uint32_t wait_limit_ns;
     uint64_t* busy;
 };
 
@@ -139,6 +141,10 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (threadIdx.x == 0) atomicExch(p.status, LIBRA_ERR_CUDA);
         return;
     }
+    if (const int ps = *p.plan_status; ps != 0) {  // malformed cu_seqlens: report and leave
+        if (threadIdx.x == 0) { atomicExch(p.status, ps); p.busy[2 * cta] = p.busy[2 * cta + 1] = 0; }
+        return;
+    }
     if (threadIdx.x == 0) {
         mbar_init(bar_kvfull, 1);
         mbar_init(bar_kvempty, 1);
@@ -155,7 +161,8 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         mbar_init(bar_dkvfull, 1);
         mbar_init(bar_dkvempty, 128 * kDkvGroups);
         mbar_init(bar_phalf, 128 * kDkvGroups);
-        *abort_flag = 0;
+        abort_flag[0] = 0;
+        abort_flag[1] = (int)p.wait_limit_ns;
         fence_mbar_init();
         p.busy[2 * cta] = globaltimer_ns();
     }
@@ -594,14 +601,14 @@ template <int D>
 static int launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const CUtensorMap& tdo,
                       const CUtensorMap& tdq,
                       const DkvParams& pa, int Wa, const DqParams& pb, int Wb, libra_plan_t* mp, cudaStream_t s) {
-    static bool configured = false;
-    if (!configured) {
+    constexpr int kSlot = D == 128 ? 2 : 3;
+    if (!cfg_done(kSlot)) {   // per device
         if (set_smem(k_attn_bwd_dkdv<D>, DkvSmem<D>::kBytes) != LIBRA_OK) return LIBRA_ERR_CUDA;
         if (set_smem(k_attn_bwd_dq<D>, DqSmem<D>::kBytes) != LIBRA_OK) return LIBRA_ERR_CUDA;
         if (kDkvGroups > 2 && !regs_pool_ok(k_attn_bwd_dkdv<D>, 128 * kDkvGroups, kDkvRegsCompute, 128, kDkvRegsOther))
             return LIBRA_ERR_UNSUPPORTED;
         if (!regs_pool_ok(k_attn_bwd_dq<D>, 128 * kDqGroups, kDqRegsCompute, 128, kDqRegsOther)) return LIBRA_ERR_UNSUPPORTED;
-        configured = true;
+        cfg_mark(kSlot);
     }
     if (mp->timing) cudaEventRecord(mp->ev[1][0], s);
     k_attn_bwd_dkdv<D><<<Wa, kBwdThreads, DkvSmem<D>::kBytes, s>>>(tq, tk, tv, tdo, pa);
@@ -653,6 +660,7 @@ extern "C" int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const v
          (uintptr_t)dq_dev | (uintptr_t)dk_dev | (uintptr_t)dv_dev) & 15)
         return LIBRA_ERR_INVALID_ARG;
     if ((uintptr_t)workspace_dev & 255) return LIBRA_ERR_INVALID_ARG;
+    if (int rcd = check_plan_device(plan); rcd != LIBRA_OK) return rcd;
 
     const int D = dims->head_dim;
     const int64_t T = plan->T;
@@ -660,6 +668,7 @@ extern "C" int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const v
     float* dvec = reinterpret_cast<float*>(workspace_dev);
     float* lse2 = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(workspace_dev) + ws.stat_bytes);
     cudaStream_t s = (cudaStream_t)stream;
+    cudaMemsetAsync(plan->d_status + 2, 0, sizeof(int), s);   // the word reports the most recent launch
 
     CUtensorMap tq, tk, tv, tdo, tdq;
     int rc = make_thd_map(&tq, q_dev, T, dims->hq, D, kBlk);
@@ -696,6 +705,8 @@ extern "C" int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const v
     pa.scale = scale;
     pa.scale_log2 = scale * 1.4426950408889634f;
     pa.status = plan->d_status + 2;
+    pa.plan_status = plan->d_status;
+    pa.wait_limit_ns = plan->wait_limit_ns;
     pa.busy = dkv_dir.d_busy;
     DqParams pb;
     pb.dq = reinterpret_cast<__nv_bfloat16*>(dq_dev);
@@ -712,6 +723,8 @@ extern "C" int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const v
     pb.scale = scale;
     pb.scale_log2 = scale * 1.4426950408889634f;
     pb.status = plan->d_status + 2;
+    pb.plan_status = plan->d_status;
+    pb.wait_limit_ns = plan->wait_limit_ns;
     pb.busy = dq_dir.d_busy2;
     libra_plan_t* mp = const_cast<libra_plan_t*>(plan);
     return D == 128 ? launch_bwd<128>(tq, tk, tv, tdo, tdq, pa, dkv_dir.W, pb, dq_dir.W, mp, s)

@@ -62,6 +62,8 @@ struct DqParams {
     int hq, hkv, H;
     float scale, scale_log2;
     int* status;
+    const int* plan_status;
+    uint32_t wait_limit_ns;
     uint64_t* busy;
 };
 
@@ -143,6 +145,10 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         if (threadIdx.x == 0) atomicExch(p.status, LIBRA_ERR_CUDA);
         return;
     }
+    if (const int ps = *p.plan_status; ps != 0) {  // malformed cu_seqlens: report and leave
+        if (threadIdx.x == 0) { atomicExch(p.status, ps); p.busy[2 * cta] = p.busy[2 * cta + 1] = 0; }
+        return;
+    }
     if (threadIdx.x == 0) {
         mbar_init(bar_qfull, 1);
         mbar_init(bar_qempty, 1);                // the thread that stores dQ through the Q tile
@@ -159,7 +165,8 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         mbar_init(bar_dpfull, 1);
         mbar_init(bar_dsready, 128 * kDqGroups);
         mbar_init(bar_dqfull, 1);
-        *abort_flag = 0;
+        abort_flag[0] = 0;
+        abort_flag[1] = (int)p.wait_limit_ns;
         fence_mbar_init();
         p.busy[2 * cta] = globaltimer_ns();
     }

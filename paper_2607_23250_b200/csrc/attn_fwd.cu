@@ -56,6 +56,8 @@ struct FwdParams {
     int hq, hkv, H;
     float scale_log2;  // softmax scale * log2(e)
     int* status;       // word to flag LIBRA_ERR_TIMEOUT in
+    const int* plan_status;  // the planner's verdict on cu_seqlens: non-zero = do not run
+    uint32_t wait_limit_ns;  // budget of one device-side wait
     uint64_t* busy;    // [2 * gridDim.x]
 };
 
@@ -119,6 +121,11 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     const int lane = threadIdx.x & 31;
     const int cta = blockIdx.x;
 
+    // A plan whose cu_seqlens failed the planner's check is never executed: report and leave.
+    if (const int ps = *p.plan_status; ps != 0) {
+        if (threadIdx.x == 0) { atomicExch(p.status, ps); p.busy[2 * cta] = p.busy[2 * cta + 1] = 0; }
+        return;
+    }
     if (threadIdx.x == 0) {
         for (int i = 0; i < L::kStages; ++i) { mbar_init(&bar_full[i], 1); mbar_init(&bar_empty[i], 1); }
         mbar_init(bar_qfull, 1);
@@ -129,7 +136,8 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             mbar_init(&bar_odone[g], 1);
             mbar_init(&bar_phalf[g], kBM);
         }
-        *abort_flag = 0;
+        abort_flag[0] = 0;
+        abort_flag[1] = (int)p.wait_limit_ns;
         fence_mbar_init();
         p.busy[2 * cta] = globaltimer_ns();
     }
@@ -534,12 +542,12 @@ template <int D>
 static int launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& prm, int W,
                       cudaStream_t s) {
     using L = FwdSmem<D>;
-    static bool configured = false;
-    if (!configured) {
+    constexpr int kSlot = D == 128 ? 0 : 1;
+    if (!cfg_done(kSlot)) {   // per device: the attribute belongs to the device's copy of the kernel
         if (cudaFuncSetAttribute(k_attn_fwd<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kAlloc) != cudaSuccess)
             return LIBRA_ERR_CUDA;
         if (!regs_pool_ok(k_attn_fwd<D>, 256, LIBRA_FWD_REG_INC, 128, LIBRA_FWD_REG_DEC)) return LIBRA_ERR_UNSUPPORTED;
-        configured = true;
+        cfg_mark(kSlot);
     }
     k_attn_fwd<D><<<W, kFwdThreads, L::kAlloc, s>>>(tq, tk, tv, prm);
     count_launch();
@@ -569,6 +577,7 @@ extern "C" int libra_attn_pool_fwd(const void* q_dev, const void* k_dev, const v
     if (dims->hq % d.H) return LIBRA_ERR_INVALID_ARG;
     if (d.W > plan->sm_count) return LIBRA_ERR_UNSUPPORTED;  // one CTA per SM owns all 512 TMEM columns
     if (((uintptr_t)q_dev | (uintptr_t)k_dev | (uintptr_t)v_dev | (uintptr_t)out_dev) & 15) return LIBRA_ERR_INVALID_ARG;
+    if (int rcd = check_plan_device(plan); rcd != LIBRA_OK) return rcd;
 
     CUtensorMap tq, tk, tv;
     int rc = make_thd_map(&tq, q_dev, plan->T, dims->hq, dims->head_dim, kBM);
@@ -589,8 +598,11 @@ extern "C" int libra_attn_pool_fwd(const void* q_dev, const void* k_dev, const v
     const float scale = dims->softmax_scale > 0.f ? dims->softmax_scale : 1.0f / sqrtf((float)dims->head_dim);
     prm.scale_log2 = scale * 1.4426950408889634f;
     prm.status = plan->d_status + 1;
+    prm.plan_status = plan->d_status;
+    prm.wait_limit_ns = plan->wait_limit_ns;
     prm.busy = d.d_busy;
     cudaStream_t s = (cudaStream_t)stream;
+    cudaMemsetAsync(plan->d_status + 1, 0, sizeof(int), s);   // the word reports the most recent launch
     libra_plan_t* mp = const_cast<libra_plan_t*>(plan);
     if (mp->timing) cudaEventRecord(mp->ev[0][0], s);
     rc = dims->head_dim == 128 ? launch_fwd<128>(tq, tk, tv, prm, d.W, s) : launch_fwd<64>(tq, tk, tv, prm, d.W, s);

@@ -42,12 +42,22 @@ struct libra_plan {
     int32_t* d_tok_end = nullptr;    // [T] one past the last token of that sample
     int* d_status = nullptr;         // [4] word 0: plan status; word 1: fwd; word 2: bwd
     libra::PlanDir dir[2];           // 0 = query-major, 1 = key-major
+    uint32_t wait_limit_ns = 2000000000u;  // budget of one device-side wait (libra_plan_set_wait_limit_ns)
     int timing = 0;                  // record events around the main kernels
     cudaEvent_t ev[3][2] = {{nullptr, nullptr}, {nullptr, nullptr}, {nullptr, nullptr}};  // [kernel][begin, end]
     int ev_valid[3] = {0, 0, 0};
 };
 
 namespace libra {
+// Per-device one-time kernel configuration (dynamic shared memory size, register-pool check).  The
+// attributes are per device, so the flag is kept per device ordinal; `slot` is a small integer the
+// caller picks per kernel family.  Returns true when this (device, slot) has been configured.
+constexpr int kMaxDevices = 64;
+constexpr int kCfgSlots = 16;
+bool cfg_done(int slot);
+void cfg_mark(int slot);
+// LIBRA_ERR_PLAN_MISMATCH when the current device is not the one the plan was built on.
+int check_plan_device(const libra_plan* plan);
 extern std::atomic<int64_t> g_launches;
 inline void count_launch(int n = 1) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 }  // namespace libra

@@ -12,6 +12,23 @@ namespace libra {
 
 std::atomic<int64_t> g_launches{0};
 
+static std::atomic<int> g_cfg[kMaxDevices][kCfgSlots];
+bool cfg_done(int slot) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return false;
+    return g_cfg[dev][slot].load(std::memory_order_acquire) != 0;
+}
+void cfg_mark(int slot) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return;
+    g_cfg[dev][slot].store(1, std::memory_order_release);
+}
+int check_plan_device(const libra_plan* plan) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return LIBRA_ERR_NO_DEVICE;
+    return dev == plan->device ? LIBRA_OK : LIBRA_ERR_PLAN_MISMATCH;
+}
+
 // ---- kernels --------------------------------------------------------------------------------
 
 // cu_seqlens checks: starts at 0, non-decreasing, ends at T.
@@ -26,7 +43,9 @@ __global__ void k_validate(const int32_t* __restrict__ cu, int n, int64_t T, int
 }
 
 // For every token: the bounds [start, end) of the sample that holds it.
-// upper_bound keeps every index inside [0, n] whatever cu contains.
+// The search keeps every index inside [0, n] whatever cu contains, and the bounds are clamped to
+// start <= t < end <= T, so that a malformed cu_seqlens (flagged by k_validate) can never make a
+// later kernel form an address outside its tensors.
 __global__ void k_token_bounds(const int32_t* __restrict__ cu, int n, int64_t T, int32_t* __restrict__ tok_start,
                                int32_t* __restrict__ tok_end) {
     const int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
@@ -36,8 +55,9 @@ __global__ void k_token_bounds(const int32_t* __restrict__ cu, int n, int64_t T,
         const int mid = (lo + hi) >> 1;
         if (cu[mid] <= t) lo = mid; else hi = mid;
     }
-    tok_start[t] = cu[lo];
-    tok_end[t] = cu[lo + 1];
+    const int64_t a = cu[lo], e = cu[lo + 1];
+    tok_start[t] = (int32_t)(a < 0 ? 0 : (a > t ? t : a));
+    tok_end[t] = (int32_t)(e < t + 1 ? t + 1 : (e > T ? T : e));
 }
 
 // Weight of block b (Eq. 6): a token at position p of a sample of length len contributes
@@ -177,8 +197,9 @@ __global__ void k_scatter_lists(const int32_t* __restrict__ cta_of_tile, const i
 
 // Execution order inside a worker's list.  The placement fixes WHICH tiles a worker runs; the order
 // it runs them in is free.  Sorting every list by (head shard, block) makes all workers sweep
-// the same head and neighbouring blocks at about the same time, so K/V re-reads and the
-// backward's dQ atomics hit L2 instead of DRAM.  One thread block per worker, rank sort.
+// the same head and neighbouring blocks at about the same time, so that the tiles several workers
+// read (K/V in the forward and the dQ kernel, Q/dO in the dK/dV kernel) are more often found in L2.
+// One thread block per worker, rank sort.
 __global__ void k_exec_order(const int32_t* __restrict__ cta_offsets, const int32_t* __restrict__ cta_tiles, int H,
                              int64_t NB, int32_t* __restrict__ cta_exec) {
     const int r = blockIdx.x;
@@ -440,6 +461,12 @@ extern "C" int libra_plan_set_timing(libra_plan_t* plan, int enabled) {
                 if (!plan->ev[a][b] && cudaEventCreate(&plan->ev[a][b]) != cudaSuccess) return LIBRA_ERR_CUDA;
     }
     plan->timing = enabled ? 1 : 0;
+    return LIBRA_OK;
+}
+
+extern "C" int libra_plan_set_wait_limit_ns(libra_plan_t* plan, uint64_t ns) {
+    if (!plan || ns > 4000000000ull) return LIBRA_ERR_INVALID_ARG;
+    plan->wait_limit_ns = ns ? (uint32_t)ns : 2000000000u;
     return LIBRA_OK;
 }
 

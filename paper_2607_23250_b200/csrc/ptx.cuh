@@ -46,25 +46,39 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 }
 
 // Wall-clock budget of one wait.  A healthy kernel never waits longer than microseconds to
-// milliseconds; the limit only ends a wait that can no longer be satisfied.
+// milliseconds; the limit only ends a wait that can no longer be satisfied.  The kernels keep two
+// control words in shared memory: ctl[0] = abort flag, ctl[1] = the budget in nanoseconds (set by
+// the host per launch, LIBRA_WAIT_LIMIT_NS when the plan does not override it).
 #ifndef LIBRA_WAIT_LIMIT_NS
-#define LIBRA_WAIT_LIMIT_NS 2000000000ull
+#define LIBRA_WAIT_LIMIT_NS 2000000000u
 #endif
 
 // Returns true when the phase with the given parity has completed, false on timeout or when
-// another thread has already flagged an abort in *abort_flag (shared memory).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+// another thread has already flagged an abort in ctl[0] (shared memory).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* ctl) {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = globaltimer_ns();
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 0x3ff) == 0) {
-            if (*abort_flag) return false;
-            if (globaltimer_ns() - t0 > LIBRA_WAIT_LIMIT_NS) {
-                *abort_flag = 1;
+            if (ctl[0]) return false;
+            if (globaltimer_ns() - t0 > (uint64_t)(uint32_t)ctl[1]) {
+                ctl[0] = 1;
                 return false;
             }
         }
+    }
+    return true;
+}
+// The same wait for the teardown of a CTA that has given up: it ignores the abort flag (which is
+// set by then) and has its own budget, so that copies and MMAs already in flight can land before
+// shared memory and TMEM are released.
+__device__ __forceinline__ bool mbar_wait_drain(uint64_t* bar, uint32_t parity, uint64_t budget_ns) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = globaltimer_ns();
+    uint32_t spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 0xff) == 0 && globaltimer_ns() - t0 > budget_ns) return false;
     }
     return true;
 }
@@ -82,7 +96,7 @@ __device__ __forceinline__ bool elect_one() {
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* m) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(m)) : "memory");
 }
-// 3-D tiled load (no multicast): coordinates (c0 = innermost element, c1, c2).
+// 3-D tiled load into this CTA's shared memory: coordinates (c0 = innermost element, c1, c2).
 __device__ __forceinline__ void tma_load_3d(void* smem_dst, const CUtensorMap* m, uint64_t* bar, int c0,
                                             int c1, int c2) {
     asm volatile(

@@ -154,7 +154,8 @@ __global__ void __launch_bounds__(1024) k_tap_place(
     int64_t sum_f = 0;
     for (int w = 0; w < nwarps; ++w) sum_f += s_sum[w];
     if (sum_f > (INT64_MAX / ((int64_t)(tau_den + tau_num) * 2)) / W) {  // the integer cap test would overflow
-        if (r == 0) *status = LIBRA_ERR_OVERFLOW;
+        if (r == 0) *status = LIBRA_ERR_OVERFLOW;   // the exchange kernels see the flag and add nothing
+        for (int64_t t = r; t < NB * H; t += blockDim.x) sigma[t] = q_home[t / H];   // defined output: every tile stays home
         return;
     }
     const int64_t cap_rhs = (int64_t)(tau_den + tau_num) * sum_f;
@@ -211,11 +212,12 @@ __global__ void __launch_bounds__(1024) k_tap_place(
 // Forward / backward send-byte matrices [src][dst].
 __global__ void k_tap_exchange_qo(const int32_t* __restrict__ sigma, const int32_t* __restrict__ q_home,
                                   const int64_t* __restrict__ v_qo, int64_t NT, int H, int W,
-                                  unsigned long long* __restrict__ fwd, unsigned long long* __restrict__ bwd) {
+                                  const int* __restrict__ status, unsigned long long* __restrict__ fwd,
+                                  unsigned long long* __restrict__ bwd) {
     const int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-    if (t >= NT) return;
+    if (t >= NT || *status != 0) return;   // a placement that gave up left sigma unwritten
     const int q = q_home[t / H], r = sigma[t];
-    if (q == r) return;
+    if (q == r || r < 0 || r >= W || q < 0 || q >= W) return;
     const unsigned long long v = (unsigned long long)(v_qo[t / H] / 2);
     atomicAdd(&fwd[(size_t)q * W + r], v);   // Q out
     atomicAdd(&fwd[(size_t)r * W + q], v);   // output back
@@ -223,11 +225,11 @@ __global__ void k_tap_exchange_qo(const int32_t* __restrict__ sigma, const int32
     atomicAdd(&bwd[(size_t)r * W + q], v);   // dQ along the output path
 }
 __global__ void k_tap_exchange_kv(TapGeom g, const uint32_t* __restrict__ Cbits, int words,
-                                  const int32_t* __restrict__ res_smp, int W, unsigned long long* __restrict__ fwd,
-                                  unsigned long long* __restrict__ bwd) {
+                                  const int32_t* __restrict__ res_smp, int W, const int* __restrict__ status,
+                                  unsigned long long* __restrict__ fwd, unsigned long long* __restrict__ bwd) {
     const int64_t idx = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
     const int64_t NG = (int64_t)g.n * g.H;
-    if (idx >= NG * W) return;
+    if (idx >= NG * W || *status != 0) return;
     const int r = (int)(idx / NG);
     const int grp = (int)(idx % NG), j = grp / g.H;
     if (!((Cbits[(size_t)r * words + (grp >> 5)] >> (grp & 31)) & 1u) || res_smp[j] == r) return;
@@ -279,6 +281,10 @@ extern "C" int libra_tap_plan(const int32_t* cu_seqlens_dev, int n_samples, cons
     if (NT <= 0) return LIBRA_ERR_INVALID_ARG;
     const int64_t NB = NT / H;
     if (NT >= INT32_MAX || NB > 65536) return LIBRA_ERR_UNSUPPORTED;  // the rank sort is quadratic in blocks
+    {   // the work total (at most H * T (T + 1) / 2) must itself fit 64 bits before the device can test the cap
+        const long double Tl = (long double)seq_offsets_host[P] - (long double)seq_offsets_host[0];
+        if ((long double)H * Tl * (Tl + 1) / 2 > 4.0e18L) return LIBRA_ERR_OVERFLOW;
+    }
     cudaStream_t s = (cudaStream_t)stream;
     const int words = (int)(((int64_t)n_samples * H + 31) / 32);
 
@@ -332,11 +338,11 @@ extern "C" int libra_tap_plan(const int32_t* cu_seqlens_dev, int n_samples, cons
         k_tap_place<<<1, ((W + 31) / 32) * 32, 0, s>>>(f_blk, ord, q_home, v_qo, j0, j1, v_smp, res_smp, NB, H, W,
                                                         n_samples, o->tau_num, o->tau_den, cbits, words, sigma_dev,
                                                         loads_dev, comm_total_dev, status_dev);
-        k_tap_exchange_qo<<<(unsigned)((NT + 255) / 256), 256, 0, s>>>(sigma_dev, q_home, v_qo, NT, H, W,
+        k_tap_exchange_qo<<<(unsigned)((NT + 255) / 256), 256, 0, s>>>(sigma_dev, q_home, v_qo, NT, H, W, status_dev,
                                                                        (unsigned long long*)fwd_bytes_dev,
                                                                        (unsigned long long*)bwd_bytes_dev);
         const int64_t pairs = (int64_t)n_samples * H * W;
-        k_tap_exchange_kv<<<(unsigned)((pairs + 255) / 256), 256, 0, s>>>(g, cbits, words, res_smp, W,
+        k_tap_exchange_kv<<<(unsigned)((pairs + 255) / 256), 256, 0, s>>>(g, cbits, words, res_smp, W, status_dev,
                                                                           (unsigned long long*)fwd_bytes_dev,
                                                                           (unsigned long long*)bwd_bytes_dev);
         count_launch(6);

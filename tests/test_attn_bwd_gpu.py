@@ -90,3 +90,10 @@ def test_single_token_pool():
     # a length-1 sample has dQ = dK = 0 and dV = sum over the group of dO
     assert np.abs(got[0]).max() < 1e-6 and np.abs(got[1]).max() < 1e-6
     assert rel_to_max(got[2], ref[2]) <= TOL_G
+
+
+@pytest.mark.parametrize("hq,hkv", [(64, 4), (128, 4)], ids=["G16", "G32"])
+def test_wide_query_head_groups(hq, hkv):
+    """Sixteen and thirty-two query heads per kv head at head_dim 128: dK / dV sum over the whole group."""
+    got, ref, cu = _run([700, 1, 300, 129, 411], hq, hkv, 128, seed=31)
+    _check(got, ref, cu)

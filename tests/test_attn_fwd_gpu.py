@@ -25,7 +25,7 @@ def _run(lengths, hq, hkv, d, seed=0, H=None, W=0, qscale=1.0, kshift=0.0):
     plan = lb.libra_plan_tiles(cu, H or hq, 256, n_workers=W, directions=lb.LIBRA_DIR_Q)
     out, lse = lb.libra_attn_pool_fwd(q, k, v, plan)
     torch.cuda.synchronize()
-    st = lb._lib.libra_busy_times(plan._h, lb.LIBRA_DIR_Q, np.zeros(plan.info()["n_workers"], np.uint64).ctypes.data_as(lb._vp))
+    st = lb._lib.libra_busy_times(plan._h, lb.KERNEL_FWD, np.zeros(plan.info()["n_workers"], np.uint64).ctypes.data_as(lb._vp))
     assert st == 0, f"kernel status {st}"
     o_ref, l_ref = oracle.attn_fwd(t["q"].float().numpy(), t["k"].float().numpy(), t["v"].float().numpy(), cu_np)
     o = out.float().cpu().numpy()
@@ -84,4 +84,12 @@ def test_peaked_softmax_and_score_offset():
 
 def test_single_token_pool():
     o, l, o_ref, l_ref, cu = _run([1], 1, 1, 64, seed=6)
+    _check(o, l, o_ref, l_ref, cu)
+
+
+@pytest.mark.parametrize("hq,hkv", [(64, 4), (128, 4)], ids=["G16", "G32"])
+def test_wide_query_head_groups(hq, hkv):
+    """Sixteen and thirty-two query heads per kv head (the 235B-shaped and the micro-benchmark head counts of
+    the paper's Table 1) at head_dim 128, several samples, ragged tail."""
+    o, l, o_ref, l_ref, cu = _run([700, 1, 300, 129, 411], hq, hkv, 128, seed=31, H=hq // 2)
     _check(o, l, o_ref, l_ref, cu)

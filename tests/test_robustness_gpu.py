@@ -1,0 +1,82 @@
+"""Error paths that must be reported, never executed: a malformed cu_seqlens, a planner that gives up, a plan used
+on the wrong arguments.  Nothing here provokes a fault or a hang: the guards under test skip the work."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2607_23250_b200 import pools
+
+pytestmark = pytest.mark.gpu
+
+
+def test_malformed_cu_seqlens_is_flagged_and_attention_does_no_work():
+    from paper_2607_23250_b200 import binding as lb
+    T, hq, hkv, d = 472, 2, 1, 128
+    cu = torch.tensor([0, 5000, 100, T], dtype=torch.int32).cuda()        # not monotone, offset beyond T
+    plan = lb.libra_plan_tiles(cu, hq, 256, tile_kv=128, n_heads_kv=hkv, total_tokens=T)
+    assert plan.status() == lb.ERR_BAD_SEQLENS
+    t = pools.make_tensors(T, hq, hkv, d, seed=1, device="cuda")
+    sentinel = 7.0
+    out = torch.full_like(t["q"], sentinel)
+    lse = torch.full((hq, T), sentinel, dtype=torch.float32, device="cuda")
+    lb.libra_attn_pool_fwd(t["q"], t["k"], t["v"], plan, out=out, lse=lse)
+    with pytest.raises(lb.LibraError) as err:
+        plan.busy_times(lb.KERNEL_FWD)
+    assert err.value.code == lb.ERR_BAD_SEQLENS
+    assert bool((out == sentinel).all()) and bool((lse == sentinel).all())     # untouched
+    dq, dk, dv = (torch.full_like(x, sentinel) for x in (t["q"], t["k"], t["v"]))
+    lb.libra_attn_pool_bwd(t["q"], t["k"], t["v"], out, lse, t["dout"], plan, dq=dq, dk=dk, dv=dv)
+    for kern in (lb.KERNEL_BWD_DKDV, lb.KERNEL_BWD_DQ):
+        with pytest.raises(lb.LibraError) as err:
+            plan.busy_times(kern)
+        assert err.value.code == lb.ERR_BAD_SEQLENS
+    for g in (dq, dk, dv):
+        assert bool((g == sentinel).all())
+    plan.destroy()
+    # a good plan on the same GPU right afterwards works and reports OK
+    cu = torch.tensor([0, 300, T], dtype=torch.int32).cuda()
+    plan = lb.libra_plan_tiles(cu, hq, 256, tile_kv=128, n_heads_kv=hkv)
+    assert plan.status() == 0
+    out, lse = lb.libra_attn_pool_fwd(t["q"], t["k"], t["v"], plan)
+    plan.busy_times(lb.KERNEL_FWD)
+    assert bool(torch.isfinite(out).all())
+    plan.destroy()
+
+
+def test_token_bounds_of_a_malformed_plan_stay_inside_the_pool():
+    """The per-token sample bounds are clamped, so even the exported weights of a bad plan are finite sums."""
+    from paper_2607_23250_b200 import binding as lb
+    T = 1000
+    cu = torch.tensor([0, 900000, 50, T], dtype=torch.int32).cuda()
+    plan = lb.libra_plan_tiles(cu, 1, 256, tile_kv=128, n_heads_kv=1, total_tokens=T)
+    assert plan.status() == lb.ERR_BAD_SEQLENS
+    for direction in (lb.LIBRA_DIR_Q, lb.LIBRA_DIR_KV):
+        w = plan.export(direction)["weight"]
+        assert (w >= 0).all() and int(w.sum()) <= T * (T + 1) // 2
+    plan.destroy()
+
+
+def test_pool_planner_overflow_leaves_defined_outputs():
+    """One sample so long that the integer soft-cap test could overflow: the planner reports OVERFLOW, every tile
+    stays at its Q-home and the byte matrices stay zero.  Needs offsets only, no tensors."""
+    from paper_2607_23250_b200 import binding as lb
+    L = 1_200_000          # 64 shards x L (L + 1) / 2 pairs = 4.6e13 > the bound of about 4.4e13 at 1024 workers
+    cu = torch.tensor([0, L], dtype=torch.int32).cuda()
+    res = lb.libra_tap_plan(cu, [0, L], cp=1024, block=32768, n_shards=64, hq=64, hkv=4, head_dim=128)
+    torch.cuda.synchronize()
+    assert int(res["status"].item()) == lb.ERR_OVERFLOW
+    assert int(res["fwd_bytes"].abs().sum().item()) == 0 and int(res["bwd_bytes"].abs().sum().item()) == 0
+    sigma = res["sigma"].cpu().numpy()
+    assert sigma.min() >= 0 and sigma.max() < 1024
+
+
+def test_plan_of_another_device_or_shape_is_refused():
+    from paper_2607_23250_b200 import binding as lb
+    cu = torch.tensor([0, 256], dtype=torch.int32).cuda()
+    plan = lb.libra_plan_tiles(cu, 2, 256, tile_kv=128, n_heads_kv=1)
+    q = torch.zeros((512, 2, 128), dtype=torch.bfloat16, device="cuda")         # T differs from the plan's
+    k = torch.zeros((512, 1, 128), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(lb.LibraError) as err:
+        lb.libra_attn_pool_fwd(q, k, k, plan)
+    assert err.value.code == lb.ERR_PLAN_MISMATCH
+    plan.destroy()
