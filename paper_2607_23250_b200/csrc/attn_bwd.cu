@@ -11,8 +11,12 @@
 // dK/dV kernel: a unit is 128 keys x one kv head; K and V stay in shared memory, dK and dV in
 // TMEM, while the CTA streams every (query head of the group, 128-row query block) that sees the
 // keys.  Keys sit in TMEM lanes:
-//   S^T  = K Q^T   (SS)   P^T  = exp2(S^T c - LSE)   -> bf16 over S^T     dV += P^T dO   (A in TMEM)
-//   dP^T = V dO^T  (SS)   dS^T = P^T o (dP^T - D)    -> bf16 over dP^T    dK += dS^T Q   (A in TMEM)
+//   S^T  = K Q^T   (SS)   P^T  = exp2(S^T c - LSE)   -> bf16, own columns     dV += P^T dO   (A in TMEM)
+//   dP^T = V dO^T  (SS)   dS^T = P^T o (dP^T - D)    -> bf16, own columns     dK += dS^T Q   (A in TMEM)
+// TMEM: X | P^T | dS^T | dK | dV = 128 + 64 + 64 + D + D columns.  S^T and dP^T take turns in the one fp32
+// region X: it is free again as soon as the compute groups have READ it, not when the MMA that consumes the
+// bf16 result has run, so dP^T(it) is issued right after S^T(it) has been read and S^T(it+1) right after
+// dP^T(it) has been read, while dV(it) and dK(it) read P^T / dS^T from their own columns.
 // P^T is handed to the dV MMA in two halves, so half of dV(it) runs under the second half's exponentials.
 // dQ kernel (attn_bwd_dq.cuh): a unit is 128 query rows x one head; Q and dO are copied once per unit from
 // shared memory into TMEM, dQ accumulates in TMEM, the CTA streams the key blocks the rows see (as the
@@ -25,18 +29,18 @@
 
 namespace libra {
 
-#ifndef LIBRA_DKV_GROUPS
-#define LIBRA_DKV_GROUPS 2
-#endif
-constexpr int kDkvGroups = LIBRA_DKV_GROUPS;            // compute warpgroups: each owns 128 / kDkvGroups query columns
-constexpr int kDkvCW = 128 / kDkvGroups;                // S^T / dP^T columns per compute thread
-constexpr int kDkvTmaWarp = 4 * kDkvGroups, kDkvMmaWarp = 4 * kDkvGroups + 1;
-// two groups: 10 warps at 168 registers; four groups: the producer / MMA warps get a warpgroup of their own
-// (two of its warps idle) and hand registers to the compute groups, as in the dQ kernel
-constexpr int kBwdThreads = kDkvGroups == 2 ? 320 : (4 * kDkvGroups + 4) * 32;
-constexpr int kDkvRegsCompute = 104, kDkvRegsOther = 40;
+#define PROF_DECL
+#define PROF(k)
+#define PROF_FLUSH(cond, base)
+
+// warps 0-3, 4-7: exp groups (64 query columns each), 8-11: dS group, 12: TMA thread, 13: MMA thread,
+// 14-15 only hand their registers over
+constexpr int kBwdThreads = 512;
+constexpr int kDkvTmaWarp = 12, kDkvMmaWarp = 13;
+constexpr int kDkvRegsDs = 200, kDkvRegsOther = 56;   // setmaxnreg: the dS group keeps a whole row of dP^T in registers
 constexpr int kBlk = 128;
 constexpr int kSmemMax = 232448;  // 227 KB per CTA on sm_100
+constexpr uint64_t kDrainNs = 2000000;  // teardown after a give-up: budget for work already in flight to land
 
 __device__ __forceinline__ void bulk_load_1d(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
@@ -44,25 +48,6 @@ __device__ __forceinline__ void bulk_load_1d(void* smem_dst, const void* gsrc, u
                  "l"(reinterpret_cast<uint64_t>(gsrc)), "r"(bytes), "r"(smem_u32(bar))
                  : "memory");
 }
-
-#ifdef LIBRA_PROF
-// Profiling build only: per-CTA cycle sums of the phases of one thread per role.
-__device__ unsigned long long g_bwd_prof[1024 * 24];
-struct Prof {
-    long long last;
-    unsigned long long acc[8];
-    __device__ void start() { last = clock64(); for (int i = 0; i < 8; ++i) acc[i] = 0; }
-    __device__ void mark(int k) { const long long now = clock64(); acc[k] += now - last; last = now; }
-    __device__ void flush(int cta, int base) { for (int i = 0; i < 8; ++i) g_bwd_prof[cta * 24 + base + i] = acc[i]; }
-};
-#define PROF_DECL Prof prof; prof.start();
-#define PROF(k) prof.mark(k);
-#define PROF_FLUSH(cond, base) if (cond) prof.flush(cta, base);
-#else
-#define PROF_DECL
-#define PROF(k)
-#define PROF_FLUSH(cond, base)
-#endif
 
 // =================================================================================================
 // dK / dV kernel
@@ -72,15 +57,18 @@ template <int D>
 struct DkvSmem {
     static constexpr int kHalfBytes = 128 * 128;
     static constexpr int kTileBytes = kHalfBytes * (D / 64);  // 128 x D bf16
+    static constexpr int kQStages = 3;   // Q(it) lives from S(it) to dK(it), which runs behind dP(it+1)
+    static constexpr int kDoStages = 2;  // dO(it) lives from dP(it) to dV(it)
     static constexpr int kKOff = 0;
     static constexpr int kVOff = kTileBytes;
-    static constexpr int kQOff = 2 * kTileBytes;   // 2 stages
-    static constexpr int kDoOff = 4 * kTileBytes;  // 2 stages
-    static constexpr int kStatOff = 6 * kTileBytes;  // per Q stage: lse2[128], dvec[128]
-    static constexpr int kBarOff = kStatOff + 2 * 1024;
-    // kv_full, kv_empty, q_full[2], q_empty[2], do_full[2], do_empty[2], s_full, p_ready, dp_full,
-    // ds_ready, dkv_full, dkv_empty, p_half
-    static constexpr int kNumBars = 17;
+    static constexpr int kQOff = 2 * kTileBytes;
+    static constexpr int kDoOff = kQOff + kQStages * kTileBytes;
+    static constexpr int kLseOff = kDoOff + kDoStages * kTileBytes;  // per Q stage:  lse2[128]
+    static constexpr int kDvecOff = kLseOff + kQStages * 512;        // per dO stage: dvec[128]
+    static constexpr int kBarOff = kDvecOff + kDoStages * 512;
+    // kv_full, kv_empty, q_full[3], q_empty[3], do_full[2], do_empty[2], s_full, x_free1, dp_full, x_free2,
+    // p_half, p_ready, p_free, ds_ready, dkv_full, dkv_empty, drain
+    static constexpr int kNumBars = 2 + 2 * kQStages + 2 * kDoStages + 11;
     static constexpr int kMiscOff = kBarOff + kNumBars * 8;
     static constexpr int kBytes = kMiscOff + 16;
     static_assert(kBytes <= kSmemMax, "exceeds the shared memory of an sm_100 CTA");
@@ -109,27 +97,39 @@ __device__ __forceinline__ int last_q_block(const int32_t* tok_end, int64_t T, i
     return (tok_end[last_key] - 1) / kBlk;
 }
 
+__device__ __forceinline__ void tmem_ld128(uint32_t taddr, uint32_t* r) {
+    tmem_ld32(taddr, r);
+    tmem_ld32(taddr + 32, r + 32);
+    tmem_ld32(taddr + 64, r + 64);
+    tmem_ld32(taddr + 96, r + 96);
+}
+
 template <int D>
 __global__ void __launch_bounds__(kBwdThreads, 1)
 k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                 const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
                 const DkvParams p) {
     using L = DkvSmem<D>;
+    constexpr int QS = L::kQStages, DS = L::kDoStages;
     extern __shared__ __align__(1024) uint8_t smem[];
     uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBarOff);
     uint64_t* bar_kvfull = bars + 0;
     uint64_t* bar_kvempty = bars + 1;
-    uint64_t* bar_qfull = bars + 2;    // [2]
-    uint64_t* bar_qempty = bars + 4;   // [2]
-    uint64_t* bar_dofull = bars + 6;   // [2]
-    uint64_t* bar_doempty = bars + 8;  // [2]
-    uint64_t* bar_sfull = bars + 10;
-    uint64_t* bar_pready = bars + 11;
-    uint64_t* bar_dpfull = bars + 12;
-    uint64_t* bar_dsready = bars + 13;
-    uint64_t* bar_dkvfull = bars + 14;
-    uint64_t* bar_dkvempty = bars + 15;
-    uint64_t* bar_phalf = bars + 16;   // the first half of every group's P^T columns is in TMEM
+    uint64_t* bar_qfull = bars + 2;               // [QS]
+    uint64_t* bar_qempty = bar_qfull + QS;        // [QS] dK(it) has run: Q stage free, dS^T columns free
+    uint64_t* bar_dofull = bar_qempty + QS;       // [DS]
+    uint64_t* bar_doempty = bar_dofull + DS;      // [DS] dV(it) has run: dO stage free
+    uint64_t* bar_sfull = bar_doempty + DS;
+    uint64_t* bar_xfree1 = bar_sfull + 1;   // S^T(it) has been read out of region X: dP^T(it) may overwrite it
+    uint64_t* bar_dpfull = bar_sfull + 2;
+    uint64_t* bar_xfree2 = bar_sfull + 3;   // dP^T(it) has been read out: S^T(it+1) may overwrite it
+    uint64_t* bar_phalf = bar_sfull + 4;    // P^T of the first 32 queries of each exp group is in TMEM
+    uint64_t* bar_pready = bar_sfull + 5;   // all of P^T(it) is in TMEM
+    uint64_t* bar_pfree = bar_sfull + 6;    // dV(it) has run and the dS group has read P^T(it): columns free
+    uint64_t* bar_dsready = bar_sfull + 7;
+    uint64_t* bar_dkvfull = bar_sfull + 8;
+    uint64_t* bar_dkvempty = bar_sfull + 9;
+    uint64_t* bar_drain = bar_sfull + 10;   // teardown after a give-up: every MMA issued so far has completed
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::kMiscOff);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kMiscOff + 4);
 
@@ -148,23 +148,26 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     if (threadIdx.x == 0) {
         mbar_init(bar_kvfull, 1);
         mbar_init(bar_kvempty, 1);
-        for (int s = 0; s < 2; ++s) {
-            mbar_init(&bar_qfull[s], 1);
-            mbar_init(&bar_qempty[s], 1);
-            mbar_init(&bar_dofull[s], 1);
-            mbar_init(&bar_doempty[s], 1);
-        }
+        for (int s = 0; s < QS; ++s) { mbar_init(&bar_qfull[s], 1); mbar_init(&bar_qempty[s], 1); }
+        for (int s = 0; s < DS; ++s) { mbar_init(&bar_dofull[s], 1); mbar_init(&bar_doempty[s], 1); }
         mbar_init(bar_sfull, 1);
-        mbar_init(bar_pready, 128 * kDkvGroups);
+        mbar_init(bar_xfree1, 256);
         mbar_init(bar_dpfull, 1);
-        mbar_init(bar_dsready, 128 * kDkvGroups);
+        mbar_init(bar_xfree2, 128);
+        mbar_init(bar_phalf, 256);
+        mbar_init(bar_pready, 256);
+        mbar_init(bar_pfree, 129);       // the dS group's 128 threads + the commit behind dV(it)
+        mbar_init(bar_dsready, 128);
         mbar_init(bar_dkvfull, 1);
-        mbar_init(bar_dkvempty, 128 * kDkvGroups);
-        mbar_init(bar_phalf, 128 * kDkvGroups);
+        mbar_init(bar_dkvempty, 256);
+        mbar_init(bar_drain, 1);
         abort_flag[0] = 0;
         abort_flag[1] = (int)p.wait_limit_ns;
         fence_mbar_init();
         p.busy[2 * cta] = globaltimer_ns();
+#ifdef LIBRA_TRACE
+        if (cta == 0) g_trace[0] = clock64();
+#endif
     }
     if (warp == kDkvMmaWarp) {
         tmem_alloc(tmem_slot, 512);
@@ -180,17 +183,17 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    constexpr uint32_t kColS = 0, kColDP = 128, kColDK = 256, kColDV = 256 + D;
+    constexpr uint32_t kColX = 0, kColP = 128, kColDS = 192, kColDK = 256, kColDV = 256 + D;
 
     const int unit_begin = p.cta_offsets[cta];
     const int unit_end = p.cta_offsets[cta + 1];
     const int G = p.hq / p.hkv;
 
     if (warp > kDkvMmaWarp) {
-        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kDkvRegsOther));  // only with four groups
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kDkvRegsOther));
     } else if (warp == kDkvTmaWarp) {
         // ---------------- TMA producer ----------------
-        if constexpr (kDkvGroups > 2) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kDkvRegsOther));
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kDkvRegsOther));
         if (elect_one()) {  // one elected thread runs the whole role
             uint32_t ucnt = 0, it_all = 0;
             bool ok = true;
@@ -202,78 +205,86 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const int nblk = last_q_block(p.tok_end, p.T, k0) - i_lo + 1;
                 ok = mbar_wait(bar_kvempty, (ucnt & 1) ^ 1, abort_flag);
                 if (!ok) break;
-                {
-                    mbar_arrive_expect_tx(bar_kvfull, 2 * L::kTileBytes);
-                    for (int half = 0; half < D / 64; ++half) {
-                        tma_load_3d(smem + L::kKOff + half * L::kHalfBytes, &tm_k, bar_kvfull, half * 64, kvh, (int)k0);
-                        tma_load_3d(smem + L::kVOff + half * L::kHalfBytes, &tm_v, bar_kvfull, half * 64, kvh, (int)k0);
-                    }
+                mbar_arrive_expect_tx(bar_kvfull, 2 * L::kTileBytes);
+                for (int half = 0; half < D / 64; ++half) {
+                    tma_load_3d(smem + L::kKOff + half * L::kHalfBytes, &tm_k, bar_kvfull, half * 64, kvh, (int)k0);
+                    tma_load_3d(smem + L::kVOff + half * L::kHalfBytes, &tm_v, bar_kvfull, half * 64, kvh, (int)k0);
                 }
                 ++ucnt;
                 const int n_it = G * nblk;
                 for (int it = 0; it < n_it && ok; ++it, ++it_all) {
                     const int h = kvh * G + it / nblk;
                     const int qb = (i_lo + it % nblk) * kBlk;
-                    const uint32_t st = it_all & 1, par = ((it_all >> 1) & 1) ^ 1;
-                    ok = mbar_wait(&bar_qempty[st], par, abort_flag);
+                    const uint32_t qs = it_all % QS, ds = it_all % DS;
+                    ok = mbar_wait(&bar_qempty[qs], ((it_all / QS) & 1) ^ 1, abort_flag);
                     if (!ok) break;
-                    {
-                        mbar_arrive_expect_tx(&bar_qfull[st], L::kTileBytes + 1024);
-                        for (int half = 0; half < D / 64; ++half)
-                            tma_load_3d(smem + L::kQOff + st * L::kTileBytes + half * L::kHalfBytes, &tm_q, &bar_qfull[st],
-                                        half * 64, h, qb);
-                        bulk_load_1d(smem + L::kStatOff + st * 1024, p.lse2 + (size_t)h * p.Tpad + qb, 512, &bar_qfull[st]);
-                        bulk_load_1d(smem + L::kStatOff + st * 1024 + 512, p.dvec + (size_t)h * p.Tpad + qb, 512,
-                                     &bar_qfull[st]);
+                    mbar_arrive_expect_tx(&bar_qfull[qs], L::kTileBytes + 512);
+                    for (int half = 0; half < D / 64; ++half)
+                        tma_load_3d(smem + L::kQOff + qs * L::kTileBytes + half * L::kHalfBytes, &tm_q, &bar_qfull[qs],
+                                    half * 64, h, qb);
+                    bulk_load_1d(smem + L::kLseOff + qs * 512, p.lse2 + (size_t)h * p.Tpad + qb, 512, &bar_qfull[qs]);
+                    ok = mbar_wait(&bar_doempty[ds], ((it_all / DS) & 1) ^ 1, abort_flag);
+                    if (!ok) {   // the Q load just issued is still in flight
+                        mbar_wait_drain(&bar_qfull[qs], (it_all / QS) & 1, kDrainNs);
+                        break;
                     }
-                    ok = mbar_wait(&bar_doempty[st], par, abort_flag);
-                    if (!ok) break;
-                    {
-                        mbar_arrive_expect_tx(&bar_dofull[st], L::kTileBytes);
-                        for (int half = 0; half < D / 64; ++half)
-                            tma_load_3d(smem + L::kDoOff + st * L::kTileBytes + half * L::kHalfBytes, &tm_do,
-                                        &bar_dofull[st], half * 64, h, qb);
-                    }
+                    mbar_arrive_expect_tx(&bar_dofull[ds], L::kTileBytes + 512);
+                    for (int half = 0; half < D / 64; ++half)
+                        tma_load_3d(smem + L::kDoOff + ds * L::kTileBytes + half * L::kHalfBytes, &tm_do,
+                                    &bar_dofull[ds], half * 64, h, qb);
+                    bulk_load_1d(smem + L::kDvecOff + ds * 512, p.dvec + (size_t)h * p.Tpad + qb, 512, &bar_dofull[ds]);
                 }
+            }
+            if (!ok || abort_flag[0]) {
+                // Give-up path: nothing new is issued; let the copies already issued land before the CTA's
+                // shared memory is released (each armed phase completes when its bytes have arrived).
+                if (ucnt > 0) mbar_wait_drain(bar_kvfull, (ucnt - 1) & 1, kDrainNs);
+                for (uint32_t b = 1; b <= (uint32_t)QS && b <= it_all; ++b)
+                    mbar_wait_drain(&bar_qfull[(it_all - b) % QS], ((it_all - b) / QS) & 1, kDrainNs);
+                for (uint32_t b = 1; b <= (uint32_t)DS && b <= it_all; ++b)
+                    mbar_wait_drain(&bar_dofull[(it_all - b) % DS], ((it_all - b) / DS) & 1, kDrainNs);
             }
         }
         __syncwarp();
     } else if (warp == kDkvMmaWarp) {
         // ---------------- MMA issuer ----------------
-        if constexpr (kDkvGroups > 2) asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kDkvRegsOther));
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kDkvRegsOther));
         if (elect_one()) {  // one elected thread runs the whole role
             constexpr uint32_t idesc_s = make_idesc(128, 128, 0, 0);  // S^T, dP^T: both operands K-major
             constexpr uint32_t idesc_acc = make_idesc(128, D, 0, 1);  // dV, dK: A from TMEM, B MN-major
             const uint32_t sb = smem_u32(smem);
             uint32_t ucnt = 0, it_all = 0;
             bool ok = true;
-            PROF_DECL
             TRACE_DECL(17, cta == 0)
             // Base descriptors are built once; every MMA only adds a constant to them.
             const uint64_t kdesc0 = make_sdesc(sb, 16, 1024);             // K-major view of a tile at offset 0
             const uint64_t mdesc0 = make_sdesc(sb, L::kHalfBytes, 1024);  // MN-major view
-            // C[tmem] = A(K-major tile) * B(K-major tile)^T over the head dimension; offsets from smem base
-            auto issue_kmajor = [&](uint32_t d_col, uint32_t a_off, uint32_t b_off) {
+            // X[tmem] = A(K-major tile) * B(K-major tile)^T over the head dimension; offsets from smem base
+            auto issue_kmajor = [&](uint32_t a_off, uint32_t b_off) {
                 const uint64_t da = sdesc_advance(kdesc0, a_off), db = sdesc_advance(kdesc0, b_off);
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
                     const uint32_t off = (kk / 4) * L::kHalfBytes + (kk % 4) * 32;
-                    mma_ss(tmem_base + d_col, sdesc_advance(da, off), sdesc_advance(db, off), idesc_s, kk > 0);
+                    mma_ss(tmem_base + kColX, sdesc_advance(da, off), sdesc_advance(db, off), idesc_s, kk > 0);
                 }
             };
-            // C[tmem] (+)= A(TMEM, bf16 packed: group c's queries at columns a_col + CW c ..) * B(MN-major tile).
-            // `half` 0 / 1 issues the key steps that read the first / second half of every group's columns
-            // (the compute groups hand P^T over in two halves), 2 issues all of them.
-            auto issue_acc = [&](uint32_t d_col, uint32_t a_col, uint32_t b_off, bool accumulate, int half) {
+            // C[tmem] (+)= A(TMEM, bf16 packed: queries 2 c and 2 c + 1 in column a_col + c) * B(MN-major tile)
+            auto issue_acc = [&](uint32_t d_col, uint32_t a_col, uint32_t b_off, bool accumulate) {
                 const uint64_t db = sdesc_advance(mdesc0, b_off);
-                constexpr int kPerGroup = kDkvCW / 16;  // key steps of 16 queries per group
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    const int within = kk % kPerGroup;
-                    if (half != 2 && (within >= kPerGroup / 2) != (half == 1)) continue;
-                    mma_ts(tmem_base + d_col, tmem_base + a_col + (kk / kPerGroup) * kDkvCW + within * 8,
-                           sdesc_advance(db, kk * 2048), idesc_acc, (accumulate || kk > 0) ? 1u : 0u);
-                }
+                for (int kk = 0; kk < 8; ++kk)
+                    mma_ts(tmem_base + d_col, tmem_base + a_col + kk * 8, sdesc_advance(db, kk * 2048), idesc_acc,
+                           (accumulate || kk > 0) ? 1u : 0u);
+            };
+            // dK(i) += dS^T(i) Q(i), i a CTA-wide iteration index
+            auto issue_dk = [&](uint32_t i, bool accumulate) -> bool {
+                if (!mbar_wait(bar_dsready, i & 1, abort_flag)) return false;
+                tc_fence_after();
+                TRACE(13)
+                issue_acc(kColDK, kColDS, L::kQOff + (i % QS) * L::kTileBytes, accumulate);
+                tc_commit(&bar_qempty[i % QS]);   // also tells the dS group that dS^T may be rewritten
+                TRACE(14)
+                return true;
             };
             for (int idx = unit_begin; idx < unit_end && ok; ++idx) {
                 const int t = p.cta_tiles[idx];
@@ -283,101 +294,158 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const int n_it = G * nblk;
                 ok = mbar_wait(bar_kvfull, ucnt & 1, abort_flag);
                 if (!ok) break;
-                // S(0), dP(0)
-                ok = mbar_wait(&bar_qfull[it_all & 1], (it_all >> 1) & 1, abort_flag);
+                // S(0): region X is free once dP of the previous unit's last iteration has been read
+                ok = mbar_wait(&bar_qfull[it_all % QS], (it_all / QS) & 1, abort_flag);
+                if (ok && it_all > 0) ok = mbar_wait(bar_xfree2, (it_all - 1) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                {
-                    issue_kmajor(kColS, L::kKOff, L::kQOff + (it_all & 1) * L::kTileBytes);
-                    tc_commit(bar_sfull);
-                }
-                ok = mbar_wait(&bar_dofull[it_all & 1], (it_all >> 1) & 1, abort_flag);
-                if (!ok) break;
-                {
-                    issue_kmajor(kColDP, L::kVOff, L::kDoOff + (it_all & 1) * L::kTileBytes);
-                    tc_commit(bar_dpfull);
-                }
+                issue_kmajor(L::kKOff, L::kQOff + (it_all % QS) * L::kTileBytes);
+                tc_commit(bar_sfull);
                 for (int it = 0; it < n_it && ok; ++it, ++it_all) {
                     TRACE(20)
-                    const uint32_t st = it_all & 1;
+                    const uint32_t ds = it_all % DS;
                     const uint32_t nx = it_all + 1;
                     const bool more = it + 1 < n_it;
+                    // dP(it) over S(it), as soon as the exp group holds S(it) in registers
+                    ok = mbar_wait(&bar_dofull[ds], (it_all / DS) & 1, abort_flag);
+                    if (ok) ok = mbar_wait(bar_xfree1, it_all & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_kmajor(L::kVOff, L::kDoOff + ds * L::kTileBytes);
+                    tc_commit(bar_dpfull);
+                    if (!more) tc_commit(bar_kvempty);   // the unit's last readers of K and V: the next unit's K / V
+                    TRACE(15)                            // load overlaps the rest of this iteration
+                    // dK(it-1): its dS^T was finished while S(it) ran
+                    if (it > 0) { ok = issue_dk(it_all - 1, it > 1); if (!ok) break; }
+                    // S(it+1) over dP(it), as soon as the dS group holds dP(it) in registers
+                    if (more) {
+                        ok = mbar_wait(&bar_qfull[nx % QS], (nx / QS) & 1, abort_flag);
+                        if (ok) ok = mbar_wait(bar_xfree2, it_all & 1, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_kmajor(L::kKOff, L::kQOff + (nx % QS) * L::kTileBytes);
+                        tc_commit(bar_sfull);
+                        TRACE(12)
+                    }
                     // dV(it) += P^T dO
-                    PROF(7)
-                    ok = mbar_wait(bar_phalf, it_all & 1, abort_flag);   // first half of P^T
-                    if (ok && it == 0 && ucnt > 0)                        // previous unit's dK/dV must have been read out
+                    ok = mbar_wait(bar_pready, it_all & 1, abort_flag);
+                    if (ok && it == 0 && ucnt > 0)   // the previous unit's dK / dV must have been read out
                         ok = mbar_wait(bar_dkvempty, (ucnt - 1) & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    issue_acc(kColDV, kColS, L::kDoOff + st * L::kTileBytes, it > 0, 0);
-                    ok = mbar_wait(bar_pready, it_all & 1, abort_flag);  // second half, while those MMAs run
-                    if (!ok) break;
-                    PROF(0)
-                    tc_fence_after();
-                    {
-                        TRACE(10)
-                        issue_acc(kColDV, kColS, L::kDoOff + st * L::kTileBytes, it > 0, 1);
-                        tc_commit(&bar_doempty[st]);
-                        TRACE(11)
-                    }
-                    // S(it+1)
-                    if (more) {
-                        PROF(7)
-                        ok = mbar_wait(&bar_qfull[nx & 1], (nx >> 1) & 1, abort_flag);
-                        if (!ok) break;
-                        PROF(1)
-                        {
-                            issue_kmajor(kColS, L::kKOff, L::kQOff + (nx & 1) * L::kTileBytes);
-                            tc_commit(bar_sfull);
-                            TRACE(12)
-                        }
-                    }
-                    // dK(it) += dS^T Q
-                    PROF(7)
-                    ok = mbar_wait(bar_dsready, it_all & 1, abort_flag);
-                    if (!ok) break;
-                    PROF(2)
-                    tc_fence_after();
-                    {
-                        TRACE(13)
-                        issue_acc(kColDK, kColDP, L::kQOff + st * L::kTileBytes, it > 0, 2);
-                        tc_commit(&bar_qempty[st]);
-                        TRACE(14)
-                    }
-                    // dP(it+1)
-                    if (more) {
-                        PROF(7)
-                        ok = mbar_wait(&bar_dofull[nx & 1], (nx >> 1) & 1, abort_flag);
-                        if (!ok) break;
-                        PROF(3)
-                        {
-                            issue_kmajor(kColDP, L::kVOff, L::kDoOff + (nx & 1) * L::kTileBytes);
-                            tc_commit(bar_dpfull);
-                            TRACE(15)
-                        }
-                    }
+                    TRACE(10)
+                    issue_acc(kColDV, kColP, L::kDoOff + ds * L::kTileBytes, it > 0);
+                    tc_commit(&bar_doempty[ds]);
+                    tc_commit(bar_pfree);
+                    TRACE(11)
                 }
-                if (ok) {
-                    tc_commit(bar_dkvfull);
-                    tc_commit(bar_kvempty);
-                }
+                if (ok) ok = issue_dk(it_all - 1, n_it > 1);   // the unit's last dK
+                if (ok) tc_commit(bar_dkvfull);
                 ++ucnt;
             }
-            PROF_FLUSH(true, 8)
+            if (!ok || abort_flag[0]) {   // give-up path: wait for the MMAs already issued before TMEM is freed
+                tc_commit(bar_drain);
+                mbar_wait_drain(bar_drain, 0, kDrainNs);
+            }
         }
         __syncwarp();
-    } else {
-        // ---------------- compute groups ----------------
-        if constexpr (kDkvGroups > 2) asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kDkvRegsCompute));
-        constexpr int CW = kDkvCW;
-        const int c = warp >> 2;  // which CW query columns of each key row this group owns
+    } else if (warp >= 8) {
+        // ---------------- dS group ----------------
+        // Thread r owns key row r (TMEM lane r) and all 128 query columns of dP^T; it turns dP^T and P^T (read back
+        // as bf16) into dS^T.  The reads of region X are made by different warps for S^T and dP^T, so each happens
+        // as soon as its MMA has landed.
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kDkvRegsDs));
         const int r = (warp & 3) * 32 + lane;
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
-        const uint32_t t_s = tmem_base + lane_addr + kColS + CW * c;
-        const uint32_t t_dp = tmem_base + lane_addr + kColDP + CW * c;
+        const uint32_t t_x = tmem_base + lane_addr + kColX;
+        const uint32_t t_p = tmem_base + lane_addr + kColP;
+        const uint32_t t_ds = tmem_base + lane_addr + kColDS;
+        uint32_t it_all = 0;
+        bool ok = true;
+        TRACE_DECL(1 + warp, cta == 0 && lane == 0)
+        for (int idx = unit_begin; idx < unit_end && ok; ++idx) {
+            const int t = p.cta_tiles[idx];
+            const int64_t k0 = (int64_t)(t / p.hkv) * kBlk;
+            const int i_lo = (int)(k0 / kBlk);
+            const int nblk = last_q_block(p.tok_end, p.T, k0) - i_lo + 1;
+            const int n_it = G * nblk;
+            // ---- dS group: dS^T = P^T o (dP^T - D) ----
+            for (int it = 0; it < n_it && ok; ++it, ++it_all) {
+                const uint32_t ds = it_all % DS;
+                const float* dvec = reinterpret_cast<const float*>(smem + L::kDvecOff + ds * 512);
+                ok = mbar_wait(&bar_dofull[ds], (it_all / DS) & 1, abort_flag) &&
+                     mbar_wait(bar_dpfull, it_all & 1, abort_flag);
+                if (!ok) break;
+                TRACE(4)
+                tc_fence_after();
+                uint32_t xs[64];   // (dP^T - D) as packed bf16 pairs
+                {
+                    uint32_t dpv[128];
+                    tmem_ld128(t_x, dpv);
+                    tmem_ld_wait();
+                    tc_fence_before();
+                    mbar_arrive(bar_xfree2);   // dP^T(it) is in registers: S^T(it+1) may take the columns
+                    TRACE(9)
+                    const uint64_t neg1 = f2_pack(-1.f, -1.f);
+#pragma unroll
+                    for (int j = 0; j < 128; j += 4) {   // packed pairs: dP - D = fma(D, -1, dP)
+                        const ulonglong2 d4 = *reinterpret_cast<const ulonglong2*>(dvec + j);
+                        float a0, a1, b0, b1;
+                        f2_unpack(f2_fma(d4.x, neg1, f2_pack(__uint_as_float(dpv[j]), __uint_as_float(dpv[j + 1]))), a0, a1);
+                        f2_unpack(f2_fma(d4.y, neg1, f2_pack(__uint_as_float(dpv[j + 2]), __uint_as_float(dpv[j + 3]))), b0, b1);
+                        xs[j >> 1] = pack_bf16x2(a0, a1);
+                        xs[(j >> 1) + 1] = pack_bf16x2(b0, b1);
+                    }
+                }
+                TRACE(22)
+                // dS^T(it-1) must have been consumed by dK(it-1) before its columns are rewritten
+                if (it_all > 0) {
+                    ok = mbar_wait(&bar_qempty[(it_all - 1) % QS], ((it_all - 1) / QS) & 1, abort_flag);
+                    if (!ok) break;
+                }
+                TRACE(16)
+                // P^T arrives in the order the exp groups finish it: the first 32 queries of each group's 64
+                // (columns 0..15 and 32..47 of the packed P^T), then the rest.  dS^T = P^T o (dP^T - D) in bf16 pairs.
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    ok = mbar_wait(half == 0 ? bar_phalf : bar_pready, it_all & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    if (half == 0) { TRACE(17) } else { TRACE(19) }
+                    uint32_t pa[16], pb[16];
+                    tmem_ld16(t_p + half * 16, pa);
+                    tmem_ld16(t_p + 32 + half * 16, pb);
+                    tmem_ld_wait();
+                    if (half == 1) {           // all of P^T(it) is in registers
+                        tc_fence_before();
+                        mbar_arrive(bar_pfree);
+                        TRACE(21)
+                    }
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        pa[j] = mul_bf16x2(pa[j], xs[half * 16 + j]);
+                        pb[j] = mul_bf16x2(pb[j], xs[32 + half * 16 + j]);
+                    }
+                    tmem_st16(t_ds + half * 16, pa);
+                    tmem_st16(t_ds + 32 + half * 16, pb);
+                }
+                if (!ok) break;
+                tmem_st_wait();
+                tc_fence_before();
+                mbar_arrive(bar_dsready);
+                TRACE(5)
+            }
+        }
+    } else {
+        // ---------------- exp groups ----------------
+        // Thread r of group grp owns key row r and the query columns [64 grp, 64 grp + 64) of S^T.
+        const int grp = warp >> 2;
+        const int r = (warp & 3) * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t t_x = tmem_base + lane_addr + kColX;
+        const uint32_t t_p = tmem_base + lane_addr + kColP;
         uint32_t ucnt = 0, it_all = 0;
         bool ok = true;
-        PROF_DECL
         TRACE_DECL(1 + warp, cta == 0 && lane == 0)
         for (int idx = unit_begin; idx < unit_end && ok; ++idx) {
             const int t = p.cta_tiles[idx];
@@ -388,115 +456,92 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const int n_it = G * nblk;
             const int64_t key = k0 + r;
             const bool key_ok = key < p.T;
+            // ---- exp groups: P^T = exp2(S^T * c - LSE), zero where the query does not see the key ----
+            const int c0 = 64 * grp;   // this group's query columns
+            const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2), neg1 = f2_pack(-1.f, -1.f);
             const int kend = key_ok ? p.tok_end[key] : 0;
             const int min_kend = p.tok_end[k0];
             const bool partial = k0 + kBlk > p.T;
             for (int it = 0; it < n_it && ok; ++it, ++it_all) {
                 const int qb = (i_lo + it % nblk) * kBlk;
-                const uint32_t st = it_all & 1, par = (it_all >> 1) & 1;
-                const float* lse2 = reinterpret_cast<const float*>(smem + L::kStatOff + st * 1024) + CW * c;
-                const float* dvec = lse2 + 128;
+                const uint32_t qs = it_all % QS;
+                const float* lse2 = reinterpret_cast<const float*>(smem + L::kLseOff + qs * 512) + c0;
                 const bool need_mask = (qb == k0) || (qb + kBlk - 1 >= min_kend) || partial;
-                const int j_lo = (int)(key - qb) - CW * c;  // first visible column of this group's range
-                const int j_hi = kend - 1 - qb - CW * c;    // last visible column
-                // ---- exp phase: P^T = exp2(S^T * c - LSE) ----
-                ok = mbar_wait(&bar_qfull[st], par, abort_flag) && mbar_wait(bar_sfull, it_all & 1, abort_flag);
+                const int j_lo = (int)(key - qb) - c0;   // first visible column of this group's range
+                const int j_hi = kend - 1 - qb - c0;     // last visible column
+                ok = mbar_wait(&bar_qfull[qs], (it_all / QS) & 1, abort_flag) &&
+                     mbar_wait(bar_sfull, it_all & 1, abort_flag);
                 if (!ok) break;
-                PROF(0)
                 TRACE(2)
                 tc_fence_after();
-                uint32_t sv[CW];
-#pragma unroll
-                for (int j = 0; j < CW; j += 32) tmem_ld32(t_s + j, sv + j);
+                uint32_t sv[64];
+                tmem_ld32(t_x + c0, sv);
+                tmem_ld32(t_x + c0 + 32, sv + 32);
                 tmem_ld_wait();
-                float pf[CW];
-                // two halves: the dV key steps over the first half of this group's queries start while the second
-                // half's exponentials are computed (S(it+1) has to wait for all of dV(it), which overwrites nothing
-                // but reads P^T from the columns S(it+1) goes to)
+                tc_fence_before();
+                mbar_arrive(bar_xfree1);   // S^T(it) is in registers: dP^T(it) may take the columns
+                TRACE(6)
+                // P^T(it-1) must have been consumed (dV(it-1), the dS group) before its columns are rewritten
+                if (it_all > 0) {
+                    ok = mbar_wait(bar_pfree, (it_all - 1) & 1, abort_flag);
+                    if (!ok) break;
+                }
+                TRACE(7)
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
-                    constexpr int HW = CW / 2;
-                    const int b0 = half * HW;
+                    float pf[32];
 #pragma unroll
-                    for (int j = b0; j < b0 + HW; j += 4) {
-                        const float4 l4 = *reinterpret_cast<const float4*>(lse2 + j);
-                        pf[j] = ex2_sel(fmaf(__uint_as_float(sv[j]), p.scale_log2, -l4.x), j);
-                        pf[j + 1] = ex2_sel(fmaf(__uint_as_float(sv[j + 1]), p.scale_log2, -l4.y), j + 1);
-                        pf[j + 2] = ex2_sel(fmaf(__uint_as_float(sv[j + 2]), p.scale_log2, -l4.z), j + 2);
-                        pf[j + 3] = ex2_sel(fmaf(__uint_as_float(sv[j + 3]), p.scale_log2, -l4.w), j + 3);
+                    for (int j = 0; j < 32; j += 4) {   // packed pairs: S * c - LSE
+                        const int jj = half * 32 + j;
+                        const ulonglong2 l4 = *reinterpret_cast<const ulonglong2*>(lse2 + jj);
+                        float x0, x1, x2, x3;
+                        f2_unpack(f2_fma(f2_pack(__uint_as_float(sv[jj]), __uint_as_float(sv[jj + 1])), scale2,
+                                         f2_mul(l4.x, neg1)), x0, x1);
+                        f2_unpack(f2_fma(f2_pack(__uint_as_float(sv[jj + 2]), __uint_as_float(sv[jj + 3])), scale2,
+                                         f2_mul(l4.y, neg1)), x2, x3);
+                        pf[j] = ex2_sel(x0, jj);
+                        pf[j + 1] = ex2_sel(x1, jj + 1);
+                        pf[j + 2] = ex2_sel(x2, jj + 2);
+                        pf[j + 3] = ex2_sel(x3, jj + 3);
                     }
-                    if (need_mask) {
+                    if (need_mask) {   // one uniform branch per half: the exponentials above stay one straight run
 #pragma unroll
-                        for (int j = b0; j < b0 + HW; ++j)
-                            if (j < j_lo || j > j_hi) pf[j] = 0.f;
+                        for (int j = 0; j < 32; ++j)
+                            if (half * 32 + j < j_lo || half * 32 + j > j_hi) pf[j] = 0.f;
                     }
-                    uint32_t pk[HW / 2];
+                    uint32_t pk[16];
 #pragma unroll
-                    for (int j = 0; j < HW; j += 2) pk[j >> 1] = pack_bf16x2(pf[b0 + j], pf[b0 + j + 1]);
-                    // packed P^T of this group sits in the first CW / 2 columns of its own S^T range
-                    if constexpr (HW == 32) tmem_st16(t_s + b0 / 2, pk); else tmem_st8(t_s + b0 / 2, pk);
-                    if (half == 0) {
-                        tmem_st_wait();
-                        tc_fence_before();
-                        mbar_arrive(bar_phalf);
-                    }
+                    for (int j = 0; j < 32; j += 2) pk[j >> 1] = pack_bf16x2(pf[j], pf[j + 1]);
+                    tmem_st16(t_p + c0 / 2 + half * 16, pk);
+                    tmem_st_wait();
+                    tc_fence_before();
+                    mbar_arrive(half == 0 ? bar_phalf : bar_pready);
+                    if (half == 0) { TRACE(8) }
                 }
-                tmem_st_wait();
-                tc_fence_before();
-                mbar_arrive(bar_pready);
-                PROF(1)
                 TRACE(3)
-                // ---- dS phase: dS^T = P^T o (dP^T - D), packed over this half's own dP^T columns ----
-                ok = mbar_wait(bar_dpfull, it_all & 1, abort_flag);
-                if (!ok) break;
-                PROF(2)
-                TRACE(4)
-                tc_fence_after();
-                uint32_t dpv[CW];
-#pragma unroll
-                for (int j = 0; j < CW; j += 32) tmem_ld32(t_dp + j, dpv + j);
-                tmem_ld_wait();
-                {
-                    uint32_t pk[CW / 2];
-#pragma unroll
-                    for (int j = 0; j < CW; j += 4) {
-                        const float4 d4 = *reinterpret_cast<const float4*>(dvec + j);
-                        pk[j >> 1] = pack_bf16x2(pf[j] * (__uint_as_float(dpv[j]) - d4.x),
-                                                 pf[j + 1] * (__uint_as_float(dpv[j + 1]) - d4.y));
-                        pk[(j >> 1) + 1] = pack_bf16x2(pf[j + 2] * (__uint_as_float(dpv[j + 2]) - d4.z),
-                                                       pf[j + 3] * (__uint_as_float(dpv[j + 3]) - d4.w));
-                    }
-                    if constexpr (CW == 64) tmem_st32(t_dp, pk); else tmem_st16(t_dp, pk);
-                }
-                tmem_st_wait();
-                tc_fence_before();
-                mbar_arrive(bar_dsready);
-                PROF(3)
-                TRACE(5)
             }
             if (!ok) break;
-            // ---- unit epilogue: dK * scale and dV to global ----
-            ok = mbar_wait(bar_dkvfull, ucnt & 1, abort_flag);
+            ++ucnt;
+            // ---- unit epilogue: dK * scale and dV to global (each exp group stores half of the columns) ----
+            ok = mbar_wait(bar_dkvfull, (ucnt - 1) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
-            constexpr int kCols = D / kDkvGroups;  // columns of dK and dV this group stores
-            const uint32_t t_dk = tmem_base + lane_addr + kColDK + c * kCols;
-            const uint32_t t_dv = tmem_base + lane_addr + kColDV + c * kCols;
-            const size_t gofs = ((size_t)key * p.hkv + kvh) * D + c * kCols;
+            constexpr int kCols = D / 2;
+            const uint32_t t_dk = tmem_base + lane_addr + kColDK + grp * kCols;
+            const uint32_t t_dv = tmem_base + lane_addr + kColDV + grp * kCols;
+            const size_t gofs = ((size_t)key * p.hkv + kvh) * D + grp * kCols;
 #pragma unroll
             for (int which = 0; which < 2; ++which) {
                 const float mul = which == 0 ? p.scale : 1.0f;
                 __nv_bfloat16* gdst = (which == 0 ? p.dk : p.dv) + gofs;
-                constexpr int kChunk = kCols < 32 ? kCols : 32;
 #pragma unroll
-                for (int cc = 0; cc < kCols; cc += kChunk) {
-                    uint32_t v[kChunk];
-                    if constexpr (kChunk == 32) tmem_ld32((which == 0 ? t_dk : t_dv) + cc, v);
-                    else tmem_ld16((which == 0 ? t_dk : t_dv) + cc, v);
+                for (int cc = 0; cc < kCols; cc += 32) {
+                    uint32_t v[32];
+                    tmem_ld32((which == 0 ? t_dk : t_dv) + cc, v);
                     tmem_ld_wait();
                     if (key_ok) {
 #pragma unroll
-                        for (int i = 0; i < kChunk; i += 8) {
+                        for (int i = 0; i < 32; i += 8) {
                             uint4 w;
                             w.x = pack_bf16x2(__uint_as_float(v[i]) * mul, __uint_as_float(v[i + 1]) * mul);
                             w.y = pack_bf16x2(__uint_as_float(v[i + 2]) * mul, __uint_as_float(v[i + 3]) * mul);
@@ -509,10 +554,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             }
             tc_fence_before();
             mbar_arrive(bar_dkvempty);
-            ++ucnt;
-            PROF(4)
         }
-        PROF_FLUSH(threadIdx.x == 0, 0)
     }
 
     // ---------------- teardown ----------------
@@ -520,7 +562,10 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     __syncthreads();
     if (warp == kDkvMmaWarp) tmem_dealloc(tmem_base, 512);
     if (threadIdx.x == 0) {
-        if (*abort_flag) atomicExch(p.status, LIBRA_ERR_TIMEOUT);
+        if (abort_flag[0]) atomicExch(p.status, LIBRA_ERR_TIMEOUT);
+#ifdef LIBRA_TRACE
+        if (cta == 0) g_trace[1] = clock64();
+#endif
         p.busy[2 * cta + 1] = globaltimer_ns();
     }
 }
@@ -605,8 +650,7 @@ static int launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtens
     if (!cfg_done(kSlot)) {   // per device
         if (set_smem(k_attn_bwd_dkdv<D>, DkvSmem<D>::kBytes) != LIBRA_OK) return LIBRA_ERR_CUDA;
         if (set_smem(k_attn_bwd_dq<D>, DqSmem<D>::kBytes) != LIBRA_OK) return LIBRA_ERR_CUDA;
-        if (kDkvGroups > 2 && !regs_pool_ok(k_attn_bwd_dkdv<D>, 128 * kDkvGroups, kDkvRegsCompute, 128, kDkvRegsOther))
-            return LIBRA_ERR_UNSUPPORTED;
+        if (!regs_pool_ok(k_attn_bwd_dkdv<D>, 128, kDkvRegsDs, 128, kDkvRegsOther)) return LIBRA_ERR_UNSUPPORTED;
         if (!regs_pool_ok(k_attn_bwd_dq<D>, 128 * kDqGroups, kDqRegsCompute, 128, kDqRegsOther)) return LIBRA_ERR_UNSUPPORTED;
         cfg_mark(kSlot);
     }
@@ -626,12 +670,6 @@ using namespace libra;
 #ifdef LIBRA_TRACE
 extern "C" int libra_debug_trace(long long* host, int n) {
     return cudaMemcpyFromSymbol(host, libra::g_trace, sizeof(long long) * n) == cudaSuccess ? 0 : -4;
-}
-#endif
-
-#ifdef LIBRA_PROF
-extern "C" int libra_debug_bwd_prof(unsigned long long* host, int n) {
-    return cudaMemcpyFromSymbol(host, libra::g_bwd_prof, sizeof(unsigned long long) * n) == cudaSuccess ? 0 : -4;
 }
 #endif
 

@@ -319,6 +319,13 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
     return r;
 }
 
+// Element-wise product of two packed bf16 pairs, rounded to nearest even.
+__device__ __forceinline__ uint32_t mul_bf16x2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+
 #ifdef LIBRA_TRACE
 // Trace build only: raw (event id, clock) pairs of one thread per role in CTA 0.
 __device__ long long g_trace[18 * 4096 * 2];
