@@ -1,16 +1,18 @@
 #!/usr/bin/env python
 """Benchmark of the pool-attention hot path (plan reused; forward + backward per step).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 2] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config 2] [--impl ours|reference] [--sweep]
 
 One step = one forward + backward pass of causal, sample-masked attention over one synthetic
 pool (default: the Qwen3-8B-shaped pool, 4 packed sequences x 32768 tokens, Hq 32 / Hkv 8 /
 d 128).  The metric is useful TFLOP/s: 14 * d * Hq * sum_j l_j (l_j + 1) / 2 per step divided
-by the step time (4 d per causal pair forward, 10 d backward).  With N > 1 (torchrun) every
-rank runs its own pool of the same shape (weak scaling, no data-path collective).
+by the step time (4 d per causal pair forward, 10 d backward).  With N > 1 (torchrun) the SAME
+pool is split over the ranks by attention heads (kv heads with their query heads; strong
+scaling, no data-path collective while N <= Hkv); `--replicas` runs one independent pool per
+rank instead (weak scaling).
 
 Prints one JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded sample
-of the same workload instead.
+of the same workload instead.  `--sweep` prints a table over head shards x tile weights x pools.
 """
 from __future__ import annotations
 
@@ -31,6 +33,7 @@ sys.path.insert(0, ROOT)
 from paper_2607_23250_b200 import pools, sharding  # noqa: E402
 
 METRIC = "useful attention TFLOP/s fwd+bwd (sum of per-sample causal FLOPs)"
+KERNELS = ("fwd", "bwd_dkdv", "bwd_dq", "bwd_prep")
 
 
 def useful_flops(lengths, hq, d):
@@ -146,6 +149,103 @@ def time_oracle(spec, lengths, steps=1, warmup=0):
                 seconds_per_step=sec)
 
 
+# ---- one pool on this rank's GPU ---------------------------------------------------------------
+
+class Pool:
+    """Device tensors, plan and buffers of one pool (or of this rank's head slice of it)."""
+
+    def __init__(self, lb, spec, dev, shard=None, weight_model="pairs", heads=0, seed=0):
+        import torch
+        self.lb, self.spec, self.dev, self.shard = lb, spec, dev, shard
+        self.lengths = pools.pool_lengths(spec)
+        cu_np = pools.cu_seqlens(self.lengths)
+        T, d = spec.total_tokens, spec.head_dim
+        t = pools.make_tensors(T, spec.hq, spec.hkv, d, seed=seed, device=str(dev))
+        if shard is not None and shard.world > 1:
+            q, k, v, dout = sharding.slice_heads(shard, t["q"], t["k"], t["v"], t["dout"])
+            del t
+        else:
+            q, k, v, dout = t["q"], t["k"], t["v"], t["dout"]
+        self.inp = dict(q=q, k=k, v=v, dout=dout)
+        self.hq, self.hkv, self.T, self.d = q.shape[1], k.shape[1], T, d
+        self.ff, self.fb = useful_flops(self.lengths, self.hq, d)
+        self.cu = torch.from_numpy(cu_np).to(dev)
+        self.heads = heads or self.hq
+        self.blocks = weight_model == "blocks"
+        self.plan = None
+        self.out = dict(out=torch.empty_like(q), lse=torch.empty((self.hq, T), dtype=torch.float32, device=dev),
+                        dq=torch.empty_like(q), dk=torch.empty_like(k), dv=torch.empty_like(v))
+
+    def make_plan(self, blocks=None):
+        lb = self.lb
+        blocks = self.blocks if blocks is None else blocks
+        return lb.libra_plan_tiles(self.cu, self.heads, 256, tile_kv=128, n_heads_kv=self.hkv, total_tokens=self.T,
+                                   weight_model=lb.LIBRA_WEIGHT_BLOCKS if blocks else lb.LIBRA_WEIGHT_PAIRS,
+                                   unit_cost_q=12 if blocks else 0, unit_cost_kv=6 if blocks else 0)
+
+    def build(self):
+        import torch
+        self.make_plan().destroy()                     # first call pays for the module load
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        self.plan = self.make_plan()                   # built once, outside the timed steps (the paper reuses it across layers)
+        e1.record()
+        torch.cuda.synchronize()
+        assert self.plan.status() == 0
+        self.ws = torch.empty(self.lb.libra_attn_pool_bwd_workspace_bytes(self.plan, self.inp["q"], self.inp["k"]),
+                              dtype=torch.uint8, device=self.dev)
+        return e0.elapsed_time(e1)
+
+    def step_on(self, i, o, plan=None):
+        lb, plan = self.lb, plan or self.plan
+        lb.libra_attn_pool_fwd(i["q"], i["k"], i["v"], plan, out=o["out"], lse=o["lse"])
+        lb.libra_attn_pool_bwd(i["q"], i["k"], i["v"], o["out"], o["lse"], i["dout"], plan, dq=o["dq"], dk=o["dk"],
+                               dv=o["dv"], workspace=self.ws)
+
+    def step(self, plan=None):
+        self.step_on(self.inp, self.out, plan)
+
+    def timed(self, steps, warmup, barrier, plan=None):
+        """(ms per step, per-kernel mean ms, busy max/mean per kernel) of `steps` steps between two events; the
+        library records its own events around every kernel inside the same loop."""
+        import torch
+        lb, plan = self.lb, plan or self.plan
+        for _ in range(warmup):
+            self.step(plan)
+        barrier()
+        plan.set_timing(True)                          # fresh record: only the timed steps below
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            self.step(plan)
+        e1.record()
+        barrier()
+        ms = e0.elapsed_time(e1) / steps
+        kern = {n: statistics.mean(plan.kernel_times_ms(k)) for n, k in
+                zip(KERNELS, (lb.KERNEL_FWD, lb.KERNEL_BWD_DKDV, lb.KERNEL_BWD_DQ, lb.KERNEL_BWD_PREP))}
+        plan.set_timing(False)
+        busy = {}
+        for n, k in zip(KERNELS[:3], (lb.KERNEL_FWD, lb.KERNEL_BWD_DKDV, lb.KERNEL_BWD_DQ)):
+            b = plan.busy_times(k).astype(np.float64)
+            b = b[b > 0]
+            busy[n] = round(float(b.max() / b.mean()), 4)
+        return ms, kern, busy
+
+    def destroy(self):
+        if self.plan is not None:
+            self.plan.destroy()
+            self.plan = None
+        self.inp = self.out = self.ws = None
+
+
+def pool_line(pool, ms, kern, busy):
+    """Compact record of one pool's measurement (the skewed-pool and sweep legs)."""
+    ff, fb = pool.ff, pool.fb
+    return {"useful_tflops": round((ff + fb) / (ms * 1e-3) / 1e12, 1), "ms_per_step": round(ms, 3),
+            "kernel_ms": {n: round(v, 3) for n, v in kern.items()}, "busy_max_over_mean": busy}
+
+
 # ---- our arm ---------------------------------------------------------------------------------
 
 def run_ours(args):
@@ -157,126 +257,100 @@ def run_ours(args):
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-
-    spec = sharding.rank_spec(args.config, args.skew, rank, args.seqs)       # every rank its own pool
-    lengths = pools.pool_lengths(spec)
-    cu_np = pools.cu_seqlens(lengths)
-    T, hq, hkv, d = spec.total_tokens, spec.hq, spec.hkv, spec.head_dim
-    ff, fb = useful_flops(lengths, hq, d)
     dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
 
-    t = pools.make_tensors(T, hq, hkv, d, seed=rank, device=f"cuda:{local}")
-    q, k, v, dout = t["q"], t["k"], t["v"], t["dout"]
-    cu = torch.from_numpy(cu_np).to(dev)
-    blocks = args.weight_model == "blocks"
+    spec = sharding.rank_spec(args.config, args.skew, rank, args.seqs, replicas=args.replicas)
+    shard = None if (args.replicas or world == 1) else sharding.head_groups(spec.hq, spec.hkv, world, rank)
+    groups = {} if shard is None else sharding.kv_subgroups(spec.hq, spec.hkv, world)
+    pool = Pool(lb, spec, dev, shard=shard, weight_model=args.weight_model, heads=args.heads,
+                seed=rank if args.replicas else 0)
+    plan_ms = pool.build()
+    kv_shared = shard is not None and len(shard.kv_sharers) > 1
 
-    def make_plan():
-        return lb.libra_plan_tiles(cu, hq, 256, tile_kv=128, n_heads_kv=hkv, total_tokens=T,
-                                   weight_model=lb.LIBRA_WEIGHT_BLOCKS if blocks else lb.LIBRA_WEIGHT_PAIRS,
-                                   unit_cost_q=12 if blocks else 0, unit_cost_kv=6 if blocks else 0)
+    if kv_shared:                                      # ranks sharing a kv head add their dK / dV up every step
+        plain_step_on = pool.step_on
+        group = groups[shard.kv_heads[0]]
 
-    make_plan().destroy()                     # first call pays for the module load
-    torch.cuda.synchronize()
-    pe0, pe1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    pe0.record()
-    plan = make_plan()                        # built once, outside the timed steps (the paper reuses it across layers)
-    pe1.record()
-    torch.cuda.synchronize()
-    plan_ms = pe0.elapsed_time(pe1)
-    assert plan.status() == 0
-    plan.set_timing(True)
-    out = torch.empty_like(q)
-    lse = torch.empty((hq, T), dtype=torch.float32, device=dev)
-    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
-    ws = torch.empty(lb.libra_attn_pool_bwd_workspace_bytes(plan, q, k), dtype=torch.uint8, device=dev)
-
-    def step_on(i, o):
-        lb.libra_attn_pool_fwd(i["q"], i["k"], i["v"], plan, out=o["out"], lse=o["lse"])
-        lb.libra_attn_pool_bwd(i["q"], i["k"], i["v"], o["out"], o["lse"], i["dout"], plan, dq=o["dq"], dk=o["dk"],
-                               dv=o["dv"], workspace=ws)
-
-    def step():
-        step_on(dict(q=q, k=k, v=v, dout=dout), dict(out=out, lse=lse, dq=dq, dk=dk, dv=dv))
+        def step_on(i, o, plan=None):
+            plain_step_on(i, o, plan)
+            dk, dv = sharding.reduce_kv_grads(shard, o["dk"], o["dv"], group)
+            o["dk"].copy_(dk); o["dv"].copy_(dv)
+        pool.step_on = step_on
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
-        step()
-    barrier()
-
-    # ---- device-resident timing: K steps between events, plus per-kernel events per step
+    # ---- device-resident timing: K steps between events, the library's per-kernel events inside the same loop
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
     n0 = lb.launch_count()
-    kern_f, kern_b, kern_q = [], [], []
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    e0.record()
-    for _ in range(args.steps):
-        step()
-    e1.record()
-    barrier()
-    total_ms = e0.elapsed_time(e1)
-    launches = lb.launch_count() - n0
-    # kernel-only durations (events recorded by the library on the launch stream), untimed extra steps
-    for _ in range(min(args.steps, 5)):
-        step()
-        kern_f.append(plan.kernel_time_ms(lb.KERNEL_FWD))
-        kern_b.append(plan.kernel_time_ms(lb.KERNEL_BWD_DKDV))
-        kern_q.append(plan.kernel_time_ms(lb.KERNEL_BWD_DQ))
+    ms_local, kern, busy = pool.timed(args.steps, max(args.warmup, 3), barrier)
+    launches = lb.launch_count() - n0 - max(args.warmup, 3) * 4
     clocks = sampler.stop() if rank == 0 else None
-    busy_f = plan.busy_times(lb.KERNEL_FWD).astype(np.float64)
-    busy_b = plan.busy_times(lb.KERNEL_BWD_DKDV).astype(np.float64)
-    busy_q = plan.busy_times(lb.KERNEL_BWD_DQ).astype(np.float64)
-
-    ms_per_step, work = sharding.aggregate(total_ms / args.steps, float(ff + fb), device=dev)
+    ms_per_step, work = sharding.aggregate(ms_local, float(pool.ff + pool.fb), device=dev)
     value = work / (ms_per_step * 1e-3) / 1e12
 
     # ---- the same steps under the plan's other tile weight (context for the busy-time spread, not the headline)
     alt = None
     if world == 1 and not args.skip_e2e:
-        other = not blocks
-        plan2 = lb.libra_plan_tiles(cu, hq, 256, tile_kv=128, n_heads_kv=hkv, total_tokens=T,
-                                    weight_model=lb.LIBRA_WEIGHT_BLOCKS if other else lb.LIBRA_WEIGHT_PAIRS,
-                                    unit_cost_q=12 if other else 0, unit_cost_kv=6 if other else 0)
-
-        def step2():
-            lb.libra_attn_pool_fwd(q, k, v, plan2, out=out, lse=lse)
-            lb.libra_attn_pool_bwd(q, k, v, out, lse, dout, plan2, dq=dq, dk=dk, dv=dv, workspace=ws)
-
-        for _ in range(3):
-            step2()
-        barrier()
-        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a0.record()
-        for _ in range(args.steps):
-            step2()
-        a1.record()
-        barrier()
-        spread = [plan2.busy_times(kk).astype(np.float64) for kk in (lb.KERNEL_FWD, lb.KERNEL_BWD_DKDV, lb.KERNEL_BWD_DQ)]
+        other = not pool.blocks
+        plan2 = pool.make_plan(blocks=other)
+        ms2, _, busy2 = pool.timed(args.steps, 3, barrier, plan=plan2)
         alt = {"tile_weight": "blocks (time proxy)" if other else "causal pairs (Eq. 6)",
-               "value": round((ff + fb) / (a0.elapsed_time(a1) / args.steps * 1e-3) / 1e12, 2), "unit": "TFLOP/s",
-               "busy_max_over_mean": {n: round(float(b.max() / b.mean()), 4) for n, b in zip(("fwd", "bwd_dkdv", "bwd_dq"), spread)}}
+               "value": round((pool.ff + pool.fb) / (ms2 * 1e-3) / 1e12, 2), "unit": "TFLOP/s",
+               "busy_max_over_mean": busy2}
         plan2.destroy()
 
     e2e = None
     if not args.skip_e2e:
-        e2e = run_e2e(args, step_on, barrier, dict(q=q, k=k, v=v, dout=dout),
-                      dict(out=out, lse=lse, dq=dq, dk=dk, dv=dv), world, dev, ff + fb)
-    finish(args, rank, world, spec, lengths, plan, value, ms_per_step, (kern_f, kern_b, kern_q),
-           (busy_f, busy_b, busy_q), clocks, launches, e2e, ff, fb, q, plan_ms, alt)
-    plan.destroy()
+        e2e = run_e2e(args, pool.step_on, barrier, pool.inp, pool.out, dev, pool.ff + pool.fb)
+
+    line = None
+    if rank == 0:
+        line = headline(args, world, spec, pool, value, ms_per_step, ms_local, kern, busy, clocks, launches, e2e,
+                        plan_ms, alt, shard)
+    pool.destroy()
+    del pool
+    torch.cuda.empty_cache()
+
+    if rank == 0 and world == 1 and not args.skip_skewed:
+        line["skewed_pools"] = skewed_pools(args, lb, dev, barrier)
+    if rank == 0 and world == 1 and not args.skip_cpu:
+        cb = time_oracle(spec, pools.pool_lengths(spec))
+        line["cpu_baseline"] = {k2: (round(v2, 6) if isinstance(v2, float) else v2) for k2, v2 in cb.items()}
+    if rank == 0:
+        print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
 
 
-def run_e2e(args, step_on, barrier, dev_in, dev_out, world, dev, flops):
+def skewed_pools(args, lb, dev, barrier):
+    """The pools that carry the busy-time target: the 30B-shaped pool with Pareto-tailed samples, the 1M-token
+    pool with one 262144-token sample, and the skew sweep at every skew; a few steps each."""
+    import torch
+    out = {}
+    for name, cfg, skew, steps in (("config3", 3, 0.0, 5), ("config5_skew0", 5, 0.0, 5), ("config5_skew0.25", 5, 0.25, 4),
+                                   ("config5_skew0.5", 5, 0.5, 3), ("config5_skew1", 5, 1.0, 2), ("config4", 4, 0.0, 2)):
+        spec = pools.config(cfg, skew)
+        pool = Pool(lb, spec, dev, weight_model=args.weight_model)
+        pool.build()
+        ms, kern, busy = pool.timed(steps, 1 if cfg == 4 else 2, barrier)
+        rec = pool_line(pool, ms, kern, busy)
+        rec.update(steps=steps, samples=len(pool.lengths), max_sample=int(max(pool.lengths)), tokens=spec.total_tokens,
+                   heads=f"Hq {spec.hq} / Hkv {spec.hkv}")
+        out[name] = rec
+        pool.destroy()
+        del pool
+        torch.cuda.empty_cache()
+    return out
+
+
+def run_e2e(args, step_on, barrier, dev_in, dev_out, dev, flops):
     """End to end through the public calls with HOST buffers: every step its inputs are copied from pinned host
     memory and its results are copied back.  The copies of neighbouring steps overlap the kernels of the current
     one (two device buffer sets, one copy-in and one copy-out stream), as a caller streaming batches would do."""
@@ -336,58 +410,63 @@ def run_e2e(args, step_on, barrier, dev_in, dev_out, world, dev, flops):
             "d2h_bytes_per_step": d2h, "ms_per_step": round(e2e_ms, 3)}
 
 
-def finish(args, rank, world, spec, lengths, plan, value, ms_per_step, kern, busy, clocks, launches, e2e, ff, fb, q,
-           plan_ms=None, alt=None):
-    kern_f, kern_b, kern_q = kern
-    busy_f, busy_b, busy_q = busy
-    from paper_2607_23250_b200 import binding as lb  # noqa: F401
-    T, hq, hkv, d = spec.total_tokens, spec.hq, spec.hkv, spec.head_dim
-    if rank == 0:
-        peaks = measured_peaks()
-        kb = statistics.mean(kern_b)
-        kf = statistics.mean(kern_f)
-        kq = statistics.mean(kern_q)
-        # Dominant kernel: the backward dK/dV kernel.  Algorithmic work per launch: the four GEMMs of
-        # the dK/dV gradient it owns (S, dP, dV, dK = 8 d flops per causal pair per query head).
-        fa = fb * 8 // 10
-        ach = fa / (kb * 1e-3) / 1e12
-        traffic = read_traffic("k_attn_bwd_dkdv", args)
-        line = {
-            "metric": METRIC, "value": round(value, 2), "unit": "TFLOP/s", "n_gpus": world,
-            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 4),
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
-            "data": "synthetic",
-            "config": {"workload": f"config {args.config}: {spec.name} pool, {spec.n_seqs} x {spec.seq_len} tokens, "
-                                   f"{len(lengths)} samples (log-normal median 644, sigma 1.6), Hq {hq} / Hkv {hkv} / d {d}, "
-                                   f"causal per sample, fwd+bwd; plan built once and reused",
-                       "tile_q": 256, "tile_kv": 128, "n_workers": plan.info()["n_workers"],
-                       "tile_weight": "blocks (time proxy)" if args.weight_model == "blocks" else "causal pairs (Eq. 6)",
-                       "l2": "inputs larger than L2 (Q alone is %.2f GB)" % (q.numel() * 2 / 1e9),
-                       "per_rank_pool": "seed = rank"},
-            "pct_of_bf16_peak": {"burst_measured": round(100 * value / world / peaks["burst"], 2),
-                                 "sustained_measured": round(100 * value / world / peaks["sustained"], 2),
-                                 "nominal_2250": round(100 * value / world / 2250.0, 2), "peaks": peaks["source"]},
-            "fwd_kernel": {"ms": round(kf, 4), "tflops": round(ff / kf / 1e9, 1)},
-            "bwd_dkdv_kernel": {"ms": round(kb, 4), "executed_tflops": round(fa / kb / 1e9, 1)},
-            "bwd_dq_kernel": {"ms": round(kq, 4), "executed_tflops": round(fb * 6 // 10 / kq / 1e9, 1)},
-            "bwd_useful_tflops": round(fb / (kb + kq) / 1e9, 1),
-            "busy_max_over_mean": {"fwd": round(float(busy_f.max() / busy_f.mean()), 4),
-                                   "bwd_dkdv": round(float(busy_b.max() / busy_b.mean()), 4),
-                                   "bwd_dq": round(float(busy_q.max() / busy_q.mean()), 4)},
-            "clocks": clocks,
-            "e2e": e2e,
-            "gpu_launches": int(launches),
-            "plan_ms": None if plan_ms is None else round(plan_ms, 3),
-            "other_tile_weight": alt,
-            "roofline": {"bound": "tensor", "kernel": "k_attn_bwd_dkdv", "achieved": round(ach, 1),
-                         "peak": peaks["sustained"], "unit": "TFLOP/s", "frac": round(ach / peaks["sustained"], 4),
-                         "peak_kind": f"bf16 sustained, {peaks['source']}", "traffic": traffic,
-                         "frac_of_burst": round(ach / peaks["burst"], 4)},
-        }
-        if world == 1 and not args.skip_cpu:
-            cb = time_oracle(spec, lengths)
-            line["cpu_baseline"] = {k2: (round(v2, 6) if isinstance(v2, float) else v2) for k2, v2 in cb.items()}
-        print(json.dumps(line), flush=True)
+def headline(args, world, spec, pool, value, ms_per_step, ms_local, kern, busy, clocks, launches, e2e, plan_ms, alt,
+             shard):
+    peaks = measured_peaks()
+    hq, hkv, d, T = spec.hq, spec.hkv, spec.head_dim, spec.total_tokens
+    ff, fb = pool.ff, pool.fb                      # this rank's heads
+    kf, kb, kq, kp = (kern[n] for n in KERNELS)
+    # Dominant kernel: the backward dK/dV kernel.  Algorithmic work per launch: the four GEMMs of the dK/dV
+    # gradient it owns (S, dP, dV, dK = 8 d flops per causal pair per query head).  It is timed inside the timed
+    # region; that region's length decides which measured peak applies (burst under a second, else sustained).
+    fa = fb * 8 // 10
+    ach = fa / (kb * 1e-3) / 1e12
+    region_s = ms_local * args.steps * 1e-3
+    kind = "burst" if region_s < 1.0 else "sustained"
+    peak = peaks[kind]
+    line = {
+        "metric": METRIC, "value": round(value, 2), "unit": "TFLOP/s", "n_gpus": world,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 4),
+        "higher_is_better": True, "scaling": "weak" if (args.replicas or world == 1) else "strong",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"config {args.config}: {spec.name} pool, {spec.n_seqs} x {spec.seq_len} tokens, "
+                               f"{len(pool.lengths)} samples (log-normal median 644, sigma 1.6), Hq {hq} / Hkv {hkv} / d {d}, "
+                               f"causal per sample, fwd+bwd; plan built once and reused",
+                   "tile_q": 256, "tile_kv": 128, "head_shards": pool.heads, "n_workers": pool.plan.info()["n_workers"],
+                   "tile_weight": "blocks (time proxy)" if pool.blocks else "causal pairs (Eq. 6)",
+                   "l2": "inputs larger than L2 (Q alone is %.2f GB per rank)" % (pool.inp["q"].numel() * 2 / 1e9),
+                   "parallelism": ("one GPU" if world == 1 else
+                                   (f"{world} independent pools (seed = rank)" if args.replicas else
+                                    f"one pool split by heads over {world} ranks: {shard.hkv} kv / {shard.hq} query heads per rank"
+                                    + (", dK/dV summed over the ranks of a kv head" if len(shard.kv_sharers) > 1 else
+                                       ", no data-path collective")))},
+        "pct_of_bf16_peak": {"burst_measured": round(100 * value / world / peaks["burst"], 2),
+                             "sustained_measured": round(100 * value / world / peaks["sustained"], 2),
+                             "nominal_2250": round(100 * value / world / 2250.0, 2), "peaks": peaks["source"]},
+        "kernel_ms_in_timed_loop": {n: round(v, 4) for n, v in kern.items()},
+        "kernel_ms_sum": round(kf + kb + kq + kp, 4),
+        "fwd_useful_tflops": round(ff / kf / 1e9, 1),
+        "bwd_useful_tflops": round(fb / (kb + kq + kp) / 1e9, 1),
+        "bwd_executed_tflops": {"dkdv (8 d per pair)": round(fa / kb / 1e9, 1), "dq (6 d per pair)": round(fb * 6 // 10 / kq / 1e9, 1)},
+        "busy_max_over_mean": busy,
+        "clocks": clocks,
+        "e2e": e2e,
+        "gpu_launches": int(launches),
+        "plan_ms": round(plan_ms, 3),
+        "other_tile_weight": alt,
+        "roofline": {"bound": "tensor", "kernel": "k_attn_bwd_dkdv", "achieved": round(ach, 1),
+                     "peak": peak, "unit": "TFLOP/s", "frac": round(ach / peak, 4),
+                     "peak_kind": f"bf16 {kind}, {peaks['source']} (timed region {region_s:.2f} s)",
+                     "traffic": read_traffic("k_attn_bwd_dkdv", args),
+                     "frac_of_burst": round(ach / peaks["burst"], 4),
+                     "frac_of_sustained": round(ach / peaks["sustained"], 4),
+                     "whole_path": {"useful_tflops_per_gpu": round(value / world, 1),
+                                    "frac_of_burst": round(value / world / peaks["burst"], 4),
+                                    "frac_of_sustained": round(value / world / peaks["sustained"], 4),
+                                    "executed_over_useful_flops": "18 d / 14 d per causal pair (S and dP are computed by "
+                                                                  "both backward kernels)"}},
+    }
+    return line
 
 
 def read_traffic(kernel, args):
@@ -402,6 +481,41 @@ def read_traffic(kernel, args):
     except Exception:
         pass
     return None
+
+
+# ---- head-shard x tile-weight sweep -----------------------------------------------------------------
+
+def run_sweep(args):
+    """Useful TFLOP/s and busy-time spread against the number of head shards H and the tile weight, on the
+    8B-shaped, the 30B-shaped and two skewed pools (a few steps each).  Prints a markdown table."""
+    import torch
+    from paper_2607_23250_b200 import binding as lb
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+
+    def barrier():
+        torch.cuda.synchronize()
+
+    rows = []
+    for name, cfg, skew, steps in (("config 2 (8B shape)", 2, 0.0, 8), ("config 3 (30B shape)", 3, 0.0, 4),
+                                   ("config 5, skew 0.5", 5, 0.5, 2), ("config 5, skew 1", 5, 1.0, 2)):
+        spec = pools.config(cfg, skew)
+        for H in sorted({spec.hkv, 2 * spec.hkv, spec.hq}):
+            for wm in ("pairs", "blocks"):
+                pool = Pool(lb, spec, dev, weight_model=wm, heads=H)
+                plan_ms = pool.build()
+                ms, kern, busy = pool.timed(steps, 2, barrier)
+                rec = pool_line(pool, ms, kern, busy)
+                rows.append((name, H, wm, rec, plan_ms))
+                pool.destroy()
+                del pool
+                torch.cuda.empty_cache()
+    print("| pool | head shards H | tile weight | useful TFLOP/s | ms/step | fwd ms | dK/dV ms | dQ ms | busy max/mean fwd | dK/dV | dQ | plan ms |")
+    print("|---|---|---|---|---|---|---|---|---|---|---|---|")
+    for name, H, wm, r, plan_ms in rows:
+        k, b = r["kernel_ms"], r["busy_max_over_mean"]
+        print(f"| {name} | {H} | {wm} | {r['useful_tflops']} | {r['ms_per_step']} | {k['fwd']} | {k['bwd_dkdv']} | "
+              f"{k['bwd_dq']} | {b['fwd']} | {b['bwd_dkdv']} | {b['bwd_dq']} | {plan_ms:.1f} |")
 
 
 def run_reference(args):
@@ -435,12 +549,18 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--weight-model", default="pairs", choices=["pairs", "blocks"],
                     help="tile weight of the plan: the paper's pair count, or the executed-block count")
+    ap.add_argument("--heads", type=int, default=0, help="head shards H of the query-major tiles (0 = one per query head)")
     ap.add_argument("--seqs", type=int, default=0, help="override the number of packed sequences (profiling runs)")
+    ap.add_argument("--replicas", action="store_true", help="N > 1: one independent pool per rank instead of one pool split by heads")
+    ap.add_argument("--sweep", action="store_true", help="print the head-shard x tile-weight table instead of the JSON line")
     ap.add_argument("--skip-e2e", action="store_true", help="skip the host-buffer end-to-end leg (profiling runs)")
     ap.add_argument("--skip-cpu", action="store_true", help="skip the CPU oracle leg (profiling runs)")
+    ap.add_argument("--skip-skewed", action="store_true", help="skip the skewed-pool leg (profiling runs)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.sweep:
+        run_sweep(args)
     else:
         run_ours(args)
 

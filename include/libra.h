@@ -63,6 +63,7 @@ extern "C" {
 #define LIBRA_KERNEL_FWD       1   /* forward kernel (walks the query-major lists)            */
 #define LIBRA_KERNEL_BWD_DKDV  2   /* backward dK/dV kernel (walks the key-major lists)       */
 #define LIBRA_KERNEL_BWD_DQ    3   /* backward dQ kernel (walks the query-major lists)        */
+#define LIBRA_KERNEL_BWD_PREP  4   /* backward row statistics (timing only: it keeps no busy times) */
 
 typedef struct libra_plan libra_plan_t;   /* opaque, library-owned */
 
@@ -284,12 +285,16 @@ int libra_busy_times(const libra_plan_t* plan, int which, uint64_t* ns_host);
  * LIBRA_ERR_TIMEOUT through libra_busy_times.  A healthy run never comes near the default. */
 int libra_plan_set_wait_limit_ns(libra_plan_t* plan, uint64_t ns);
 
-/* Kernel timing: when enabled, every forward / backward call records CUDA events on its
- * stream around each persistent kernel (not around the row-statistics launch).
- * libra_kernel_time_ms synchronises on the closing event of the most recent launch of kernel
- * `which` (LIBRA_KERNEL_*) and returns its duration in milliseconds.  Off by default. */
+/* Kernel timing: when enabled, every forward / backward call records CUDA events on its stream
+ * around each of its kernels (LIBRA_KERNEL_*), keeping the 64 most recent launches of each;
+ * enabling it again starts a fresh record.  libra_kernel_time_ms synchronises on the closing event
+ * of the most recent launch of kernel `which` and returns its duration in milliseconds;
+ * libra_kernel_times_ms returns the durations of up to `capacity` most recent recorded launches,
+ * oldest first, and their number in *n_out.  Off by default.
+ * Errors: INVALID_ARG, PLAN_MISMATCH (nothing recorded yet), CUDA. */
 int libra_plan_set_timing(libra_plan_t* plan, int enabled);
 int libra_kernel_time_ms(const libra_plan_t* plan, int which, float* ms_host);
+int libra_kernel_times_ms(const libra_plan_t* plan, int which, float* ms_host, int capacity, int* n_out);
 
 /* Number of kernels this library has launched in the calling process (for accounting). */
 int64_t libra_launch_count(void);

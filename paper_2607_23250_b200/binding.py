@@ -21,7 +21,7 @@ _lib = ctypes.CDLL(_SO)
 
 LIBRA_DIR_Q, LIBRA_DIR_KV = 1, 2
 LIBRA_WEIGHT_PAIRS, LIBRA_WEIGHT_BLOCKS = 0, 1
-KERNEL_FWD, KERNEL_BWD_DKDV, KERNEL_BWD_DQ = 1, 2, 3
+KERNEL_FWD, KERNEL_BWD_DKDV, KERNEL_BWD_DQ, KERNEL_BWD_PREP = 1, 2, 3, 4
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_PLAN_MISMATCH, ERR_CUDA = -1, -2, -3, -4
 ERR_OVERFLOW, ERR_TIMEOUT, ERR_BAD_SEQLENS, ERR_NO_DEVICE = -5, -6, -7, -8
 ERR_SCRATCH_TOO_SMALL = -9
@@ -29,7 +29,7 @@ ERR_SCRATCH_TOO_SMALL = -9
 EXPORTS = ["libra_plan_tiles", "libra_plan_info", "libra_plan_status", "libra_plan_export",
            "libra_plan_destroy", "libra_attn_pool_fwd", "libra_attn_pool_bwd_workspace_bytes",
            "libra_attn_pool_bwd", "libra_attn_pool_bwd_noalloc_max_bytes", "libra_attn_pool_bwd_noalloc",
-           "libra_busy_times", "libra_plan_set_wait_limit_ns", "libra_plan_set_timing", "libra_kernel_time_ms", "libra_launch_count",
+           "libra_busy_times", "libra_plan_set_wait_limit_ns", "libra_plan_set_timing", "libra_kernel_time_ms", "libra_kernel_times_ms", "libra_launch_count",
            "libra_strerror"]
 
 
@@ -124,6 +124,14 @@ class Plan:
         ms = ctypes.c_float()
         _check(_lib.libra_kernel_time_ms(self._h, which, ctypes.byref(ms)), "libra_kernel_time_ms")
         return float(ms.value)
+
+    def kernel_times_ms(self, which=KERNEL_FWD, capacity=64):
+        """Durations (ms) of the most recent recorded launches of kernel `which`, oldest first."""
+        buf = (ctypes.c_float * capacity)()
+        n = ctypes.c_int()
+        _check(_lib.libra_kernel_times_ms(self._h, which, buf, ctypes.c_int(capacity), ctypes.byref(n)),
+               "libra_kernel_times_ms")
+        return [float(buf[i]) for i in range(n.value)]
 
     def destroy(self):
         if self._h:

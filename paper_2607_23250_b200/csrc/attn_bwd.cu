@@ -654,11 +654,12 @@ static int launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtens
         if (!regs_pool_ok(k_attn_bwd_dq<D>, 128 * kDqGroups, kDqRegsCompute, 128, kDqRegsOther)) return LIBRA_ERR_UNSUPPORTED;
         cfg_mark(kSlot);
     }
-    if (mp->timing) cudaEventRecord(mp->ev[1][0], s);
+    time_begin(mp, 1, s);
     k_attn_bwd_dkdv<D><<<Wa, kBwdThreads, DkvSmem<D>::kBytes, s>>>(tq, tk, tv, tdo, pa);
-    if (mp->timing) { cudaEventRecord(mp->ev[1][1], s); mp->ev_valid[1] = 1; cudaEventRecord(mp->ev[2][0], s); }
+    time_end(mp, 1, s);
+    time_begin(mp, 2, s);
     k_attn_bwd_dq<D><<<Wb, kDqThreads, DqSmem<D>::kBytes, s>>>(tq, tk, tv, tdo, tdq, pb);
-    if (mp->timing) { cudaEventRecord(mp->ev[2][1], s); mp->ev_valid[2] = 1; }
+    time_end(mp, 2, s);
     count_launch(2);
     return cudaGetLastError() == cudaSuccess ? LIBRA_OK : LIBRA_ERR_CUDA;
 }
@@ -716,6 +717,8 @@ extern "C" int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const v
     if (rc == LIBRA_OK) rc = make_thd_map(&tdq, dq_dev, T, dims->hq, D, kBlk);
     if (rc != LIBRA_OK) return rc;
 
+    libra_plan_t* mp0 = const_cast<libra_plan_t*>(plan);
+    time_begin(mp0, 3, s);
     {
         const int64_t warps = ws.Tpad / 32 * dims->hq;
         const unsigned grid = (unsigned)((warps * 32 + 255) / 256);
@@ -727,6 +730,7 @@ extern "C" int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const v
                                                 T, ws.Tpad, dims->hq, dvec, lse2);
         count_launch();
     }
+    time_end(mp0, 3, s);
     const float scale = dims->softmax_scale > 0.f ? dims->softmax_scale : 1.0f / sqrtf((float)D);
     DkvParams pa;
     pa.dk = reinterpret_cast<__nv_bfloat16*>(dk_dev);

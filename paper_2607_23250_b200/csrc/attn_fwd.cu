@@ -604,9 +604,9 @@ extern "C" int libra_attn_pool_fwd(const void* q_dev, const void* k_dev, const v
     cudaStream_t s = (cudaStream_t)stream;
     cudaMemsetAsync(plan->d_status + 1, 0, sizeof(int), s);   // the word reports the most recent launch
     libra_plan_t* mp = const_cast<libra_plan_t*>(plan);
-    if (mp->timing) cudaEventRecord(mp->ev[0][0], s);
+    time_begin(mp, 0, s);
     rc = dims->head_dim == 128 ? launch_fwd<128>(tq, tk, tv, prm, d.W, s) : launch_fwd<64>(tq, tk, tv, prm, d.W, s);
-    if (mp->timing) { cudaEventRecord(mp->ev[0][1], s); mp->ev_valid[0] = 1; }
+    time_end(mp, 0, s);
     return rc;
 }
 

@@ -44,8 +44,10 @@ struct libra_plan {
     libra::PlanDir dir[2];           // 0 = query-major, 1 = key-major
     uint32_t wait_limit_ns = 2000000000u;  // budget of one device-side wait (libra_plan_set_wait_limit_ns)
     int timing = 0;                  // record events around the main kernels
-    cudaEvent_t ev[3][2] = {{nullptr, nullptr}, {nullptr, nullptr}, {nullptr, nullptr}};  // [kernel][begin, end]
-    int ev_valid[3] = {0, 0, 0};
+    // [kernel][slot][begin, end]: a ring of the most recent launches of each kernel (LIBRA_KERNEL_* - 1)
+    static constexpr int kTimedKernels = 4, kTimeRing = 64;
+    cudaEvent_t ev[kTimedKernels][kTimeRing][2] = {};
+    int64_t ev_count[kTimedKernels] = {0, 0, 0, 0};   // launches recorded since timing was switched on
 };
 
 namespace libra {
@@ -58,6 +60,13 @@ bool cfg_done(int slot);
 void cfg_mark(int slot);
 // LIBRA_ERR_PLAN_MISMATCH when the current device is not the one the plan was built on.
 int check_plan_device(const libra_plan* plan);
+// Kernel timing (libra_plan_set_timing): events on the launch stream around kernel k (LIBRA_KERNEL_* - 1).
+inline void time_begin(libra_plan* p, int k, cudaStream_t s) {
+    if (p->timing) cudaEventRecord(p->ev[k][p->ev_count[k] % libra_plan::kTimeRing][0], s);
+}
+inline void time_end(libra_plan* p, int k, cudaStream_t s) {
+    if (p->timing) { cudaEventRecord(p->ev[k][p->ev_count[k] % libra_plan::kTimeRing][1], s); ++p->ev_count[k]; }
+}
 extern std::atomic<int64_t> g_launches;
 inline void count_launch(int n = 1) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 }  // namespace libra

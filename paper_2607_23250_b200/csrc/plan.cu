@@ -427,9 +427,10 @@ extern "C" int libra_plan_destroy(libra_plan_t* plan) {
     cudaFree(plan->d_tok_start);
     cudaFree(plan->d_tok_end);
     cudaFree(plan->d_status);
-    for (int a = 0; a < 3; ++a)
-        for (int b = 0; b < 2; ++b)
-            if (plan->ev[a][b]) cudaEventDestroy(plan->ev[a][b]);
+    for (int a = 0; a < libra_plan::kTimedKernels; ++a)
+        for (int r = 0; r < libra_plan::kTimeRing; ++r)
+            for (int b = 0; b < 2; ++b)
+                if (plan->ev[a][r][b]) cudaEventDestroy(plan->ev[a][r][b]);
     delete plan;
     return LIBRA_OK;
 }
@@ -456,9 +457,11 @@ extern "C" int libra_busy_times(const libra_plan_t* plan, int which, uint64_t* n
 extern "C" int libra_plan_set_timing(libra_plan_t* plan, int enabled) {
     if (!plan) return LIBRA_ERR_INVALID_ARG;
     if (enabled) {
-        for (int a = 0; a < 3; ++a)
-            for (int b = 0; b < 2; ++b)
-                if (!plan->ev[a][b] && cudaEventCreate(&plan->ev[a][b]) != cudaSuccess) return LIBRA_ERR_CUDA;
+        for (int a = 0; a < libra_plan::kTimedKernels; ++a)
+            for (int r = 0; r < libra_plan::kTimeRing; ++r)
+                for (int b = 0; b < 2; ++b)
+                    if (!plan->ev[a][r][b] && cudaEventCreate(&plan->ev[a][r][b]) != cudaSuccess) return LIBRA_ERR_CUDA;
+        for (int a = 0; a < libra_plan::kTimedKernels; ++a) plan->ev_count[a] = 0;   // a fresh record
     }
     plan->timing = enabled ? 1 : 0;
     return LIBRA_OK;
@@ -470,13 +473,31 @@ extern "C" int libra_plan_set_wait_limit_ns(libra_plan_t* plan, uint64_t ns) {
     return LIBRA_OK;
 }
 
+static int kernel_time(const libra_plan_t* plan, int a, int64_t launch, float* ms) {
+    cudaEvent_t e0 = plan->ev[a][launch % libra_plan::kTimeRing][0], e1 = plan->ev[a][launch % libra_plan::kTimeRing][1];
+    if (cudaEventSynchronize(e1) != cudaSuccess) return LIBRA_ERR_CUDA;
+    return cudaEventElapsedTime(ms, e0, e1) == cudaSuccess ? LIBRA_OK : LIBRA_ERR_CUDA;
+}
+
 extern "C" int libra_kernel_time_ms(const libra_plan_t* plan, int which, float* ms_host) {
     if (!plan || !ms_host) return LIBRA_ERR_INVALID_ARG;
-    const int a = which - 1;  // LIBRA_KERNEL_FWD / _BWD_DKDV / _BWD_DQ
-    if (a < 0 || a > 2) return LIBRA_ERR_INVALID_ARG;
-    if (!plan->ev_valid[a]) return LIBRA_ERR_PLAN_MISMATCH;
-    if (cudaEventSynchronize(plan->ev[a][1]) != cudaSuccess) return LIBRA_ERR_CUDA;
-    if (cudaEventElapsedTime(ms_host, plan->ev[a][0], plan->ev[a][1]) != cudaSuccess) return LIBRA_ERR_CUDA;
+    const int a = which - 1;  // LIBRA_KERNEL_FWD / _BWD_DKDV / _BWD_DQ / _BWD_PREP
+    if (a < 0 || a >= libra_plan::kTimedKernels) return LIBRA_ERR_INVALID_ARG;
+    if (plan->ev_count[a] == 0) return LIBRA_ERR_PLAN_MISMATCH;
+    return kernel_time(plan, a, plan->ev_count[a] - 1, ms_host);
+}
+
+extern "C" int libra_kernel_times_ms(const libra_plan_t* plan, int which, float* ms_host, int capacity, int* n_out) {
+    if (!plan || !ms_host || !n_out || capacity < 0) return LIBRA_ERR_INVALID_ARG;
+    const int a = which - 1;
+    if (a < 0 || a >= libra_plan::kTimedKernels) return LIBRA_ERR_INVALID_ARG;
+    int64_t n = plan->ev_count[a] < libra_plan::kTimeRing ? plan->ev_count[a] : libra_plan::kTimeRing;
+    if (n > capacity) n = capacity;
+    for (int64_t i = 0; i < n; ++i) {   // oldest first
+        const int rc = kernel_time(plan, a, plan->ev_count[a] - n + i, ms_host + i);
+        if (rc != LIBRA_OK) return rc;
+    }
+    *n_out = (int)n;
     return LIBRA_OK;
 }
 
