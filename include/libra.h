@@ -285,6 +285,20 @@ int libra_busy_times(const libra_plan_t* plan, int which, uint64_t* ns_host);
  * LIBRA_ERR_TIMEOUT through libra_busy_times.  A healthy run never comes near the default. */
 int libra_plan_set_wait_limit_ns(libra_plan_t* plan, uint64_t ns);
 
+/* Test aid (no counterpart in the paper): while enabled, the producer role of the attention kernels launched
+ * with this plan issues no loads at all, so every consumer's first wait runs out of its budget on an
+ * otherwise healthy GPU.  This is how the give-up path is exercised without a fault or an endless loop: set a
+ * short budget with libra_plan_set_wait_limit_ns, launch, and libra_busy_times reports LIBRA_ERR_TIMEOUT; the
+ * outputs of such a launch are undefined.  Off by default. */
+int libra_plan_inject_stall(libra_plan_t* plan, int enabled);
+
+/* Self-test of the bounded wait: launches one small CTA that waits, through the same routine as every
+ * barrier wait of the attention kernels, on a barrier nothing ever arrives on, with a budget of limit_ns
+ * (1 ns .. 0.1 s) and nothing else in flight.  *status_host receives LIBRA_ERR_TIMEOUT when the wait gave up
+ * as designed (LIBRA_OK would mean it claimed completion), *waited_ns_host (nullable) how long it waited.
+ * Synchronous; allocates and frees 8 bytes of device memory.  Errors: INVALID_ARG, CUDA. */
+int libra_selftest_wait_timeout(uint32_t limit_ns, int* status_host, int* waited_ns_host);
+
 /* Kernel timing: when enabled, every forward / backward call records CUDA events on its stream
  * around each of its kernels (LIBRA_KERNEL_*), keeping the 64 most recent launches of each;
  * enabling it again starts a fresh record.  libra_kernel_time_ms synchronises on the closing event

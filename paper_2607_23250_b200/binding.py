@@ -29,7 +29,7 @@ ERR_SCRATCH_TOO_SMALL = -9
 EXPORTS = ["libra_plan_tiles", "libra_plan_info", "libra_plan_status", "libra_plan_export",
            "libra_plan_destroy", "libra_attn_pool_fwd", "libra_attn_pool_bwd_workspace_bytes",
            "libra_attn_pool_bwd", "libra_attn_pool_bwd_noalloc_max_bytes", "libra_attn_pool_bwd_noalloc",
-           "libra_busy_times", "libra_plan_set_wait_limit_ns", "libra_plan_set_timing", "libra_kernel_time_ms", "libra_kernel_times_ms", "libra_launch_count",
+           "libra_busy_times", "libra_plan_set_wait_limit_ns", "libra_plan_inject_stall", "libra_plan_set_timing", "libra_kernel_time_ms", "libra_kernel_times_ms", "libra_selftest_wait_timeout", "libra_launch_count",
            "libra_strerror"]
 
 
@@ -75,6 +75,14 @@ def _stream(stream=None):
     return _vp(s.cuda_stream)
 
 
+def libra_selftest_wait_timeout(limit_ns: int):
+    """(status, nanoseconds waited) of a wait on a barrier nothing arrives on; status is ERR_TIMEOUT by design."""
+    st, ns = ctypes.c_int(), ctypes.c_int()
+    _check(_lib.libra_selftest_wait_timeout(ctypes.c_uint32(limit_ns), ctypes.byref(st), ctypes.byref(ns)),
+           "libra_selftest_wait_timeout")
+    return st.value, ns.value
+
+
 def launch_count() -> int:
     return int(_lib.libra_launch_count())
 
@@ -116,6 +124,9 @@ class Plan:
 
     def set_wait_limit_ns(self, ns: int):
         _check(_lib.libra_plan_set_wait_limit_ns(self._h, ctypes.c_uint64(ns)), "libra_plan_set_wait_limit_ns")
+
+    def inject_stall(self, enabled=True):
+        _check(_lib.libra_plan_inject_stall(self._h, 1 if enabled else 0), "libra_plan_inject_stall")
 
     def set_timing(self, enabled=True):
         _check(_lib.libra_plan_set_timing(self._h, 1 if enabled else 0), "libra_plan_set_timing")

@@ -8,9 +8,9 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 SO = os.path.join(HERE, "liblibra.so")
-SOURCES = ["plan.cu", "attn_fwd.cu", "attn_bwd.cu", "no_alloc.cu", "vrsp.cu", "tap.cu"]
+SOURCES = ["plan.cu", "attn_fwd.cu", "attn_bwd.cu", "no_alloc.cu", "vrsp.cu", "tap.cu", "selftest.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-Xcompiler", "-fPIC", "--use_fast_math", "-Xptxas", "-v"]
+              "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 
 
 def _deps():

@@ -88,6 +88,7 @@ struct DkvParams {
     int* status;
     const int* plan_status;  // the planner's verdict on cu_seqlens: non-zero = do not run
     uint32_t wait_limit_ns;
+    int inject_stall;        // test aid: the producer issues no loads, so the consumers' waits run out
     uint64_t* busy;
 };
 
@@ -197,7 +198,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         if (elect_one()) {  // one elected thread runs the whole role
             uint32_t ucnt = 0, it_all = 0;
             bool ok = true;
-            for (int idx = unit_begin; idx < unit_end && ok; ++idx) {
+            for (int idx = unit_begin; idx < unit_end && ok && !p.inject_stall; ++idx) {
                 const int t = p.cta_tiles[idx];
                 const int kvh = t % p.hkv;
                 const int64_t k0 = (int64_t)(t / p.hkv) * kBlk;
@@ -373,8 +374,8 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             for (int it = 0; it < n_it && ok; ++it, ++it_all) {
                 const uint32_t ds = it_all % DS;
                 const float* dvec = reinterpret_cast<const float*>(smem + L::kDvecOff + ds * 512);
-                ok = mbar_wait(&bar_dofull[ds], (it_all / DS) & 1, abort_flag) &&
-                     mbar_wait(bar_dpfull, it_all & 1, abort_flag);
+                ok = warp_wait(&bar_dofull[ds], (it_all / DS) & 1, abort_flag) &&
+                     warp_wait(bar_dpfull, it_all & 1, abort_flag);
                 if (!ok) break;
                 TRACE(4)
                 tc_fence_after();
@@ -400,7 +401,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 TRACE(22)
                 // dS^T(it-1) must have been consumed by dK(it-1) before its columns are rewritten
                 if (it_all > 0) {
-                    ok = mbar_wait(&bar_qempty[(it_all - 1) % QS], ((it_all - 1) / QS) & 1, abort_flag);
+                    ok = warp_wait(&bar_qempty[(it_all - 1) % QS], ((it_all - 1) / QS) & 1, abort_flag);
                     if (!ok) break;
                 }
                 TRACE(16)
@@ -408,7 +409,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 // (columns 0..15 and 32..47 of the packed P^T), then the rest.  dS^T = P^T o (dP^T - D) in bf16 pairs.
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
-                    ok = mbar_wait(half == 0 ? bar_phalf : bar_pready, it_all & 1, abort_flag);
+                    ok = warp_wait(half == 0 ? bar_phalf : bar_pready, it_all & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
                     if (half == 0) { TRACE(17) } else { TRACE(19) }
@@ -469,8 +470,8 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 const bool need_mask = (qb == k0) || (qb + kBlk - 1 >= min_kend) || partial;
                 const int j_lo = (int)(key - qb) - c0;   // first visible column of this group's range
                 const int j_hi = kend - 1 - qb - c0;     // last visible column
-                ok = mbar_wait(&bar_qfull[qs], (it_all / QS) & 1, abort_flag) &&
-                     mbar_wait(bar_sfull, it_all & 1, abort_flag);
+                ok = warp_wait(&bar_qfull[qs], (it_all / QS) & 1, abort_flag) &&
+                     warp_wait(bar_sfull, it_all & 1, abort_flag);
                 if (!ok) break;
                 TRACE(2)
                 tc_fence_after();
@@ -483,7 +484,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 TRACE(6)
                 // P^T(it-1) must have been consumed (dV(it-1), the dS group) before its columns are rewritten
                 if (it_all > 0) {
-                    ok = mbar_wait(bar_pfree, (it_all - 1) & 1, abort_flag);
+                    ok = warp_wait(bar_pfree, (it_all - 1) & 1, abort_flag);
                     if (!ok) break;
                 }
                 TRACE(7)
@@ -523,7 +524,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             if (!ok) break;
             ++ucnt;
             // ---- unit epilogue: dK * scale and dV to global (each exp group stores half of the columns) ----
-            ok = mbar_wait(bar_dkvfull, (ucnt - 1) & 1, abort_flag);
+            ok = warp_wait(bar_dkvfull, (ucnt - 1) & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
             constexpr int kCols = D / 2;
@@ -749,6 +750,7 @@ extern "C" int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const v
     pa.status = plan->d_status + 2;
     pa.plan_status = plan->d_status;
     pa.wait_limit_ns = plan->wait_limit_ns;
+    pa.inject_stall = plan->inject_stall;
     pa.busy = dkv_dir.d_busy;
     DqParams pb;
     pb.dq = reinterpret_cast<__nv_bfloat16*>(dq_dev);
@@ -767,6 +769,7 @@ extern "C" int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const v
     pb.status = plan->d_status + 2;
     pb.plan_status = plan->d_status;
     pb.wait_limit_ns = plan->wait_limit_ns;
+    pb.inject_stall = plan->inject_stall;
     pb.busy = dq_dir.d_busy2;
     libra_plan_t* mp = const_cast<libra_plan_t*>(plan);
     return D == 128 ? launch_bwd<128>(tq, tk, tv, tdo, tdq, pa, dkv_dir.W, pb, dq_dir.W, mp, s)

@@ -44,8 +44,8 @@ struct DqSmem {
     static constexpr int kVOff = kKOff + kKStages * kTileBytes;
     static constexpr int kBarOff = kVOff + kVStages * kTileBytes;
     // q_full, q_empty, do_full, do_empty, k_full[3], k_empty[3], v_full[2], v_empty[2], qt_ready,
-    // s_full, s_free, dp_full, ds_ready, dq_full, dot_ready, dq_empty, dq_staged
-    static constexpr int kNumBars = 23;
+    // s_full, s_free, dp_full, ds_ready, dq_full, dot_ready, dq_empty, dq_staged, drain
+    static constexpr int kNumBars = 24;
     static constexpr int kMiscOff = kBarOff + kNumBars * 8;
     static constexpr int kBytes = kMiscOff + 16;
     static_assert(kBytes <= kSmemMax, "exceeds the shared memory of an sm_100 CTA");
@@ -64,6 +64,7 @@ struct DqParams {
     int* status;
     const int* plan_status;
     uint32_t wait_limit_ns;
+    int inject_stall;
     uint64_t* busy;
 };
 
@@ -134,6 +135,7 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     uint64_t* bar_dotready = bars + 20;
     uint64_t* bar_dqempty = bars + 21;
     uint64_t* bar_dqstaged = bars + 22;
+    uint64_t* bar_drain = bars + 23;   // teardown after a give-up: every MMA issued so far has completed
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::kMiscOff);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kMiscOff + 4);
 
@@ -165,6 +167,7 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         mbar_init(bar_dpfull, 1);
         mbar_init(bar_dsready, 128 * kDqGroups);
         mbar_init(bar_dqfull, 1);
+        mbar_init(bar_drain, 1);
         abort_flag[0] = 0;
         abort_flag[1] = (int)p.wait_limit_ns;
         fence_mbar_init();
@@ -234,6 +237,7 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kDqRegsOther));
         if (elect_one()) {  // one elected thread runs the whole role
             uint32_t ucnt = 0, kcnt = 0, vcnt = 0;
+            uint32_t n_q = 0, n_do = 0;   // Q / dO loads armed so far (for the give-up path)
             bool ok = true;
             // Tiles a unit will need are pulled into L2 this many key blocks ahead: the shared-memory rings
             // hold one block of lead, which covers an L2 hit but not a first touch in DRAM.
@@ -253,14 +257,17 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             auto load_q_do = [&](const DqUnit& un, uint32_t cnt) -> bool {
                 if (!mbar_wait(bar_qempty, (cnt & 1) ^ 1, abort_flag)) return false;
                 mbar_arrive_expect_tx(bar_qfull, L::kTileBytes);
+                ++n_q;
                 for (int half = 0; half < D / 64; ++half)
                     tma_load_3d(smem + L::kQOff + half * L::kHalfBytes, &tm_q, bar_qfull, half * 64, un.h, (int)un.q0);
                 if (!mbar_wait(bar_doempty, (cnt & 1) ^ 1, abort_flag)) return false;
                 mbar_arrive_expect_tx(bar_dofull, L::kTileBytes);
+                ++n_do;
                 for (int half = 0; half < D / 64; ++half)
                     tma_load_3d(smem + L::kDoOff + half * L::kHalfBytes, &tm_do, bar_dofull, half * 64, un.h, (int)un.q0);
                 return true;
             };
+            if (p.inject_stall) u.valid = false;   // test aid: no loads at all
             if (u.valid) ok = load_q_do(u, 0);
             while (u.valid && ok) {
                 const DqUnit nx = units.next();
@@ -307,6 +314,15 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     }
                 }
                 u = nx;
+            }
+            if (!ok || abort_flag[0]) {
+                // Give-up path: nothing new is issued; the copies already issued land before shared memory is released.
+                if (n_q > 0) mbar_wait_drain(bar_qfull, (n_q - 1) & 1, kDrainNs);
+                if (n_do > 0) mbar_wait_drain(bar_dofull, (n_do - 1) & 1, kDrainNs);
+                for (uint32_t b = 1; b <= (uint32_t)L::kKStages && b <= kcnt; ++b)
+                    mbar_wait_drain(&bar_kfull[(kcnt - b) % L::kKStages], ((kcnt - b) / L::kKStages) & 1, kDrainNs);
+                for (uint32_t b = 1; b <= (uint32_t)L::kVStages && b <= vcnt; ++b)
+                    mbar_wait_drain(&bar_vfull[(vcnt - b) % L::kVStages], ((vcnt - b) / L::kVStages) & 1, kDrainNs);
             }
         }
         __syncwarp();
@@ -430,7 +446,10 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 ++ucnt;
                 u = nx;
             }
-            PROF_FLUSH(true, 512 * 24 + 8)
+            if (!ok || abort_flag[0]) {   // give-up path: the MMAs already issued finish before TMEM is freed
+                tc_commit(bar_drain);
+                mbar_wait_drain(bar_drain, 0, kDrainNs);
+            }
         }
         __syncwarp();
     } else {
@@ -451,7 +470,7 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         // Copies this thread's row of Q or dO (its group's duty) of the unit whose tile has landed into TMEM.
         // The caller has seen every MMA that read the previous copy complete (s_full for Q, dp_full for dO).
         auto stage = [&](uint32_t parity) -> bool {
-            if (!mbar_wait(st_op == 0 ? bar_qfull : bar_dofull, parity, abort_flag)) return false;
+            if (!warp_wait(st_op == 0 ? bar_qfull : bar_dofull, parity, abort_flag)) return false;
             if (st_half < D / 64) {
                 const uint8_t* src = smem + (st_op == 0 ? L::kQOff : L::kDoOff) + st_half * L::kHalfBytes + r * 128;
                 const uint32_t t_dst = tmem_base + lane_addr + (st_op == 0 ? kColQ : kColDO) + 32 * st_half;
@@ -510,7 +529,7 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 const int c_hi = (row_ok ? (int)(row - k0) : -1) - CW * c;  // last visible column
                 // ---- P = exp2(S c - LSE) ----
                 PROF(4)
-                ok = mbar_wait(bar_sfull, blk & 1, abort_flag);
+                ok = warp_wait(bar_sfull, blk & 1, abort_flag);
                 if (!ok) break;
                 PROF(0)
                 TRACE(10)
@@ -536,7 +555,7 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 // ---- dS = P o (dP - D), packed over this half's own dP columns ----
                 PROF(1)
                 TRACE(11)
-                ok = mbar_wait(bar_dpfull, blk & 1, abort_flag);
+                ok = warp_wait(bar_dpfull, blk & 1, abort_flag);
                 if (!ok) break;
                 PROF(2)
                 TRACE(12)
@@ -568,7 +587,7 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             }
             if (!ok) break;
             // ---- epilogue: dQ * scale to global ----
-            ok = mbar_wait(bar_dqfull, ucnt & 1, abort_flag);
+            ok = warp_wait(bar_dqfull, ucnt & 1, abort_flag);
             if (!ok) break;
             TRACE(28)
             tc_fence_after();
@@ -579,7 +598,7 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             tmem_ld_wait();
             TRACE(30)
             // The Q tile still holds the next unit's Q until every row of it has been copied to TMEM.
-            if (nx.valid) ok = mbar_wait(bar_qtready, (ucnt + 1) & 1, abort_flag);
+            if (nx.valid) ok = warp_wait(bar_qtready, (ucnt + 1) & 1, abort_flag);
             if (!ok) break;
             {
                 uint8_t* dst = smem + L::kQOff + ((c * kCols) / 64) * L::kHalfBytes + r * 128;

@@ -30,6 +30,7 @@ constexpr int kBM = 128;            // rows per slot
 constexpr int kBN = 128;            // keys per block
 constexpr int kFwdThreads = 384;  // warps 10-11 only donate registers
 constexpr float kRescaleThreshold = 8.0f;  // log2 units: O is rescaled only when the max grows by more
+constexpr uint64_t kFwdDrainNs = 2000000;  // teardown after a give-up: budget for work already in flight to land
 
 template <int D>
 struct FwdSmem {
@@ -39,8 +40,8 @@ struct FwdSmem {
     static constexpr int kQOff = 0;
     static constexpr int kRingOff = 2 * kTileBytes;
     static constexpr int kBarOff = kRingOff + kStages * kTileBytes;
-    // barriers: full[kStages], empty[kStages], q_full, q_empty, s_full[2], p_ready[2], o_done[2], p_half[2]
-    static constexpr int kNumBars = 2 * kStages + 10;
+    // barriers: full[kStages], empty[kStages], q_full, q_empty, s_full[2], p_ready[2], o_done[2], p_half[2], drain
+    static constexpr int kNumBars = 2 * kStages + 11;
     static constexpr int kMiscOff = kBarOff + kNumBars * 8;
     static constexpr int kBytes = kMiscOff + 16;
     static constexpr int kAlloc = kBytes + 1024;  // slack to align the base to 1024 B
@@ -58,6 +59,7 @@ struct FwdParams {
     int* status;       // word to flag LIBRA_ERR_TIMEOUT in
     const int* plan_status;  // the planner's verdict on cu_seqlens: non-zero = do not run
     uint32_t wait_limit_ns;  // budget of one device-side wait
+    int inject_stall;        // test aid: the producer issues no loads, so the consumers' waits run out
     uint64_t* busy;    // [2 * gridDim.x]
 };
 
@@ -73,12 +75,6 @@ __device__ __forceinline__ SlotRange slot_range(const int32_t* tok_start, int64_
     return r;
 }
 
-// Every lane polls the barrier itself: electing one lane and broadcasting its result costs a
-// divergent branch plus a shuffle on the path between two MMA groups, which is enough silence for the
-// tensor pipe to drain (a wait on an already completed barrier measured ~230 cycles that way, ~100 so).
-__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag));
-}
 
 #ifdef LIBRA_PROF
 __device__ unsigned long long g_fwd_prof[1024 * 24];
@@ -114,6 +110,7 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
     uint64_t* bar_pready = bar_qfull + 4;  // [2]
     uint64_t* bar_odone = bar_qfull + 6;   // [2]
     uint64_t* bar_phalf = bar_qfull + 8;   // [2] P of the first 64 keys is in TMEM
+    uint64_t* bar_drain = bar_qfull + 10;  // teardown after a give-up: every MMA issued so far has completed
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::kMiscOff);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kMiscOff + 4);
 
@@ -136,6 +133,7 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             mbar_init(&bar_odone[g], 1);
             mbar_init(&bar_phalf[g], kBM);
         }
+        mbar_init(bar_drain, 1);
         abort_flag[0] = 0;
         abort_flag[1] = (int)p.wait_limit_ns;
         fence_mbar_init();
@@ -170,7 +168,7 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         const bool leader = elect_one();
         uint32_t ring = 0, qcnt = 0;
         bool ok = true;
-        for (int idx = tile_begin; idx < tile_end && ok; ++idx) {
+        for (int idx = tile_begin; idx < tile_end && ok && !p.inject_stall; ++idx) {
             const int t = p.cta_tiles[idx];
             const int64_t q0 = (int64_t)(t / p.H) * (2 * kBM);
             const SlotRange r0 = slot_range(p.tok_start, p.T, q0);
@@ -206,6 +204,13 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 }
             }
         }
+        if (leader && (!ok || abort_flag[0])) {
+            // Give-up path: nothing new is issued; the copies already issued land before shared memory is released.
+            if (qcnt > 0) mbar_wait_drain(bar_qfull, (qcnt - 1) & 1, kFwdDrainNs);
+            for (uint32_t b = 1; b <= (uint32_t)L::kStages && b <= ring; ++b)
+                mbar_wait_drain(&bar_full[(ring - b) % L::kStages], ((ring - b) / L::kStages) & 1, kFwdDrainNs);
+        }
+        __syncwarp();
     } else if (warp == 9) {
         // ---------------- MMA issuer ----------------
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(LIBRA_FWD_REG_DEC));
@@ -316,7 +321,11 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 __syncwarp();
             }
         }
-        PROF_FLUSH(lane == 0, 8)
+        if (leader && (!ok || abort_flag[0])) {   // give-up path: the MMAs already issued finish before TMEM is freed
+            tc_commit(bar_drain);
+            mbar_wait_drain(bar_drain, 0, kFwdDrainNs);
+        }
+        __syncwarp();
     } else {
         // ---------------- softmax groups ----------------
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(LIBRA_FWD_REG_INC));
@@ -345,7 +354,7 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 float m_ref = -INFINITY, l_sum = 0.f;
                 for (int j = rg.lo; j <= rg.hi && ok; ++j) {
                     PROF(3)
-                    ok = mbar_wait(&bar_sfull[g], scnt & 1, abort_flag);
+                    ok = warp_wait(&bar_sfull[g], scnt & 1, abort_flag);
                     if (!ok) break;
                     TRACE(2)
                     PROF(0)
@@ -392,7 +401,7 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                     const bool first = (j == rg.lo);
                     if (!first && __any_sync(0xffffffffu, grow)) {
                         // PV(j-1) must have landed in O before it is rescaled
-                        ok = mbar_wait(&bar_odone[g], (ocnt - 1) & 1, abort_flag);
+                        ok = warp_wait(&bar_odone[g], (ocnt - 1) & 1, abort_flag);
                         if (!ok) break;
                         tc_fence_after();
 #pragma unroll
@@ -447,7 +456,7 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 if (!ok) break;
                 // epilogue: wait for the last PV, normalise, store
                 TRACE(24)
-                ok = mbar_wait(&bar_odone[g], (ocnt - 1) & 1, abort_flag);
+                ok = warp_wait(&bar_odone[g], (ocnt - 1) & 1, abort_flag);
                 if (!ok) break;
                 PROF(2)
                 TRACE(25)
@@ -600,6 +609,7 @@ extern "C" int libra_attn_pool_fwd(const void* q_dev, const void* k_dev, const v
     prm.status = plan->d_status + 1;
     prm.plan_status = plan->d_status;
     prm.wait_limit_ns = plan->wait_limit_ns;
+    prm.inject_stall = plan->inject_stall;
     prm.busy = d.d_busy;
     cudaStream_t s = (cudaStream_t)stream;
     cudaMemsetAsync(plan->d_status + 1, 0, sizeof(int), s);   // the word reports the most recent launch

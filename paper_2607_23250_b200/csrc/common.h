@@ -43,6 +43,7 @@ struct libra_plan {
     int* d_status = nullptr;         // [4] word 0: plan status; word 1: fwd; word 2: bwd
     libra::PlanDir dir[2];           // 0 = query-major, 1 = key-major
     uint32_t wait_limit_ns = 2000000000u;  // budget of one device-side wait (libra_plan_set_wait_limit_ns)
+    int inject_stall = 0;            // test aid: the producer role issues no loads (libra_plan_inject_stall)
     int timing = 0;                  // record events around the main kernels
     // [kernel][slot][begin, end]: a ring of the most recent launches of each kernel (LIBRA_KERNEL_* - 1)
     static constexpr int kTimedKernels = 4, kTimeRing = 64;

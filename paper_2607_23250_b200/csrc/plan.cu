@@ -473,6 +473,12 @@ extern "C" int libra_plan_set_wait_limit_ns(libra_plan_t* plan, uint64_t ns) {
     return LIBRA_OK;
 }
 
+extern "C" int libra_plan_inject_stall(libra_plan_t* plan, int enabled) {
+    if (!plan) return LIBRA_ERR_INVALID_ARG;
+    plan->inject_stall = enabled ? 1 : 0;
+    return LIBRA_OK;
+}
+
 static int kernel_time(const libra_plan_t* plan, int a, int64_t launch, float* ms) {
     cudaEvent_t e0 = plan->ev[a][launch % libra_plan::kTimeRing][0], e1 = plan->ev[a][launch % libra_plan::kTimeRing][1];
     if (cudaEventSynchronize(e1) != cudaSuccess) return LIBRA_ERR_CUDA;

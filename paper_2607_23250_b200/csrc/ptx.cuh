@@ -58,9 +58,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* ctl) {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = globaltimer_ns();
+    const uint32_t mask = (uint32_t)ctl[1] < 1000000u ? 0u : 0x3ffu;   // budgets under a millisecond: look every poll
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
-        if ((++spins & 0x3ff) == 0) {
+        if ((++spins & mask) == 0) {
             if (ctl[0]) return false;
             if (globaltimer_ns() - t0 > (uint64_t)(uint32_t)ctl[1]) {
                 ctl[0] = 1;
@@ -69,6 +70,12 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
         }
     }
     return true;
+}
+// The same wait for a role that runs on whole warps: every lane polls the barrier itself and the warp agrees
+// on the outcome, so that all 32 lanes either go on to the warp-wide tensor-memory instructions that follow or
+// leave together (a lane that gave up while its neighbours saw the phase complete would strand them there).
+__device__ __forceinline__ bool warp_wait(uint64_t* bar, uint32_t parity, volatile int* ctl) {
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, ctl));
 }
 // The same wait for the teardown of a CTA that has given up: it ignores the abort flag (which is
 // set by then) and has its own budget, so that copies and MMAs already in flight can land before

@@ -80,3 +80,62 @@ def test_plan_of_another_device_or_shape_is_refused():
         lb.libra_attn_pool_fwd(q, k, k, plan)
     assert err.value.code == lb.ERR_PLAN_MISMATCH
     plan.destroy()
+
+
+def test_bounded_wait_gives_up_and_reports_timeout():
+    """The wait routine of the kernels, alone: a barrier nothing arrives on, nothing in flight.  It must give
+    up after its budget, report TIMEOUT, and leave the GPU usable."""
+    from paper_2607_23250_b200 import binding as lb
+    for limit in (1_000, 2_000_000, 20_000_000):                  # 1 us, 2 ms, 20 ms
+        st, waited = lb.libra_selftest_wait_timeout(limit)
+        assert st == lb.ERR_TIMEOUT
+        assert waited >= limit and waited < limit + 50_000_000    # not before the budget, not long after it
+    x = torch.arange(8, device="cuda").sum().item()                # the context still works
+    assert x == 28
+
+
+def test_attention_kernels_give_up_cleanly_when_their_producer_stalls():
+    """The failure is made on a healthy GPU by a flag that nothing sets: with the plan's stall injection on, the
+    producer role issues no loads, so every consumer's wait runs out of its (shortened) budget.  Every CTA stops,
+    frees its tensor memory and returns; the launch reports TIMEOUT.  With the injection off and the default
+    budget restored the same plan gives correct results."""
+    import oracle
+    from paper_2607_23250_b200 import binding as lb
+    lengths = [300, 200, 524]
+    hq, hkv, d = 4, 2, 128
+    cu_np = pools.cu_seqlens(lengths)
+    T = int(cu_np[-1])
+    t = pools.make_tensors(T, hq, hkv, d, seed=3)
+    q, k, v, dout = (t[n].cuda() for n in ("q", "k", "v", "dout"))
+    cu = torch.from_numpy(cu_np).cuda()
+    plan = lb.libra_plan_tiles(cu, hq, 256, tile_kv=128, n_heads_kv=hkv)
+    assert plan.status() == 0
+    good_out, good_lse = lb.libra_attn_pool_fwd(q, k, v, plan)
+    plan.busy_times(lb.KERNEL_FWD)
+    plan.set_wait_limit_ns(200_000)                                # 0.2 ms
+    plan.inject_stall(True)
+    lb.libra_attn_pool_fwd(q, k, v, plan)
+    with pytest.raises(lb.LibraError) as err:
+        plan.busy_times(lb.KERNEL_FWD)
+    assert err.value.code == lb.ERR_TIMEOUT
+    lb.libra_attn_pool_bwd(q, k, v, good_out, good_lse, dout, plan)
+    with pytest.raises(lb.LibraError) as err:
+        plan.busy_times(lb.KERNEL_BWD_DKDV)
+    assert err.value.code == lb.ERR_TIMEOUT
+    with pytest.raises(lb.LibraError) as err:
+        plan.busy_times(lb.KERNEL_BWD_DQ)
+    assert err.value.code == lb.ERR_TIMEOUT
+    plan.inject_stall(False)
+    plan.set_wait_limit_ns(0)                                      # back to the default budget
+    out, lse = lb.libra_attn_pool_fwd(q, k, v, plan)
+    dq, dk, dv = lb.libra_attn_pool_bwd(q, k, v, out, lse, dout, plan)
+    torch.cuda.synchronize()
+    for kern in (lb.KERNEL_FWD, lb.KERNEL_BWD_DKDV, lb.KERNEL_BWD_DQ):
+        plan.busy_times(kern)                                      # status words report the most recent launches: OK
+    assert torch.equal(out, good_out) and torch.equal(lse, good_lse)
+    f = {n: t[n].float().numpy() for n in t}
+    o_ref, l_ref = oracle.attn_fwd(f["q"], f["k"], f["v"], cu_np)
+    ref = oracle.attn_bwd(f["q"], f["k"], f["v"], o_ref, l_ref, f["dout"], cu_np)
+    for g, r in zip((dq, dk, dv), ref):
+        assert np.abs(g.float().cpu().numpy() - r).max() <= 5e-2 * np.abs(r).max()
+    plan.destroy()
