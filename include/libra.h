@@ -226,8 +226,9 @@ int libra_vrsp_place(const int64_t* work_dev, int n_sequences, int pool_size, in
 /* ---- Tiled Attention Pooling across workers (Section 4.3: Eq. 5-8, Algorithm 2, exchange plan) ----
  * Plans one sequence pool: P packed sequences, each held by its own group of CP workers, W = P * CP
  * workers in all.  Everything runs in device kernels on `stream`; the paper runs it on CPU cores.
- * This is the planning half only: the transfers it describes and the head-chunk pipeline that
- * overlaps them with attention need more than one GPU and are not part of this library.
+ * libra_tap_plan places the tiles and sums the exchange volumes; libra_tap_schedule lists the transfers.
+ * Executing them (peer copies into local memory, then the attention kernels per head chunk) is host code
+ * above this library.
  *
  * Layout (a reading; the paper does not fix how a sequence is split over its CP group): sequence s
  * is tokens [seq_offsets[s], seq_offsets[s+1]) of the pool's sample list (a sequence boundary is
@@ -268,6 +269,29 @@ int libra_tap_plan(const int32_t* cu_seqlens_dev, int n_samples, const int32_t* 
                    int n_sequences, const libra_tap_opts* opts, int32_t* sigma_dev, int64_t* loads_dev,
                    int64_t* fwd_bytes_dev, int64_t* bwd_bytes_dev, int64_t* comm_total_dev,
                    int* status_dev, void* stream);
+
+/* Exchange schedule of an assignment (Section 4.3.3; the head pieces of Section 4.4 follow from it).
+ * Turns sigma (as written by libra_tap_plan, or any assignment of the pool's tiles to its workers) into
+ * transfer records of six int32 each, (kind, src, dst, tok0, ntok, shard), in device memory:
+ *   kind 0 : a tile placed away from its Q-home.  Forward: the Q rows [tok0, tok0 + ntok) of head shard `shard`
+ *            go src -> dst and the output rows come back dst -> src.  Backward: dO goes src -> dst, dQ comes
+ *            back dst -> src.  (The rows are taken to live at the Q-home, the worker holding the block's first
+ *            token; that is the case whenever the run length ceil(L / CP) is a multiple of B.)
+ *   kind 1 : a KV group (sample, shard) some tile placed at dst refers to, not wholly resident there: one record
+ *            per token run of the sample held by another worker.  Forward: K and V of the run go src -> dst,
+ *            once per destination however many tiles use the group.  Backward: the dK / dV partial sums of the
+ *            run go dst -> src and are added there.
+ * Order: kind 0 records by tile id, then kind 1 records by (dst, sample, shard, src).
+ * The Pipeliner moves every record in M equal head pieces (M divides hq / n_shards): chunk m carries the m-th
+ * piece of the shard's query heads of every kind 0 record and, of every kind 1 record, the kv heads that this
+ * piece is the first to read (query head q reads kv head q / (hq / hkv)); so one list serves all chunks and
+ * both passes.
+ * records_dev: int32[capacity * 6]; *n_records_dev receives the number of records the assignment implies
+ * (records beyond `capacity` are not written).  Scratch comes from the stream-ordered allocator.
+ * Errors: INVALID_ARG, UNSUPPORTED (W > 1024, n_samples * n_shards * W >= 2^31), CUDA. */
+int libra_tap_schedule(const int32_t* cu_seqlens_dev, int n_samples, const int32_t* seq_offsets_host,
+                       int n_sequences, const libra_tap_opts* opts, const int32_t* sigma_dev,
+                       int32_t* records_dev, int64_t capacity, int64_t* n_records_dev, void* stream);
 
 /* ---- instrumentation -------------------------------------------------------------------
  * Per-CTA busy time of the most recent launch of kernel `which` (LIBRA_KERNEL_*) that used this

@@ -29,7 +29,7 @@ ERR_SCRATCH_TOO_SMALL = -9
 EXPORTS = ["libra_plan_tiles", "libra_plan_info", "libra_plan_status", "libra_plan_export",
            "libra_plan_destroy", "libra_attn_pool_fwd", "libra_attn_pool_bwd_workspace_bytes",
            "libra_attn_pool_bwd", "libra_attn_pool_bwd_noalloc_max_bytes", "libra_attn_pool_bwd_noalloc",
-           "libra_busy_times", "libra_plan_set_wait_limit_ns", "libra_plan_inject_stall", "libra_plan_set_timing", "libra_kernel_time_ms", "libra_kernel_times_ms", "libra_selftest_wait_timeout", "libra_launch_count",
+           "libra_tap_schedule", "libra_busy_times", "libra_plan_set_wait_limit_ns", "libra_plan_inject_stall", "libra_plan_set_timing", "libra_kernel_time_ms", "libra_kernel_times_ms", "libra_selftest_wait_timeout", "libra_launch_count",
            "libra_strerror"]
 
 
@@ -283,3 +283,28 @@ def libra_tap_plan(cu_seqlens: torch.Tensor, seq_offsets, cp: int, block: int, n
                                _ptr(out["bwd_bytes"]), _ptr(out["comm_total"]), _ptr(out["status"]), _stream(stream)),
            "libra_tap_plan")
     return out
+
+
+def libra_tap_schedule(cu_seqlens: torch.Tensor, seq_offsets, sigma: torch.Tensor, cp: int, block: int, n_shards: int,
+                       hq: int, hkv: int, head_dim: int, capacity: int = 0, stream=None) -> torch.Tensor:
+    """Transfer records [n, 6] (kind, src, dst, tok0, ntok, shard) implied by assignment `sigma` (device int32).
+    Two calls when `capacity` is 0: the first only counts."""
+    assert cu_seqlens.is_cuda and cu_seqlens.dtype == torch.int32 and sigma.is_cuda and sigma.dtype == torch.int32
+    so = (ctypes.c_int32 * len(seq_offsets))(*[int(x) for x in seq_offsets])
+    P = len(seq_offsets) - 1
+    opts = TapOpts(cp, block, n_shards, hq, hkv, head_dim, 3, 100)
+    dev = cu_seqlens.device
+    n = torch.zeros(1, dtype=torch.int64, device=dev)
+
+    def call(cap):
+        rec = torch.empty((max(cap, 1), 6), dtype=torch.int32, device=dev)
+        _check(_lib.libra_tap_schedule(_ptr(cu_seqlens), ctypes.c_int(cu_seqlens.numel() - 1), so, ctypes.c_int(P),
+                                       ctypes.byref(opts), _ptr(sigma), _ptr(rec), ctypes.c_int64(cap), _ptr(n),
+                                       _stream(stream)), "libra_tap_schedule")
+        return rec
+
+    if capacity <= 0:
+        call(0)
+        capacity = int(n.item())
+    rec = call(capacity)
+    return rec[:min(capacity, int(n.item()))]

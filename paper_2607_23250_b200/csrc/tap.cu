@@ -249,6 +249,114 @@ __global__ void k_tap_exchange_kv(TapGeom g, const uint32_t* __restrict__ Cbits,
     }
 }
 
+
+// ---- exchange schedule (Section 4.3.3): the transfer records implied by an assignment ----------------------
+// Record = 6 x int32 (kind, src, dst, tok0, ntok, shard); kind 0: Q rows of a tile placed away from its Q-home
+// (output back the same way, dO / dQ in the backward pass), kind 1: the K / V rows of a selected KV group held by
+// another worker (dK / dV back the same way).  Order: kind 0 by tile id, then kind 1 by (dst, sample, shard, src).
+
+// The KV groups some tile placed at r refers to, as bit rows [W][words].
+__global__ void k_tap_mark(const int32_t* __restrict__ sigma, const int32_t* __restrict__ j_first,
+                           const int32_t* __restrict__ j_last, int64_t NT, int H, int W, int words,
+                           uint32_t* __restrict__ marks) {
+    const int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (t >= NT) return;
+    const int r = sigma[t], h = (int)(t % H);
+    if (r < 0 || r >= W) return;
+    for (int j = j_first[t / H]; j <= j_last[t / H]; ++j) {
+        const int g = j * H + h;
+        atomicOr(&marks[(size_t)r * words + (g >> 5)], 1u << (g & 31));
+    }
+}
+
+// Records slot x of the enumeration produces: slot x < NT is tile x (0 or 1), slot NT + r * NG + g is group g
+// at destination r (one per token run of the sample on another worker).
+__device__ __forceinline__ int tap_slot_count(const TapGeom& g, int64_t x, int64_t NT, int64_t NG, int W,
+                                              const int32_t* sigma, const int32_t* q_home, const uint32_t* marks,
+                                              int words, const int32_t* res_smp) {
+    if (x < NT) {
+        const int r = sigma[x];
+        return (r >= 0 && r < W && r != q_home[x / g.H]) ? 1 : 0;
+    }
+    const int64_t y = x - NT;
+    const int r = (int)(y / NG);
+    const int grp = (int)(y % NG), j = grp / g.H;
+    if (!((marks[(size_t)r * words + (grp >> 5)] >> (grp & 31)) & 1u) || res_smp[j] == r) return 0;
+    const int64_t a = g.cu[j], e = g.cu[j + 1];
+    if (e <= a) return 0;
+    const int s = tap_seq_of_token(g, a);
+    int c = 0;
+    for (int w = tap_owner(g, s, a); w <= tap_owner(g, s, e - 1); ++w) c += (w != r);
+    return c;
+}
+
+// One block: exclusive prefix sum of the slot counts (each thread takes a contiguous piece), total to n_out.
+__global__ void __launch_bounds__(1024) k_tap_sched_scan(TapGeom g, int64_t NT, int64_t NG, int W,
+                                                         const int32_t* __restrict__ sigma,
+                                                         const int32_t* __restrict__ q_home,
+                                                         const uint32_t* __restrict__ marks, int words,
+                                                         const int32_t* __restrict__ res_smp,
+                                                         int64_t* __restrict__ offs /*[slots]*/, int64_t* n_out) {
+    __shared__ int64_t part[1024];
+    const int64_t slots = NT + NG * W;
+    const int64_t per = (slots + blockDim.x - 1) / blockDim.x;
+    const int64_t x0 = threadIdx.x * per, x1 = x0 + per < slots ? x0 + per : slots;
+    int64_t sum = 0;
+    for (int64_t x = x0; x < x1; ++x) sum += tap_slot_count(g, x, NT, NG, W, sigma, q_home, marks, words, res_smp);
+    part[threadIdx.x] = sum;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int64_t run = 0;
+        for (int i = 0; i < (int)blockDim.x; ++i) { const int64_t v = part[i]; part[i] = run; run += v; }
+        *n_out = run;
+    }
+    __syncthreads();
+    int64_t run = part[threadIdx.x];
+    for (int64_t x = x0; x < x1; ++x) {
+        offs[x] = run;
+        run += tap_slot_count(g, x, NT, NG, W, sigma, q_home, marks, words, res_smp);
+    }
+}
+
+__global__ void k_tap_sched_fill(TapGeom g, int64_t NT, int64_t NG, int W, const int32_t* __restrict__ sigma,
+                                 const int32_t* __restrict__ q_home, const uint32_t* __restrict__ marks, int words,
+                                 const int32_t* __restrict__ res_smp, const int64_t* __restrict__ offs,
+                                 int64_t capacity, int32_t* __restrict__ rec) {
+    const int64_t x = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (x >= NT + NG * W) return;
+    int64_t at = offs[x];
+    if (x < NT) {
+        const int r = sigma[x];
+        const int64_t b = x / g.H;
+        if (!(r >= 0 && r < W && r != q_home[b]) || at >= capacity) return;
+        int s = 0;
+        while (s + 1 < g.P && g.blk_off[s + 1] <= b) ++s;
+        const int64_t q0 = g.seq_off[s] + (b - g.blk_off[s]) * g.B;
+        const int64_t q1 = q0 + g.B < g.seq_off[s + 1] ? q0 + g.B : g.seq_off[s + 1];
+        int32_t* o = rec + at * 6;
+        o[0] = 0; o[1] = q_home[b]; o[2] = r; o[3] = (int32_t)q0; o[4] = (int32_t)(q1 - q0); o[5] = (int32_t)(x % g.H);
+        return;
+    }
+    const int64_t y = x - NT;
+    const int r = (int)(y / NG);
+    const int grp = (int)(y % NG), j = grp / g.H;
+    if (!((marks[(size_t)r * words + (grp >> 5)] >> (grp & 31)) & 1u) || res_smp[j] == r) return;
+    const int64_t a = g.cu[j], e = g.cu[j + 1];
+    if (e <= a) return;
+    const int s = tap_seq_of_token(g, a);
+    const int64_t len = g.seq_off[s + 1] - g.seq_off[s];
+    const int64_t run = (len + g.CP - 1) / g.CP;
+    for (int w = tap_owner(g, s, a); w <= tap_owner(g, s, e - 1); ++w) {
+        if (w == r) continue;
+        if (at >= capacity) return;
+        const int64_t w0 = g.seq_off[s] + (int64_t)(w - s * g.CP) * run, w1 = w0 + run;
+        const int64_t lo = a > w0 ? a : w0, hi = e < w1 ? e : w1;
+        int32_t* o = rec + at * 6;
+        o[0] = 1; o[1] = w; o[2] = r; o[3] = (int32_t)lo; o[4] = (int32_t)(hi - lo); o[5] = grp % g.H;
+        ++at;
+    }
+}
+
 }  // namespace libra
 
 using namespace libra;
@@ -346,6 +454,72 @@ extern "C" int libra_tap_plan(const int32_t* cu_seqlens_dev, int n_samples, cons
                                                                           (unsigned long long*)fwd_bytes_dev,
                                                                           (unsigned long long*)bwd_bytes_dev);
         count_launch(6);
+        if (cudaGetLastError() != cudaSuccess) rc = LIBRA_ERR_CUDA;
+    }
+    cudaFreeAsync(scratch, s);
+    return rc;
+}
+
+extern "C" int libra_tap_schedule(const int32_t* cu_seqlens_dev, int n_samples, const int32_t* seq_offsets_host,
+                                  int n_sequences, const libra_tap_opts* o, const int32_t* sigma_dev,
+                                  int32_t* records_dev, int64_t capacity, int64_t* n_records_dev, void* stream) {
+    if (!cu_seqlens_dev || !seq_offsets_host || !o || !sigma_dev || !records_dev || !n_records_dev || capacity < 0)
+        return LIBRA_ERR_INVALID_ARG;
+    if (n_samples <= 0 || n_sequences <= 0 || o->cp <= 0 || o->block <= 0 || o->n_shards <= 0 || o->hq <= 0 ||
+        o->hkv <= 0 || o->head_dim <= 0 || o->hq % o->n_shards != 0)
+        return LIBRA_ERR_INVALID_ARG;
+    const int P = n_sequences, W = P * o->cp, H = o->n_shards;
+    if (W > 1024 || P > 4096) return LIBRA_ERR_UNSUPPORTED;
+    const int64_t NT = libra_tap_num_tiles(seq_offsets_host, P, o->block, H);
+    if (NT <= 0) return LIBRA_ERR_INVALID_ARG;
+    const int64_t NB = NT / H, NG = (int64_t)n_samples * H;
+    if (NT >= INT32_MAX || NG * W >= INT32_MAX) return LIBRA_ERR_UNSUPPORTED;
+    cudaStream_t s = (cudaStream_t)stream;
+    const int words = (int)((NG + 31) / 32);
+    int32_t* h_tab = new (std::nothrow) int32_t[2 * (P + 1)];
+    if (!h_tab) return LIBRA_ERR_CUDA;
+    int64_t nb = 0;
+    for (int q = 0; q <= P; ++q) {
+        h_tab[q] = seq_offsets_host[q];
+        h_tab[P + 1 + q] = (int32_t)nb;
+        if (q < P) nb += ((int64_t)seq_offsets_host[q + 1] - seq_offsets_host[q] + o->block - 1) / o->block;
+    }
+    uint8_t* scratch = nullptr;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { const size_t at = off; off += (bytes + 255) & ~size_t(255); return at; };
+    const size_t o_tab = take(sizeof(int32_t) * 2 * (P + 1));
+    const size_t o_f = take(sizeof(int64_t) * NB), o_vqo = take(sizeof(int64_t) * NB);
+    const size_t o_q = take(sizeof(int32_t) * NB), o_j0 = take(sizeof(int32_t) * NB), o_j1 = take(sizeof(int32_t) * NB);
+    const size_t o_vs = take(sizeof(int64_t) * n_samples), o_rs = take(sizeof(int32_t) * n_samples);
+    const size_t o_m = take(sizeof(uint32_t) * (size_t)words * W);
+    const size_t o_offs = take(sizeof(int64_t) * (size_t)(NT + NG * W));
+    if (cudaMallocAsync((void**)&scratch, off, s) != cudaSuccess) { delete[] h_tab; return LIBRA_ERR_CUDA; }
+    int rc = LIBRA_OK;
+    if (cudaMemcpyAsync(scratch + o_tab, h_tab, sizeof(int32_t) * 2 * (P + 1), cudaMemcpyHostToDevice, s) != cudaSuccess)
+        rc = LIBRA_ERR_CUDA;
+    delete[] h_tab;
+    TapGeom g;
+    g.cu = cu_seqlens_dev;
+    g.seq_off = (const int32_t*)(scratch + o_tab);
+    g.blk_off = g.seq_off + (P + 1);
+    g.n = n_samples; g.P = P; g.CP = o->cp; g.B = o->block; g.H = H; g.hq = o->hq; g.hkv = o->hkv; g.d = o->head_dim;
+    int32_t* q_home = (int32_t*)(scratch + o_q);
+    int32_t* j0 = (int32_t*)(scratch + o_j0);
+    int32_t* j1 = (int32_t*)(scratch + o_j1);
+    int32_t* res_smp = (int32_t*)(scratch + o_rs);
+    uint32_t* marks = (uint32_t*)(scratch + o_m);
+    int64_t* offs = (int64_t*)(scratch + o_offs);
+    if (rc == LIBRA_OK) {
+        cudaMemsetAsync(marks, 0, sizeof(uint32_t) * (size_t)words * W, s);
+        k_tap_blocks<<<(unsigned)((NB + 127) / 128), 128, 0, s>>>(g, NB, (int64_t*)(scratch + o_f), q_home,
+                                                                  (int64_t*)(scratch + o_vqo), j0, j1);
+        k_tap_samples<<<(n_samples + 127) / 128, 128, 0, s>>>(g, (int64_t*)(scratch + o_vs), res_smp);
+        k_tap_mark<<<(unsigned)((NT + 255) / 256), 256, 0, s>>>(sigma_dev, j0, j1, NT, H, W, words, marks);
+        k_tap_sched_scan<<<1, 1024, 0, s>>>(g, NT, NG, W, sigma_dev, q_home, marks, words, res_smp, offs, n_records_dev);
+        const int64_t slots = NT + NG * W;
+        k_tap_sched_fill<<<(unsigned)((slots + 255) / 256), 256, 0, s>>>(g, NT, NG, W, sigma_dev, q_home, marks, words,
+                                                                        res_smp, offs, capacity, records_dev);
+        count_launch(5);
         if (cudaGetLastError() != cudaSuccess) rc = LIBRA_ERR_CUDA;
     }
     cudaFreeAsync(scratch, s);

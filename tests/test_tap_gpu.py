@@ -4,6 +4,7 @@ import pytest
 import torch
 
 import oracle
+from oracle import schedule as osched
 from paper_2607_23250_b200 import pools
 
 pytestmark = pytest.mark.gpu
@@ -24,6 +25,13 @@ def _compare(cu, seq_off, cp, B, H, hq, hkv, d, tau=(3, 100)):
     assert int(got["comm_total"].item()) == want["comm_total"]
     assert np.array_equal(got["fwd_bytes"].cpu().numpy(), fwd)
     assert np.array_equal(got["bwd_bytes"].cpu().numpy(), bwd)
+    # the transfer records of the same assignment, and of one that scatters the tiles, equal the oracle's list
+    if len(want["sigma"]) <= 4096:
+        cu_dev = torch.from_numpy(np.asarray(cu, np.int32)).cuda()
+        scattered = np.array([(5 * t + 3) % W for t in range(len(want["sigma"]))], np.int32)
+        for sigma in (want["sigma"], scattered):
+            rec = lb.libra_tap_schedule(cu_dev, seq_off, torch.from_numpy(sigma).cuda(), cp, B, H, hq, hkv, d)
+            assert np.array_equal(rec.cpu().numpy().reshape(-1, 6), osched.schedule(cu, seq_off, cp, B, H, sigma))
     return want, fwd
 
 
