@@ -58,6 +58,7 @@ extern "C" {
 
 #define LIBRA_DIR_Q   1   /* query-major tiles (forward)  */
 #define LIBRA_DIR_KV  2   /* key-major tiles   (backward) */
+#define LIBRA_DIR_PAIR 4  /* pair tiles: key block x query chunk x kv head (the fused backward); only on request */
 
 /* kernels, for libra_busy_times / libra_kernel_time_ms */
 #define LIBRA_KERNEL_FWD       1   /* forward kernel (walks the query-major lists)            */
@@ -79,6 +80,8 @@ typedef struct {
     int     unit_cost_q;   /* LIBRA_WEIGHT_BLOCKS: added per row chunk of a query-major tile, in
                               eighths of a block (>= 0)                                             */
     int     unit_cost_kv;  /* same per key chunk of a key-major tile                                */
+    int     pair_chunk;    /* LIBRA_DIR_PAIR: tokens per query chunk, a multiple of the key block; 0 = 2048
+                              (doubled by the planner until there are at most 65536 pair-blocks)       */
 } libra_plan_opts;
 
 typedef struct {
@@ -137,6 +140,19 @@ int libra_plan_status(const libra_plan_t* plan);
 int libra_plan_export(const libra_plan_t* plan, int direction, int64_t* weight_host,
                       int32_t* order_host, int32_t* cta_of_tile_host, int32_t* cta_offsets_host,
                       int32_t* cta_tiles_host, int64_t* loads_host);
+
+/* Pair tiles (directions & LIBRA_DIR_PAIR; the units of the fused backward).  The paper's tile is a query block
+ * with all of its keys (Section 4.3.1); a pair tile cuts that rectangle along the key axis as well: key block j
+ * (tile_kv keys of kv head h) against query chunk c (pair_chunk tokens).  Key block j is attended by the
+ * queries from its first key to the last token of the sample that holds its last key, and has one pair-block
+ * for every query chunk this range touches, chunks ascending; pair-blocks are numbered key block by key block,
+ * tile id = pair-block * n_heads_kv + h.  The weight is still Eq. 6's count: the (query, key) pairs with the
+ * key in the block, the query in the chunk, both in one sample and the query not before the key.  Ordering,
+ * placement and lists follow Algorithm 2 as for the other directions, and libra_plan_info / libra_plan_export
+ * take LIBRA_DIR_PAIR (n_blocks = pair-blocks).  libra_plan_export_pairs copies the key block and the query
+ * chunk of every pair-block (int32[n_blocks] each, HOST, nullable) and the chunk size in tokens. */
+int libra_plan_export_pairs(const libra_plan_t* plan, int32_t* key_block_host, int32_t* query_chunk_host,
+                            int* chunk_tokens_host);
 
 /* Frees the plan's device and host memory (synchronises the device first). NULL is OK. */
 int libra_plan_destroy(libra_plan_t* plan);

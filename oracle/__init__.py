@@ -168,6 +168,27 @@ def plan(cu, n_heads, tile, n_workers, direction=0, weight_model=0, cost_block=1
     return res
 
 
+def plan_pairs(cu, n_heads, tile, chunk, n_workers):
+    """Plan over pair tiles (key block x query chunk x head) -> oracle_plan's dict + key_block, query_chunk per pair-block."""
+    cu = _arr(cu, np.int32)
+    lib = _load()
+    lib.oracle_plan_pairs_num_blocks.restype = ctypes.c_int64
+    n = len(cu) - 1
+    nu = int(lib.oracle_plan_pairs_num_blocks(_p(cu), ctypes.c_int(n), ctypes.c_int(tile), ctypes.c_int(chunk)))
+    if nu < 0:
+        raise RuntimeError("oracle_plan_pairs: bad arguments")
+    nt = nu * n_heads
+    res = dict(weight=np.empty(nt, np.int64), order=np.empty(nt, np.int32), cta_of_tile=np.empty(nt, np.int32),
+               cta_offsets=np.empty(n_workers + 1, np.int32), cta_tiles=np.empty(nt, np.int32),
+               loads=np.empty(n_workers, np.int64), key_block=np.empty(nu, np.int32), query_chunk=np.empty(nu, np.int32))
+    _check(lib.oracle_plan_pairs(_p(cu), ctypes.c_int(n), ctypes.c_int(n_heads), ctypes.c_int(tile), ctypes.c_int(chunk),
+                                 ctypes.c_int(n_workers), _p(res["weight"]), _p(res["order"]), _p(res["cta_of_tile"]),
+                                 _p(res["cta_offsets"]), _p(res["cta_tiles"]), _p(res["loads"]), _p(res["key_block"]),
+                                 _p(res["query_chunk"])), "oracle_plan_pairs")
+    res["n_blocks"] = nu
+    return res
+
+
 def vrsp_work(sample_offsets, seq_first_sample):
     """F_i = sum of squared raw-sample lengths of packed sequence i (Eq. 4)."""
     so = _arr(sample_offsets, np.int32)

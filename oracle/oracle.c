@@ -143,6 +143,60 @@ int oracle_plan(const int32_t* cu, int n, int H, int tile, int W, int direction,
 }
 
 /* ------------------------------------------------------------------------------------
+ * Plan over pair tiles (the fused backward's work units; the paper's tiles are query blocks with all their
+ * keys, Section 4.3.1 - here a tile is additionally cut along the key axis, its weight is still the causal
+ * pairs it covers, Eq. 6, and steps 3-5 are those of Algorithm 2 as in oracle_plan).
+ *
+ * Keys are cut into blocks of `tile` tokens at global positions, queries into chunks of `chunk` tokens
+ * (a multiple of `tile`).  Key block j is attended by queries from its own first key up to the last token of
+ * the sample that holds its last key; it gets one pair-block for every query chunk that range touches:
+ * chunks (j * tile) / chunk .. (end - 1) / chunk, in that order.  Pair-blocks are numbered key block by key
+ * block; tile id = pair-block * H + h.  Weight = the (query, key) pairs with the key in the block, the query
+ * in the chunk, both in the same sample, query position >= key position: counted pair by pair.
+ * Outputs as oracle_plan, plus the key block and the query chunk of every pair-block.
+ * ------------------------------------------------------------------------------------ */
+int64_t oracle_plan_pairs_num_blocks(const int32_t* cu, int n, int tile, int chunk) {
+    if (!cu || n <= 0 || tile <= 0 || chunk <= 0 || chunk % tile) return -1;
+    const int64_t T = cu[n];
+    int64_t nu = 0;
+    for (int64_t k0 = 0; k0 < T; k0 += tile) {
+        const int64_t last_key = (k0 + tile < T ? k0 + tile : T) - 1;
+        int j = 0;
+        while (!(cu[j] <= last_key && last_key < cu[j + 1])) ++j;
+        nu += (cu[j + 1] - 1) / chunk - k0 / chunk + 1;
+    }
+    return nu;
+}
+
+int oracle_plan_pairs(const int32_t* cu, int n, int H, int tile, int chunk, int W, int64_t* weight /*[NU*H]*/,
+                      int32_t* order, int32_t* cta_of_tile, int32_t* cta_offsets, int32_t* cta_tiles, int64_t* loads,
+                      int32_t* key_block /*[NU]*/, int32_t* query_chunk /*[NU]*/) {
+    if (!cu || n <= 0 || H <= 0 || tile <= 0 || chunk <= 0 || chunk % tile || W <= 0) return -1;
+    if (cu[0] != 0) return -1;
+    for (int j = 0; j < n; ++j) if (cu[j + 1] < cu[j]) return -1;
+    const int64_t T = cu[n];
+    int64_t u = 0;
+    for (int64_t k0 = 0; k0 < T; k0 += tile) {
+        const int64_t k1 = k0 + tile < T ? k0 + tile : T;
+        int jl = 0;
+        while (!(cu[jl] <= k1 - 1 && k1 - 1 < cu[jl + 1])) ++jl;          /* sample of the block's last key */
+        for (int64_t c = k0 / chunk; c <= (cu[jl + 1] - 1) / chunk; ++c, ++u) {
+            int64_t w = 0;
+            for (int64_t k = k0; k < k1; ++k) {
+                int j = 0;
+                while (!(cu[j] <= k && k < cu[j + 1])) ++j;               /* sample of key k */
+                for (int64_t q = c * chunk; q < (c + 1) * chunk && q < cu[j + 1]; ++q)
+                    if (q >= k) ++w;                                      /* same sample (q < its end), causal */
+            }
+            for (int h = 0; h < H; ++h) weight[u * H + h] = w;
+            key_block[u] = (int32_t)(k0 / tile);
+            query_chunk[u] = (int32_t)c;
+        }
+    }
+    return place_tiles(u * H, W, weight, order, cta_of_tile, cta_offsets, cta_tiles, loads);
+}
+
+/* ------------------------------------------------------------------------------------
  * Plan with the block-count weight (not in the paper; Section 3.2 only remarks that equal
  * FLOPs need not mean equal time).  A kernel spends the same time on a g x g block of the
  * score matrix whether one pair of it is visible or all, so this weight counts blocks.

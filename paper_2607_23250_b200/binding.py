@@ -19,7 +19,7 @@ if not os.path.exists(_SO):
     raise ImportError(f"{_SO} is missing: run `python -m paper_2607_23250_b200.build` (needs nvcc)")
 _lib = ctypes.CDLL(_SO)
 
-LIBRA_DIR_Q, LIBRA_DIR_KV = 1, 2
+LIBRA_DIR_Q, LIBRA_DIR_KV, LIBRA_DIR_PAIR = 1, 2, 4
 LIBRA_WEIGHT_PAIRS, LIBRA_WEIGHT_BLOCKS = 0, 1
 KERNEL_FWD, KERNEL_BWD_DKDV, KERNEL_BWD_DQ, KERNEL_BWD_PREP = 1, 2, 3, 4
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_PLAN_MISMATCH, ERR_CUDA = -1, -2, -3, -4
@@ -27,7 +27,7 @@ ERR_OVERFLOW, ERR_TIMEOUT, ERR_BAD_SEQLENS, ERR_NO_DEVICE = -5, -6, -7, -8
 ERR_SCRATCH_TOO_SMALL = -9
 
 EXPORTS = ["libra_plan_tiles", "libra_plan_info", "libra_plan_status", "libra_plan_export",
-           "libra_plan_destroy", "libra_attn_pool_fwd", "libra_attn_pool_bwd_workspace_bytes",
+           "libra_plan_export_pairs", "libra_plan_destroy", "libra_attn_pool_fwd", "libra_attn_pool_bwd_workspace_bytes",
            "libra_attn_pool_bwd", "libra_attn_pool_bwd_noalloc_max_bytes", "libra_attn_pool_bwd_noalloc",
            "libra_tap_schedule", "libra_busy_times", "libra_plan_set_wait_limit_ns", "libra_plan_inject_stall", "libra_plan_set_timing", "libra_kernel_time_ms", "libra_kernel_times_ms", "libra_selftest_wait_timeout", "libra_launch_count",
            "libra_strerror"]
@@ -36,7 +36,8 @@ EXPORTS = ["libra_plan_tiles", "libra_plan_info", "libra_plan_status", "libra_pl
 class PlanOpts(ctypes.Structure):
     _fields_ = [("n_workers", ctypes.c_int), ("directions", ctypes.c_int), ("tile_kv", ctypes.c_int),
                 ("n_heads_kv", ctypes.c_int), ("total_tokens", ctypes.c_int64), ("weight_model", ctypes.c_int),
-                ("cost_block", ctypes.c_int), ("unit_cost_q", ctypes.c_int), ("unit_cost_kv", ctypes.c_int)]
+                ("cost_block", ctypes.c_int), ("unit_cost_q", ctypes.c_int), ("unit_cost_kv", ctypes.c_int),
+                ("pair_chunk", ctypes.c_int)]
 
 
 class Dims(ctypes.Structure):
@@ -116,6 +117,13 @@ class Plan:
         res["n_blocks"] = i["n_blocks"]
         return res
 
+    def export_pairs(self):
+        """(key_block, query_chunk) of every pair-block and the chunk size in tokens (LIBRA_DIR_PAIR plans)."""
+        nb = self.info(LIBRA_DIR_PAIR)["n_blocks"]
+        kb, qc, chunk = np.empty(nb, np.int32), np.empty(nb, np.int32), ctypes.c_int()
+        _check(_lib.libra_plan_export_pairs(self._h, _np(kb), _np(qc), ctypes.byref(chunk)), "libra_plan_export_pairs")
+        return kb, qc, chunk.value
+
     def busy_times(self, which=KERNEL_FWD):
         w = self.info(LIBRA_DIR_KV if which == KERNEL_BWD_DKDV else LIBRA_DIR_Q)["n_workers"]
         out = np.zeros(w, np.uint64)
@@ -159,10 +167,10 @@ class Plan:
 def libra_plan_tiles(cu_seqlens: torch.Tensor, n_heads: int, tile_q: int, n_workers: int = 0,
                      directions: int = 0, tile_kv: int = 0, n_heads_kv: int = 0, total_tokens: int = 0,
                      stream=None, weight_model: int = 0, cost_block: int = 0, unit_cost_q: int = 0,
-                     unit_cost_kv: int = 0) -> Plan:
+                     unit_cost_kv: int = 0, pair_chunk: int = 0) -> Plan:
     assert cu_seqlens.is_cuda and cu_seqlens.dtype == torch.int32 and cu_seqlens.is_contiguous()
     opts = PlanOpts(n_workers, directions, tile_kv, n_heads_kv, total_tokens, weight_model, cost_block,
-                    unit_cost_q, unit_cost_kv)
+                    unit_cost_q, unit_cost_kv, pair_chunk)
     h = _vp()
     _check(_lib.libra_plan_tiles(_ptr(cu_seqlens), ctypes.c_int(cu_seqlens.numel() - 1), ctypes.c_int(n_heads),
                                  ctypes.c_int(tile_q), ctypes.byref(opts), _stream(stream), ctypes.byref(h)),

@@ -28,6 +28,10 @@ struct PlanDir {
     int64_t* d_loads = nullptr;        // [W]
     uint64_t* d_busy = nullptr;        // [2*W] (start, end) global-timer stamps of the last run
     uint64_t* d_busy2 = nullptr;       // [2*W] same, for the second kernel that walks this direction (dQ)
+    // pair tiles only (key block x query chunk x head): the "blocks" above are pair-blocks
+    int chunk = 0;                     // tokens per query chunk
+    int32_t* d_u_blk = nullptr;        // [NB] key block of pair-block u
+    int32_t* d_u_chunk = nullptr;      // [NB] query chunk of pair-block u
 };
 
 }  // namespace libra
@@ -41,7 +45,7 @@ struct libra_plan {
     int32_t* d_tok_start = nullptr;  // [T] first token of the sample that holds token t
     int32_t* d_tok_end = nullptr;    // [T] one past the last token of that sample
     int* d_status = nullptr;         // [4] word 0: plan status; word 1: fwd; word 2: bwd
-    libra::PlanDir dir[2];           // 0 = query-major, 1 = key-major
+    libra::PlanDir dir[3];           // 0 = query-major, 1 = key-major, 2 = pair tiles (key block x query chunk)
     uint32_t wait_limit_ns = 2000000000u;  // budget of one device-side wait (libra_plan_set_wait_limit_ns)
     int inject_stall = 0;            // test aid: the producer role issues no loads (libra_plan_inject_stall)
     int timing = 0;                  // record events around the main kernels

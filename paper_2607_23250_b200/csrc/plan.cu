@@ -220,6 +220,83 @@ __global__ void k_exec_order(const int32_t* __restrict__ cta_offsets, const int3
     }
 }
 
+// ---- pair tiles: key block x query chunk x head (the fused backward's units) ---------------------------------
+// Key block j (`tile` keys) is attended by queries from its first key to the last token of the sample that holds
+// its last key: one pair-block per query chunk that range touches, chunks ascending, numbered key block by key block.
+__global__ void k_pair_count(const int32_t* __restrict__ tok_end, int64_t T, int tile, int chunk, int64_t NKB,
+                             int32_t* __restrict__ count) {
+    const int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (j >= NKB) return;
+    const int64_t k0 = j * tile;
+    const int64_t last_key = (k0 + tile < T ? k0 + tile : T) - 1;
+    count[j] = (int32_t)(((int64_t)tok_end[last_key] - 1) / chunk - k0 / chunk + 1);
+}
+// One block: exclusive prefix sum of count[0..n) into base, total into *total.
+__global__ void __launch_bounds__(1024) k_scan_i32(const int32_t* __restrict__ count, int64_t n, int64_t* __restrict__ base,
+                                                   int64_t* __restrict__ total) {
+    __shared__ int64_t part[1024];
+    const int64_t per = (n + blockDim.x - 1) / blockDim.x;
+    const int64_t x0 = threadIdx.x * per, x1 = x0 + per < n ? x0 + per : n;
+    int64_t sum = 0;
+    for (int64_t x = x0; x < x1; ++x) sum += count[x];
+    part[threadIdx.x] = sum;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int64_t run = 0;
+        for (int i = 0; i < (int)blockDim.x; ++i) { const int64_t v = part[i]; part[i] = run; run += v; }
+        *total = run;
+    }
+    __syncthreads();
+    int64_t run = part[threadIdx.x];
+    for (int64_t x = x0; x < x1; ++x) { base[x] = run; run += count[x]; }
+}
+// Weight of pair-block (j, c): the pairs with the key in block j, the query in chunk c, both in one sample and
+// query position >= key position = sum over the block's keys of the queries of the chunk inside [key, sample end).
+__global__ void k_pair_fill(const int32_t* __restrict__ tok_end, int64_t T, int tile, int chunk, int64_t NKB,
+                            const int64_t* __restrict__ base, int32_t* __restrict__ u_blk,
+                            int32_t* __restrict__ u_chunk, int64_t* __restrict__ weight_blk) {
+    const int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (j >= NKB) return;
+    const int64_t k0 = j * tile, k1 = k0 + tile < T ? k0 + tile : T;
+    const int64_t c_lo = k0 / chunk, c_hi = ((int64_t)tok_end[k1 - 1] - 1) / chunk;
+    for (int64_t c = c_lo; c <= c_hi; ++c) {
+        const int64_t q0 = c * chunk, q1 = q0 + chunk;
+        int64_t w = 0;
+        for (int64_t k = k0; k < k1; ++k) {
+            const int64_t lo = k > q0 ? k : q0, hi = (int64_t)tok_end[k] < q1 ? (int64_t)tok_end[k] : q1;
+            if (hi > lo) w += hi - lo;
+        }
+        const int64_t u = base[j] + (c - c_lo);
+        u_blk[u] = (int32_t)j;
+        u_chunk[u] = (int32_t)c;
+        weight_blk[u] = w;
+    }
+}
+// Execution order of a worker's pair tiles: by (head, query chunk, key block), so that the workers, which get
+// the equal-weight tiles dealt out in turn, work on the same query chunk of the same head at about the same
+// time and the chunk's dQ accumulator rows and Q / dO tiles stay in L2 between their uses.
+__global__ void k_exec_order_pairs(const int32_t* __restrict__ cta_offsets, const int32_t* __restrict__ cta_tiles, int H,
+                                   const int32_t* __restrict__ u_blk, const int32_t* __restrict__ u_chunk,
+                                   int32_t* __restrict__ cta_exec) {
+    const int r = blockIdx.x;
+    const int beg = cta_offsets[r], n = cta_offsets[r + 1] - beg;
+    auto key_of = [&](int32_t t) {
+        const int32_t u = t / H;
+        return ((int64_t)(t % H) << 44) | ((int64_t)u_chunk[u] << 22) | (int64_t)u_blk[u];
+    };
+    if (n > 16384) {  // quadratic sort too slow: keep placement order
+        for (int i = threadIdx.x; i < n; i += blockDim.x) cta_exec[beg + i] = cta_tiles[beg + i];
+        return;
+    }
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        const int32_t t = cta_tiles[beg + i];
+        const int64_t key = key_of(t);
+        int rank = 0;
+        for (int j = 0; j < n; ++j) rank += key_of(cta_tiles[beg + j]) < key;
+        cta_exec[beg + rank] = t;
+    }
+}
+
 // Expanders used by libra_plan_export.
 __global__ void k_expand_weight(const int64_t* __restrict__ weight_blk, int64_t NT, int H, int64_t* __restrict__ out) {
     const int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
@@ -237,12 +314,48 @@ static inline unsigned grid_for(int64_t n, int block) { return (unsigned)((n + b
 static void free_dir(PlanDir& d) {
     cudaFree(d.d_weight_blk); cudaFree(d.d_blk_order); cudaFree(d.d_cta_of_tile); cudaFree(d.d_pos);
     cudaFree(d.d_cta_offsets); cudaFree(d.d_cta_tiles); cudaFree(d.d_cta_exec); cudaFree(d.d_loads); cudaFree(d.d_busy); cudaFree(d.d_busy2);
+    cudaFree(d.d_u_blk); cudaFree(d.d_u_chunk);
     d = PlanDir();
 }
 
-static int build_dir(libra_plan* p, PlanDir& d, int key_major, const libra_plan_opts& o) {
+// The pair-blocks of a plan: counts per key block, their prefix sums, and the total read back (one synchronous
+// 8-byte copy).  The query chunk is doubled until the pair-blocks fit the quadratic rank sort.
+static int count_pair_blocks(libra_plan* p, PlanDir& d, int64_t** base_out) {
+    const int64_t T = p->T, NKB = (T + d.tile - 1) / d.tile;
+    int32_t* count = nullptr;
+    int64_t *base = nullptr, *total = nullptr;
+    if (cudaMalloc((void**)&count, sizeof(int32_t) * NKB) != cudaSuccess ||
+        cudaMalloc((void**)&base, sizeof(int64_t) * (NKB + 1)) != cudaSuccess)
+        { cudaFree(count); cudaFree(base); return LIBRA_ERR_CUDA; }
+    total = base + NKB;
+    int rc = LIBRA_OK;
+    for (;;) {
+        k_pair_count<<<(unsigned)((NKB + 127) / 128), 128, 0, p->stream>>>(p->d_tok_end, T, d.tile, d.chunk, NKB, count);
+        k_scan_i32<<<1, 1024, 0, p->stream>>>(count, NKB, base, total);
+        count_launch(2);
+        int64_t nu = 0;
+        if (cudaMemcpyAsync(&nu, total, sizeof(int64_t), cudaMemcpyDeviceToHost, p->stream) != cudaSuccess ||
+            cudaStreamSynchronize(p->stream) != cudaSuccess) { rc = LIBRA_ERR_CUDA; break; }
+        d.NB = nu;
+        if (nu <= 65536) break;
+        if ((int64_t)d.chunk * 2 > (int64_t)1 << 30) { rc = LIBRA_ERR_UNSUPPORTED; break; }
+        d.chunk *= 2;
+    }
+    cudaFree(count);
+    if (rc != LIBRA_OK) { cudaFree(base); return rc; }
+    *base_out = base;
+    return LIBRA_OK;
+}
+
+static int build_dir(libra_plan* p, PlanDir& d, int key_major, const libra_plan_opts& o, bool pairs = false) {
     const int64_t T = p->T;
-    d.NB = (T + d.tile - 1) / d.tile;
+    int64_t* pair_base = nullptr;
+    if (pairs) {
+        const int rcp = count_pair_blocks(p, d, &pair_base);
+        if (rcp != LIBRA_OK) return rcp;
+    } else {
+        d.NB = (T + d.tile - 1) / d.tile;
+    }
     if (d.NB * (int64_t)d.H >= (int64_t)INT32_MAX) return LIBRA_ERR_OVERFLOW;
     // a worker's load is at most the weight total <= H * T^2 / 2 + ...; the placement packs load * 1024 + index
     if ((long double)d.H * (long double)T * (long double)T >= 9.0e15L) return LIBRA_ERR_OVERFLOW;
@@ -261,11 +374,21 @@ static int build_dir(libra_plan* p, PlanDir& d, int key_major, const libra_plan_
     A((void**)&d.d_loads, sizeof(int64_t) * d.W);
     A((void**)&d.d_busy, sizeof(uint64_t) * 2 * d.W);
     A((void**)&d.d_busy2, sizeof(uint64_t) * 2 * d.W);
-    if (e != cudaSuccess) return LIBRA_ERR_CUDA;
+    if (pairs) {
+        A((void**)&d.d_u_blk, sizeof(int32_t) * d.NB);
+        A((void**)&d.d_u_chunk, sizeof(int32_t) * d.NB);
+    }
+    if (e != cudaSuccess) { cudaFree(pair_base); return LIBRA_ERR_CUDA; }
     cudaStream_t s = p->stream;
     cudaMemsetAsync(d.d_busy, 0, sizeof(uint64_t) * 2 * d.W, s);
     cudaMemsetAsync(d.d_busy2, 0, sizeof(uint64_t) * 2 * d.W, s);
-    if (o.weight_model == LIBRA_WEIGHT_BLOCKS)
+    if (pairs) {
+        const int64_t NKB = (T + d.tile - 1) / d.tile;
+        k_pair_fill<<<grid_for(NKB, 128), 128, 0, s>>>(p->d_tok_end, T, d.tile, d.chunk, NKB, pair_base, d.d_u_blk,
+                                                       d.d_u_chunk, d.d_weight_blk);
+        cudaStreamSynchronize(s);   // pair_base is read by the kernel above
+        cudaFree(pair_base);
+    } else if (o.weight_model == LIBRA_WEIGHT_BLOCKS)
         k_block_weights_blocks<<<grid_for(d.NB, 128), 128, 0, s>>>(p->d_tok_start, p->d_tok_end, T, d.tile, d.NB,
                                                                    key_major, o.cost_block ? o.cost_block : 128,
                                                                    key_major ? o.unit_cost_kv : o.unit_cost_q,
@@ -285,7 +408,10 @@ static int build_dir(libra_plan* p, PlanDir& d, int key_major, const libra_plan_
                                      d.d_cta_offsets, d.d_loads);
     k_scatter_lists<<<grid_for(d.NT, 256), 256, 0, s>>>(d.d_cta_of_tile, d.d_pos, d.d_cta_offsets, d.NT,
                                                         d.d_cta_tiles);
-    k_exec_order<<<d.W, 256, 0, s>>>(d.d_cta_offsets, d.d_cta_tiles, d.H, d.NB, d.d_cta_exec);
+    if (pairs)
+        k_exec_order_pairs<<<d.W, 256, 0, s>>>(d.d_cta_offsets, d.d_cta_tiles, d.H, d.d_u_blk, d.d_u_chunk, d.d_cta_exec);
+    else
+        k_exec_order<<<d.W, 256, 0, s>>>(d.d_cta_offsets, d.d_cta_tiles, d.H, d.NB, d.d_cta_exec);
     count_launch(5);
     d.enabled = 1;
     return cudaGetLastError() == cudaSuccess ? LIBRA_OK : LIBRA_ERR_CUDA;
@@ -299,10 +425,11 @@ extern "C" int libra_plan_tiles(const int32_t* cu_seqlens_dev, int n_samples, in
                                 const libra_plan_opts* opts, void* stream, libra_plan_t** plan_out) {
     if (!cu_seqlens_dev || !plan_out || n_samples <= 0 || n_heads <= 0 || tile_q <= 0) return LIBRA_ERR_INVALID_ARG;
     *plan_out = nullptr;
-    libra_plan_opts o = {0, 0, 0, 0, 0, 0, 0, 0, 0};
+    libra_plan_opts o = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
     if (opts) o = *opts;
     if (o.n_workers < 0 || o.tile_kv < 0 || o.n_heads_kv < 0 || o.total_tokens < 0) return LIBRA_ERR_INVALID_ARG;
-    if (o.directions & ~(LIBRA_DIR_Q | LIBRA_DIR_KV)) return LIBRA_ERR_INVALID_ARG;
+    if (o.directions & ~(LIBRA_DIR_Q | LIBRA_DIR_KV | LIBRA_DIR_PAIR)) return LIBRA_ERR_INVALID_ARG;
+    if (o.pair_chunk < 0) return LIBRA_ERR_INVALID_ARG;
     if (o.weight_model != LIBRA_WEIGHT_PAIRS && o.weight_model != LIBRA_WEIGHT_BLOCKS) return LIBRA_ERR_INVALID_ARG;
     if (o.cost_block < 0 || o.unit_cost_q < 0 || o.unit_cost_kv < 0) return LIBRA_ERR_INVALID_ARG;
     int dev = 0;
@@ -346,6 +473,12 @@ extern "C" int libra_plan_tiles(const int32_t* cu_seqlens_dev, int n_samples, in
             d.tile = o.tile_kv ? o.tile_kv : 128; d.H = o.n_heads_kv ? o.n_heads_kv : n_heads; d.W = W;
             rc = build_dir(p, d, 1, o);
         }
+        if (rc == LIBRA_OK && (dirs & LIBRA_DIR_PAIR)) {
+            PlanDir& d = p->dir[2];
+            d.tile = o.tile_kv ? o.tile_kv : 128; d.H = o.n_heads_kv ? o.n_heads_kv : n_heads; d.W = W;
+            d.chunk = o.pair_chunk ? o.pair_chunk : 2048;
+            rc = d.chunk % d.tile ? LIBRA_ERR_INVALID_ARG : build_dir(p, d, 1, o, true);
+        }
     }
     if (rc != LIBRA_OK) {
         libra_plan_destroy(p);
@@ -359,6 +492,7 @@ static PlanDir* dir_of(const libra_plan_t* plan, int direction) {
     if (!plan) return nullptr;
     if (direction == LIBRA_DIR_Q) return plan->dir[0].enabled ? const_cast<PlanDir*>(&plan->dir[0]) : nullptr;
     if (direction == LIBRA_DIR_KV) return plan->dir[1].enabled ? const_cast<PlanDir*>(&plan->dir[1]) : nullptr;
+    if (direction == LIBRA_DIR_PAIR) return plan->dir[2].enabled ? const_cast<PlanDir*>(&plan->dir[2]) : nullptr;
     return nullptr;
 }
 
@@ -419,11 +553,26 @@ extern "C" int libra_plan_export(const libra_plan_t* plan, int direction, int64_
     return e == cudaSuccess ? LIBRA_OK : LIBRA_ERR_CUDA;
 }
 
+extern "C" int libra_plan_export_pairs(const libra_plan_t* plan, int32_t* key_block_host, int32_t* query_chunk_host,
+                                       int* chunk_tokens_host) {
+    if (!plan) return LIBRA_ERR_INVALID_ARG;
+    PlanDir* d = dir_of(plan, LIBRA_DIR_PAIR);
+    if (!d) return LIBRA_ERR_PLAN_MISMATCH;
+    cudaError_t e = cudaStreamSynchronize(plan->stream);
+    if (e == cudaSuccess && key_block_host)
+        e = cudaMemcpy(key_block_host, d->d_u_blk, sizeof(int32_t) * d->NB, cudaMemcpyDeviceToHost);
+    if (e == cudaSuccess && query_chunk_host)
+        e = cudaMemcpy(query_chunk_host, d->d_u_chunk, sizeof(int32_t) * d->NB, cudaMemcpyDeviceToHost);
+    if (chunk_tokens_host) *chunk_tokens_host = d->chunk;
+    return e == cudaSuccess ? LIBRA_OK : LIBRA_ERR_CUDA;
+}
+
 extern "C" int libra_plan_destroy(libra_plan_t* plan) {
     if (!plan) return LIBRA_OK;
     cudaDeviceSynchronize();
     free_dir(plan->dir[0]);
     free_dir(plan->dir[1]);
+    free_dir(plan->dir[2]);
     cudaFree(plan->d_tok_start);
     cudaFree(plan->d_tok_end);
     cudaFree(plan->d_status);

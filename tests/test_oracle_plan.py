@@ -227,3 +227,55 @@ def test_block_model_placement_vs_heap_simulation(seed):
     assert p["order"].tolist() == order
     assert p["cta_of_tile"].tolist() == owner
     assert p["loads"].tolist() == loads
+
+
+# ---- pair tiles (key block x query chunk x head): the fused backward's units ---------------------------------
+
+def _visible_pairs(cu):
+    """All (query, key) pairs of the pool: same sample, key position <= query position."""
+    out = []
+    for j in range(len(cu) - 1):
+        for q in range(cu[j], cu[j + 1]):
+            for k in range(cu[j], q + 1):
+                out.append((q, k))
+    return out
+
+
+@pytest.mark.parametrize("cu,tile,chunk", [([0, 5, 6, 16], 4, 8), ([0, 3, 3, 20, 21, 37], 4, 4), ([0, 40], 8, 16),
+                                           ([0, 1, 2, 3, 30], 4, 12), ([0, 9, 33], 16, 16)])
+def test_pair_tiles_cover_every_visible_pair_exactly_once(cu, tile, chunk):
+    H, W = 2, 3
+    res = oracle.plan_pairs(cu, H, tile, chunk, W)
+    nu = res["n_blocks"]
+    # brute force: every visible pair falls into exactly one (key block, query chunk) cell, and every cell that
+    # holds a pair is a pair-block; cells are listed key block by key block, chunks ascending
+    cells = {}
+    for q, k in _visible_pairs(cu):
+        cells[(k // tile, q // chunk)] = cells.get((k // tile, q // chunk), 0) + 1
+    listed = list(zip(res["key_block"].tolist(), res["query_chunk"].tolist()))
+    assert listed == sorted(listed) and len(set(listed)) == nu
+    assert set(cells) <= set(listed)
+    for u, cell in enumerate(listed):
+        for h in range(H):
+            assert res["weight"][u * H + h] == cells.get(cell, 0)
+    assert int(res["weight"].sum()) == H * len(_visible_pairs(cu))
+    # a listed cell without pairs can only be the diagonal chunk's neighbour of a block whose sample ends before it
+    # placement is Algorithm 2's: heaviest first, least-loaded worker, lowest index on ties
+    order = sorted(range(nu * H), key=lambda t: (-int(res["weight"][t]), t))
+    assert res["order"].tolist() == order
+    loads = [0] * W
+    for t in order:
+        r = min(range(W), key=lambda x: (loads[x], x))
+        assert res["cta_of_tile"][t] == r
+        loads[r] += int(res["weight"][t])
+    assert res["loads"].tolist() == loads
+
+
+def test_pair_tiles_with_one_chunk_per_sample_are_the_key_major_tiles():
+    """With a chunk that holds the whole pool every key block has one pair-block and its weight is the key-major
+    weight of oracle_plan (the number of queries attending each key)."""
+    cu = [0, 5, 6, 16, 40]
+    a = oracle.plan_pairs(cu, 2, 4, 64, 3)
+    b = oracle.plan(cu, 2, 4, 3, 1)
+    for key in ("weight", "order", "cta_of_tile", "cta_offsets", "cta_tiles", "loads"):
+        assert np.array_equal(a[key], b[key]), key

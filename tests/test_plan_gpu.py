@@ -99,3 +99,48 @@ def test_bad_cu_seqlens_is_reported_not_crashing():
         plan.destroy()
     with pytest.raises(lb.LibraError):
         lb.libra_plan_tiles(torch.tensor([0, 4], dtype=torch.int32).cuda(), 0, 4)
+
+
+# ---- pair tiles (key block x query chunk x head): the fused backward's units ---------------------------------
+
+def _compare_pairs(cu_np, H_kv, tile_kv, chunk, W):
+    from paper_2607_23250_b200 import binding as lb
+    cu = torch.from_numpy(cu_np).cuda()
+    plan = lb.libra_plan_tiles(cu, H_kv, 256, n_workers=W, directions=lb.LIBRA_DIR_PAIR, tile_kv=tile_kv, n_heads_kv=H_kv,
+                               pair_chunk=chunk)
+    assert plan.status() == 0
+    kb, qc, chunk_used = plan.export_pairs()
+    want = oracle.plan_pairs(cu_np, H_kv, tile_kv, chunk_used, W)       # the planner may have widened the chunk
+    got = plan.export(lb.LIBRA_DIR_PAIR)
+    assert got["n_blocks"] == want["n_blocks"] <= 65536
+    assert np.array_equal(kb, want["key_block"]) and np.array_equal(qc, want["query_chunk"])
+    for k in KEYS:
+        assert np.array_equal(got[k], want[k]), k
+    plan.destroy()
+    return chunk_used
+
+
+def test_pair_tiles_hand_example():
+    _compare_pairs(np.array([0, 5, 6, 16], dtype=np.int32), 1, 4, 8, 2)
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_pair_tiles_random_layouts(seed):
+    rng = np.random.default_rng(100 + seed)
+    lengths = pools.random_layout(rng, int(rng.integers(10, 4000)), int(rng.integers(1, 900)))
+    tile = int(rng.choice([4, 16, 128]))
+    _compare_pairs(pools.cu_seqlens(lengths), int(rng.integers(1, 5)), tile, tile * int(rng.choice([1, 2, 8])),
+                   int(rng.integers(1, 300)))
+
+
+@pytest.mark.parametrize("idx,skew", [(1, 0), (2, 0), (3, 0)])
+def test_pair_tiles_benchmark_configs(idx, skew):
+    spec = pools.config(idx, skew)
+    cu = pools.cu_seqlens(pools.pool_lengths(spec))
+    _compare_pairs(cu, spec.hkv, 128, 2048, 148)
+
+
+def test_pair_chunk_is_widened_until_the_pair_blocks_fit():
+    # a 60000-token sample at 128-token chunks would have about 110000 pair-blocks
+    cu = np.array([0, 60000], dtype=np.int32)
+    assert _compare_pairs(cu, 1, 128, 128, 7) > 128
