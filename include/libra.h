@@ -81,7 +81,7 @@ typedef struct {
                               eighths of a block (>= 0)                                             */
     int     unit_cost_kv;  /* same per key chunk of a key-major tile                                */
     int     pair_chunk;    /* LIBRA_DIR_PAIR: tokens per query chunk, a multiple of the key block; 0 = 2048
-                              (doubled by the planner until there are at most 65536 pair-blocks)       */
+                              (doubled by the planner while there are more than 262144 pair-blocks)    */
 } libra_plan_opts;
 
 typedef struct {
@@ -141,16 +141,21 @@ int libra_plan_export(const libra_plan_t* plan, int direction, int64_t* weight_h
                       int32_t* order_host, int32_t* cta_of_tile_host, int32_t* cta_offsets_host,
                       int32_t* cta_tiles_host, int64_t* loads_host);
 
-/* Pair tiles (directions & LIBRA_DIR_PAIR; the units of the fused backward).  The paper's tile is a query block
- * with all of its keys (Section 4.3.1); a pair tile cuts that rectangle along the key axis as well: key block j
- * (tile_kv keys of kv head h) against query chunk c (pair_chunk tokens).  Key block j is attended by the
- * queries from its first key to the last token of the sample that holds its last key, and has one pair-block
- * for every query chunk this range touches, chunks ascending; pair-blocks are numbered key block by key block,
- * tile id = pair-block * n_heads_kv + h.  The weight is still Eq. 6's count: the (query, key) pairs with the
- * key in the block, the query in the chunk, both in one sample and the query not before the key.  Ordering,
- * placement and lists follow Algorithm 2 as for the other directions, and libra_plan_info / libra_plan_export
- * take LIBRA_DIR_PAIR (n_blocks = pair-blocks).  libra_plan_export_pairs copies the key block and the query
- * chunk of every pair-block (int32[n_blocks] each, HOST, nullable) and the chunk size in tokens. */
+/* Pair tiles (directions & LIBRA_DIR_PAIR; the units of the fused backward; no counterpart in the paper beyond
+ * the tile idea itself).  The paper's tile is a query block with all of its keys (Section 4.3.1); a pair tile
+ * cuts that rectangle along the key axis as well.  The score matrix is cut into tile_kv x tile_kv cells at
+ * global positions; a cell is live when a query of its row block attends a key of its key block.  Pair-block
+ * (c, j) is key block j against the row blocks of query chunk c (pair_chunk tokens), present when one of those
+ * cells is live; pair-blocks are numbered chunk by chunk, key blocks ascending inside a chunk; tile id =
+ * h * n_blocks + pair-block (head-major).  The weight is the time proxy of LIBRA_WEIGHT_BLOCKS: the live cells
+ * of the pair-block.  Placement uses Algorithm 2's greedy rule (least-loaded worker, lowest index on ties) but
+ * takes the tiles in id order instead of heaviest first: the plan then equals the schedule of a first-in-first-
+ * out work queue, the workers stay on neighbouring tiles, and the rows of Q, dO and the dQ accumulator that
+ * those tiles share stay in L2 between their uses; since no tile is large, the loads still end up within one
+ * tile weight of each other.  libra_plan_info / libra_plan_export take LIBRA_DIR_PAIR (n_blocks = pair-blocks,
+ * order = identity).  libra_plan_export_pairs copies the key block and the query chunk of every pair-block
+ * (int32[n_blocks] each, HOST, nullable) and the chunk size in tokens (the planner doubles pair_chunk while
+ * there are more than 262144 pair-blocks). */
 int libra_plan_export_pairs(const libra_plan_t* plan, int32_t* key_block_host, int32_t* query_chunk_host,
                             int* chunk_tokens_host);
 

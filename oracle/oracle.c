@@ -143,28 +143,45 @@ int oracle_plan(const int32_t* cu, int n, int H, int tile, int W, int direction,
 }
 
 /* ------------------------------------------------------------------------------------
- * Plan over pair tiles (the fused backward's work units; the paper's tiles are query blocks with all their
- * keys, Section 4.3.1 - here a tile is additionally cut along the key axis, its weight is still the causal
- * pairs it covers, Eq. 6, and steps 3-5 are those of Algorithm 2 as in oracle_plan).
+ * Plan over pair tiles (the fused backward's work units).  The paper's tile is a query block with all of its
+ * keys (Section 4.3.1); a pair tile cuts that rectangle along the key axis too.  Not in the paper: the weight
+ * is the time proxy of oracle_plan_blocks (cells of the score matrix that hold a visible pair), and the tiles
+ * are placed in tile-id order instead of heaviest first, by the same greedy rule (least-loaded worker, lowest
+ * index on ties).  Placing in id order makes the static plan the schedule a first-in-first-out work queue
+ * would give, so the workers stay on neighbouring tiles, which share their query-side tensors.
  *
- * Keys are cut into blocks of `tile` tokens at global positions, queries into chunks of `chunk` tokens
- * (a multiple of `tile`).  Key block j is attended by queries from its own first key up to the last token of
- * the sample that holds its last key; it gets one pair-block for every query chunk that range touches:
- * chunks (j * tile) / chunk .. (end - 1) / chunk, in that order.  Pair-blocks are numbered key block by key
- * block; tile id = pair-block * H + h.  Weight = the (query, key) pairs with the key in the block, the query
- * in the chunk, both in the same sample, query position >= key position: counted pair by pair.
- * Outputs as oracle_plan, plus the key block and the query chunk of every pair-block.
+ * Cells: the score matrix cut into `tile` x `tile` cells at global positions; cell (i, j) is live if some
+ * query of row block i attends some key of key block j (same sample, query not before the key).
+ * Pair-block (c, j): key block j against query chunk c (`chunk` tokens, a multiple of `tile`), present when
+ * one of the chunk's row blocks has a live cell with j.  Pair-blocks are numbered chunk by chunk, key blocks
+ * ascending inside a chunk; tile id = h * NU + u (head-major); weight = live cells of the pair-block.
  * ------------------------------------------------------------------------------------ */
+static int pair_cells(const int32_t* cu, int n, int tile, uint8_t** live_out, int64_t* nb_out) {
+    const int64_t T = cu[n];
+    const int64_t NB = (T + tile - 1) / tile;
+    uint8_t* live = (uint8_t*)calloc((size_t)(NB * NB), 1);          /* [row block][key block] */
+    if (!live) return -2;
+    for (int j = 0; j < n; ++j)
+        for (int64_t k = cu[j]; k < cu[j + 1]; ++k)                   /* key k is attended by queries k .. end - 1 */
+            for (int64_t i = k / tile; i <= (cu[j + 1] - 1) / tile; ++i) live[i * NB + k / tile] = 1;
+    *live_out = live;
+    *nb_out = NB;
+    return 0;
+}
+
 int64_t oracle_plan_pairs_num_blocks(const int32_t* cu, int n, int tile, int chunk) {
     if (!cu || n <= 0 || tile <= 0 || chunk <= 0 || chunk % tile) return -1;
-    const int64_t T = cu[n];
+    uint8_t* live; int64_t NB;
+    if (pair_cells(cu, n, tile, &live, &NB)) return -2;
+    const int64_t R = chunk / tile;
     int64_t nu = 0;
-    for (int64_t k0 = 0; k0 < T; k0 += tile) {
-        const int64_t last_key = (k0 + tile < T ? k0 + tile : T) - 1;
-        int j = 0;
-        while (!(cu[j] <= last_key && last_key < cu[j + 1])) ++j;
-        nu += (cu[j + 1] - 1) / chunk - k0 / chunk + 1;
-    }
+    for (int64_t c = 0; c * R < NB; ++c)
+        for (int64_t j = 0; j < NB; ++j) {
+            int any = 0;
+            for (int64_t i = c * R; i < (c + 1) * R && i < NB; ++i) any |= live[i * NB + j];
+            nu += any;
+        }
+    free(live);
     return nu;
 }
 
@@ -174,26 +191,41 @@ int oracle_plan_pairs(const int32_t* cu, int n, int H, int tile, int chunk, int 
     if (!cu || n <= 0 || H <= 0 || tile <= 0 || chunk <= 0 || chunk % tile || W <= 0) return -1;
     if (cu[0] != 0) return -1;
     for (int j = 0; j < n; ++j) if (cu[j + 1] < cu[j]) return -1;
-    const int64_t T = cu[n];
-    int64_t u = 0;
-    for (int64_t k0 = 0; k0 < T; k0 += tile) {
-        const int64_t k1 = k0 + tile < T ? k0 + tile : T;
-        int jl = 0;
-        while (!(cu[jl] <= k1 - 1 && k1 - 1 < cu[jl + 1])) ++jl;          /* sample of the block's last key */
-        for (int64_t c = k0 / chunk; c <= (cu[jl + 1] - 1) / chunk; ++c, ++u) {
-            int64_t w = 0;
-            for (int64_t k = k0; k < k1; ++k) {
-                int j = 0;
-                while (!(cu[j] <= k && k < cu[j + 1])) ++j;               /* sample of key k */
-                for (int64_t q = c * chunk; q < (c + 1) * chunk && q < cu[j + 1]; ++q)
-                    if (q >= k) ++w;                                      /* same sample (q < its end), causal */
-            }
-            for (int h = 0; h < H; ++h) weight[u * H + h] = w;
-            key_block[u] = (int32_t)(k0 / tile);
-            query_chunk[u] = (int32_t)c;
+    uint8_t* live; int64_t NB;
+    if (pair_cells(cu, n, tile, &live, &NB)) return -2;
+    const int64_t R = chunk / tile;
+    int64_t nu = 0;
+    for (int64_t c = 0; c * R < NB; ++c)
+        for (int64_t j = 0; j < NB; ++j) {
+            int64_t cells = 0;
+            for (int64_t i = c * R; i < (c + 1) * R && i < NB; ++i) cells += live[i * NB + j];
+            if (!cells) continue;
+            key_block[nu] = (int32_t)j;
+            query_chunk[nu] = (int32_t)c;
+            weight[nu] = cells;                                        /* head 0 for now, copied below */
+            ++nu;
         }
+    free(live);
+    const int64_t NT = nu * H;
+    for (int h = H - 1; h >= 0; --h)
+        for (int64_t u = nu - 1; u >= 0; --u) weight[(int64_t)h * nu + u] = weight[u];
+    /* placement in tile-id order: each tile to the least-loaded worker, lowest index on ties */
+    for (int r = 0; r < W; ++r) loads[r] = 0;
+    for (int r = 0; r <= W; ++r) cta_offsets[r] = 0;
+    for (int64_t t = 0; t < NT; ++t) {
+        int best = 0;
+        for (int r = 1; r < W; ++r) if (loads[r] < loads[best]) best = r;
+        order[t] = (int32_t)t;
+        cta_of_tile[t] = best;
+        loads[best] += weight[t];
+        cta_offsets[best + 1] += 1;
     }
-    return place_tiles(u * H, W, weight, order, cta_of_tile, cta_offsets, cta_tiles, loads);
+    for (int r = 0; r < W; ++r) cta_offsets[r + 1] += cta_offsets[r];
+    int32_t* fill = (int32_t*)calloc((size_t)W, sizeof(int32_t));
+    if (!fill) return -2;
+    for (int64_t t = 0; t < NT; ++t) { const int r = cta_of_tile[t]; cta_tiles[cta_offsets[r] + fill[r]++] = (int32_t)t; }
+    free(fill);
+    return 0;
 }
 
 /* ------------------------------------------------------------------------------------

@@ -125,7 +125,8 @@ __global__ void k_rank_blocks(const int64_t* __restrict__ weight_blk, int64_t NB
 // host from the weight total), so load * 1024 + index fits 64 bits.
 template <int PER>
 __global__ void __launch_bounds__(32) k_place(const int64_t* __restrict__ weight_blk,
-                                              const int32_t* __restrict__ blk_order, int64_t NT, int H, int W,
+                                              const int32_t* __restrict__ blk_order /* null: tiles in id order, id =
+                                              head * NB + block */, int64_t NB, int64_t NT, int H, int W,
                                               int32_t* __restrict__ cta_of_tile, int32_t* __restrict__ pos,
                                               int32_t* __restrict__ cta_offsets, int64_t* __restrict__ loads) {
     const int lane = threadIdx.x;
@@ -147,9 +148,14 @@ __global__ void __launch_bounds__(32) k_place(const int64_t* __restrict__ weight
         int64_t w_l = 0;
         int32_t t_l = 0;
         if (xl < NT) {
-            const int32_t blk = blk_order[xl / H];
-            w_l = weight_blk[blk];
-            t_l = (int32_t)((int64_t)blk * H + xl % H);
+            if (blk_order) {
+                const int32_t blk = blk_order[xl / H];
+                w_l = weight_blk[blk];
+                t_l = (int32_t)((int64_t)blk * H + xl % H);
+            } else {
+                w_l = weight_blk[xl % NB];
+                t_l = (int32_t)xl;
+            }
         }
         const int lim = (int)((NT - x0 < 32) ? NT - x0 : 32);
         for (int i = 0; i < lim; ++i) {
@@ -221,15 +227,27 @@ __global__ void k_exec_order(const int32_t* __restrict__ cta_offsets, const int3
 }
 
 // ---- pair tiles: key block x query chunk x head (the fused backward's units) ---------------------------------
-// Key block j (`tile` keys) is attended by queries from its first key to the last token of the sample that holds
-// its last key: one pair-block per query chunk that range touches, chunks ascending, numbered key block by key block.
-__global__ void k_pair_count(const int32_t* __restrict__ tok_end, int64_t T, int tile, int chunk, int64_t NKB,
-                             int32_t* __restrict__ count) {
-    const int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-    if (j >= NKB) return;
-    const int64_t k0 = j * tile;
-    const int64_t last_key = (k0 + tile < T ? k0 + tile : T) - 1;
-    count[j] = (int32_t)(((int64_t)tok_end[last_key] - 1) / chunk - k0 / chunk + 1);
+// The score matrix in tile x tile cells: cell (i, j) is live when a query of row block i attends a key of key
+// block j; for a key block the live cells are the row blocks j .. last(j), last(j) = the block of the last token
+// of the sample that holds the key block's last key.  Pair-block (c, j) = key block j against the R = chunk / tile
+// row blocks of query chunk c, present when one of them is live; numbered chunk by chunk, key blocks ascending.
+// last(j) never decreases with j, so the key blocks of a chunk are the range first(c) .. min(NKB, (c+1) R) - 1.
+__device__ __forceinline__ int64_t pair_last_row_block(const int32_t* tok_end, int64_t T, int tile, int64_t j) {
+    const int64_t last_key = ((j + 1) * tile < T ? (j + 1) * tile : T) - 1;
+    return ((int64_t)tok_end[last_key] - 1) / tile;
+}
+__global__ void k_pair_chunks(const int32_t* __restrict__ tok_end, int64_t T, int tile, int R, int64_t NKB, int64_t NC,
+                              int32_t* __restrict__ first_j, int32_t* __restrict__ count) {
+    const int64_t c = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
+    if (c >= NC) return;
+    int64_t lo = 0, hi = NKB;   // first j with last(j) / R >= c
+    while (lo < hi) {
+        const int64_t mid = (lo + hi) >> 1;
+        if (pair_last_row_block(tok_end, T, tile, mid) / R >= c) hi = mid; else lo = mid + 1;
+    }
+    const int64_t last = (c + 1) * R - 1 < NKB - 1 ? (c + 1) * R - 1 : NKB - 1;
+    first_j[c] = (int32_t)lo;
+    count[c] = (int32_t)(last >= lo ? last - lo + 1 : 0);
 }
 // One block: exclusive prefix sum of count[0..n) into base, total into *total.
 __global__ void __launch_bounds__(1024) k_scan_i32(const int32_t* __restrict__ count, int64_t n, int64_t* __restrict__ base,
@@ -250,61 +268,32 @@ __global__ void __launch_bounds__(1024) k_scan_i32(const int32_t* __restrict__ c
     int64_t run = part[threadIdx.x];
     for (int64_t x = x0; x < x1; ++x) { base[x] = run; run += count[x]; }
 }
-// Weight of pair-block (j, c): the pairs with the key in block j, the query in chunk c, both in one sample and
-// query position >= key position = sum over the block's keys of the queries of the chunk inside [key, sample end).
-__global__ void k_pair_fill(const int32_t* __restrict__ tok_end, int64_t T, int tile, int chunk, int64_t NKB,
+// Weight of pair-block (c, j): its live cells, min(last(j), c R + R - 1) - max(j, c R) + 1.
+__global__ void k_pair_fill(const int32_t* __restrict__ tok_end, int64_t T, int tile, int R, int64_t NC,
+                            const int32_t* __restrict__ first_j, const int32_t* __restrict__ count,
                             const int64_t* __restrict__ base, int32_t* __restrict__ u_blk,
                             int32_t* __restrict__ u_chunk, int64_t* __restrict__ weight_blk) {
-    const int64_t j = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-    if (j >= NKB) return;
-    const int64_t k0 = j * tile, k1 = k0 + tile < T ? k0 + tile : T;
-    const int64_t c_lo = k0 / chunk, c_hi = ((int64_t)tok_end[k1 - 1] - 1) / chunk;
-    for (int64_t c = c_lo; c <= c_hi; ++c) {
-        const int64_t q0 = c * chunk, q1 = q0 + chunk;
-        int64_t w = 0;
-        for (int64_t k = k0; k < k1; ++k) {
-            const int64_t lo = k > q0 ? k : q0, hi = (int64_t)tok_end[k] < q1 ? (int64_t)tok_end[k] : q1;
-            if (hi > lo) w += hi - lo;
-        }
-        const int64_t u = base[j] + (c - c_lo);
+    const int64_t c = blockIdx.x;
+    if (c >= NC) return;
+    for (int x = threadIdx.x; x < count[c]; x += blockDim.x) {
+        const int64_t j = first_j[c] + x, u = base[c] + x;
+        const int64_t last = pair_last_row_block(tok_end, T, tile, j);
+        const int64_t i0 = j > c * R ? j : c * R, i1 = last < c * R + R - 1 ? last : c * R + R - 1;
         u_blk[u] = (int32_t)j;
         u_chunk[u] = (int32_t)c;
-        weight_blk[u] = w;
-    }
-}
-// Execution order of a worker's pair tiles: by (head, query chunk, key block), so that the workers, which get
-// the equal-weight tiles dealt out in turn, work on the same query chunk of the same head at about the same
-// time and the chunk's dQ accumulator rows and Q / dO tiles stay in L2 between their uses.
-__global__ void k_exec_order_pairs(const int32_t* __restrict__ cta_offsets, const int32_t* __restrict__ cta_tiles, int H,
-                                   const int32_t* __restrict__ u_blk, const int32_t* __restrict__ u_chunk,
-                                   int32_t* __restrict__ cta_exec) {
-    const int r = blockIdx.x;
-    const int beg = cta_offsets[r], n = cta_offsets[r + 1] - beg;
-    auto key_of = [&](int32_t t) {
-        const int32_t u = t / H;
-        return ((int64_t)(t % H) << 44) | ((int64_t)u_chunk[u] << 22) | (int64_t)u_blk[u];
-    };
-    if (n > 16384) {  // quadratic sort too slow: keep placement order
-        for (int i = threadIdx.x; i < n; i += blockDim.x) cta_exec[beg + i] = cta_tiles[beg + i];
-        return;
-    }
-    for (int i = threadIdx.x; i < n; i += blockDim.x) {
-        const int32_t t = cta_tiles[beg + i];
-        const int64_t key = key_of(t);
-        int rank = 0;
-        for (int j = 0; j < n; ++j) rank += key_of(cta_tiles[beg + j]) < key;
-        cta_exec[beg + rank] = t;
+        weight_blk[u] = i1 - i0 + 1;
     }
 }
 
 // Expanders used by libra_plan_export.
-__global__ void k_expand_weight(const int64_t* __restrict__ weight_blk, int64_t NT, int H, int64_t* __restrict__ out) {
+__global__ void k_expand_weight(const int64_t* __restrict__ weight_blk, int64_t NT, int H, int64_t NB_headmajor,
+                                int64_t* __restrict__ out) {
     const int64_t t = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-    if (t < NT) out[t] = weight_blk[t / H];
+    if (t < NT) out[t] = NB_headmajor ? weight_blk[t % NB_headmajor] : weight_blk[t / H];
 }
 __global__ void k_expand_order(const int32_t* __restrict__ blk_order, int64_t NT, int H, int32_t* __restrict__ out) {
     const int64_t x = blockIdx.x * (int64_t)blockDim.x + threadIdx.x;
-    if (x < NT) out[x] = (int32_t)((int64_t)blk_order[x / H] * H + x % H);
+    if (x < NT) out[x] = blk_order ? (int32_t)((int64_t)blk_order[x / H] * H + x % H) : (int32_t)x;
 }
 
 // ---- host ---------------------------------------------------------------------------------
@@ -318,48 +307,48 @@ static void free_dir(PlanDir& d) {
     d = PlanDir();
 }
 
-// The pair-blocks of a plan: counts per key block, their prefix sums, and the total read back (one synchronous
-// 8-byte copy).  The query chunk is doubled until the pair-blocks fit the quadratic rank sort.
-static int count_pair_blocks(libra_plan* p, PlanDir& d, int64_t** base_out) {
+// The pair-blocks of a plan: counts per query chunk, their prefix sums, and the total read back (one synchronous
+// 8-byte copy).  The query chunk is doubled while there are more than 262144 pair-blocks (the placement is
+// sequential, about a third of a microsecond per tile).
+struct PairTables { int32_t* first_j = nullptr; int32_t* count = nullptr; int64_t* base = nullptr; int64_t NC = 0; };
+static void free_pair_tables(PairTables& t) { cudaFree(t.first_j); cudaFree(t.count); cudaFree(t.base); t = PairTables(); }
+static int count_pair_blocks(libra_plan* p, PlanDir& d, PairTables& tb) {
     const int64_t T = p->T, NKB = (T + d.tile - 1) / d.tile;
-    int32_t* count = nullptr;
-    int64_t *base = nullptr, *total = nullptr;
-    if (cudaMalloc((void**)&count, sizeof(int32_t) * NKB) != cudaSuccess ||
-        cudaMalloc((void**)&base, sizeof(int64_t) * (NKB + 1)) != cudaSuccess)
-        { cudaFree(count); cudaFree(base); return LIBRA_ERR_CUDA; }
-    total = base + NKB;
-    int rc = LIBRA_OK;
     for (;;) {
-        k_pair_count<<<(unsigned)((NKB + 127) / 128), 128, 0, p->stream>>>(p->d_tok_end, T, d.tile, d.chunk, NKB, count);
-        k_scan_i32<<<1, 1024, 0, p->stream>>>(count, NKB, base, total);
+        const int R = d.chunk / d.tile;
+        tb.NC = (NKB + R - 1) / R;
+        if (cudaMalloc((void**)&tb.first_j, sizeof(int32_t) * tb.NC) != cudaSuccess ||
+            cudaMalloc((void**)&tb.count, sizeof(int32_t) * tb.NC) != cudaSuccess ||
+            cudaMalloc((void**)&tb.base, sizeof(int64_t) * (tb.NC + 1)) != cudaSuccess)
+            { free_pair_tables(tb); return LIBRA_ERR_CUDA; }
+        k_pair_chunks<<<(unsigned)((tb.NC + 127) / 128), 128, 0, p->stream>>>(p->d_tok_end, T, d.tile, R, NKB, tb.NC,
+                                                                             tb.first_j, tb.count);
+        k_scan_i32<<<1, 1024, 0, p->stream>>>(tb.count, tb.NC, tb.base, tb.base + tb.NC);
         count_launch(2);
         int64_t nu = 0;
-        if (cudaMemcpyAsync(&nu, total, sizeof(int64_t), cudaMemcpyDeviceToHost, p->stream) != cudaSuccess ||
-            cudaStreamSynchronize(p->stream) != cudaSuccess) { rc = LIBRA_ERR_CUDA; break; }
+        if (cudaMemcpyAsync(&nu, tb.base + tb.NC, sizeof(int64_t), cudaMemcpyDeviceToHost, p->stream) != cudaSuccess ||
+            cudaStreamSynchronize(p->stream) != cudaSuccess) { free_pair_tables(tb); return LIBRA_ERR_CUDA; }
         d.NB = nu;
-        if (nu <= 65536) break;
-        if ((int64_t)d.chunk * 2 > (int64_t)1 << 30) { rc = LIBRA_ERR_UNSUPPORTED; break; }
+        if (nu <= 262144) return LIBRA_OK;
+        free_pair_tables(tb);
+        if ((int64_t)d.chunk * 2 > (int64_t)1 << 30) return LIBRA_ERR_UNSUPPORTED;
         d.chunk *= 2;
     }
-    cudaFree(count);
-    if (rc != LIBRA_OK) { cudaFree(base); return rc; }
-    *base_out = base;
-    return LIBRA_OK;
 }
 
 static int build_dir(libra_plan* p, PlanDir& d, int key_major, const libra_plan_opts& o, bool pairs = false) {
     const int64_t T = p->T;
-    int64_t* pair_base = nullptr;
+    PairTables tb;
     if (pairs) {
-        const int rcp = count_pair_blocks(p, d, &pair_base);
+        const int rcp = count_pair_blocks(p, d, tb);
         if (rcp != LIBRA_OK) return rcp;
     } else {
         d.NB = (T + d.tile - 1) / d.tile;
     }
-    if (d.NB * (int64_t)d.H >= (int64_t)INT32_MAX) return LIBRA_ERR_OVERFLOW;
+    if (d.NB * (int64_t)d.H >= (int64_t)INT32_MAX) { free_pair_tables(tb); return LIBRA_ERR_OVERFLOW; }
     // a worker's load is at most the weight total <= H * T^2 / 2 + ...; the placement packs load * 1024 + index
     if ((long double)d.H * (long double)T * (long double)T >= 9.0e15L) return LIBRA_ERR_OVERFLOW;
-    if (d.NB > 65536) return LIBRA_ERR_UNSUPPORTED;  // the rank sort is quadratic in blocks
+    if (!pairs && d.NB > 65536) return LIBRA_ERR_UNSUPPORTED;  // the rank sort is quadratic in blocks
     if (d.W > 1024) return LIBRA_ERR_UNSUPPORTED;
     d.NT = d.NB * d.H;
     cudaError_t e = cudaSuccess;
@@ -378,16 +367,15 @@ static int build_dir(libra_plan* p, PlanDir& d, int key_major, const libra_plan_
         A((void**)&d.d_u_blk, sizeof(int32_t) * d.NB);
         A((void**)&d.d_u_chunk, sizeof(int32_t) * d.NB);
     }
-    if (e != cudaSuccess) { cudaFree(pair_base); return LIBRA_ERR_CUDA; }
+    if (e != cudaSuccess) { free_pair_tables(tb); return LIBRA_ERR_CUDA; }
     cudaStream_t s = p->stream;
     cudaMemsetAsync(d.d_busy, 0, sizeof(uint64_t) * 2 * d.W, s);
     cudaMemsetAsync(d.d_busy2, 0, sizeof(uint64_t) * 2 * d.W, s);
     if (pairs) {
-        const int64_t NKB = (T + d.tile - 1) / d.tile;
-        k_pair_fill<<<grid_for(NKB, 128), 128, 0, s>>>(p->d_tok_end, T, d.tile, d.chunk, NKB, pair_base, d.d_u_blk,
-                                                       d.d_u_chunk, d.d_weight_blk);
-        cudaStreamSynchronize(s);   // pair_base is read by the kernel above
-        cudaFree(pair_base);
+        k_pair_fill<<<(unsigned)tb.NC, 128, 0, s>>>(p->d_tok_end, T, d.tile, d.chunk / d.tile, tb.NC, tb.first_j, tb.count,
+                                                    tb.base, d.d_u_blk, d.d_u_chunk, d.d_weight_blk);
+        cudaStreamSynchronize(s);   // the tables are read by the kernel above
+        free_pair_tables(tb);
     } else if (o.weight_model == LIBRA_WEIGHT_BLOCKS)
         k_block_weights_blocks<<<grid_for(d.NB, 128), 128, 0, s>>>(p->d_tok_start, p->d_tok_end, T, d.tile, d.NB,
                                                                    key_major, o.cost_block ? o.cost_block : 128,
@@ -396,20 +384,21 @@ static int build_dir(libra_plan* p, PlanDir& d, int key_major, const libra_plan_
     else
         k_block_weights<<<grid_for(d.NB, 128), 128, 0, s>>>(p->d_tok_start, p->d_tok_end, T, d.tile, d.NB, key_major,
                                                             d.d_weight_blk);
-    k_rank_blocks<<<grid_for(d.NB, 256), 256, 0, s>>>(d.d_weight_blk, d.NB, d.d_blk_order);
+    const int32_t* ord = pairs ? nullptr : d.d_blk_order;   // pair tiles are placed in id order
+    if (!pairs) k_rank_blocks<<<grid_for(d.NB, 256), 256, 0, s>>>(d.d_weight_blk, d.NB, d.d_blk_order);
     if (d.W <= 160)
-        k_place<5><<<1, 32, 0, s>>>(d.d_weight_blk, d.d_blk_order, d.NT, d.H, d.W, d.d_cta_of_tile, d.d_pos,
+        k_place<5><<<1, 32, 0, s>>>(d.d_weight_blk, ord, d.NB, d.NT, d.H, d.W, d.d_cta_of_tile, d.d_pos,
                                     d.d_cta_offsets, d.d_loads);
     else if (d.W <= 320)
-        k_place<10><<<1, 32, 0, s>>>(d.d_weight_blk, d.d_blk_order, d.NT, d.H, d.W, d.d_cta_of_tile, d.d_pos,
+        k_place<10><<<1, 32, 0, s>>>(d.d_weight_blk, ord, d.NB, d.NT, d.H, d.W, d.d_cta_of_tile, d.d_pos,
                                      d.d_cta_offsets, d.d_loads);
     else
-        k_place<32><<<1, 32, 0, s>>>(d.d_weight_blk, d.d_blk_order, d.NT, d.H, d.W, d.d_cta_of_tile, d.d_pos,
+        k_place<32><<<1, 32, 0, s>>>(d.d_weight_blk, ord, d.NB, d.NT, d.H, d.W, d.d_cta_of_tile, d.d_pos,
                                      d.d_cta_offsets, d.d_loads);
     k_scatter_lists<<<grid_for(d.NT, 256), 256, 0, s>>>(d.d_cta_of_tile, d.d_pos, d.d_cta_offsets, d.NT,
                                                         d.d_cta_tiles);
-    if (pairs)
-        k_exec_order_pairs<<<d.W, 256, 0, s>>>(d.d_cta_offsets, d.d_cta_tiles, d.H, d.d_u_blk, d.d_u_chunk, d.d_cta_exec);
+    if (pairs)   // placed in id order: the lists already are in execution order
+        cudaMemcpyAsync(d.d_cta_exec, d.d_cta_tiles, sizeof(int32_t) * d.NT, cudaMemcpyDeviceToDevice, s);
     else
         k_exec_order<<<d.W, 256, 0, s>>>(d.d_cta_offsets, d.d_cta_tiles, d.H, d.NB, d.d_cta_exec);
     count_launch(5);
@@ -530,13 +519,15 @@ extern "C" int libra_plan_export(const libra_plan_t* plan, int direction, int64_
     if (weight_host || order_host) ok(cudaMalloc(&tmp, sizeof(int64_t) * (d->NT ? d->NT : 1)));
     if (e != cudaSuccess) return LIBRA_ERR_CUDA;
     if (weight_host) {
-        k_expand_weight<<<grid_for(d->NT, 256), 256, 0, s>>>(d->d_weight_blk, d->NT, d->H, (int64_t*)tmp);
+        k_expand_weight<<<grid_for(d->NT, 256), 256, 0, s>>>(d->d_weight_blk, d->NT, d->H, d->d_u_blk ? d->NB : 0,
+                                                             (int64_t*)tmp);
         count_launch();
         ok(cudaMemcpyAsync(weight_host, tmp, sizeof(int64_t) * d->NT, cudaMemcpyDeviceToHost, s));
         ok(cudaStreamSynchronize(s));
     }
     if (order_host) {
-        k_expand_order<<<grid_for(d->NT, 256), 256, 0, s>>>(d->d_blk_order, d->NT, d->H, (int32_t*)tmp);
+        k_expand_order<<<grid_for(d->NT, 256), 256, 0, s>>>(d->d_u_blk ? nullptr : d->d_blk_order, d->NT, d->H,
+                                                            (int32_t*)tmp);
         count_launch();
         ok(cudaMemcpyAsync(order_host, tmp, sizeof(int32_t) * d->NT, cudaMemcpyDeviceToHost, s));
         ok(cudaStreamSynchronize(s));

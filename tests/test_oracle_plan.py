@@ -242,40 +242,39 @@ def _visible_pairs(cu):
 
 
 @pytest.mark.parametrize("cu,tile,chunk", [([0, 5, 6, 16], 4, 8), ([0, 3, 3, 20, 21, 37], 4, 4), ([0, 40], 8, 16),
-                                           ([0, 1, 2, 3, 30], 4, 12), ([0, 9, 33], 16, 16)])
-def test_pair_tiles_cover_every_visible_pair_exactly_once(cu, tile, chunk):
+                                           ([0, 1, 2, 3, 30], 4, 12), ([0, 9, 33], 16, 16), ([0, 70], 4, 16)])
+def test_pair_tiles_are_the_live_cells_of_the_score_matrix(cu, tile, chunk):
     H, W = 2, 3
     res = oracle.plan_pairs(cu, H, tile, chunk, W)
     nu = res["n_blocks"]
-    # brute force: every visible pair falls into exactly one (key block, query chunk) cell, and every cell that
-    # holds a pair is a pair-block; cells are listed key block by key block, chunks ascending
-    cells = {}
-    for q, k in _visible_pairs(cu):
-        cells[(k // tile, q // chunk)] = cells.get((k // tile, q // chunk), 0) + 1
-    listed = list(zip(res["key_block"].tolist(), res["query_chunk"].tolist()))
-    assert listed == sorted(listed) and len(set(listed)) == nu
-    assert set(cells) <= set(listed)
+    # brute force over every visible pair: the live cells, grouped by (query chunk, key block)
+    cells = {(q // tile, k // tile) for q, k in _visible_pairs(cu)}
+    groups = {}
+    for i, j in cells:
+        groups[(i * tile // chunk, j)] = groups.get((i * tile // chunk, j), 0) + 1
+    listed = list(zip(res["query_chunk"].tolist(), res["key_block"].tolist()))
+    assert listed == sorted(groups)                                  # chunk by chunk, key blocks ascending
     for u, cell in enumerate(listed):
         for h in range(H):
-            assert res["weight"][u * H + h] == cells.get(cell, 0)
-    assert int(res["weight"].sum()) == H * len(_visible_pairs(cu))
-    # a listed cell without pairs can only be the diagonal chunk's neighbour of a block whose sample ends before it
-    # placement is Algorithm 2's: heaviest first, least-loaded worker, lowest index on ties
-    order = sorted(range(nu * H), key=lambda t: (-int(res["weight"][t]), t))
-    assert res["order"].tolist() == order
-    loads = [0] * W
-    for t in order:
+            assert res["weight"][h * nu + u] == groups[cell]          # head-major ids, the same weight for every head
+    assert int(res["weight"].sum()) == H * len(cells)
+    # placement: in tile-id order, least-loaded worker, lowest index on ties
+    assert res["order"].tolist() == list(range(nu * H))
+    loads, lists = [0] * W, [[] for _ in range(W)]
+    for t in range(nu * H):
         r = min(range(W), key=lambda x: (loads[x], x))
         assert res["cta_of_tile"][t] == r
         loads[r] += int(res["weight"][t])
+        lists[r].append(t)
     assert res["loads"].tolist() == loads
+    assert res["cta_tiles"].tolist() == [t for l in lists for t in l]
+    assert max(loads) - min(loads) <= int(res["weight"].max())     # list scheduling: no worker is a whole tile ahead
 
 
-def test_pair_tiles_with_one_chunk_per_sample_are_the_key_major_tiles():
-    """With a chunk that holds the whole pool every key block has one pair-block and its weight is the key-major
-    weight of oracle_plan (the number of queries attending each key)."""
-    cu = [0, 5, 6, 16, 40]
-    a = oracle.plan_pairs(cu, 2, 4, 64, 3)
-    b = oracle.plan(cu, 2, 4, 3, 1)
-    for key in ("weight", "order", "cta_of_tile", "cta_offsets", "cta_tiles", "loads"):
-        assert np.array_equal(a[key], b[key]), key
+def test_pair_tiles_of_one_long_sample_in_closed_form():
+    """One sample of n row blocks, chunks of R blocks: key block j meets chunk c in min(n, (c+1)R) - max(j, cR) cells."""
+    tile, R, n = 8, 4, 11
+    res = oracle.plan_pairs([0, n * tile], 1, tile, R * tile, 5)
+    want = [(c, j, min(n, (c + 1) * R) - max(j, c * R)) for c in range((n + R - 1) // R) for j in range(min(n, (c + 1) * R))]
+    got = list(zip(res["query_chunk"].tolist(), res["key_block"].tolist(), res["weight"].tolist()))
+    assert got == want

@@ -112,7 +112,7 @@ def _compare_pairs(cu_np, H_kv, tile_kv, chunk, W):
     kb, qc, chunk_used = plan.export_pairs()
     want = oracle.plan_pairs(cu_np, H_kv, tile_kv, chunk_used, W)       # the planner may have widened the chunk
     got = plan.export(lb.LIBRA_DIR_PAIR)
-    assert got["n_blocks"] == want["n_blocks"] <= 65536
+    assert got["n_blocks"] == want["n_blocks"] <= 262144
     assert np.array_equal(kb, want["key_block"]) and np.array_equal(qc, want["query_chunk"])
     for k in KEYS:
         assert np.array_equal(got[k], want[k]), k
@@ -141,6 +141,6 @@ def test_pair_tiles_benchmark_configs(idx, skew):
 
 
 def test_pair_chunk_is_widened_until_the_pair_blocks_fit():
-    # a 60000-token sample at 128-token chunks would have about 110000 pair-blocks
+    # a 60000-token sample at 16-token blocks and chunks would have about 7 million pair-blocks
     cu = np.array([0, 60000], dtype=np.int32)
-    assert _compare_pairs(cu, 1, 128, 128, 7) > 128
+    assert _compare_pairs(cu, 1, 16, 16, 7) > 16
