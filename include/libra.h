@@ -65,6 +65,8 @@ extern "C" {
 #define LIBRA_KERNEL_BWD_DKDV  2   /* backward dK/dV kernel (walks the key-major lists)       */
 #define LIBRA_KERNEL_BWD_DQ    3   /* backward dQ kernel (walks the query-major lists)        */
 #define LIBRA_KERNEL_BWD_PREP  4   /* backward row statistics (timing only: it keeps no busy times) */
+#define LIBRA_KERNEL_BWD_FUSED 5   /* fused backward kernel incl. clearing its accumulators (walks the pair tiles) */
+#define LIBRA_KERNEL_BWD_POST  6   /* fused backward: scaling and rounding of the accumulators (timing only)   */
 
 typedef struct libra_plan libra_plan_t;   /* opaque, library-owned */
 

@@ -21,7 +21,7 @@ _lib = ctypes.CDLL(_SO)
 
 LIBRA_DIR_Q, LIBRA_DIR_KV, LIBRA_DIR_PAIR = 1, 2, 4
 LIBRA_WEIGHT_PAIRS, LIBRA_WEIGHT_BLOCKS = 0, 1
-KERNEL_FWD, KERNEL_BWD_DKDV, KERNEL_BWD_DQ, KERNEL_BWD_PREP = 1, 2, 3, 4
+KERNEL_FWD, KERNEL_BWD_DKDV, KERNEL_BWD_DQ, KERNEL_BWD_PREP, KERNEL_BWD_FUSED, KERNEL_BWD_POST = 1, 2, 3, 4, 5, 6
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_PLAN_MISMATCH, ERR_CUDA = -1, -2, -3, -4
 ERR_OVERFLOW, ERR_TIMEOUT, ERR_BAD_SEQLENS, ERR_NO_DEVICE = -5, -6, -7, -8
 ERR_SCRATCH_TOO_SMALL = -9
@@ -125,7 +125,8 @@ class Plan:
         return kb, qc, chunk.value
 
     def busy_times(self, which=KERNEL_FWD):
-        w = self.info(LIBRA_DIR_KV if which == KERNEL_BWD_DKDV else LIBRA_DIR_Q)["n_workers"]
+        w = self.info(LIBRA_DIR_PAIR if which == KERNEL_BWD_FUSED else
+                      (LIBRA_DIR_KV if which == KERNEL_BWD_DKDV else LIBRA_DIR_Q))["n_workers"]
         out = np.zeros(w, np.uint64)
         _check(_lib.libra_busy_times(self._h, which, _np(out)), "libra_busy_times")
         return out

@@ -574,6 +574,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
 }  // namespace libra
 
 #include "attn_bwd_dq.cuh"
+#include "attn_bwd_fused.cuh"
 
 namespace libra {
 
@@ -627,14 +628,25 @@ __global__ void k_bwd_prep(const __nv_bfloat16* __restrict__ out, const __nv_bfl
 
 struct BwdWorkspace {
     size_t stat_bytes, total;
+    size_t dq_acc_bytes, dkv_acc_bytes;   // fused form only: fp32 accumulators of dQ and of dK, dV (each)
     int64_t Tpad;
 };
-static BwdWorkspace bwd_workspace(int64_t T, int hq) {
+static BwdWorkspace bwd_workspace(int64_t T, int hq, int hkv = 0, int d = 0, bool fused = false) {
     BwdWorkspace w;
     w.Tpad = (T + 127) / 128 * 128;
     w.stat_bytes = ((size_t)hq * w.Tpad * sizeof(float) + 255) & ~(size_t)255;
     w.total = 2 * w.stat_bytes;
+    w.dq_acc_bytes = w.dkv_acc_bytes = 0;
+    if (fused) {
+        w.dq_acc_bytes = ((size_t)T * hq * d * sizeof(float) + 255) & ~(size_t)255;
+        w.dkv_acc_bytes = ((size_t)T * hkv * d * sizeof(float) + 255) & ~(size_t)255;
+        w.total += w.dq_acc_bytes + 2 * w.dkv_acc_bytes;
+    }
     return w;
+}
+// The fused backward runs when the plan carries pair tiles and the head dimension is 128.
+static bool use_fused(const libra_plan_t* plan, const libra_dims* dims) {
+    return plan->dir[2].enabled && dims->head_dim == 128;
 }
 
 template <typename Kernel>
@@ -676,8 +688,64 @@ extern "C" int libra_debug_trace(long long* host, int n) {
 #endif
 
 extern "C" size_t libra_attn_pool_bwd_workspace_bytes(const libra_plan_t* plan, const libra_dims* dims) {
-    if (!plan || !dims || dims->hq <= 0 || (dims->head_dim != 64 && dims->head_dim != 128)) return 0;
-    return bwd_workspace(plan->T, dims->hq).total;
+    if (!plan || !dims || dims->hq <= 0 || dims->hkv <= 0 || (dims->head_dim != 64 && dims->head_dim != 128)) return 0;
+    return bwd_workspace(plan->T, dims->hq, dims->hkv, dims->head_dim, use_fused(plan, dims)).total;
+}
+
+// fp32 tensor [T, H, 128] viewed as (128, H, T); box = 32 floats x 1 head x 32 rows, 128-byte swizzle.
+static int make_f32_thd_map(CUtensorMap* m, const void* base, int64_t T, int H) {
+    // three dimensions through the same driver entry point as the bf16 maps
+    return libra::make_f32_3d_map(m, base, T, H, 128, 32, 32);
+}
+
+static int launch_fused(const void* q_dev, const void* k_dev, const void* v_dev, const void* dout_dev, void* dq_dev,
+                        void* dk_dev, void* dv_dev, uint8_t* ws_dev, const BwdWorkspace& ws, const libra_plan_t* plan,
+                        const libra_dims* dims, float scale, cudaStream_t s) {
+    const PlanDir& d = plan->dir[2];
+    const int64_t T = plan->T;
+    if (d.tile != kBlk || d.H != dims->hkv) return LIBRA_ERR_PLAN_MISMATCH;
+    if (d.W > plan->sm_count) return LIBRA_ERR_UNSUPPORTED;
+    float* dvec = reinterpret_cast<float*>(ws_dev);
+    float* lse2 = reinterpret_cast<float*>(ws_dev + ws.stat_bytes);
+    float* dq_acc = reinterpret_cast<float*>(ws_dev + 2 * ws.stat_bytes);
+    float* dk_acc = reinterpret_cast<float*>(ws_dev + 2 * ws.stat_bytes + ws.dq_acc_bytes);
+    float* dv_acc = reinterpret_cast<float*>(ws_dev + 2 * ws.stat_bytes + ws.dq_acc_bytes + ws.dkv_acc_bytes);
+    CUtensorMap tq, tk, tv, tdo, tacc;
+    int rc = make_thd_map(&tq, q_dev, T, dims->hq, 128, kBlk);
+    if (rc == LIBRA_OK) rc = make_thd_map(&tk, k_dev, T, dims->hkv, 128, kBlk);
+    if (rc == LIBRA_OK) rc = make_thd_map(&tv, v_dev, T, dims->hkv, 128, kBlk);
+    if (rc == LIBRA_OK) rc = make_thd_map(&tdo, dout_dev, T, dims->hq, 128, kBlk);
+    if (rc == LIBRA_OK) rc = make_f32_thd_map(&tacc, dq_acc, T, dims->hq);
+    if (rc != LIBRA_OK) return rc;
+    if (!cfg_done(4)) {
+        if (set_smem(k_attn_bwd_fused, FusedSmem::kBytes) != LIBRA_OK) return LIBRA_ERR_CUDA;
+        if (!regs_pool_ok(k_attn_bwd_fused, 128, kFuRegsDs, 128, kFuRegsOther)) return LIBRA_ERR_UNSUPPORTED;
+        cfg_mark(4);
+    }
+    libra_plan_t* mp = const_cast<libra_plan_t*>(plan);
+    FusedParams fp;
+    fp.dq_acc = dq_acc; fp.dk_acc = dk_acc; fp.dv_acc = dv_acc;
+    fp.lse2 = lse2; fp.dvec = dvec;
+    fp.cta_offsets = d.d_cta_offsets; fp.cta_tiles = d.d_cta_exec;
+    fp.u_blk = d.d_u_blk; fp.u_chunk = d.d_u_chunk; fp.tok_end = plan->d_tok_end;
+    fp.T = T; fp.Tpad = ws.Tpad; fp.NU = d.NB;
+    fp.hq = dims->hq; fp.hkv = dims->hkv; fp.R = d.chunk / d.tile;
+    fp.scale_log2 = scale * 1.4426950408889634f;
+    fp.status = plan->d_status + 2; fp.plan_status = plan->d_status;
+    fp.wait_limit_ns = plan->wait_limit_ns; fp.inject_stall = plan->inject_stall;
+    fp.busy = d.d_busy;
+    time_begin(mp, 4, s);
+    cudaMemsetAsync(dq_acc, 0, ws.dq_acc_bytes + 2 * ws.dkv_acc_bytes, s);   // the three accumulators are contiguous
+    k_attn_bwd_fused<<<d.W, kFusedThreads, FusedSmem::kBytes, s>>>(tq, tk, tv, tdo, tacc, fp);
+    time_end(mp, 4, s);
+    time_begin(mp, 5, s);
+    const int64_t nq8 = T * dims->hq * 128 / 8, nk8 = T * dims->hkv * 128 / 8;
+    k_bwd_fused_finish<<<(unsigned)((nq8 + 255) / 256), 256, 0, s>>>(dq_acc, (__nv_bfloat16*)dq_dev, nq8, scale);
+    k_bwd_fused_finish<<<(unsigned)((nk8 + 255) / 256), 256, 0, s>>>(dk_acc, (__nv_bfloat16*)dk_dev, nk8, scale);
+    k_bwd_fused_finish<<<(unsigned)((nk8 + 255) / 256), 256, 0, s>>>(dv_acc, (__nv_bfloat16*)dv_dev, nk8, 1.0f);
+    time_end(mp, 5, s);
+    count_launch(4);
+    return cudaGetLastError() == cudaSuccess ? LIBRA_OK : LIBRA_ERR_CUDA;
 }
 
 extern "C" int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const void* v_dev, const void* out_dev,
@@ -691,11 +759,15 @@ extern "C" int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const v
     if (dims->head_dim != 64 && dims->head_dim != 128) return LIBRA_ERR_UNSUPPORTED;
     const PlanDir& dq_dir = plan->dir[0];
     const PlanDir& dkv_dir = plan->dir[1];
-    if (!dq_dir.enabled || !dkv_dir.enabled || plan->T != dims->total_tokens) return LIBRA_ERR_PLAN_MISMATCH;
-    if (dkv_dir.tile != kBlk || dq_dir.tile != 2 * kBlk) return LIBRA_ERR_UNSUPPORTED;
-    if (dkv_dir.H != dims->hkv) return LIBRA_ERR_PLAN_MISMATCH;
-    if (dims->hq % dq_dir.H) return LIBRA_ERR_INVALID_ARG;
-    if (dkv_dir.W > plan->sm_count || dq_dir.W > plan->sm_count) return LIBRA_ERR_UNSUPPORTED;
+    const bool fused = use_fused(plan, dims);
+    if (plan->T != dims->total_tokens) return LIBRA_ERR_PLAN_MISMATCH;
+    if (!fused) {
+        if (!dq_dir.enabled || !dkv_dir.enabled) return LIBRA_ERR_PLAN_MISMATCH;
+        if (dkv_dir.tile != kBlk || dq_dir.tile != 2 * kBlk) return LIBRA_ERR_UNSUPPORTED;
+        if (dkv_dir.H != dims->hkv) return LIBRA_ERR_PLAN_MISMATCH;
+        if (dims->hq % dq_dir.H) return LIBRA_ERR_INVALID_ARG;
+        if (dkv_dir.W > plan->sm_count || dq_dir.W > plan->sm_count) return LIBRA_ERR_UNSUPPORTED;
+    }
     if (((uintptr_t)q_dev | (uintptr_t)k_dev | (uintptr_t)v_dev | (uintptr_t)out_dev | (uintptr_t)dout_dev |
          (uintptr_t)dq_dev | (uintptr_t)dk_dev | (uintptr_t)dv_dev) & 15)
         return LIBRA_ERR_INVALID_ARG;
@@ -704,7 +776,7 @@ extern "C" int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const v
 
     const int D = dims->head_dim;
     const int64_t T = plan->T;
-    const BwdWorkspace ws = bwd_workspace(T, dims->hq);
+    const BwdWorkspace ws = bwd_workspace(T, dims->hq, dims->hkv, D, fused);
     float* dvec = reinterpret_cast<float*>(workspace_dev);
     float* lse2 = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(workspace_dev) + ws.stat_bytes);
     cudaStream_t s = (cudaStream_t)stream;
@@ -733,6 +805,9 @@ extern "C" int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const v
     }
     time_end(mp0, 3, s);
     const float scale = dims->softmax_scale > 0.f ? dims->softmax_scale : 1.0f / sqrtf((float)D);
+    if (fused)
+        return launch_fused(q_dev, k_dev, v_dev, dout_dev, dq_dev, dk_dev, dv_dev, reinterpret_cast<uint8_t*>(workspace_dev),
+                            ws, plan, dims, scale, s);
     DkvParams pa;
     pa.dk = reinterpret_cast<__nv_bfloat16*>(dk_dev);
     pa.dv = reinterpret_cast<__nv_bfloat16*>(dv_dev);

@@ -547,6 +547,19 @@ int make_f32_2d_map(CUtensorMap* m, const void* base, int64_t rows, int64_t cols
     return r == CUDA_SUCCESS ? LIBRA_OK : LIBRA_ERR_CUDA;
 }
 
+int make_f32_3d_map(CUtensorMap* m, const void* base, int64_t T, int H, int d, int box_cols, int box_rows) {
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return LIBRA_ERR_CUDA;
+    cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)H, (cuuint64_t)T};
+    cuuint64_t strides[2] = {(cuuint64_t)d * 4, (cuuint64_t)H * d * 4};
+    cuuint32_t box[3] = {(cuuint32_t)box_cols, 1, (cuuint32_t)box_rows};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(base), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? LIBRA_OK : LIBRA_ERR_CUDA;
+}
+
 template <int D>
 static int launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtensorMap& tv, const FwdParams& prm, int W,
                       cudaStream_t s) {

@@ -50,9 +50,9 @@ struct libra_plan {
     int inject_stall = 0;            // test aid: the producer role issues no loads (libra_plan_inject_stall)
     int timing = 0;                  // record events around the main kernels
     // [kernel][slot][begin, end]: a ring of the most recent launches of each kernel (LIBRA_KERNEL_* - 1)
-    static constexpr int kTimedKernels = 4, kTimeRing = 64;
+    static constexpr int kTimedKernels = 6, kTimeRing = 64;
     cudaEvent_t ev[kTimedKernels][kTimeRing][2] = {};
-    int64_t ev_count[kTimedKernels] = {0, 0, 0, 0};   // launches recorded since timing was switched on
+    int64_t ev_count[kTimedKernels] = {0, 0, 0, 0, 0, 0};   // launches recorded since timing was switched on
 };
 
 namespace libra {
@@ -82,6 +82,8 @@ namespace libra {
 int make_thd_map(CUtensorMap* m, const void* base, int64_t T, int H, int d, int box_rows);
 // fp32 matrix [rows, cols] (cols contiguous); box = box_cols x box_rows, 128-byte swizzle.
 int make_f32_2d_map(CUtensorMap* m, const void* base, int64_t rows, int64_t cols, int box_cols, int box_rows);
+// fp32 tensor [T, H, d] viewed as (d, H, T); box = box_cols x 1 x box_rows, 128-byte swizzle.
+int make_f32_3d_map(CUtensorMap* m, const void* base, int64_t T, int H, int d, int box_cols, int box_rows);
 }  // namespace libra
 
 // setmaxnreg moves registers inside the pool the CTA got at launch (registers per thread as compiled x

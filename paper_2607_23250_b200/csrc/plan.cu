@@ -577,9 +577,11 @@ extern "C" int libra_plan_destroy(libra_plan_t* plan) {
 
 extern "C" int libra_busy_times(const libra_plan_t* plan, int which, uint64_t* ns_host) {
     if (!plan || !ns_host) return LIBRA_ERR_INVALID_ARG;
-    if (which < LIBRA_KERNEL_FWD || which > LIBRA_KERNEL_BWD_DQ) return LIBRA_ERR_INVALID_ARG;
-    // the forward and the dQ kernel walk the query-major lists, the dK/dV kernel the key-major ones
-    PlanDir* d = dir_of(plan, which == LIBRA_KERNEL_BWD_DKDV ? LIBRA_DIR_KV : LIBRA_DIR_Q);
+    if ((which < LIBRA_KERNEL_FWD || which > LIBRA_KERNEL_BWD_DQ) && which != LIBRA_KERNEL_BWD_FUSED) return LIBRA_ERR_INVALID_ARG;
+    // the forward and the dQ kernel walk the query-major lists, the dK/dV kernel the key-major ones, the fused
+    // backward the pair tiles
+    PlanDir* d = dir_of(plan, which == LIBRA_KERNEL_BWD_FUSED ? LIBRA_DIR_PAIR
+                                                              : (which == LIBRA_KERNEL_BWD_DKDV ? LIBRA_DIR_KV : LIBRA_DIR_Q));
     if (!d) return LIBRA_ERR_PLAN_MISMATCH;
     if (cudaDeviceSynchronize() != cudaSuccess) return LIBRA_ERR_CUDA;
     uint64_t* tmp = new (std::nothrow) uint64_t[2 * (size_t)d->W];
