@@ -2,6 +2,7 @@
 """Benchmark of the pool-attention hot path (plan reused; forward + backward per step).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config 2] [--impl ours|reference] [--sweep]
+                    [--backward fused|two-kernel]
 
 One step = one forward + backward pass of causal, sample-masked attention over one synthetic
 pool (default: the Qwen3-8B-shaped pool, 4 packed sequences x 32768 tokens, Hq 32 / Hkv 8 /
@@ -9,7 +10,8 @@ d 128).  The metric is useful TFLOP/s: 14 * d * Hq * sum_j l_j (l_j + 1) / 2 per
 by the step time (4 d per causal pair forward, 10 d backward).  With N > 1 (torchrun) the SAME
 pool is split over the ranks by attention heads (kv heads with their query heads; strong
 scaling, no data-path collective while N <= Hkv); `--replicas` runs one independent pool per
-rank instead (weak scaling).
+rank instead (weak scaling).  The backward runs in its fused form (one kernel over pair tiles, five GEMMs per cell)
+unless `--backward two-kernel` asks for the dK/dV + dQ pair of kernels (seven GEMMs per cell, bit-reproducible).
 
 Prints one JSON line (rank 0).  `--impl reference` times the CPU oracle on a bounded sample
 of the same workload instead.  `--sweep` prints a table over head shards x tile weights x pools.
@@ -33,7 +35,15 @@ sys.path.insert(0, ROOT)
 from paper_2607_23250_b200 import pools, sharding  # noqa: E402
 
 METRIC = "useful attention TFLOP/s fwd+bwd (sum of per-sample causal FLOPs)"
-KERNELS = ("fwd", "bwd_dkdv", "bwd_dq", "bwd_prep")
+
+
+def kernel_ids(lb, fused):
+    """name -> library kernel id of the launches of one step, and the names that keep per-CTA busy times."""
+    if fused:
+        return ({"fwd": lb.KERNEL_FWD, "bwd_prep": lb.KERNEL_BWD_PREP, "bwd_fused": lb.KERNEL_BWD_FUSED,
+                 "bwd_post": lb.KERNEL_BWD_POST}, ("fwd", "bwd_fused"))
+    return ({"fwd": lb.KERNEL_FWD, "bwd_prep": lb.KERNEL_BWD_PREP, "bwd_dkdv": lb.KERNEL_BWD_DKDV,
+             "bwd_dq": lb.KERNEL_BWD_DQ}, ("fwd", "bwd_dkdv", "bwd_dq"))
 
 
 def useful_flops(lengths, hq, d):
@@ -154,9 +164,10 @@ def time_oracle(spec, lengths, steps=1, warmup=0):
 class Pool:
     """Device tensors, plan and buffers of one pool (or of this rank's head slice of it)."""
 
-    def __init__(self, lb, spec, dev, shard=None, weight_model="pairs", heads=0, seed=0):
+    def __init__(self, lb, spec, dev, shard=None, weight_model="pairs", heads=0, seed=0, fused=True):
         import torch
         self.lb, self.spec, self.dev, self.shard = lb, spec, dev, shard
+        self.fused = fused and spec.head_dim == 128      # the fused backward exists for head_dim 128
         self.lengths = pools.pool_lengths(spec)
         cu_np = pools.cu_seqlens(self.lengths)
         T, d = spec.total_tokens, spec.head_dim
@@ -179,7 +190,9 @@ class Pool:
     def make_plan(self, blocks=None):
         lb = self.lb
         blocks = self.blocks if blocks is None else blocks
-        return lb.libra_plan_tiles(self.cu, self.heads, 256, tile_kv=128, n_heads_kv=self.hkv, total_tokens=self.T,
+        directions = lb.LIBRA_DIR_Q | (lb.LIBRA_DIR_PAIR if self.fused else lb.LIBRA_DIR_KV)
+        return lb.libra_plan_tiles(self.cu, self.heads, 256, directions=directions, tile_kv=128, n_heads_kv=self.hkv,
+                                   total_tokens=self.T,
                                    weight_model=lb.LIBRA_WEIGHT_BLOCKS if blocks else lb.LIBRA_WEIGHT_PAIRS,
                                    unit_cost_q=12 if blocks else 0, unit_cost_kv=6 if blocks else 0)
 
@@ -207,14 +220,16 @@ class Pool:
         self.step_on(self.inp, self.out, plan)
 
     def timed(self, steps, warmup, barrier, plan=None):
-        """(ms per step, per-kernel mean ms, busy max/mean per kernel) of `steps` steps between two events; the
-        library records its own events around every kernel inside the same loop."""
+        """(ms per step, per-kernel mean ms, busy max/mean per kernel, launches) of `steps` steps between two events;
+        the library records its own events around every kernel inside the same loop."""
         import torch
         lb, plan = self.lb, plan or self.plan
         for _ in range(warmup):
             self.step(plan)
         barrier()
         plan.set_timing(True)                          # fresh record: only the timed steps below
+        ids, with_busy = kernel_ids(lb, self.fused)
+        n0 = lb.launch_count()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for _ in range(steps):
@@ -222,12 +237,12 @@ class Pool:
         e1.record()
         barrier()
         ms = e0.elapsed_time(e1) / steps
-        kern = {n: statistics.mean(plan.kernel_times_ms(k)) for n, k in
-                zip(KERNELS, (lb.KERNEL_FWD, lb.KERNEL_BWD_DKDV, lb.KERNEL_BWD_DQ, lb.KERNEL_BWD_PREP))}
+        self.launches = lb.launch_count() - n0
+        kern = {n: statistics.mean(plan.kernel_times_ms(k)) for n, k in ids.items()}
         plan.set_timing(False)
         busy = {}
-        for n, k in zip(KERNELS[:3], (lb.KERNEL_FWD, lb.KERNEL_BWD_DKDV, lb.KERNEL_BWD_DQ)):
-            b = plan.busy_times(k).astype(np.float64)
+        for n in with_busy:
+            b = plan.busy_times(ids[n]).astype(np.float64)
             b = b[b > 0]
             busy[n] = round(float(b.max() / b.mean()), 4)
         return ms, kern, busy
@@ -265,7 +280,7 @@ def run_ours(args):
     shard = None if (args.replicas or world == 1) else sharding.head_groups(spec.hq, spec.hkv, world, rank)
     groups = {} if shard is None else sharding.kv_subgroups(spec.hq, spec.hkv, world)
     pool = Pool(lb, spec, dev, shard=shard, weight_model=args.weight_model, heads=args.heads,
-                seed=rank if args.replicas else 0)
+                seed=rank if args.replicas else 0, fused=args.backward == "fused")
     plan_ms = pool.build()
     kv_shared = shard is not None and len(shard.kv_sharers) > 1
 
@@ -288,9 +303,8 @@ def run_ours(args):
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    n0 = lb.launch_count()
     ms_local, kern, busy = pool.timed(args.steps, max(args.warmup, 3), barrier)
-    launches = lb.launch_count() - n0 - max(args.warmup, 3) * 4
+    launches = pool.launches
     clocks = sampler.stop() if rank == 0 else None
     ms_per_step, work = sharding.aggregate(ms_local, float(pool.ff + pool.fb), device=dev)
     value = work / (ms_per_step * 1e-3) / 1e12
@@ -337,7 +351,7 @@ def skewed_pools(args, lb, dev, barrier):
     for name, cfg, skew, steps in (("config3", 3, 0.0, 5), ("config5_skew0", 5, 0.0, 5), ("config5_skew0.25", 5, 0.25, 4),
                                    ("config5_skew0.5", 5, 0.5, 3), ("config5_skew1", 5, 1.0, 2), ("config4", 4, 0.0, 2)):
         spec = pools.config(cfg, skew)
-        pool = Pool(lb, spec, dev, weight_model=args.weight_model)
+        pool = Pool(lb, spec, dev, weight_model=args.weight_model, fused=args.backward == "fused")
         pool.build()
         ms, kern, busy = pool.timed(steps, 1 if cfg == 4 else 2, barrier)
         rec = pool_line(pool, ms, kern, busy)
@@ -415,12 +429,22 @@ def headline(args, world, spec, pool, value, ms_per_step, ms_local, kern, busy, 
     peaks = measured_peaks()
     hq, hkv, d, T = spec.hq, spec.hkv, spec.head_dim, spec.total_tokens
     ff, fb = pool.ff, pool.fb                      # this rank's heads
-    kf, kb, kq, kp = (kern[n] for n in KERNELS)
-    # Dominant kernel: the backward dK/dV kernel.  Algorithmic work per launch: the four GEMMs of the dK/dV
-    # gradient it owns (S, dP, dV, dK = 8 d flops per causal pair per query head).  It is timed inside the timed
-    # region; that region's length decides which measured peak applies (burst under a second, else sustained).
-    fa = fb * 8 // 10
-    ach = fa / (kb * 1e-3) / 1e12
+    kf = kern["fwd"]
+    bwd_ms = sum(v for n, v in kern.items() if n != "fwd")
+    # Dominant kernel: the backward's main kernel.  Algorithmic work per launch of the fused kernel: the five GEMMs
+    # of the gradient (S, dP, dV, dK, dQ = 10 d flops per causal pair per query head, all of them useful); of the
+    # dK/dV kernel of the two-kernel form: the four GEMMs it owns (8 d).  It is timed inside the timed region; that
+    # region's length decides which measured peak applies (burst under a second, else sustained).
+    if pool.fused:
+        dom, dom_ms, fa = "k_attn_bwd_fused", kern["bwd_fused"], fb
+        executed = {"fused (10 d per pair)": round(fb / kern["bwd_fused"] / 1e9, 1)}
+        ratio = "14 d / 14 d per causal pair (every GEMM of the gradient is computed once)"
+    else:
+        dom, dom_ms, fa = "k_attn_bwd_dkdv", kern["bwd_dkdv"], fb * 8 // 10
+        executed = {"dkdv (8 d per pair)": round(fa / kern["bwd_dkdv"] / 1e9, 1),
+                    "dq (6 d per pair)": round(fb * 6 // 10 / kern["bwd_dq"] / 1e9, 1)}
+        ratio = "18 d / 14 d per causal pair (S and dP are computed by both backward kernels)"
+    ach = fa / (dom_ms * 1e-3) / 1e12
     region_s = ms_local * args.steps * 1e-3
     kind = "burst" if region_s < 1.0 else "sustained"
     peak = peaks[kind]
@@ -432,6 +456,8 @@ def headline(args, world, spec, pool, value, ms_per_step, ms_local, kern, busy, 
         "config": {"workload": f"config {args.config}: {spec.name} pool, {spec.n_seqs} x {spec.seq_len} tokens, "
                                f"{len(pool.lengths)} samples (log-normal median 644, sigma 1.6), Hq {hq} / Hkv {hkv} / d {d}, "
                                f"causal per sample, fwd+bwd; plan built once and reused",
+                   "backward": ("fused: one kernel over pair tiles (key block x %d-token query chunk x kv head), fp32 "
+                                "accumulators" % pool.plan.export_pairs()[2]) if pool.fused else "two kernels (dK/dV, dQ)",
                    "tile_q": 256, "tile_kv": 128, "head_shards": pool.heads, "n_workers": pool.plan.info()["n_workers"],
                    "tile_weight": "blocks (time proxy)" if pool.blocks else "causal pairs (Eq. 6)",
                    "l2": "inputs larger than L2 (Q alone is %.2f GB per rank)" % (pool.inp["q"].numel() * 2 / 1e9),
@@ -444,27 +470,26 @@ def headline(args, world, spec, pool, value, ms_per_step, ms_local, kern, busy, 
                              "sustained_measured": round(100 * value / world / peaks["sustained"], 2),
                              "nominal_2250": round(100 * value / world / 2250.0, 2), "peaks": peaks["source"]},
         "kernel_ms_in_timed_loop": {n: round(v, 4) for n, v in kern.items()},
-        "kernel_ms_sum": round(kf + kb + kq + kp, 4),
+        "kernel_ms_sum": round(kf + bwd_ms, 4),
         "fwd_useful_tflops": round(ff / kf / 1e9, 1),
-        "bwd_useful_tflops": round(fb / (kb + kq + kp) / 1e9, 1),
-        "bwd_executed_tflops": {"dkdv (8 d per pair)": round(fa / kb / 1e9, 1), "dq (6 d per pair)": round(fb * 6 // 10 / kq / 1e9, 1)},
+        "bwd_useful_tflops": round(fb / bwd_ms / 1e9, 1),
+        "bwd_executed_tflops": executed,
         "busy_max_over_mean": busy,
         "clocks": clocks,
         "e2e": e2e,
         "gpu_launches": int(launches),
         "plan_ms": round(plan_ms, 3),
         "other_tile_weight": alt,
-        "roofline": {"bound": "tensor", "kernel": "k_attn_bwd_dkdv", "achieved": round(ach, 1),
+        "roofline": {"bound": "tensor", "kernel": dom, "achieved": round(ach, 1),
                      "peak": peak, "unit": "TFLOP/s", "frac": round(ach / peak, 4),
                      "peak_kind": f"bf16 {kind}, {peaks['source']} (timed region {region_s:.2f} s)",
-                     "traffic": read_traffic("k_attn_bwd_dkdv", args),
+                     "traffic": read_traffic(dom, args),
                      "frac_of_burst": round(ach / peaks["burst"], 4),
                      "frac_of_sustained": round(ach / peaks["sustained"], 4),
                      "whole_path": {"useful_tflops_per_gpu": round(value / world, 1),
                                     "frac_of_burst": round(value / world / peaks["burst"], 4),
                                     "frac_of_sustained": round(value / world / peaks["sustained"], 4),
-                                    "executed_over_useful_flops": "18 d / 14 d per causal pair (S and dP are computed by "
-                                                                  "both backward kernels)"}},
+                                    "executed_over_useful_flops": ratio}},
     }
     return line
 
@@ -502,20 +527,21 @@ def run_sweep(args):
         spec = pools.config(cfg, skew)
         for H in sorted({spec.hkv, 2 * spec.hkv, spec.hq}):
             for wm in ("pairs", "blocks"):
-                pool = Pool(lb, spec, dev, weight_model=wm, heads=H)
-                plan_ms = pool.build()
-                ms, kern, busy = pool.timed(steps, 2, barrier)
-                rec = pool_line(pool, ms, kern, busy)
-                rows.append((name, H, wm, rec, plan_ms))
-                pool.destroy()
-                del pool
-                torch.cuda.empty_cache()
-    print("| pool | head shards H | tile weight | useful TFLOP/s | ms/step | fwd ms | dK/dV ms | dQ ms | busy max/mean fwd | dK/dV | dQ | plan ms |")
-    print("|---|---|---|---|---|---|---|---|---|---|---|---|")
-    for name, H, wm, r, plan_ms in rows:
-        k, b = r["kernel_ms"], r["busy_max_over_mean"]
-        print(f"| {name} | {H} | {wm} | {r['useful_tflops']} | {r['ms_per_step']} | {k['fwd']} | {k['bwd_dkdv']} | "
-              f"{k['bwd_dq']} | {b['fwd']} | {b['bwd_dkdv']} | {b['bwd_dq']} | {plan_ms:.1f} |")
+                for fused in (False, True):
+                    pool = Pool(lb, spec, dev, weight_model=wm, heads=H, fused=fused)
+                    plan_ms = pool.build()
+                    ms, kern, busy = pool.timed(steps, 2, barrier)
+                    rec = pool_line(pool, ms, kern, busy)
+                    rows.append((name, H, wm, "fused" if fused else "two-kernel", rec, plan_ms))
+                    pool.destroy()
+                    del pool
+                    torch.cuda.empty_cache()
+    print("| pool | head shards H (forward, dQ) | tile weight | backward | useful TFLOP/s | ms/step | kernel ms | busy max/mean | plan ms |")
+    print("|---|---|---|---|---|---|---|---|---|")
+    for name, H, wm, form, r, plan_ms in rows:
+        k = ", ".join(f"{n} {v}" for n, v in r["kernel_ms"].items())
+        b = ", ".join(f"{n} {v}" for n, v in r["busy_max_over_mean"].items())
+        print(f"| {name} | {H} | {wm} | {form} | {r['useful_tflops']} | {r['ms_per_step']} | {k} | {b} | {plan_ms:.1f} |")
 
 
 def run_reference(args):
@@ -549,6 +575,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--weight-model", default="pairs", choices=["pairs", "blocks"],
                     help="tile weight of the plan: the paper's pair count, or the executed-block count")
+    ap.add_argument("--backward", default="fused", choices=["fused", "two-kernel"],
+                    help="backward form: one fused kernel over pair tiles (default) or the dK/dV + dQ kernels")
     ap.add_argument("--heads", type=int, default=0, help="head shards H of the query-major tiles (0 = one per query head)")
     ap.add_argument("--seqs", type=int, default=0, help="override the number of packed sequences (profiling runs)")
     ap.add_argument("--replicas", action="store_true", help="N > 1: one independent pool per rank instead of one pool split by heads")

@@ -177,8 +177,10 @@ int libra_attn_pool_fwd(const void* q_dev, const void* k_dev, const void* v_dev,
                         const int32_t* cu_seqlens_dev, const libra_plan_t* plan,
                         void* out_dev, float* lse_dev, const libra_dims* dims, void* stream);
 
-/* Bytes of caller-owned device scratch libra_attn_pool_bwd needs (the row statistics D and
- * LSE in log2 units, padded to a multiple of 128 rows); 0 on bad arguments. */
+/* Bytes of caller-owned device scratch libra_attn_pool_bwd needs; 0 on bad arguments.  Two-kernel form: the row
+ * statistics D and LSE in log2 units, padded to a multiple of 128 rows (2 * hq * round_up(T, 128) floats).
+ * Fused form (see below): in addition the fp32 accumulators of dQ (T * hq * 128 floats) and of dK and dV
+ * (T * hkv * 128 floats each). */
 size_t libra_attn_pool_bwd_workspace_bytes(const libra_plan_t* plan, const libra_dims* dims);
 
 /* Backward: the gradient of <dout, out> with respect to q, k, v, given out and lse from the
@@ -187,12 +189,20 @@ size_t libra_attn_pool_bwd_workspace_bytes(const libra_plan_t* plan, const libra
  *     P_ik = exp(scale <q_i,k_k> - lse_i), D_i = <dout_i, out_i>, dS_ik = P_ik (<dout_i,v_k> - D_i)
  *     dq_i = scale sum_k dS_ik k_k;  dk_k = scale sum_{h,i} dS_ik q_i;  dv_k = sum_{h,i} P_ik dout_i
  * (sums over the query heads h of the kv head's group and the rows i >= k of the sample).
- * Three launches: row statistics, a dK/dV kernel that walks the plan's key-major lists, and a
- * dQ kernel that walks its query-major lists; no atomics, so results are run-to-run identical.
- * Needs a plan with both directions: LIBRA_DIR_KV with tile_kv == 128 and n_heads_kv == hkv,
- * LIBRA_DIR_Q with tile_q == 256 and n_heads dividing hq.  `workspace_dev` must hold
- * libra_attn_pool_bwd_workspace_bytes bytes, 256-byte aligned; it is fully written inside the
- * call.  Errors: INVALID_ARG, UNSUPPORTED, PLAN_MISMATCH, CUDA.
+ * The plan decides between two forms of the same computation.
+ *   Two-kernel form (plan without pair tiles, or head_dim 64): three launches: row statistics, a dK/dV kernel
+ *   that walks the plan's key-major lists, and a dQ kernel that walks its query-major lists (S and dP are computed
+ *   by both, seven GEMMs per 128 x 128 cell); no atomics, so results are run-to-run identical.  Needs LIBRA_DIR_KV
+ *   with tile_kv == 128 and n_heads_kv == hkv, and LIBRA_DIR_Q with tile_q == 256 and n_heads dividing hq.
+ *   Fused form (plan with LIBRA_DIR_PAIR, tile_kv == 128, n_heads_kv == hkv, and head_dim 128): row statistics, one
+ *   kernel that walks the pair-tile lists and computes S, dP, dV, dK and dQ of a cell together (five GEMMs per
+ *   cell), and a conversion pass.  dK and dV of a pair tile accumulate on chip and are added to fp32 accumulators
+ *   in the workspace when the tile ends; dQ of every cell is added to its fp32 accumulator by bulk reduce-adds.
+ *   The accumulators are rounded to bf16 once, at the end, so the result is at least as accurate as the two-kernel
+ *   form's, but the order of the floating-point additions varies from run to run: results agree to rounding, not
+ *   bit for bit.  The other directions of the plan are not used by this form.
+ * `workspace_dev` must hold libra_attn_pool_bwd_workspace_bytes bytes, 256-byte aligned; every byte the call reads
+ * is written (or cleared) inside the call.  Errors: INVALID_ARG, UNSUPPORTED, PLAN_MISMATCH, CUDA.
  */
 int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const void* v_dev,
                         const void* out_dev, const float* lse_dev, const void* dout_dev,

@@ -29,9 +29,6 @@
 
 namespace libra {
 
-#define PROF_DECL
-#define PROF(k)
-#define PROF_FLUSH(cond, base)
 
 // warps 0-3, 4-7: exp groups (64 query columns each), 8-11: dS group, 12: TMA thread, 13: MMA thread,
 // 14-15 only hand their registers over
@@ -166,9 +163,6 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         abort_flag[1] = (int)p.wait_limit_ns;
         fence_mbar_init();
         p.busy[2 * cta] = globaltimer_ns();
-#ifdef LIBRA_TRACE
-        if (cta == 0) g_trace[0] = clock64();
-#endif
     }
     if (warp == kDkvMmaWarp) {
         tmem_alloc(tmem_slot, 512);
@@ -256,7 +250,6 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const uint32_t sb = smem_u32(smem);
             uint32_t ucnt = 0, it_all = 0;
             bool ok = true;
-            TRACE_DECL(17, cta == 0)
             // Base descriptors are built once; every MMA only adds a constant to them.
             const uint64_t kdesc0 = make_sdesc(sb, 16, 1024);             // K-major view of a tile at offset 0
             const uint64_t mdesc0 = make_sdesc(sb, L::kHalfBytes, 1024);  // MN-major view
@@ -281,10 +274,8 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             auto issue_dk = [&](uint32_t i, bool accumulate) -> bool {
                 if (!mbar_wait(bar_dsready, i & 1, abort_flag)) return false;
                 tc_fence_after();
-                TRACE(13)
                 issue_acc(kColDK, kColDS, L::kQOff + (i % QS) * L::kTileBytes, accumulate);
                 tc_commit(&bar_qempty[i % QS]);   // also tells the dS group that dS^T may be rewritten
-                TRACE(14)
                 return true;
             };
             for (int idx = unit_begin; idx < unit_end && ok; ++idx) {
@@ -303,7 +294,6 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 issue_kmajor(L::kKOff, L::kQOff + (it_all % QS) * L::kTileBytes);
                 tc_commit(bar_sfull);
                 for (int it = 0; it < n_it && ok; ++it, ++it_all) {
-                    TRACE(20)
                     const uint32_t ds = it_all % DS;
                     const uint32_t nx = it_all + 1;
                     const bool more = it + 1 < n_it;
@@ -315,7 +305,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     issue_kmajor(L::kVOff, L::kDoOff + ds * L::kTileBytes);
                     tc_commit(bar_dpfull);
                     if (!more) tc_commit(bar_kvempty);   // the unit's last readers of K and V: the next unit's K / V
-                    TRACE(15)                            // load overlaps the rest of this iteration
+                                                         // load overlaps the rest of this iteration
                     // dK(it-1): its dS^T was finished while S(it) ran
                     if (it > 0) { ok = issue_dk(it_all - 1, it > 1); if (!ok) break; }
                     // S(it+1) over dP(it), as soon as the dS group holds dP(it) in registers
@@ -326,7 +316,6 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         tc_fence_after();
                         issue_kmajor(L::kKOff, L::kQOff + (nx % QS) * L::kTileBytes);
                         tc_commit(bar_sfull);
-                        TRACE(12)
                     }
                     // dV(it) += P^T dO
                     ok = mbar_wait(bar_pready, it_all & 1, abort_flag);
@@ -334,11 +323,9 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         ok = mbar_wait(bar_dkvempty, (ucnt - 1) & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    TRACE(10)
                     issue_acc(kColDV, kColP, L::kDoOff + ds * L::kTileBytes, it > 0);
                     tc_commit(&bar_doempty[ds]);
                     tc_commit(bar_pfree);
-                    TRACE(11)
                 }
                 if (ok) ok = issue_dk(it_all - 1, n_it > 1);   // the unit's last dK
                 if (ok) tc_commit(bar_dkvfull);
@@ -356,14 +343,12 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         // as bf16) into dS^T.  The reads of region X are made by different warps for S^T and dP^T, so each happens
         // as soon as its MMA has landed.
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kDkvRegsDs));
-        const int r = (warp & 3) * 32 + lane;
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t t_x = tmem_base + lane_addr + kColX;
         const uint32_t t_p = tmem_base + lane_addr + kColP;
         const uint32_t t_ds = tmem_base + lane_addr + kColDS;
         uint32_t it_all = 0;
         bool ok = true;
-        TRACE_DECL(1 + warp, cta == 0 && lane == 0)
         for (int idx = unit_begin; idx < unit_end && ok; ++idx) {
             const int t = p.cta_tiles[idx];
             const int64_t k0 = (int64_t)(t / p.hkv) * kBlk;
@@ -377,7 +362,6 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 ok = warp_wait(&bar_dofull[ds], (it_all / DS) & 1, abort_flag) &&
                      warp_wait(bar_dpfull, it_all & 1, abort_flag);
                 if (!ok) break;
-                TRACE(4)
                 tc_fence_after();
                 uint32_t xs[64];   // (dP^T - D) as packed bf16 pairs
                 {
@@ -386,7 +370,6 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     tmem_ld_wait();
                     tc_fence_before();
                     mbar_arrive(bar_xfree2);   // dP^T(it) is in registers: S^T(it+1) may take the columns
-                    TRACE(9)
                     const uint64_t neg1 = f2_pack(-1.f, -1.f);
 #pragma unroll
                     for (int j = 0; j < 128; j += 4) {   // packed pairs: dP - D = fma(D, -1, dP)
@@ -398,13 +381,11 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                         xs[(j >> 1) + 1] = pack_bf16x2(b0, b1);
                     }
                 }
-                TRACE(22)
                 // dS^T(it-1) must have been consumed by dK(it-1) before its columns are rewritten
                 if (it_all > 0) {
                     ok = warp_wait(&bar_qempty[(it_all - 1) % QS], ((it_all - 1) / QS) & 1, abort_flag);
                     if (!ok) break;
                 }
-                TRACE(16)
                 // P^T arrives in the order the exp groups finish it: the first 32 queries of each group's 64
                 // (columns 0..15 and 32..47 of the packed P^T), then the rest.  dS^T = P^T o (dP^T - D) in bf16 pairs.
 #pragma unroll
@@ -412,7 +393,6 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     ok = warp_wait(half == 0 ? bar_phalf : bar_pready, it_all & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    if (half == 0) { TRACE(17) } else { TRACE(19) }
                     uint32_t pa[16], pb[16];
                     tmem_ld16(t_p + half * 16, pa);
                     tmem_ld16(t_p + 32 + half * 16, pb);
@@ -420,7 +400,6 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     if (half == 1) {           // all of P^T(it) is in registers
                         tc_fence_before();
                         mbar_arrive(bar_pfree);
-                        TRACE(21)
                     }
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
@@ -434,7 +413,6 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 tmem_st_wait();
                 tc_fence_before();
                 mbar_arrive(bar_dsready);
-                TRACE(5)
             }
         }
     } else {
@@ -447,7 +425,6 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         const uint32_t t_p = tmem_base + lane_addr + kColP;
         uint32_t ucnt = 0, it_all = 0;
         bool ok = true;
-        TRACE_DECL(1 + warp, cta == 0 && lane == 0)
         for (int idx = unit_begin; idx < unit_end && ok; ++idx) {
             const int t = p.cta_tiles[idx];
             const int kvh = t % p.hkv;
@@ -473,7 +450,6 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 ok = warp_wait(&bar_qfull[qs], (it_all / QS) & 1, abort_flag) &&
                      warp_wait(bar_sfull, it_all & 1, abort_flag);
                 if (!ok) break;
-                TRACE(2)
                 tc_fence_after();
                 uint32_t sv[64];
                 tmem_ld32(t_x + c0, sv);
@@ -481,13 +457,11 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                 tmem_ld_wait();
                 tc_fence_before();
                 mbar_arrive(bar_xfree1);   // S^T(it) is in registers: dP^T(it) may take the columns
-                TRACE(6)
                 // P^T(it-1) must have been consumed (dV(it-1), the dS group) before its columns are rewritten
                 if (it_all > 0) {
                     ok = warp_wait(bar_pfree, (it_all - 1) & 1, abort_flag);
                     if (!ok) break;
                 }
-                TRACE(7)
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
                     float pf[32];
@@ -517,9 +491,7 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     tmem_st_wait();
                     tc_fence_before();
                     mbar_arrive(half == 0 ? bar_phalf : bar_pready);
-                    if (half == 0) { TRACE(8) }
                 }
-                TRACE(3)
             }
             if (!ok) break;
             ++ucnt;
@@ -564,9 +536,6 @@ k_attn_bwd_dkdv(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     if (warp == kDkvMmaWarp) tmem_dealloc(tmem_base, 512);
     if (threadIdx.x == 0) {
         if (abort_flag[0]) atomicExch(p.status, LIBRA_ERR_TIMEOUT);
-#ifdef LIBRA_TRACE
-        if (cta == 0) g_trace[1] = clock64();
-#endif
         p.busy[2 * cta + 1] = globaltimer_ns();
     }
 }
@@ -681,11 +650,6 @@ static int launch_bwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtens
 
 using namespace libra;
 
-#ifdef LIBRA_TRACE
-extern "C" int libra_debug_trace(long long* host, int n) {
-    return cudaMemcpyFromSymbol(host, libra::g_trace, sizeof(long long) * n) == cudaSuccess ? 0 : -4;
-}
-#endif
 
 extern "C" size_t libra_attn_pool_bwd_workspace_bytes(const libra_plan_t* plan, const libra_dims* dims) {
     if (!plan || !dims || dims->hq <= 0 || dims->hkv <= 0 || (dims->head_dim != 64 && dims->head_dim != 128)) return 0;
@@ -719,7 +683,12 @@ static int launch_fused(const void* q_dev, const void* k_dev, const void* v_dev,
     if (rc != LIBRA_OK) return rc;
     if (!cfg_done(4)) {
         if (set_smem(k_attn_bwd_fused, FusedSmem::kBytes) != LIBRA_OK) return LIBRA_ERR_CUDA;
-        if (!regs_pool_ok(k_attn_bwd_fused, 128, kFuRegsDs, 128, kFuRegsOther)) return LIBRA_ERR_UNSUPPORTED;
+        {   // the register pool: what warps 12-15 release must cover what the exp and dS groups ask for
+            cudaFuncAttributes a;
+            if (cudaFuncGetAttributes(&a, k_attn_bwd_fused) != cudaSuccess) return LIBRA_ERR_CUDA;
+            const long long wanted = 256LL * (kFuRegsExp - a.numRegs) + 128LL * (kFuRegsDs - a.numRegs);
+            if (a.numRegs < kFuRegsOther || wanted > 128LL * (a.numRegs - kFuRegsOther)) return LIBRA_ERR_UNSUPPORTED;
+        }
         cfg_mark(4);
     }
     libra_plan_t* mp = const_cast<libra_plan_t*>(plan);

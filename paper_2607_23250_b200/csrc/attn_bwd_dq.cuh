@@ -18,9 +18,6 @@
 
 namespace libra {
 
-#ifndef LIBRA_TRACE_DQ
-#define LIBRA_TRACE_DQ 1   // trace builds: 0 leaves the trace buffer to the dK/dV kernel
-#endif
 #ifndef LIBRA_DQ_PREFETCH
 #define LIBRA_DQ_PREFETCH 0
 #endif
@@ -337,8 +334,6 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             const uint64_t mdesc0 = make_sdesc(sb, L::kHalfBytes, 1024);  // MN-major view
             uint32_t kcnt = 0, vcnt = 0, blk = 0;
             bool ok = true;
-            PROF_DECL
-            TRACE_DECL(0, cta == 0 && LIBRA_TRACE_DQ)
             // C[tmem d_col] = A[tmem a_col, bf16 packed over the head dimension] * B(K-major tile at b_off)^T
             auto issue_qk = [&](uint32_t d_col, uint32_t a_col, uint32_t b_off) {
                 const uint64_t db = sdesc_advance(kdesc0, b_off);
@@ -350,29 +345,21 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             };
             // S(j) from K ring entry kidx
             auto do_s = [&](uint32_t kidx) -> bool {
-                PROF(7)
                 if (!mbar_wait(&bar_kfull[kidx % L::kKStages], (kidx / L::kKStages) & 1, abort_flag)) return false;
-                PROF(0)
-                TRACE(1)
                 {
                     issue_qk(kColS, kColQ, L::kKOff + (kidx % L::kKStages) * L::kTileBytes);
                     tc_commit(bar_sfull);
                 }
-                TRACE(2)
                 return true;
             };
             auto do_dp = [&]() -> bool {
                 const uint32_t vs = vcnt % L::kVStages;
-                PROF(7)
                 if (!mbar_wait(&bar_vfull[vs], (vcnt / L::kVStages) & 1, abort_flag)) return false;
-                PROF(1)
-                TRACE(3)
                 {
                     issue_qk(kColDP, kColDO, L::kVOff + vs * L::kTileBytes);
                     tc_commit(bar_dpfull);
                     tc_commit(&bar_vempty[vs]);
                 }
-                TRACE(4)
                 ++vcnt;
                 return true;
             };
@@ -393,20 +380,16 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     const bool last = j == hi;
                     // S(j+1) as soon as the compute groups have read S(j)
                     if (!last) {
-                        PROF(7)
                         ok = mbar_wait(bar_sfree, blk & 1, abort_flag);
                         if (!ok) break;
-                        PROF(3)
                         tc_fence_after();
                         ok = do_s(kbase + (j + 1 - lo));
                         if (!ok) break;
                     }
                     // dQ += dS(j) K_j
-                    PROF(7)
                     ok = mbar_wait(bar_dsready, blk & 1, abort_flag);
                     if (ok && j == lo && ucnt > 0) ok = mbar_wait(bar_dqempty, (ucnt - 1) & 1, abort_flag);  // dQ read out
                     if (!ok) break;
-                    PROF(4)
                     tc_fence_after();
                     const uint32_t kidx = kbase + (j - lo);
                     {
@@ -424,22 +407,15 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                     } else if (nx.valid) {
                         // first block of the next unit, behind the last dQ of this one: its Q and dO rows
                         // were copied into TMEM while that dQ ran
-                        PROF(7)
-                        TRACE(21)
                         ok = mbar_wait(bar_sfree, blk & 1, abort_flag);
                         if (ok) ok = mbar_wait(bar_qtready, (ucnt + 1) & 1, abort_flag);
                         if (!ok) break;
-                        PROF(2)
-                        TRACE(22)
                         tc_fence_after();
                         ok = do_s(kbase + (hi - lo + 1));
-                        TRACE(23)
                         if (ok) ok = mbar_wait(bar_dotready, (ucnt + 1) & 1, abort_flag);
                         if (!ok) break;
-                        TRACE(24)
                         tc_fence_after();
                         ok = do_dp();
-                        TRACE(25)
                     }
                 }
                 kcnt = kbase + (hi - lo + 1);
@@ -465,8 +441,6 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
         const uint32_t t_dp = tmem_base + lane_addr + kColDP + CW * c;
         uint32_t ucnt = 0, blk = 0;
         bool ok = true;
-        PROF_DECL
-        TRACE_DECL(1 + warp, cta == 0 && lane == 0 && LIBRA_TRACE_DQ)
         // Copies this thread's row of Q or dO (its group's duty) of the unit whose tile has landed into TMEM.
         // The caller has seen every MMA that read the previous copy complete (s_full for Q, dp_full for dO).
         auto stage = [&](uint32_t parity) -> bool {
@@ -528,11 +502,8 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 const int c_lo = (row_ok ? kstart - k0 : kBlk) - CW * c;    // first visible column of this group's range
                 const int c_hi = (row_ok ? (int)(row - k0) : -1) - CW * c;  // last visible column
                 // ---- P = exp2(S c - LSE) ----
-                PROF(4)
                 ok = warp_wait(bar_sfull, blk & 1, abort_flag);
                 if (!ok) break;
-                PROF(0)
-                TRACE(10)
                 tc_fence_after();
                 uint32_t sv[CW];
 #pragma unroll
@@ -540,7 +511,6 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 tmem_ld_wait();
                 tc_fence_before();
                 mbar_arrive(bar_sfree);  // S(j+1) may overwrite the columns
-                TRACE(14)
                 float pf[CW];
 #pragma unroll
                 for (int i = 0; i < CW; i += 2) {
@@ -553,12 +523,8 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                         if (i < c_lo || i > c_hi) pf[i] = 0.f;
                 }
                 // ---- dS = P o (dP - D), packed over this half's own dP columns ----
-                PROF(1)
-                TRACE(11)
                 ok = warp_wait(bar_dpfull, blk & 1, abort_flag);
                 if (!ok) break;
-                PROF(2)
-                TRACE(12)
                 tc_fence_after();
                 uint32_t dpv[CW];
 #pragma unroll
@@ -578,25 +544,19 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
                 // Last block of the unit: every S and dP MMA that read this unit's Q / dO copy has completed, so
                 // the next unit's row goes into TMEM now, while the tensor pipe runs the last dQ.
                 if (j == hi && nx.valid) {
-                    TRACE(26)
                     ok = stage((ucnt + 1) & 1);
-                    TRACE(27)
                 }
-                PROF(3)
-                TRACE(13)
             }
             if (!ok) break;
             // ---- epilogue: dQ * scale to global ----
             ok = warp_wait(bar_dqfull, ucnt & 1, abort_flag);
             if (!ok) break;
-            TRACE(28)
             tc_fence_after();
             constexpr int kCols = D / kDqGroups;   // this group's dQ columns: kCols * 2 bytes of every row
             const uint32_t t_dq = tmem_base + lane_addr + kColDQ + c * kCols;
             uint32_t v[kCols];
             if constexpr (kCols == 32) tmem_ld32(t_dq, v); else tmem_ld16(t_dq, v);
             tmem_ld_wait();
-            TRACE(30)
             // The Q tile still holds the next unit's Q until every row of it has been copied to TMEM.
             if (nx.valid) ok = warp_wait(bar_qtready, (ucnt + 1) & 1, abort_flag);
             if (!ok) break;
@@ -617,12 +577,10 @@ k_attn_bwd_dq(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
             mbar_arrive(bar_dqstaged);
             tc_fence_before();
             mbar_arrive(bar_dqempty);  // the next unit's first dQ MMA may overwrite the accumulator
-            TRACE(29)
             ++ucnt;
             u = nx;
             cx = cx_next;
         }
-        PROF_FLUSH(threadIdx.x == 0, 512 * 24)
     }
 
     // ---------------- teardown ----------------

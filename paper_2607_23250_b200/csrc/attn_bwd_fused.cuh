@@ -14,9 +14,12 @@
 //   S^T  = K Q^T   (SS) -> X     P^T  = exp2(S^T c - LSE)      -> bf16, own TMEM columns    dV += P^T dO  (A in TMEM)
 //   dP^T = V dO^T  (SS) -> X     dS^T = P^T o (dP^T - D)       -> bf16, own TMEM columns    dK += dS^T Q  (A in TMEM)
 //                                                               and the same tile in shared memory:
-//   dQ   = dS K    (SS, A = the shared-memory dS^T read along its contiguous query axis) -> X
-// TMEM: X | P^T | dS^T | dK | dV = 128 + 64 + 64 + 128 + 128 columns; the fp32 region X is used three times per
-// iteration and is free again as soon as it has been READ: by the exp groups (S^T, then dQ) and the dS group (dP^T).
+//   dQ   = dS K    (SS, A = the shared-memory dS^T read along its contiguous query axis) -> Y
+// TMEM: X | Y | dK | dV = 128 + 128 + 128 + 128 columns.  X holds S^T, then dP^T (fp32), and is free again as soon
+// as it has been READ, so S^T(it+1) and dP^T(it+1) run ahead.  Y holds P^T and dS^T (bf16, 64 columns each) and,
+// once dV(it) and dK(it) have consumed them, receives dQ(it) (fp32, 128 columns: the MMAs run in issue order, so
+// the overwrite needs no extra barrier); P^T(it+1), already computed in registers, is written as soon as dQ(it) has
+// been read out.
 // Roles (512 threads): warps 0-3 and 4-7 exp groups (64 query columns of S^T each; 64 head-dim columns of dQ
 // each), 8-11 dS group, 12 TMA thread, 13 MMA thread, 14-15 only hand their registers over.
 #pragma once
@@ -25,7 +28,9 @@ namespace libra {
 
 constexpr int kFusedThreads = 512;
 constexpr int kFuTmaWarp = 12, kFuMmaWarp = 13;
-constexpr int kFuRegsDs = 200, kFuRegsOther = 56;
+// setmaxnreg budgets: 512 threads x 128 compiled registers = 256 x 144 (exp groups: P^T(it) and dQ(it-1) held
+// together) + 128 x 144 (dS group) + 128 x 80
+constexpr int kFuRegsExp = 144, kFuRegsDs = 144, kFuRegsOther = 80;
 
 struct FusedSmem {
     static constexpr int kTile = 32768;        // 128 x 128 bf16
@@ -36,13 +41,13 @@ struct FusedSmem {
     static constexpr int kQOff = 2 * kTile;
     static constexpr int kDoOff = kQOff + kQStages * kTile;
     static constexpr int kDsOff = kDoOff + kTile;          // dS^T tile (bf16, the operand layout of K / V tiles)
-    static constexpr int kStageOff = kDsOff + kTile;       // dQ staging: per warp two tiles of 32 rows x 32 floats, swizzled
+    static constexpr int kStageOff = kDsOff + kTile;       // dQ staging: per exp warp a tile of 32 rows x 32 floats, swizzled
     static constexpr int kLseOff = kStageOff + 2 * kHalf;  // per Q stage: lse2[128]
     static constexpr int kDvecOff = kLseOff + kQStages * 512;   // two buffers: dvec(it+1) lands while dvec(it) is read
     static constexpr int kBarOff = kDvecOff + 2 * 512;
     // kv_full, kv_empty, q_full[2], q_empty[2], do_full, do_empty, s_full, x_free1, dp_full, x_free2, dq_full,
-    // x_free3, p_half, p_ready, p_free, ds_ready, dss_free, dkv_full, dkv_empty, drain
-    static constexpr int kNumBars = 2 + 2 * kQStages + 18;
+    // y_free, p_half, p_ready, ds_ready, dkv_full, dkv_empty, drain
+    static constexpr int kNumBars = 2 + 2 * kQStages + 16;
     static constexpr int kMiscOff = kBarOff + kNumBars * 8;
     static constexpr int kBytes = kMiscOff + 16;
     static_assert(kBytes <= kSmemMax, "exceeds the shared memory of an sm_100 CTA");
@@ -96,6 +101,39 @@ __device__ __forceinline__ void tma_reduce_add_3d(const CUtensorMap* m, const vo
                  : "memory");
 }
 
+// dQ of one iteration: out of Y (query rows in lanes; this thread's 64 head-dim columns at `taddr`) into registers,
+// after which Y is released.
+__device__ __forceinline__ bool fused_read_dq(uint64_t* bar_dqfull, uint64_t* bar_yfree, uint32_t i, volatile int* ctl,
+                                              uint32_t taddr, uint32_t (&dqv)[64]) {
+    if (!warp_wait(bar_dqfull, i & 1, ctl)) return false;
+    tc_fence_after();
+    tmem_ld32(taddr, dqv);
+    tmem_ld32(taddr + 32, dqv + 32);
+    tmem_ld_wait();
+    tc_fence_before();
+    mbar_arrive(bar_yfree);
+    return true;
+}
+// ... and from the registers through the warp's staging tile (32 rows of 128 bytes, 128-byte swizzle) into the fp32
+// accumulator: one bulk tensor reduce-add of 32 head-dim columns (from column col0), rows row0 .. row0 + 31 of head h.
+// The reduce that last used the tile must have finished reading it.
+__device__ __forceinline__ void fused_stage_dq(const CUtensorMap* tm, uint8_t* stage, const uint32_t* dq, int lane,
+                                               int col0, int h, int row0) {
+    if (lane == 0) tma_store_wait_read();
+    __syncwarp();
+#pragma unroll
+    for (int ch = 0; ch < 8; ++ch) {
+        const int at = lane * 128 + ((ch ^ (lane & 7)) << 4);
+        *reinterpret_cast<uint4*>(stage + at) = make_uint4(dq[4 * ch], dq[4 * ch + 1], dq[4 * ch + 2], dq[4 * ch + 3]);
+    }
+    fence_proxy_async_smem();
+    __syncwarp();
+    if (lane == 0) {
+        tma_reduce_add_3d(tm, stage, col0, h, row0);
+        tma_store_commit();
+    }
+}
+
 __global__ void __launch_bounds__(kFusedThreads, 1)
 k_attn_bwd_fused(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
@@ -114,17 +152,15 @@ k_attn_bwd_fused(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     uint64_t* bar_sfull = b2 + 2;
     uint64_t* bar_xfree1 = b2 + 3;     // S^T(it) has been read out of X: dP^T(it) may overwrite it
     uint64_t* bar_dpfull = b2 + 4;
-    uint64_t* bar_xfree2 = b2 + 5;     // dP^T(it) has been read out: dQ(it) may overwrite it
-    uint64_t* bar_dqfull = b2 + 6;
-    uint64_t* bar_xfree3 = b2 + 7;     // dQ(it) has been read out: S^T(it+1) may overwrite it
+    uint64_t* bar_xfree2 = b2 + 5;     // dP^T(it) has been read out: S^T(it+1) may overwrite it
+    uint64_t* bar_dqfull = b2 + 6;     // dQ(it) is in Y (so dV(it), dK(it) and dQ(it) have all run)
+    uint64_t* bar_yfree = b2 + 7;      // dQ(it) has been read out of Y: P^T(it+1), then dS^T(it+1), may be written
     uint64_t* bar_phalf = b2 + 8;
     uint64_t* bar_pready = b2 + 9;
-    uint64_t* bar_pfree = b2 + 10;     // dV(it) has run and the dS group has read P^T(it)
-    uint64_t* bar_dsready = b2 + 11;   // dS^T(it) is in TMEM and in shared memory
-    uint64_t* bar_dssfree = b2 + 12;   // dQ(it) has run: the shared-memory dS^T tile is free
-    uint64_t* bar_dkvfull = b2 + 13;
-    uint64_t* bar_dkvempty = b2 + 14;
-    uint64_t* bar_drain = b2 + 15;
+    uint64_t* bar_dsready = b2 + 10;   // dS^T(it) is in TMEM and in shared memory
+    uint64_t* bar_dkvfull = b2 + 11;
+    uint64_t* bar_dkvempty = b2 + 12;
+    uint64_t* bar_drain = b2 + 13;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::kMiscOff);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kMiscOff + 4);
 
@@ -151,12 +187,10 @@ k_attn_bwd_fused(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         mbar_init(bar_dpfull, 1);
         mbar_init(bar_xfree2, 128);
         mbar_init(bar_dqfull, 1);
-        mbar_init(bar_xfree3, 128);
+        mbar_init(bar_yfree, 256);
         mbar_init(bar_phalf, 256);
         mbar_init(bar_pready, 256);
-        mbar_init(bar_pfree, 129);        // the dS group's 128 threads + the commit behind dV(it)
         mbar_init(bar_dsready, 128);
-        mbar_init(bar_dssfree, 1);
         mbar_init(bar_dkvfull, 1);
         mbar_init(bar_dkvempty, 256);
         mbar_init(bar_drain, 1);
@@ -180,7 +214,7 @@ k_attn_bwd_fused(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    constexpr uint32_t kColX = 0, kColP = 128, kColDS = 192, kColDK = 256, kColDV = 384;
+    constexpr uint32_t kColX = 0, kColY = 128, kColP = 128, kColDS = 192, kColDK = 256, kColDV = 384;
 
     const int unit_begin = p.cta_offsets[cta];
     const int unit_end = p.cta_offsets[cta + 1];
@@ -242,7 +276,6 @@ k_attn_bwd_fused(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             const uint32_t sb = smem_u32(smem);
             uint32_t ucnt = 0, it_all = 0;
             bool ok = true;
-            TRACE_DECL(17, cta == 0)
             const uint64_t kdesc0 = make_sdesc(sb, 16, 1024);          // K-major view of a tile at offset 0
             const uint64_t mdesc0 = make_sdesc(sb, L::kHalf, 1024);    // MN-major view
             auto issue_kmajor = [&](uint32_t a_off, uint32_t b_off) {
@@ -260,37 +293,37 @@ k_attn_bwd_fused(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                     mma_ts(tmem_base + d_col, tmem_base + a_col + kk * 8, sdesc_advance(db, kk * 2048), idesc_acc,
                            (accumulate || kk > 0) ? 1u : 0u);
             };
-            // dK(i) += dS^T(i) Q(i) from the TMEM copy of dS^T, i a CTA-wide iteration index (its dsready has been seen)
-            auto issue_dk = [&](uint32_t i, bool accumulate) {
-                issue_acc(kColDK, kColDS, L::kQOff + (i % QS) * L::kTile, accumulate);
-                tc_commit(&bar_qempty[i % QS]);   // also tells the dS group that the TMEM dS^T may be rewritten
-            };
             for (int idx = unit_begin; idx < unit_end && ok; ++idx) {
                 const FusedUnit u = fused_unit(p, p.cta_tiles[idx]);
                 const int n_it = G * u.n_blk;
                 ok = mbar_wait(bar_kvfull, ucnt & 1, abort_flag);
                 if (!ok) break;
-                // S(0): X is free once dQ of the previous unit's last iteration has been read
+                // S(0): X is free once dP of the previous unit's last iteration has been read
                 ok = mbar_wait(&bar_qfull[it_all % QS], (it_all / QS) & 1, abort_flag);
-                if (ok && it_all > 0) ok = mbar_wait(bar_xfree3, (it_all - 1) & 1, abort_flag);
+                if (ok && it_all > 0) ok = mbar_wait(bar_xfree2, (it_all - 1) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
                 issue_kmajor(L::kKOff, L::kQOff + (it_all % QS) * L::kTile);
                 tc_commit(bar_sfull);
                 for (int it = 0; it < n_it && ok; ++it, ++it_all) {
-                    TRACE(20)
                     const uint32_t nx = it_all + 1;
                     const bool more = it + 1 < n_it;
-                    // dP(it) over S(it)
+                    // dP(it) over S(it), as soon as the exp groups hold S(it) in registers
                     ok = mbar_wait(bar_dofull, it_all & 1, abort_flag);
                     if (ok) ok = mbar_wait(bar_xfree1, it_all & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
                     issue_kmajor(L::kVOff, L::kDoOff);
                     tc_commit(bar_dpfull);
-                    TRACE(15)
-                    // dK(it-1): its dS^T was seen ready when dQ(it-1) was issued
-                    if (it > 0) issue_dk(it_all - 1, it > 1);
+                    // S(it+1) over dP(it), as soon as the dS group holds dP(it) in registers
+                    if (more) {
+                        ok = mbar_wait(&bar_qfull[nx % QS], (nx / QS) & 1, abort_flag);
+                        if (ok) ok = mbar_wait(bar_xfree2, it_all & 1, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_kmajor(L::kKOff, L::kQOff + (nx % QS) * L::kTile);
+                        tc_commit(bar_sfull);
+                    }
                     // dV(it) += P^T dO
                     ok = mbar_wait(bar_pready, it_all & 1, abort_flag);
                     if (ok && it == 0 && ucnt > 0) ok = mbar_wait(bar_dkvempty, (ucnt - 1) & 1, abort_flag);
@@ -298,37 +331,21 @@ k_attn_bwd_fused(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                     tc_fence_after();
                     issue_acc(kColDV, kColP, L::kDoOff, it > 0);
                     tc_commit(bar_doempty);
-                    tc_commit(bar_pfree);
-                    TRACE(11)
-                    // dQ(it) = dS K over dP(it): dS^T is in shared memory, dP^T has been read out of X
+                    // dK(it) += dS^T Q from the TMEM copy of dS^T, then dQ(it) = dS K from the shared-memory copy,
+                    // into Y over P^T and dS^T: dV(it) and dK(it) precede it in issue order
                     ok = mbar_wait(bar_dsready, it_all & 1, abort_flag);
-                    if (ok) ok = mbar_wait(bar_xfree2, it_all & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
+                    issue_acc(kColDK, kColDS, L::kQOff + (it_all % QS) * L::kTile, it > 0);
+                    tc_commit(&bar_qempty[it_all % QS]);
                     {
                         const uint64_t da = sdesc_advance(mdesc0, L::kDsOff), db = sdesc_advance(mdesc0, L::kKOff);
 #pragma unroll
                         for (int kk = 0; kk < 8; ++kk)   // 16 keys per step
-                            mma_ss(tmem_base + kColX, sdesc_advance(da, kk * 2048), sdesc_advance(db, kk * 2048), idesc_dq, kk > 0);
+                            mma_ss(tmem_base + kColY, sdesc_advance(da, kk * 2048), sdesc_advance(db, kk * 2048), idesc_dq, kk > 0);
                         tc_commit(bar_dqfull);
-                        tc_commit(bar_dssfree);
-                        if (!more) tc_commit(bar_kvempty);   // the unit's last reader of K and V
-                        TRACE(16)
+                        if (!more) { tc_commit(bar_kvempty); tc_commit(bar_dkvfull); }   // the unit's last MMAs
                     }
-                    // S(it+1) over dQ(it), as soon as the exp groups hold dQ(it) in registers
-                    if (more) {
-                        ok = mbar_wait(&bar_qfull[nx % QS], (nx / QS) & 1, abort_flag);
-                        if (ok) ok = mbar_wait(bar_xfree3, it_all & 1, abort_flag);
-                        if (!ok) break;
-                        tc_fence_after();
-                        issue_kmajor(L::kKOff, L::kQOff + (nx % QS) * L::kTile);
-                        tc_commit(bar_sfull);
-                        TRACE(12)
-                    }
-                }
-                if (ok) {
-                    issue_dk(it_all - 1, n_it > 1);   // the unit's last dK
-                    tc_commit(bar_dkvfull);
                 }
                 ++ucnt;
             }
@@ -351,7 +368,6 @@ k_attn_bwd_fused(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         uint8_t* ds_row = smem + L::kDsOff + r * 128;
         uint32_t it_all = 0;
         bool ok = true;
-        TRACE_DECL(1 + warp, cta == 0 && lane == 0)
         for (int idx = unit_begin; idx < unit_end && ok; ++idx) {
             const FusedUnit u = fused_unit(p, p.cta_tiles[idx]);
             const int n_it = G * u.n_blk;
@@ -359,32 +375,33 @@ k_attn_bwd_fused(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 const float* dvec = reinterpret_cast<const float*>(smem + L::kDvecOff + (it_all & 1) * 512);
                 ok = warp_wait(bar_dofull, it_all & 1, abort_flag) && warp_wait(bar_dpfull, it_all & 1, abort_flag);
                 if (!ok) break;
-                TRACE(4)
                 tc_fence_after();
                 uint32_t xs[64];   // (dP^T - D) as packed bf16 pairs
                 {
-                    uint32_t dpv[128];
-                    tmem_ld128(t_x, dpv);
-                    tmem_ld_wait();
-                    tc_fence_before();
-                    mbar_arrive(bar_xfree2);   // dP^T(it) is in registers: dQ(it) may take the columns
                     const uint64_t neg1 = f2_pack(-1.f, -1.f);
 #pragma unroll
-                    for (int j = 0; j < 128; j += 4) {
-                        const ulonglong2 d4 = *reinterpret_cast<const ulonglong2*>(dvec + j);
-                        float a0, a1, b0, b1;
-                        f2_unpack(f2_fma(d4.x, neg1, f2_pack(__uint_as_float(dpv[j]), __uint_as_float(dpv[j + 1]))), a0, a1);
-                        f2_unpack(f2_fma(d4.y, neg1, f2_pack(__uint_as_float(dpv[j + 2]), __uint_as_float(dpv[j + 3]))), b0, b1);
-                        xs[j >> 1] = pack_bf16x2(a0, a1);
-                        xs[(j >> 1) + 1] = pack_bf16x2(b0, b1);
+                    for (int part = 0; part < 2; ++part) {   // 64 columns at a time keeps the live registers down
+                        uint32_t dpv[64];
+                        tmem_ld32(t_x + part * 64, dpv);
+                        tmem_ld32(t_x + part * 64 + 32, dpv + 32);
+                        tmem_ld_wait();
+                        if (part == 1) {
+                            tc_fence_before();
+                            mbar_arrive(bar_xfree2);   // dP^T(it) is in registers: S^T(it+1) may take the columns
+                        }
+#pragma unroll
+                        for (int j = 0; j < 64; j += 4) {
+                            const ulonglong2 d4 = *reinterpret_cast<const ulonglong2*>(dvec + part * 64 + j);
+                            float a0, a1, b0, b1;
+                            f2_unpack(f2_fma(d4.x, neg1, f2_pack(__uint_as_float(dpv[j]), __uint_as_float(dpv[j + 1]))), a0, a1);
+                            f2_unpack(f2_fma(d4.y, neg1, f2_pack(__uint_as_float(dpv[j + 2]), __uint_as_float(dpv[j + 3]))), b0, b1);
+                            xs[part * 32 + (j >> 1)] = pack_bf16x2(a0, a1);
+                            xs[part * 32 + (j >> 1) + 1] = pack_bf16x2(b0, b1);
+                        }
                     }
                 }
-                // the previous dS^T must have been consumed: by dK(it-1) (TMEM copy) and by dQ(it-1) (shared-memory copy)
-                if (it_all > 0) {
-                    ok = warp_wait(&bar_qempty[(it_all - 1) % QS], ((it_all - 1) / QS) & 1, abort_flag) &&
-                         warp_wait(bar_dssfree, (it_all - 1) & 1, abort_flag);
-                    if (!ok) break;
-                }
+                // P^T(it) only appears in Y after dQ(it-1) has been read out of it, and dQ(it-1) ran behind dK(it-1): by
+                // the time P^T(it) is seen, both copies of dS^T(it-1) have been consumed
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
                     ok = warp_wait(half == 0 ? bar_phalf : bar_pready, it_all & 1, abort_flag);
@@ -394,10 +411,6 @@ k_attn_bwd_fused(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                     tmem_ld16(t_p + half * 16, pa);
                     tmem_ld16(t_p + 32 + half * 16, pb);
                     tmem_ld_wait();
-                    if (half == 1) {
-                        tc_fence_before();
-                        mbar_arrive(bar_pfree);
-                    }
 #pragma unroll
                     for (int j = 0; j < 16; ++j) {
                         pa[j] = mul_bf16x2(pa[j], xs[half * 16 + j]);
@@ -421,65 +434,24 @@ k_attn_bwd_fused(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 fence_proxy_async_smem();     // the MMA reads the shared-memory tile through the async proxy
                 tc_fence_before();
                 mbar_arrive(bar_dsready);
-                TRACE(5)
-                // ---- dQ(it): out of X (query rows in lanes), through the two staging tiles in four rounds of 32
-                // head-dim columns, added to the fp32 accumulator by bulk tensor reduces ----
-                ok = warp_wait(bar_dqfull, it_all & 1, abort_flag);
-                if (!ok) break;
-                TRACE(6)
-                tc_fence_after();
-                uint32_t dqv[128];
-                tmem_ld128(t_x, dqv);
-                tmem_ld_wait();
-                tc_fence_before();
-                mbar_arrive(bar_xfree3);   // dQ(it) is in registers: S^T(it+1) may take the columns
-                const int h = u.kvh * G + it / u.n_blk;
-                const int qb = (u.i0 + it % u.n_blk) * kBlk;
-                // Each warp stages its own 32 rows (two 4 KB tiles used in turn) and one of its lanes issues the
-                // reduce, so no block-wide barrier is on this path.
-#ifdef LIBRA_X_NOSTAGE
-                if (dqv[5] == 0x12345678u) p.dq_acc[0] = 1.f;
-#else
-#pragma unroll
-                for (int round = 0; round < 4; ++round) {
-                    uint8_t* stage = smem + L::kStageOff + ((warp & 3) * 2 + (round & 1)) * 4096;
-                    // the reduce that last read this staging tile (two rounds ago) must have finished reading it
-                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-                    __syncwarp();
-#pragma unroll
-                    for (int ch = 0; ch < 8; ++ch)   // 32 floats of row `lane`: eight 16-byte chunks, 128-byte swizzle
-                        *reinterpret_cast<uint4*>(stage + lane * 128 + ((ch ^ (lane & 7)) << 4)) =
-                            make_uint4(dqv[round * 32 + 4 * ch], dqv[round * 32 + 4 * ch + 1], dqv[round * 32 + 4 * ch + 2],
-                                       dqv[round * 32 + 4 * ch + 3]);
-                    fence_proxy_async_smem();
-                    __syncwarp();
-#ifndef LIBRA_X_NOREDUCE
-                    if (lane == 0) {
-                        tma_reduce_add_3d(&tm_dqacc, stage, round * 32, h, qb + (warp & 3) * 32);
-                        tma_store_commit();
-                    }
-#endif
-                }
-#endif
-                TRACE(8)
             }
         }
-        // every bulk reduce this thread issued has completed before the CTA leaves
-        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     } else {
         // ---------------- exp groups ----------------
         // Thread r of group grp owns key row r and the query columns [64 grp, 64 grp + 64) of S^T; when dQ comes
-        // back in X (query rows in lanes) it owns query row r and the head-dim columns [64 grp, 64 grp + 64).
+        // back in Y (query rows in lanes) it owns query row r and the head-dim columns [64 grp, 64 grp + 64).
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kFuRegsExp));
         const int grp = warp >> 2;
         const int r = (warp & 3) * 32 + lane;
         const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
         const uint32_t t_x = tmem_base + lane_addr + kColX;
         const uint32_t t_p = tmem_base + lane_addr + kColP;
+        const uint32_t t_y = tmem_base + lane_addr + kColY;
         const int c0 = 64 * grp;
         const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2), neg1 = f2_pack(-1.f, -1.f);
+        uint8_t* stage = smem + L::kStageOff + warp * 4096;   // this warp's staging tile: 32 rows x 32 floats
         uint32_t ucnt = 0, it_all = 0;
         bool ok = true;
-        TRACE_DECL(1 + warp, cta == 0 && lane == 0)
         for (int idx = unit_begin; idx < unit_end && ok; ++idx) {
             const FusedUnit u = fused_unit(p, p.cta_tiles[idx]);
             const int n_it = G * u.n_blk;
@@ -488,7 +460,9 @@ k_attn_bwd_fused(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             const int kend = key_ok ? p.tok_end[key] : 0;
             const int min_kend = p.tok_end[u.k0];
             const bool partial = u.k0 + kBlk > p.T;
+            int prev_h = 0, prev_qb = 0;
             for (int it = 0; it < n_it && ok; ++it, ++it_all) {
+                const int h = u.kvh * G + it / u.n_blk;
                 const int qb = (u.i0 + it % u.n_blk) * kBlk;
                 const uint32_t qs = it_all % QS;
                 const float* lse2 = reinterpret_cast<const float*>(smem + L::kLseOff + qs * 512) + c0;
@@ -497,51 +471,74 @@ k_attn_bwd_fused(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                 const int j_hi = kend - 1 - qb - c0;
                 ok = warp_wait(&bar_qfull[qs], (it_all / QS) & 1, abort_flag) && warp_wait(bar_sfull, it_all & 1, abort_flag);
                 if (!ok) break;
-                TRACE(2)
                 tc_fence_after();
-                uint32_t sv[64];
-                tmem_ld32(t_x + c0, sv);
-                tmem_ld32(t_x + c0 + 32, sv + 32);
-                tmem_ld_wait();
-                tc_fence_before();
-                mbar_arrive(bar_xfree1);
-                if (it_all > 0) {
-                    ok = warp_wait(bar_pfree, (it_all - 1) & 1, abort_flag);
+                uint32_t pk[32];   // P^T(it) of this thread's 64 queries, packed, kept until Y is free
+                {
+                    uint32_t sv[64];
+                    tmem_ld32(t_x + c0, sv);
+                    tmem_ld32(t_x + c0 + 32, sv + 32);
+                    tmem_ld_wait();
+                    tc_fence_before();
+                    mbar_arrive(bar_xfree1);
+#pragma unroll
+                    for (int half = 0; half < 2; ++half) {
+                        float pf[32];
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            const int jj = half * 32 + j;
+                            const ulonglong2 l4 = *reinterpret_cast<const ulonglong2*>(lse2 + jj);
+                            float x0, x1, x2, x3;
+                            f2_unpack(f2_fma(f2_pack(__uint_as_float(sv[jj]), __uint_as_float(sv[jj + 1])), scale2,
+                                             f2_mul(l4.x, neg1)), x0, x1);
+                            f2_unpack(f2_fma(f2_pack(__uint_as_float(sv[jj + 2]), __uint_as_float(sv[jj + 3])), scale2,
+                                             f2_mul(l4.y, neg1)), x2, x3);
+                            pf[j] = ex2_approx(x0);
+                            pf[j + 1] = ex2_approx(x1);
+                            pf[j + 2] = ex2_approx(x2);
+                            pf[j + 3] = ex2_approx(x3);
+                        }
+                        if (need_mask) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (half * 32 + j < j_lo || half * 32 + j > j_hi) pf[j] = 0.f;
+                        }
+#pragma unroll
+                        for (int j = 0; j < 32; j += 2) pk[half * 16 + (j >> 1)] = pack_bf16x2(pf[j], pf[j + 1]);
+                    }
+                }
+                // dQ(it-1) leaves Y (its MMA ran behind dV(it-1) and dK(it-1), so P^T(it-1) and dS^T(it-1) are spent)
+                uint32_t dqv[64];   // this thread's share of dQ(it-1): head-dim columns c0 .. c0 + 63 of query row r
+                if (it > 0) {
+                    ok = fused_read_dq(bar_dqfull, bar_yfree, it_all - 1, abort_flag, t_y + c0, dqv);
                     if (!ok) break;
                 }
-#pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    float pf[32];
-#pragma unroll
-                    for (int j = 0; j < 32; j += 4) {
-                        const int jj = half * 32 + j;
-                        const ulonglong2 l4 = *reinterpret_cast<const ulonglong2*>(lse2 + jj);
-                        float x0, x1, x2, x3;
-                        f2_unpack(f2_fma(f2_pack(__uint_as_float(sv[jj]), __uint_as_float(sv[jj + 1])), scale2,
-                                         f2_mul(l4.x, neg1)), x0, x1);
-                        f2_unpack(f2_fma(f2_pack(__uint_as_float(sv[jj + 2]), __uint_as_float(sv[jj + 3])), scale2,
-                                         f2_mul(l4.y, neg1)), x2, x3);
-                        pf[j] = ex2_approx(x0);
-                        pf[j + 1] = ex2_approx(x1);
-                        pf[j + 2] = ex2_approx(x2);
-                        pf[j + 3] = ex2_approx(x3);
-                    }
-                    if (need_mask) {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (half * 32 + j < j_lo || half * 32 + j > j_hi) pf[j] = 0.f;
-                    }
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int j = 0; j < 32; j += 2) pk[j >> 1] = pack_bf16x2(pf[j], pf[j + 1]);
-                    tmem_st16(t_p + c0 / 2 + half * 16, pk);
-                    tmem_st_wait();
-                    tc_fence_before();
-                    mbar_arrive(half == 0 ? bar_phalf : bar_pready);
+                if (it_all > 0) {   // every exp thread has read its part of the last dQ: Y is free
+                    ok = warp_wait(bar_yfree, (it_all - 1) & 1, abort_flag);
+                    if (!ok) break;
                 }
-                TRACE(3)
+                tc_fence_after();
+                tmem_st16(t_p + c0 / 2, pk);
+                tmem_st16(t_p + c0 / 2 + 16, pk + 16);
+                tmem_st_wait();
+                tc_fence_before();
+                mbar_arrive(bar_phalf);
+                mbar_arrive(bar_pready);
+                if (it > 0) {
+                    fused_stage_dq(&tm_dqacc, stage, dqv, lane, c0, prev_h, prev_qb + (warp & 3) * 32);
+                    fused_stage_dq(&tm_dqacc, stage, dqv + 32, lane, c0 + 32, prev_h, prev_qb + (warp & 3) * 32);
+                }
+                prev_h = h;
+                prev_qb = qb;
             }
             if (!ok) break;
+            // the unit's last dQ, then its dK and dV
+            {
+                uint32_t dqv[64];
+                ok = fused_read_dq(bar_dqfull, bar_yfree, it_all - 1, abort_flag, t_y + c0, dqv);
+                if (!ok) break;
+                fused_stage_dq(&tm_dqacc, stage, dqv, lane, c0, prev_h, prev_qb + (warp & 3) * 32);
+                fused_stage_dq(&tm_dqacc, stage, dqv + 32, lane, c0 + 32, prev_h, prev_qb + (warp & 3) * 32);
+            }
             ++ucnt;
             // ---- unit epilogue: dK and dV of the pair tile are added to the fp32 accumulators ----
             ok = warp_wait(bar_dkvfull, (ucnt - 1) & 1, abort_flag);
@@ -571,6 +568,8 @@ k_attn_bwd_fused(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             tc_fence_before();
             mbar_arrive(bar_dkvempty);
         }
+        // every bulk reduce this warp issued has completed before the CTA leaves
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
     }
 
     // ---------------- teardown ----------------

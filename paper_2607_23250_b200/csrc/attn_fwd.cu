@@ -76,23 +76,6 @@ __device__ __forceinline__ SlotRange slot_range(const int32_t* tok_start, int64_
 }
 
 
-#ifdef LIBRA_PROF
-__device__ unsigned long long g_fwd_prof[1024 * 24];
-struct FProf {
-    long long last;
-    unsigned long long acc[8];
-    __device__ void start() { last = clock64(); for (int i = 0; i < 8; ++i) acc[i] = 0; }
-    __device__ void mark(int k) { const long long now = clock64(); acc[k] += now - last; last = now; }
-    __device__ void flush(int cta, int base) { for (int i = 0; i < 8; ++i) g_fwd_prof[cta * 24 + base + i] = acc[i]; }
-};
-#define PROF_DECL FProf prof; prof.start();
-#define PROF(k) prof.mark(k);
-#define PROF_FLUSH(cond, base) if (cond) prof.flush(cta, base);
-#else
-#define PROF_DECL
-#define PROF(k)
-#define PROF_FLUSH(cond, base)
-#endif
 
 template <int D>
 __global__ void __launch_bounds__(kFwdThreads, 1)
@@ -221,8 +204,6 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         uint32_t ring = 0, qcnt = 0;
         uint32_t pcnt[2] = {0, 0};
         bool ok = true;
-        PROF_DECL
-        TRACE_DECL(0, cta == 0 && leader)
         // Base descriptors are built once; every MMA only adds a constant to them.
         const uint64_t desc_q = make_sdesc(smem_base + L::kQOff, 16, 1024);                  // K-major Q slot 0
         const uint64_t desc_k = make_sdesc(smem_base + L::kRingOff, 16, 1024);               // K-major ring stage 0
@@ -254,12 +235,8 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             const bool act1 = r[1].lo <= r[1].hi;
             const int lo = r[0].lo, hi = act1 ? r[1].hi : r[0].hi;
             for (int hh = 0; hh < heads_per_shard && ok; ++hh) {
-                PROF(7)
-                TRACE(21)
                 ok = warp_wait(bar_qfull, qcnt & 1, abort_flag);
                 if (!ok) break;
-                PROF(0)
-                TRACE(22)
                 ++qcnt;
                 // prologue: S(lo)
                 uint32_t st = ring % L::kStages;
@@ -272,42 +249,33 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                     tc_commit(&bar_empty[st]);
                     if (lo == hi) tc_commit(bar_qempty);  // no later MMA of this tile reads Q
                 }
-                TRACE(23)
                 ++ring;
                 for (int j = lo; j <= hi && ok; ++j) {
-                    TRACE(20)
                     const uint32_t st_v = ring % L::kStages;
-                    PROF(7)
                     ok = warp_wait(&bar_full[st_v], (ring / L::kStages) & 1, abort_flag);
                     if (!ok) break;
-                    PROF(1)
                     ++ring;
                     uint32_t st_k = 0;
                     if (j + 1 <= hi) {
                         st_k = ring % L::kStages;
                         ok = warp_wait(&bar_full[st_k], (ring / L::kStages) & 1, abort_flag);
                         if (!ok) break;
-                        PROF(2)
                         ++ring;
                     }
                     for (int g = 0; g < 2 && ok; ++g) {
                         if (j >= r[g].lo && j <= r[g].hi) {
-                            PROF(7)
                             ok = warp_wait(&bar_phalf[g], pcnt[g] & 1, abort_flag);   // P of keys 0..63
                             if (!ok) break;
                             tc_fence_after();
                             if (leader) issue_pv(g, st_v, j != r[g].lo, 0, kBN / 32);
                             ok = warp_wait(&bar_pready[g], pcnt[g] & 1, abort_flag);  // the rest, while those MMAs run
                             if (!ok) break;
-                            PROF(3 + g)
                             ++pcnt[g];
                             tc_fence_after();
                             if (leader) issue_pv(g, st_v, j != r[g].lo, kBN / 32, kBN / 16);
-                            TRACE(10 + g)
                         }
                         if (j + 1 <= hi && j + 1 >= r[g].lo && j + 1 <= r[g].hi) {
                             if (leader) issue_s(g, st_k);
-                            TRACE(12 + g)
                         }
                     }
                     if (!ok) break;
@@ -336,8 +304,6 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
         const uint32_t t_o = tmem_base + lane_addr + 2 * kBN + g * D;
         uint32_t scnt = 0, ocnt = 0;
         bool ok = true;
-        PROF_DECL
-        TRACE_DECL(1 + g, cta == 0 && (warp & 3) == 0 && lane == 0)
         for (int idx = tile_begin; idx < tile_end && ok; ++idx) {
             const int t = p.cta_tiles[idx];
             const int64_t qs = (int64_t)(t / p.H) * (2 * kBM) + g * kBM;
@@ -353,11 +319,8 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 const int h = (t % p.H) * heads_per_shard + hh;
                 float m_ref = -INFINITY, l_sum = 0.f;
                 for (int j = rg.lo; j <= rg.hi && ok; ++j) {
-                    PROF(3)
                     ok = warp_wait(&bar_sfull[g], scnt & 1, abort_flag);
                     if (!ok) break;
-                    TRACE(2)
-                    PROF(0)
                     ++scnt;
                     tc_fence_after();
                     uint32_t sr[kBN];
@@ -366,7 +329,6 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                     tmem_ld32(t_s + 64, sr + 64);
                     tmem_ld32(t_s + 96, sr + 96);
                     tmem_ld_wait();
-                    PROF(4)
                     const int k0 = j * kBN;
                     const bool need_mask = (k0 + kBN - 1 > qs) || (k0 < max_kstart) || !row_ok;
                     if (need_mask) {
@@ -414,7 +376,6 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                             tmem_st32(t_o + c, orow);
                         }
                     }
-                    PROF(5)
                     l_sum *= factor;
                     m_ref = m_new;
                     const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
@@ -445,21 +406,15 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                         f2_unpack(f2_add(f2_add(psum2[0], psum2[1]), f2_add(psum2[2], psum2[3])), a, b);
                         l_sum += a + b;
                     }
-                    PROF(6)
                     tmem_st_wait();
                     tc_fence_before();
                     mbar_arrive(&bar_pready[g]);
-                    TRACE(3)
-                    PROF(1)
                     ++ocnt;
                 }
                 if (!ok) break;
                 // epilogue: wait for the last PV, normalise, store
-                TRACE(24)
                 ok = warp_wait(&bar_odone[g], (ocnt - 1) & 1, abort_flag);
                 if (!ok) break;
-                PROF(2)
-                TRACE(25)
                 tc_fence_after();
                 const float inv_l = (l_sum > 0.f) ? 1.0f / l_sum : 0.f;
                 __nv_bfloat16* orow_ptr = p.out + ((size_t)row * p.hq + h) * D;
@@ -485,11 +440,8 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 // the next PV into this slot's O may only start after these reads: it is issued
                 // after this group's next p_ready arrival, which follows in program order
                 tc_fence_before();
-                TRACE(26)
             }
         }
-        PROF_FLUSH(threadIdx.x == 0, 0)
-        PROF_FLUSH(threadIdx.x == 128, 16)
     }
 
     // ---------------- teardown ----------------
@@ -580,11 +532,6 @@ static int launch_fwd(const CUtensorMap& tq, const CUtensorMap& tk, const CUtens
 
 using namespace libra;
 
-#ifdef LIBRA_PROF
-extern "C" int libra_debug_fwd_prof(unsigned long long* host, int n) {
-    return cudaMemcpyFromSymbol(host, libra::g_fwd_prof, sizeof(unsigned long long) * n) == cudaSuccess ? 0 : -4;
-}
-#endif
 
 extern "C" int libra_attn_pool_fwd(const void* q_dev, const void* k_dev, const void* v_dev,
                                    const int32_t* cu_seqlens_dev, const libra_plan_t* plan, void* out_dev,
@@ -633,8 +580,3 @@ extern "C" int libra_attn_pool_fwd(const void* q_dev, const void* k_dev, const v
     return rc;
 }
 
-#ifdef LIBRA_TRACE
-extern "C" int libra_debug_trace_fwd(long long* host, int n) {
-    return cudaMemcpyFromSymbol(host, libra::g_trace, sizeof(long long) * n) == cudaSuccess ? 0 : -4;
-}
-#endif

@@ -333,24 +333,5 @@ __device__ __forceinline__ uint32_t mul_bf16x2(uint32_t a, uint32_t b) {
     return d;
 }
 
-#ifdef LIBRA_TRACE
-// Trace build only: raw (event id, clock) pairs of one thread per role in CTA 0.
-__device__ long long g_trace[18 * 4096 * 2];
-struct Trace {
-    int n, role, on;
-    __device__ void init(int r, bool enable) { n = 0; role = r; on = enable; }
-    __device__ void ev(int id) {
-        if (on && n < 4096) { g_trace[(role * 4096 + n) * 2] = id; g_trace[(role * 4096 + n) * 2 + 1] = clock64(); ++n; }
-    }
-};
-#define TRACE_DECL(role, cond) Trace tr; tr.init(role, cond);
-#ifndef LIBRA_TRACE_MASK
-#define LIBRA_TRACE_MASK 0xffffffffu
-#endif
-#define TRACE(id) if ((LIBRA_TRACE_MASK >> (id)) & 1u) tr.ev(id);
-#else
-#define TRACE_DECL(role, cond)
-#define TRACE(id)
-#endif
 
 }  // namespace libra

@@ -1,6 +1,7 @@
 """Full-size parity: the Qwen3-8B-shaped pool in the launch configuration the benchmark times, the 30B-shaped
 pool with Pareto-tailed samples, the 1M-token pool with one 262144-token sample (Hq 64 / Hkv 4: sixteen query
-heads per kv head, tensors beyond 2^32 bytes) and the skew sweep of 65536-token sequences at every skew.
+heads per kv head, tensors beyond 2^32 bytes) and the skew sweep of 65536-token sequences at every skew.  The
+"fused" cases run the same pools with a pair-tile plan, which makes the backward call take its fused form.
 
 The whole oracle would take minutes here, so outputs are sampled: rows of O / LSE / dQ and
 columns of dK / dV are recomputed one by one by the CPU oracle on the (sample, kv-head group)
@@ -25,25 +26,30 @@ def _rel(got, want, floor=1e-3):
     return float(np.abs(np.asarray(got, np.float64) - want).max() / max(np.abs(want).max(), floor))
 
 
-@pytest.fixture(scope="module", params=[(2, 0.0), (3, 0.0), (4, 0.0), (5, 0.0), (5, 0.25), (5, 0.5), (5, 1.0)],
-                ids=["config2", "config3", "config4", "config5_skew0", "config5_skew0.25", "config5_skew0.5",
-                     "config5_skew1"])
+@pytest.fixture(scope="module",
+                params=[(2, 0.0, False), (2, 0.0, True), (3, 0.0, False), (3, 0.0, True), (4, 0.0, False), (4, 0.0, True),
+                        (5, 0.0, False), (5, 0.25, False), (5, 0.5, False), (5, 1.0, False), (5, 1.0, True)],
+                ids=["config2", "config2_fused", "config3", "config3_fused", "config4", "config4_fused",
+                     "config5_skew0", "config5_skew0.25", "config5_skew0.5", "config5_skew1", "config5_skew1_fused"])
 def run(request):
     from paper_2607_23250_b200 import binding as lb
-    spec = pools.config(*request.param)
+    fused = request.param[2]
+    spec = pools.config(*request.param[:2])
     lengths = pools.pool_lengths(spec)
     cu_np = pools.cu_seqlens(lengths)
     T, hq, hkv, d = spec.total_tokens, spec.hq, spec.hkv, spec.head_dim
     t = pools.make_tensors(T, hq, hkv, d, seed=0, device="cuda")
     cu = torch.from_numpy(cu_np).cuda()
-    plan = lb.libra_plan_tiles(cu, hq, 256, tile_kv=128, n_heads_kv=hkv, total_tokens=T)   # as bench.py
+    directions = lb.LIBRA_DIR_Q | (lb.LIBRA_DIR_PAIR if fused else lb.LIBRA_DIR_KV)
+    plan = lb.libra_plan_tiles(cu, hq, 256, directions=directions, tile_kv=128, n_heads_kv=hkv,
+                               total_tokens=T)                                             # as bench.py
     assert plan.status() == 0
     out, lse = lb.libra_attn_pool_fwd(t["q"], t["k"], t["v"], plan)
     dq, dk, dv = lb.libra_attn_pool_bwd(t["q"], t["k"], t["v"], out, lse, t["dout"], plan)
     torch.cuda.synchronize()
-    for kern in (lb.KERNEL_FWD, lb.KERNEL_BWD_DKDV, lb.KERNEL_BWD_DQ):
+    for kern in (lb.KERNEL_FWD,) + ((lb.KERNEL_BWD_FUSED,) if fused else (lb.KERNEL_BWD_DKDV, lb.KERNEL_BWD_DQ)):
         plan.busy_times(kern)
-    res = dict(spec=spec, lengths=lengths, cu=cu_np, t=t, out=out, lse=lse, dq=dq, dk=dk, dv=dv, plan=plan, lb=lb)
+    res = dict(fused=fused, spec=spec, lengths=lengths, cu=cu_np, t=t, out=out, lse=lse, dq=dq, dk=dk, dv=dv, plan=plan, lb=lb)
     yield res
     plan.destroy()
     del res
@@ -67,6 +73,8 @@ def _sub(run, j, kvh, heads=None, lo=0):
 def test_plan_matches_oracle_at_full_size(run):
     lb, plan, spec = run["lb"], run["plan"], run["spec"]
     for direction, d_or, tile, H in ((lb.LIBRA_DIR_Q, 0, 256, spec.hq), (lb.LIBRA_DIR_KV, 1, 128, spec.hkv)):
+        if direction == lb.LIBRA_DIR_KV and run["fused"]:
+            continue
         got = plan.export(direction)
         want = oracle.plan(run["cu"], H, tile, plan.info(direction)["n_workers"], d_or)
         for key in ("weight", "order", "cta_of_tile", "cta_offsets", "cta_tiles", "loads"):
@@ -166,8 +174,14 @@ def test_whole_tensor_properties(run):
     firsts = torch.from_numpy(cu[:-1].astype(np.int64)).cuda()
     v_first = t["v"][firsts].float().repeat_interleave(G, dim=1)
     assert torch.equal(run["out"][firsts].float(), v_first)
-    # same call again gives bit-identical results (no atomics anywhere on the path)
     lb, plan = run["lb"], run["plan"]
     dq2, dk2, dv2 = lb.libra_attn_pool_bwd(t["q"], t["k"], t["v"], run["out"], run["lse"], t["dout"], plan)
     torch.cuda.synchronize()
-    assert torch.equal(dq2, run["dq"]) and torch.equal(dk2, run["dk"]) and torch.equal(dv2, run["dv"])
+    if not run["fused"]:
+        # the two-kernel form has no atomics anywhere: the same call again gives bit-identical results
+        assert torch.equal(dq2, run["dq"]) and torch.equal(dk2, run["dk"]) and torch.equal(dv2, run["dv"])
+    else:
+        # the fused form adds into fp32 accumulators in a varying order: equal up to the final bf16 rounding
+        for a, b in ((dq2, run["dq"]), (dk2, run["dk"]), (dv2, run["dv"])):
+            diff = float((a[:: 7].float() - b[:: 7].float()).abs().max())
+            assert diff <= 2.0 ** -7 * float(b[:: 7].float().abs().max())

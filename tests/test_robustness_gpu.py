@@ -139,3 +139,36 @@ def test_attention_kernels_give_up_cleanly_when_their_producer_stalls():
     for g, r in zip((dq, dk, dv), ref):
         assert np.abs(g.float().cpu().numpy() - r).max() <= 5e-2 * np.abs(r).max()
     plan.destroy()
+
+
+def test_fused_backward_gives_up_cleanly_when_its_producer_stalls():
+    """The same injected stall for the fused backward (plan with pair tiles): TIMEOUT is reported, the context
+    stays usable, and the next launch with the injection off is correct."""
+    import oracle
+    from paper_2607_23250_b200 import binding as lb
+    lengths = [300, 200, 524]
+    hq, hkv, d = 4, 2, 128
+    cu_np = pools.cu_seqlens(lengths)
+    t = pools.make_tensors(int(cu_np[-1]), hq, hkv, d, seed=4)
+    q, k, v, dout = (t[n].cuda() for n in ("q", "k", "v", "dout"))
+    plan = lb.libra_plan_tiles(torch.from_numpy(cu_np).cuda(), hq, 256, directions=lb.LIBRA_DIR_Q | lb.LIBRA_DIR_PAIR,
+                               tile_kv=128, n_heads_kv=hkv)
+    assert plan.status() == 0
+    out, lse = lb.libra_attn_pool_fwd(q, k, v, plan)
+    plan.set_wait_limit_ns(200_000)                                # 0.2 ms
+    plan.inject_stall(True)
+    lb.libra_attn_pool_bwd(q, k, v, out, lse, dout, plan)
+    with pytest.raises(lb.LibraError) as err:
+        plan.busy_times(lb.KERNEL_BWD_FUSED)
+    assert err.value.code == lb.ERR_TIMEOUT
+    plan.inject_stall(False)
+    plan.set_wait_limit_ns(0)
+    dq, dk, dv = lb.libra_attn_pool_bwd(q, k, v, out, lse, dout, plan)
+    torch.cuda.synchronize()
+    plan.busy_times(lb.KERNEL_BWD_FUSED)
+    f = {n: t[n].float().numpy() for n in t}
+    o_ref, l_ref = oracle.attn_fwd(f["q"], f["k"], f["v"], cu_np)
+    ref = oracle.attn_bwd(f["q"], f["k"], f["v"], o_ref, l_ref, f["dout"], cu_np)
+    for g, r in zip((dq, dk, dv), ref):
+        assert np.abs(g.float().cpu().numpy() - r).max() <= 5e-2 * np.abs(r).max()
+    plan.destroy()
