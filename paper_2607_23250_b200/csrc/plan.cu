@@ -118,11 +118,13 @@ __global__ void k_rank_blocks(const int64_t* __restrict__ weight_blk, int64_t NB
     if (b < NB) blk_order[rank] = (int32_t)b;
 }
 
-// Sequential placement by one warp.  Worker r's load lives in lane r % 32, register r / 32.
-// Per tile: every lane finds its lightest worker, two warp reductions find the warp's
-// (load, index) minimum, the owning lane adds the weight.  Ties go to the lowest index
-// because the comparison is lexicographic on (load, index).  Loads stay below 2^53 (checked on the
-// host from the weight total), so load * 1024 + index fits 64 bits.
+// Sequential placement by one warp.  Worker r's load lives in lane r / PER, register r % PER, so among equal
+// loads the lowest worker index is the lowest slot of the lowest lane.  Per tile: one warp reduction finds the
+// lightest load, a ballot finds the lowest lane that holds it, and that lane adds the weight to its lightest slot
+// and picks its new lightest.  The reduction runs on 32-bit loads relative to a moving base (the loads of a greedy
+// placement never spread by more than the heaviest tile, which is checked to be below 2^31 first; the base follows
+// the minimum whenever that passes 2^30), exact 64-bit loads are kept beside them.  With a heavier tile than that the
+// same steps run on the 64-bit loads themselves (two reductions per tile).
 template <int PER>
 __global__ void __launch_bounds__(32) k_place(const int64_t* __restrict__ weight_blk,
                                               const int32_t* __restrict__ blk_order /* null: tiles in id order, id =
@@ -130,18 +132,27 @@ __global__ void __launch_bounds__(32) k_place(const int64_t* __restrict__ weight
                                               int32_t* __restrict__ cta_of_tile, int32_t* __restrict__ pos,
                                               int32_t* __restrict__ cta_offsets, int64_t* __restrict__ loads) {
     const int lane = threadIdx.x;
-    // key[k] = load * 1024 + worker index of worker lane + 32 k (all ones: no such worker); the lane's
-    // lightest worker is kept up to date, so a placement only recomputes it in the lane that changed
-    uint64_t key[PER];
+    int64_t wmax = 0;
+    for (int64_t b = lane; b < NB; b += 32) wmax = weight_blk[b] > wmax ? weight_blk[b] : wmax;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const int64_t other = __shfl_xor_sync(0xffffffffu, wmax, o);
+        wmax = other > wmax ? other : wmax;
+    }
+    const bool narrow = wmax < ((int64_t)1 << 31);
+    int64_t load[PER];      // exact loads of workers lane * PER + k
+    uint32_t rel[PER];      // narrow form: load - base; all ones: no such worker
     int32_t cnt[PER];
 #pragma unroll
-    for (int i = 0; i < PER; ++i) {
-        key[i] = (lane + 32 * i < W) ? (uint64_t)(lane + 32 * i) : ~0ull;
-        cnt[i] = 0;
+    for (int k = 0; k < PER; ++k) {
+        load[k] = 0;
+        cnt[k] = 0;
+        rel[k] = (lane * PER + k < W) ? 0u : 0xffffffffu;
     }
-    uint64_t best = key[0];
-#pragma unroll
-    for (int k = 1; k < PER; ++k) best = key[k] < best ? key[k] : best;
+    // the lane's lightest slot (lowest slot among equals)
+    uint32_t best = rel[0];
+    int64_t best64 = rel[0] == 0xffffffffu ? INT64_MAX : 0;
+    int slot = 0;
     for (int64_t x0 = 0; x0 < NT; x0 += 32) {
         // each lane fetches one upcoming tile, then they are broadcast one by one
         const int64_t xl = x0 + lane;
@@ -161,30 +172,50 @@ __global__ void __launch_bounds__(32) k_place(const int64_t* __restrict__ weight
         for (int i = 0; i < lim; ++i) {
             const int64_t w = __shfl_sync(0xffffffffu, w_l, i);
             const int32_t t = __shfl_sync(0xffffffffu, t_l, i);
-            // lexicographic (load, worker) minimum over the warp: two hardware reductions, high word first,
-            // then the low word among the lanes that tie on it
-            const uint32_t hi = (uint32_t)(best >> 32), lo = (uint32_t)best;
-            const uint32_t mhi = __reduce_min_sync(0xffffffffu, hi);
-            const uint32_t mlo = __reduce_min_sync(0xffffffffu, hi == mhi ? lo : 0xffffffffu);
-            const int32_t bidx = (int32_t)(mlo & 1023u);
-            if ((bidx & 31) == lane) {
+            unsigned tie;
+            if (narrow) {
+                uint32_t m = __reduce_min_sync(0xffffffffu, best);
+                if (m > (1u << 30)) {   // move the base up to the minimum (uniform branch)
+#pragma unroll
+                    for (int k = 0; k < PER; ++k)
+                        if (rel[k] != 0xffffffffu) rel[k] -= m;
+                    if (best != 0xffffffffu) best -= m;
+                    m = 0;
+                }
+                tie = __ballot_sync(0xffffffffu, best == m);
+            } else {
+                const uint32_t hi = (uint32_t)((uint64_t)best64 >> 32), lo = (uint32_t)best64;
+                const uint32_t mhi = __reduce_min_sync(0xffffffffu, hi);
+                const uint32_t mlo = __reduce_min_sync(0xffffffffu, hi == mhi ? lo : 0xffffffffu);
+                tie = __ballot_sync(0xffffffffu, hi == mhi && lo == mlo);
+            }
+            if (lane == __ffs(tie) - 1) {
                 int32_t my_pos = 0;
 #pragma unroll
                 for (int k = 0; k < PER; ++k) {
-                    if (k == (bidx >> 5)) { key[k] += (uint64_t)w << 10; my_pos = cnt[k]++; }
+                    if (k == slot) { load[k] += w; rel[k] += (uint32_t)w; my_pos = cnt[k]++; }
                 }
-                best = key[0];
-#pragma unroll
-                for (int k = 1; k < PER; ++k) best = key[k] < best ? key[k] : best;
-                cta_of_tile[t] = bidx;
+                cta_of_tile[t] = lane * PER + slot;
                 pos[t] = my_pos;
+                if (narrow) {
+                    best = rel[0];
+                    slot = 0;
+#pragma unroll
+                    for (int k = 1; k < PER; ++k)
+                        if (rel[k] < best) { best = rel[k]; slot = k; }
+                } else {
+                    best64 = INT64_MAX;
+#pragma unroll
+                    for (int k = PER - 1; k >= 0; --k)
+                        if (lane * PER + k < W && load[k] <= best64) { best64 = load[k]; slot = k; }
+                }
             }
         }
     }
 #pragma unroll
-    for (int i = 0; i < PER; ++i) {
-        const int r = lane + 32 * i;
-        if (r < W) { loads[r] = (int64_t)(key[i] >> 10); cta_offsets[r + 1] = cnt[i]; }
+    for (int k = 0; k < PER; ++k) {
+        const int r = lane * PER + k;
+        if (r < W) { loads[r] = load[k]; cta_offsets[r + 1] = cnt[k]; }
     }
     __syncwarp();
     if (lane == 0) {  // counts -> offsets
