@@ -1,12 +1,15 @@
 // Backward pool attention for sm_100a.
 //
-// Three launches: (1) prep: D_i = <dO_i, O_i> and LSE in log2 units, padded to a multiple of 128
-// rows; (2) the dK/dV kernel over key-major tiles; (3) the dQ kernel over query-major tiles.
-// Splitting dQ off costs two extra GEMMs per block pair (S and dP are recomputed) but needs no
-// cross-CTA reduction at all: no fp32 dQ accumulator, no atomics, no shared-memory staging, and
-// the result is deterministic.  Both kernels are persistent and warp-specialised (compute warpgroups,
-// one TMA thread, one MMA-issuing thread; the dQ kernel also has a store thread) and keep their
-// accumulators in TMEM.
+// Two forms of the same computation; the plan decides (see libra_attn_pool_bwd in the public header).
+// Fused form (attn_bwd_fused.cuh, plans with pair tiles, head_dim 128): row statistics, ONE kernel that computes
+// S, dP, dV, dK and dQ of every 128 x 128 cell together (five GEMMs) with fp32 accumulators in global memory,
+// and a conversion pass.
+// Two-kernel form (this file and attn_bwd_dq.cuh): (1) prep: D_i = <dO_i, O_i> and LSE in log2 units, padded
+// to a multiple of 128 rows; (2) the dK/dV kernel over key-major tiles; (3) the dQ kernel over query-major
+// tiles.  Splitting dQ off costs two extra GEMMs per cell (S and dP are recomputed) but needs no cross-CTA
+// reduction at all: no fp32 accumulator, no atomics, and the result is deterministic.  All kernels are persistent
+// and warp-specialised (compute warpgroups, one TMA thread, one MMA-issuing thread; the dQ kernel also has a
+// store thread) and keep their accumulators in TMEM.
 //
 // dK/dV kernel: a unit is 128 keys x one kv head; K and V stay in shared memory, dK and dV in
 // TMEM, while the CTA streams every (query head of the group, 128-row query block) that sees the
