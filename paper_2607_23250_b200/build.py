@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 SO = os.path.join(HERE, "liblibra.so")
-SOURCES = ["plan.cu", "attn_fwd.cu", "attn_bwd.cu", "no_alloc.cu", "vrsp.cu", "tap.cu", "selftest.cu"]
+SOURCES = ["plan.cu", "attn_fwd.cu", "attn_bwd.cu", "attn_d256.cu", "no_alloc.cu", "vrsp.cu", "tap.cu", "selftest.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xptxas", "-v"]
 

@@ -42,13 +42,6 @@ constexpr int kBlk = 128;
 constexpr int kSmemMax = 232448;  // 227 KB per CTA on sm_100
 constexpr uint64_t kDrainNs = 2000000;  // teardown after a give-up: budget for work already in flight to land
 
-__device__ __forceinline__ void bulk_load_1d(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                     smem_u32(smem_dst)),
-                 "l"(reinterpret_cast<uint64_t>(gsrc)), "r"(bytes), "r"(smem_u32(bar))
-                 : "memory");
-}
-
 // =================================================================================================
 // dK / dV kernel
 // =================================================================================================
@@ -655,7 +648,9 @@ using namespace libra;
 
 
 extern "C" size_t libra_attn_pool_bwd_workspace_bytes(const libra_plan_t* plan, const libra_dims* dims) {
-    if (!plan || !dims || dims->hq <= 0 || dims->hkv <= 0 || (dims->head_dim != 64 && dims->head_dim != 128)) return 0;
+    if (!plan || !dims || dims->hq <= 0 || dims->hkv <= 0 ||
+        (dims->head_dim != 64 && dims->head_dim != 128 && dims->head_dim != 256))
+        return 0;
     return bwd_workspace(plan->T, dims->hq, dims->hkv, dims->head_dim, use_fused(plan, dims)).total;
 }
 
@@ -728,7 +723,7 @@ extern "C" int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const v
         !dk_dev || !dv_dev || !workspace_dev || !dims)
         return LIBRA_ERR_INVALID_ARG;
     if (dims->hq <= 0 || dims->hkv <= 0 || dims->hq % dims->hkv) return LIBRA_ERR_INVALID_ARG;
-    if (dims->head_dim != 64 && dims->head_dim != 128) return LIBRA_ERR_UNSUPPORTED;
+    if (dims->head_dim != 64 && dims->head_dim != 128 && dims->head_dim != 256) return LIBRA_ERR_UNSUPPORTED;
     const PlanDir& dq_dir = plan->dir[0];
     const PlanDir& dkv_dir = plan->dir[1];
     const bool fused = use_fused(plan, dims);
@@ -754,6 +749,17 @@ extern "C" int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const v
     cudaStream_t s = (cudaStream_t)stream;
     cudaMemsetAsync(plan->d_status + 2, 0, sizeof(int), s);   // the word reports the most recent launch
 
+    const float scale = dims->softmax_scale > 0.f ? dims->softmax_scale : 1.0f / sqrtf((float)D);
+    if (D == 256) {   // row statistics, then the three passes of the 256-wide kernel
+        libra_plan_t* mp256 = const_cast<libra_plan_t*>(plan);
+        time_begin(mp256, 3, s);
+        const int64_t warps = ws.Tpad / 32 * dims->hq;
+        k_bwd_prep<256><<<(unsigned)((warps * 32 + 255) / 256), 256, 0, s>>>(
+            (const __nv_bfloat16*)out_dev, (const __nv_bfloat16*)dout_dev, lse_dev, T, ws.Tpad, dims->hq, dvec, lse2);
+        count_launch();
+        time_end(mp256, 3, s);
+        return launch_bwd_d256(q_dev, k_dev, v_dev, dout_dev, dq_dev, dk_dev, dv_dev, lse2, dvec, ws.Tpad, plan, dims, scale, s);
+    }
     CUtensorMap tq, tk, tv, tdo, tdq;
     int rc = make_thd_map(&tq, q_dev, T, dims->hq, D, kBlk);
     if (rc == LIBRA_OK) rc = make_thd_map(&tk, k_dev, T, dims->hkv, D, kBlk);
@@ -776,7 +782,6 @@ extern "C" int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const v
         count_launch();
     }
     time_end(mp0, 3, s);
-    const float scale = dims->softmax_scale > 0.f ? dims->softmax_scale : 1.0f / sqrtf((float)D);
     if (fused)
         return launch_fused(q_dev, k_dev, v_dev, dout_dev, dq_dev, dk_dev, dv_dev, reinterpret_cast<uint8_t*>(workspace_dev),
                             ws, plan, dims, scale, s);

@@ -539,7 +539,7 @@ extern "C" int libra_attn_pool_fwd(const void* q_dev, const void* k_dev, const v
     if (!q_dev || !k_dev || !v_dev || !cu_seqlens_dev || !plan || !out_dev || !lse_dev || !dims)
         return LIBRA_ERR_INVALID_ARG;
     if (dims->hq <= 0 || dims->hkv <= 0 || dims->hq % dims->hkv) return LIBRA_ERR_INVALID_ARG;
-    if (dims->head_dim != 64 && dims->head_dim != 128) return LIBRA_ERR_UNSUPPORTED;
+    if (dims->head_dim != 64 && dims->head_dim != 128 && dims->head_dim != 256) return LIBRA_ERR_UNSUPPORTED;
     const PlanDir& d = plan->dir[0];
     if (!d.enabled || plan->T != dims->total_tokens) return LIBRA_ERR_PLAN_MISMATCH;
     if (d.tile != 2 * kBM) return LIBRA_ERR_UNSUPPORTED;
@@ -548,6 +548,16 @@ extern "C" int libra_attn_pool_fwd(const void* q_dev, const void* k_dev, const v
     if (((uintptr_t)q_dev | (uintptr_t)k_dev | (uintptr_t)v_dev | (uintptr_t)out_dev) & 15) return LIBRA_ERR_INVALID_ARG;
     if (int rcd = check_plan_device(plan); rcd != LIBRA_OK) return rcd;
 
+    const float scale = dims->softmax_scale > 0.f ? dims->softmax_scale : 1.0f / sqrtf((float)dims->head_dim);
+    cudaStream_t s = (cudaStream_t)stream;
+    libra_plan_t* mp = const_cast<libra_plan_t*>(plan);
+    if (dims->head_dim == 256) {
+        cudaMemsetAsync(plan->d_status + 1, 0, sizeof(int), s);
+        time_begin(mp, 0, s);
+        const int rc256 = launch_fwd_d256(q_dev, k_dev, v_dev, out_dev, lse_dev, plan, dims, scale, s);
+        time_end(mp, 0, s);
+        return rc256;
+    }
     CUtensorMap tq, tk, tv;
     int rc = make_thd_map(&tq, q_dev, plan->T, dims->hq, dims->head_dim, kBM);
     if (rc == LIBRA_OK) rc = make_thd_map(&tk, k_dev, plan->T, dims->hkv, dims->head_dim, kBN);
@@ -564,16 +574,13 @@ extern "C" int libra_attn_pool_fwd(const void* q_dev, const void* k_dev, const v
     prm.hq = dims->hq;
     prm.hkv = dims->hkv;
     prm.H = d.H;
-    const float scale = dims->softmax_scale > 0.f ? dims->softmax_scale : 1.0f / sqrtf((float)dims->head_dim);
     prm.scale_log2 = scale * 1.4426950408889634f;
     prm.status = plan->d_status + 1;
     prm.plan_status = plan->d_status;
     prm.wait_limit_ns = plan->wait_limit_ns;
     prm.inject_stall = plan->inject_stall;
     prm.busy = d.d_busy;
-    cudaStream_t s = (cudaStream_t)stream;
     cudaMemsetAsync(plan->d_status + 1, 0, sizeof(int), s);   // the word reports the most recent launch
-    libra_plan_t* mp = const_cast<libra_plan_t*>(plan);
     time_begin(mp, 0, s);
     rc = dims->head_dim == 128 ? launch_fwd<128>(tq, tk, tv, prm, d.W, s) : launch_fwd<64>(tq, tk, tv, prm, d.W, s);
     time_end(mp, 0, s);

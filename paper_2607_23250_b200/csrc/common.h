@@ -84,6 +84,13 @@ int make_thd_map(CUtensorMap* m, const void* base, int64_t T, int H, int d, int 
 int make_f32_2d_map(CUtensorMap* m, const void* base, int64_t rows, int64_t cols, int box_cols, int box_rows);
 // fp32 tensor [T, H, d] viewed as (d, H, T); box = box_cols x 1 x box_rows, 128-byte swizzle.
 int make_f32_3d_map(CUtensorMap* m, const void* base, int64_t T, int H, int d, int box_cols, int box_rows);
+// head_dim 256 (attn_d256.cu): the forward over the plan's query-major lists; the three gradient passes over
+// its key-major (dV, dK) and query-major (dQ) lists, given the row statistics lse2 / dvec [Hq, Tpad].
+int launch_fwd_d256(const void* q, const void* k, const void* v, void* out, float* lse, const libra_plan* plan,
+                    const libra_dims* dims, float scale, cudaStream_t s);
+int launch_bwd_d256(const void* q, const void* k, const void* v, const void* dout, void* dq, void* dk, void* dv,
+                    const float* lse2, const float* dvec, int64_t Tpad, const libra_plan* plan, const libra_dims* dims,
+                    float scale, cudaStream_t s);
 }  // namespace libra
 
 // setmaxnreg moves registers inside the pool the CTA got at launch (registers per thread as compiled x

@@ -48,7 +48,7 @@ extern "C" int libra_attn_pool_bwd_noalloc(const void* q_dev, const void* k_dev,
     if (!plan || !dims) return LIBRA_ERR_INVALID_ARG;
     // the same verdicts, in the same order, as the regular entry point gives for bad dimensions
     if (dims->hq <= 0 || dims->hkv <= 0 || dims->hq % dims->hkv) return LIBRA_ERR_INVALID_ARG;
-    if (dims->head_dim != 64 && dims->head_dim != 128) return LIBRA_ERR_UNSUPPORTED;
+    if (dims->head_dim != 64 && dims->head_dim != 128 && dims->head_dim != 256) return LIBRA_ERR_UNSUPPORTED;
     const size_t need = libra_attn_pool_bwd_workspace_bytes(plan, dims);
     if (need == 0) return LIBRA_ERR_INVALID_ARG;
     if (need > kMaxScratchFloats * sizeof(float)) return LIBRA_ERR_SCRATCH_TOO_SMALL;
