@@ -345,11 +345,13 @@ def run_ours(args):
 
 def skewed_pools(args, lb, dev, barrier):
     """The pools that carry the busy-time target: the 30B-shaped pool with Pareto-tailed samples, the 1M-token
-    pool with one 262144-token sample, and the skew sweep at every skew; a few steps each."""
+    pool with one 262144-token sample, and the skew sweep at every skew; a few steps each.  Last, the pool in the
+    micro-benchmark head shape (Hq 128 / Hkv 4 / d 256), which runs the 256-wide kernels."""
     import torch
     out = {}
     for name, cfg, skew, steps in (("config3", 3, 0.0, 5), ("config5_skew0", 5, 0.0, 5), ("config5_skew0.25", 5, 0.25, 4),
-                                   ("config5_skew0.5", 5, 0.5, 3), ("config5_skew1", 5, 1.0, 2), ("config4", 4, 0.0, 2)):
+                                   ("config5_skew0.5", 5, 0.5, 3), ("config5_skew1", 5, 1.0, 2), ("config4", 4, 0.0, 2),
+                                   ("config6_d256", 6, 0.0, 2)):
         spec = pools.config(cfg, skew)
         pool = Pool(lb, spec, dev, weight_model=args.weight_model, fused=args.backward == "fused")
         pool.build()
@@ -439,6 +441,12 @@ def headline(args, world, spec, pool, value, ms_per_step, ms_local, kern, busy, 
         dom, dom_ms, fa = "k_attn_bwd_fused", kern["bwd_fused"], fb
         executed = {"fused (10 d per pair)": round(fb / kern["bwd_fused"] / 1e9, 1)}
         ratio = "14 d / 14 d per causal pair (every GEMM of the gradient is computed once)"
+    elif d == 256:
+        # the 256-wide kernel: dV pass (S, dV) + dK pass (S, dP, dK) = 10 d executed, dQ pass (S, dP, dQ) = 6 d
+        dom, dom_ms, fa = "k_attn_d256 (dV and dK passes)", kern["bwd_dkdv"], fb
+        executed = {"dv + dk passes (10 d per pair)": round(fa / kern["bwd_dkdv"] / 1e9, 1),
+                    "dq pass (6 d per pair)": round(fb * 6 // 10 / kern["bwd_dq"] / 1e9, 1)}
+        ratio = "20 d / 14 d per causal pair (three gradient passes, each recomputes S)"
     else:
         dom, dom_ms, fa = "k_attn_bwd_dkdv", kern["bwd_dkdv"], fb * 8 // 10
         executed = {"dkdv (8 d per pair)": round(fa / kern["bwd_dkdv"] / 1e9, 1),
@@ -457,7 +465,8 @@ def headline(args, world, spec, pool, value, ms_per_step, ms_local, kern, busy, 
                                f"{len(pool.lengths)} samples (log-normal median 644, sigma 1.6), Hq {hq} / Hkv {hkv} / d {d}, "
                                f"causal per sample, fwd+bwd; plan built once and reused",
                    "backward": ("fused: one kernel over pair tiles (key block x %d-token query chunk x kv head), fp32 "
-                                "accumulators" % pool.plan.export_pairs()[2]) if pool.fused else "two kernels (dK/dV, dQ)",
+                                "accumulators" % pool.plan.export_pairs()[2]) if pool.fused else
+                               ("three passes of the 256-wide kernel (dV, dK, dQ)" if d == 256 else "two kernels (dK/dV, dQ)"),
                    "tile_q": 256, "tile_kv": 128, "head_shards": pool.heads, "n_workers": pool.plan.info()["n_workers"],
                    "tile_weight": "blocks (time proxy)" if pool.blocks else "causal pairs (Eq. 6)",
                    "l2": "inputs larger than L2 (Q alone is %.2f GB per rank)" % (pool.inp["q"].numel() * 2 / 1e9),

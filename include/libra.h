@@ -33,7 +33,7 @@ extern "C" {
 
 #define LIBRA_OK                 0
 #define LIBRA_ERR_INVALID_ARG   (-1)  /* null pointer, non-positive size, H does not divide Hq, ... */
-#define LIBRA_ERR_UNSUPPORTED   (-2)  /* head_dim not in {64,128}, tile size the kernels cannot run */
+#define LIBRA_ERR_UNSUPPORTED   (-2)  /* head_dim not in {64,128,256}, tile size the kernels cannot run */
 #define LIBRA_ERR_PLAN_MISMATCH (-3)  /* plan was built for another T / head count / direction      */
 #define LIBRA_ERR_CUDA          (-4)  /* a CUDA runtime or driver call failed                        */
 #define LIBRA_ERR_OVERFLOW      (-5)  /* tile ids or loads would not fit their integer types         */
@@ -90,7 +90,7 @@ typedef struct {
     int64_t total_tokens;  /* T */
     int     n_samples;     /* n */
     int     hq, hkv;       /* query / kv heads, hkv divides hq */
-    int     head_dim;      /* 64 or 128 */
+    int     head_dim;      /* 64, 128 or 256 */
     float   softmax_scale; /* 0 = 1/sqrt(head_dim) */
 } libra_dims;
 
@@ -169,7 +169,9 @@ int libra_plan_destroy(libra_plan_t* plan);
  * mask of Section 2.3):  for row i of a sample starting at s, with keys s..i,
  *     out_i = sum_k softmax_k(scale * <q_i, k_k>) v_k,   lse_i = ln sum_k exp(scale * <q_i, k_k>)
  * bf16 inputs, fp32 accumulation and softmax, bf16 out (round to nearest even), fp32 lse
- * (natural log).  One persistent kernel walks the plan's query-major tile lists.
+ * (natural log).  One persistent kernel walks the plan's query-major tile lists.  head_dim 256 (the
+ * micro-benchmark head shape of Table 1) runs a kernel of its own: one 128-row slot at a time against
+ * 64-key blocks, the 256-column output accumulator taking half of the tensor memory.
  * Requires a plan with LIBRA_DIR_Q, tile_q == 256 and n_heads dividing hq.
  * Errors: INVALID_ARG, UNSUPPORTED, PLAN_MISMATCH (plan T != dims->total_tokens), CUDA.
  */
@@ -190,7 +192,7 @@ size_t libra_attn_pool_bwd_workspace_bytes(const libra_plan_t* plan, const libra
  *     dq_i = scale sum_k dS_ik k_k;  dk_k = scale sum_{h,i} dS_ik q_i;  dv_k = sum_{h,i} P_ik dout_i
  * (sums over the query heads h of the kv head's group and the rows i >= k of the sample).
  * The plan decides between two forms of the same computation.
- *   Two-kernel form (plan without pair tiles, or head_dim 64): three launches: row statistics, a dK/dV kernel
+ *   Two-kernel form (plan without pair tiles, or head_dim other than 128): three launches: row statistics, a dK/dV kernel
  *   that walks the plan's key-major lists, and a dQ kernel that walks its query-major lists (S and dP are computed
  *   by both, seven GEMMs per 128 x 128 cell); no atomics, so results are run-to-run identical.  Needs LIBRA_DIR_KV
  *   with tile_kv == 128 and n_heads_kv == hkv, and LIBRA_DIR_Q with tile_q == 256 and n_heads dividing hq.
@@ -201,6 +203,9 @@ size_t libra_attn_pool_bwd_workspace_bytes(const libra_plan_t* plan, const libra
  *   The accumulators are rounded to bf16 once, at the end, so the result is at least as accurate as the two-kernel
  *   form's, but the order of the floating-point additions varies from run to run: results agree to rounding, not
  *   bit for bit.  The other directions of the plan are not used by this form.
+ *   At head_dim 256 the two-kernel form takes three passes of one kernel after the row statistics (dV and dK
+ *   over the key-major lists, dQ over the query-major lists; S is recomputed by each: eight GEMMs per cell), because
+ *   the accumulators of dK and dV together would fill the tensor memory.  Same plan, results and determinism.
  * `workspace_dev` must hold libra_attn_pool_bwd_workspace_bytes bytes, 256-byte aligned; every byte the call reads
  * is written (or cleared) inside the call.  Errors: INVALID_ARG, UNSUPPORTED, PLAN_MISMATCH, CUDA.
  */

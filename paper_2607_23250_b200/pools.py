@@ -95,7 +95,9 @@ def cu_seqlens(lengths) -> np.ndarray:
 # ---- the benchmark's configurations -------------------------------------------------
 
 def config(index: int, skew: float = 0.0, seed: int = 0) -> PoolSpec:
-    """The five pool shapes of the benchmark (index 1..5); `skew` selects s for index 5."""
+    """The five pool shapes of the benchmark (index 1..5; `skew` selects s for index 5) and, as index 6, a pool in the
+    micro-benchmark head shape of the paper's Table 1 (Hq 128 / Hkv 4 / d 256): two packed 32768-token sequences,
+    the share of one worker of a 256K sequence at CP = 8."""
     if index == 1:
         return PoolSpec("tiny", 1, 1, 4096, 4, 4, 64, seed=seed)
     if index == 2:
@@ -108,6 +110,8 @@ def config(index: int, skew: float = 0.0, seed: int = 0) -> PoolSpec:
     if index == 5:
         return PoolSpec(f"skew-{skew:g}", 5, 8, 65536, 32, 8, 128,
                         big="frac" if skew > 0 else "none", big_frac=skew, seed=seed)
+    if index == 6:
+        return PoolSpec("microbenchmark-heads", 6, 2, 32768, 128, 4, 256, seed=seed)
     raise ValueError(f"no config {index}")
 
 

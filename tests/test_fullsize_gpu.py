@@ -1,7 +1,8 @@
 """Full-size parity: the Qwen3-8B-shaped pool in the launch configuration the benchmark times, the 30B-shaped
 pool with Pareto-tailed samples, the 1M-token pool with one 262144-token sample (Hq 64 / Hkv 4: sixteen query
 heads per kv head, tensors beyond 2^32 bytes) and the skew sweep of 65536-token sequences at every skew.  The
-"fused" cases run the same pools with a pair-tile plan, which makes the backward call take its fused form.
+"fused" cases run the same pools with a pair-tile plan, which makes the backward call take its fused form; config 6 is
+the micro-benchmark head shape (Hq 128 / Hkv 4 / d 256) on two packed 32768-token sequences.
 
 The whole oracle would take minutes here, so outputs are sampled: rows of O / LSE / dQ and
 columns of dK / dV are recomputed one by one by the CPU oracle on the (sample, kv-head group)
@@ -28,9 +29,11 @@ def _rel(got, want, floor=1e-3):
 
 @pytest.fixture(scope="module",
                 params=[(2, 0.0, False), (2, 0.0, True), (3, 0.0, False), (3, 0.0, True), (4, 0.0, False), (4, 0.0, True),
-                        (5, 0.0, False), (5, 0.25, False), (5, 0.5, False), (5, 1.0, False), (5, 1.0, True)],
+                        (5, 0.0, False), (5, 0.25, False), (5, 0.5, False), (5, 1.0, False), (5, 1.0, True),
+                        (6, 0.0, False)],
                 ids=["config2", "config2_fused", "config3", "config3_fused", "config4", "config4_fused",
-                     "config5_skew0", "config5_skew0.25", "config5_skew0.5", "config5_skew1", "config5_skew1_fused"])
+                     "config5_skew0", "config5_skew0.25", "config5_skew0.5", "config5_skew1", "config5_skew1_fused",
+                     "config6_d256"])
 def run(request):
     from paper_2607_23250_b200 import binding as lb
     fused = request.param[2]
