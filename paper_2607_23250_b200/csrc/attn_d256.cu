@@ -12,10 +12,12 @@
 //
 // dK and dV cannot share TMEM with S^T and dP^T at this width (2 x 256 accumulator columns), so the gradient takes
 // three passes and recomputes S (eight GEMMs per cell for the five of the definition).
-// TMEM: X1 (64) | X2 (64) | W (32: the bf16 result of the element-wise step, A operand of the last GEMM) | acc (256).
+// TMEM: X1 (2 x 64, double-buffered) | X2 (64) | W (32: the bf16 result of the element-wise step, A operand of the
+// last GEMM) | acc (256).
 // Roles (192 threads): warps 0-3 compute (one stationary row per thread), warp 4 one TMA thread, warp 5 one MMA
 // thread.  Per streamed block: X1 (and X2) are issued, the compute warps turn them into W, the accumulating GEMM
-// is issued; tiles are prefetched through a ring of 32 KB slots.  Masks follow the sample bounds per element.
+// is issued; X1 of the next block is issued ahead, so it runs under the element-wise step of the current one.
+// Tiles are prefetched through a ring of 32 KB slots.  Masks follow the sample bounds per element.
 #include <math.h>
 
 #include "common.h"
@@ -29,7 +31,7 @@ constexpr int kTmaWarp = 4, kMmaWarp = 5;
 constexpr int kRows = 128;       // stationary rows per unit
 constexpr int kBlk = 64;         // streamed rows per block
 constexpr int kD = 256;
-constexpr uint32_t kColX1 = 0, kColX2 = 64, kColW = 128, kColAcc = 256;
+constexpr uint32_t kColX1 = 0 /* and 64 */, kColX2 = 128, kColW = 192, kColAcc = 256;
 constexpr uint64_t kDrainNs = 2000000;
 constexpr int kSmemMax = 232448;
 enum Mode { FWD = 0, DV = 1, DK = 2, DQ = 3 };
@@ -48,11 +50,18 @@ struct Cfg {
     static constexpr int kRingOff = kStationary * kBig;
     static constexpr int kStatOff = kRingOff + kSlots * kSmall;
     static constexpr int kBarOff = kStatOff + kSlots * 512;
-    // full[kSlots], empty[kSlots], st_full, st_empty, x1_full, x2_full, w_ready, acc_done, acc_free, drain
-    static constexpr int kNumBars = 2 * kSlots + 8;
+    // full[kSlots], empty[kSlots], st_full, st_empty, x1_full[2], x2_full, w_ready, acc_done, acc_free, drain, acc_step
+    static constexpr int kNumBars = 2 * kSlots + 10;
     static constexpr int kMiscOff = kBarOff + kNumBars * 8;
     static constexpr int kBytes = kMiscOff + 16;
     static_assert(kBytes <= kSmemMax, "exceeds the shared memory of an sm_100 CTA");
+    // Ring slots by stream and iteration i (counted over the whole kernel): the first streamed tile alternates
+    // between slots 0 and 1; the second has slot 2 to itself when it only feeds X2 (it is free again as soon as X2 has
+    // run, so its successor loads early), else it alternates between slots 2 and 3.
+    __host__ __device__ static constexpr uint32_t slot1(uint32_t i) { return i & 1; }
+    __host__ __device__ static constexpr uint32_t phase1(uint32_t i) { return (i >> 1) & 1; }
+    __host__ __device__ static constexpr uint32_t slot2(uint32_t i) { return kHasX2 ? 2 : 2 + (i & 1); }
+    __host__ __device__ static constexpr uint32_t phase2(uint32_t i) { return kHasX2 ? (i & 1) : ((i >> 1) & 1); }
 };
 
 struct Params {
@@ -141,12 +150,13 @@ k_attn_d256(const __grid_constant__ CUtensorMap tm_sa, const __grid_constant__ C
     uint64_t* b2 = bars + 2 * S;
     uint64_t* bar_stfull = b2 + 0;
     uint64_t* bar_stempty = b2 + 1;
-    uint64_t* bar_x1full = b2 + 2;
     uint64_t* bar_x2full = b2 + 3;
     uint64_t* bar_wready = b2 + 4;
     uint64_t* bar_accdone = b2 + 5;
     uint64_t* bar_accfree = b2 + 6;
     uint64_t* bar_drain = b2 + 7;
+    uint64_t* bar_accstep = b2 + 8;    // the accumulating GEMM of an iteration has run: W may be rewritten, acc rescaled
+    uint64_t* bar_x1full = b2 + 9;     // [2] one per X1 buffer: X1 of the next block is committed a block ahead
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::kMiscOff);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + L::kMiscOff + 4);
 
@@ -166,12 +176,14 @@ k_attn_d256(const __grid_constant__ CUtensorMap tm_sa, const __grid_constant__ C
         for (int s = 0; s < S; ++s) { mbar_init(&bar_full[s], 1); mbar_init(&bar_empty[s], 1); }
         mbar_init(bar_stfull, 1);
         mbar_init(bar_stempty, 1);
-        mbar_init(bar_x1full, 1);
+        mbar_init(&bar_x1full[0], 1);
+        mbar_init(&bar_x1full[1], 1);
         mbar_init(bar_x2full, 1);
         mbar_init(bar_wready, kRows);
         mbar_init(bar_accdone, 1);
         mbar_init(bar_accfree, kRows);
         mbar_init(bar_drain, 1);
+        mbar_init(bar_accstep, 1);
         abort_flag[0] = 0;
         abort_flag[1] = (int)p.wait_limit_ns;
         fence_mbar_init();
@@ -196,7 +208,8 @@ k_attn_d256(const __grid_constant__ CUtensorMap tm_sa, const __grid_constant__ C
         // ---------------- TMA producer ----------------
         if (elect_one()) {
             Units<MODE> u(p, cta);
-            uint32_t n = 0, uc = 0;
+            uint32_t n = 0, uc = 0;          // n: iterations so far (over all units)
+            uint32_t armed[S] = {};          // per slot: 1 + parity of the phase last armed (0: never)
             bool ok = true;
             while (ok && !p.inject_stall && u.next()) {
                 ok = mbar_wait(bar_stempty, (uc & 1) ^ 1, abort_flag);
@@ -209,13 +222,15 @@ k_attn_d256(const __grid_constant__ CUtensorMap tm_sa, const __grid_constant__ C
                         tma_load_3d(smem + L::kSbOff + half * L::kBigHalf, &tm_sb, bar_stfull, half * 64, st_head, (int)u.r0);
                 }
                 ++uc;
-                for (int it = 0; it < u.n_it && ok; ++it) {
+                for (int it = 0; it < u.n_it && ok; ++it, ++n) {
                     const int sh = u.stream_head(it), row = u.stream_row(it);
-                    for (int which = 0; which < 2 && ok; ++which, ++n) {
-                        const uint32_t s = n % S;
-                        ok = mbar_wait(&bar_empty[s], ((n / S) & 1) ^ 1, abort_flag);
+                    for (int which = 0; which < 2 && ok; ++which) {
+                        const uint32_t s = which == 0 ? L::slot1(n) : L::slot2(n);
+                        const uint32_t ph = which == 0 ? L::phase1(n) : L::phase2(n);
+                        ok = mbar_wait(&bar_empty[s], ph ^ 1, abort_flag);
                         if (!ok) break;
                         mbar_arrive_expect_tx(&bar_full[s], L::kSmall + (which == 0 ? L::kStatBytes : 0));
+                        armed[s] = 1 + ph;
                         for (int half = 0; half < 4; ++half)
                             tma_load_3d(smem + L::kRingOff + s * L::kSmall + half * L::kSmallHalf, which == 0 ? &tm_t1 : &tm_t2,
                                         &bar_full[s], half * 64, sh, row);
@@ -228,8 +243,8 @@ k_attn_d256(const __grid_constant__ CUtensorMap tm_sa, const __grid_constant__ C
             }
             if (!ok || abort_flag[0]) {   // give-up path: the copies already issued land before shared memory is released
                 if (uc > 0) mbar_wait_drain(bar_stfull, (uc - 1) & 1, kDrainNs);
-                for (uint32_t b = 1; b <= (uint32_t)S && b <= n; ++b)
-                    mbar_wait_drain(&bar_full[(n - b) % S], ((n - b) / S) & 1, kDrainNs);
+                for (int b = 0; b < S; ++b)
+                    if (armed[b]) mbar_wait_drain(&bar_full[b], armed[b] - 1, kDrainNs);
             }
         }
         __syncwarp();
@@ -249,27 +264,33 @@ k_attn_d256(const __grid_constant__ CUtensorMap tm_sa, const __grid_constant__ C
                            sdesc_advance(db, (kk / 4) * L::kSmallHalf + (kk % 4) * 32), idesc_x, kk > 0);
             };
             Units<MODE> u(p, cta);
-            uint32_t n = 0, uc = 0, itc = 0;
+            uint32_t uc = 0, itc = 0;
             bool ok = true;
             while (ok && u.next()) {
                 ok = mbar_wait(bar_stfull, uc & 1, abort_flag);
+                if (ok) ok = mbar_wait(&bar_full[L::slot1(itc)], L::phase1(itc), abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                issue_x(kColX1 + (itc & 1) * 64, L::kSaOff, L::kRingOff + L::slot1(itc) * L::kSmall);
+                tc_commit(&bar_x1full[itc & 1]);
                 for (int it = 0; it < u.n_it && ok; ++it, ++itc) {
-                    const uint32_t s1 = n % S;
-                    ok = mbar_wait(&bar_full[s1], (n / S) & 1, abort_flag);
+                    const uint32_t s1 = L::slot1(itc), s2 = L::slot2(itc);
+                    ok = mbar_wait(&bar_full[s2], L::phase2(itc), abort_flag);
                     if (!ok) break;
-                    ++n;
-                    tc_fence_after();
-                    issue_x(kColX1, L::kSaOff, L::kRingOff + s1 * L::kSmall);
-                    tc_commit(bar_x1full);
-                    const uint32_t s2 = n % S;
-                    ok = mbar_wait(&bar_full[s2], (n / S) & 1, abort_flag);
-                    if (!ok) break;
-                    ++n;
                     if (L::kHasX2) {
                         tc_fence_after();
                         issue_x(kColX2, L::kSbOff, L::kRingOff + s2 * L::kSmall);
                         tc_commit(bar_x2full);
                         tc_commit(&bar_empty[s2]);   // the second streamed tile only feeds X2
+                    }
+                    if (it + 1 < u.n_it) {
+                        // X1 of the next block into the other buffer (read out two iterations ago): it runs while the
+                        // compute warps work on this block
+                        ok = mbar_wait(&bar_full[L::slot1(itc + 1)], L::phase1(itc + 1), abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_x(kColX1 + ((itc + 1) & 1) * 64, L::kSaOff, L::kRingOff + L::slot1(itc + 1) * L::kSmall);
+                        tc_commit(&bar_x1full[(itc + 1) & 1]);
                     }
                     ok = mbar_wait(bar_wready, itc & 1, abort_flag);
                     if (ok && it == 0 && uc > 0) ok = mbar_wait(bar_accfree, (uc - 1) & 1, abort_flag);
@@ -283,6 +304,7 @@ k_attn_d256(const __grid_constant__ CUtensorMap tm_sa, const __grid_constant__ C
                             mma_ts(tmem_base + kColAcc, tmem_base + kColW + kk * 8, sdesc_advance(db, kk * 2048), idesc_acc,
                                    (it > 0 || kk > 0) ? 1u : 0u);
                     }
+                    tc_commit(bar_accstep);
                     tc_commit(&bar_empty[s1]);
                     if (!L::kHasX2) tc_commit(&bar_empty[s2]);
                     if (it == u.n_it - 1) { tc_commit(bar_accdone); tc_commit(bar_stempty); }
@@ -330,18 +352,18 @@ k_attn_d256(const __grid_constant__ CUtensorMap tm_sa, const __grid_constant__ C
                 const int64_t b0 = u.stream_row(it);
                 const int c_lo = (int)(lo_abs - b0 > kBlk ? kBlk : lo_abs - b0);
                 const int c_hi = (int)(hi_abs - b0 < -1 ? -1 : hi_abs - b0);
-                const uint32_t s1 = (2 * itc) % S;
+                const uint32_t s1 = L::slot1(itc);
                 const float* st = reinterpret_cast<const float*>(smem + L::kStatOff + s1 * 512);
                 if (L::kStatBytes > 0) {   // the streamed rows' statistics arrive with their first tile
-                    ok = warp_wait(&bar_full[s1], ((2 * itc) / S) & 1, abort_flag);
+                    ok = warp_wait(&bar_full[s1], L::phase1(itc), abort_flag);
                     if (!ok) break;
                 }
-                ok = warp_wait(bar_x1full, itc & 1, abort_flag);
+                ok = warp_wait(&bar_x1full[itc & 1], (itc >> 1) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
                 uint32_t sr[kBlk];
-                tmem_ld32(t_x1, sr);
-                tmem_ld32(t_x1 + 32, sr + 32);
+                tmem_ld32(t_x1 + (itc & 1) * 64, sr);
+                tmem_ld32(t_x1 + (itc & 1) * 64 + 32, sr + 32);
                 tmem_ld_wait();
                 uint32_t pk[kBlk / 2];
                 if (MODE == FWD) {
@@ -367,18 +389,6 @@ k_attn_d256(const __grid_constant__ CUtensorMap tm_sa, const __grid_constant__ C
                     bool grow = false;
                     if (mx > m_ref + 8.0f || (m_ref == -INFINITY && mx > -INFINITY)) { m_new = mx; grow = true; }
                     const float factor = grow ? ex2_approx(m_ref - m_new) : 1.0f;
-                    if (it > 0 && __any_sync(0xffffffffu, grow)) {
-                        // the previous block's accumulation completed before this block's S was committed
-#pragma unroll
-                        for (int c = 0; c < kD; c += 32) {
-                            uint32_t orow[32];
-                            tmem_ld32(t_acc + c, orow);
-                            tmem_ld_wait();
-#pragma unroll
-                            for (int i = 0; i < 32; ++i) orow[i] = __float_as_uint(__uint_as_float(orow[i]) * factor);
-                            tmem_st32(t_acc + c, orow);
-                        }
-                    }
                     l_sum *= factor;
                     m_ref = m_new;
                     const float m_use = (m_ref == -INFINITY) ? 0.f : m_ref;
@@ -390,6 +400,21 @@ k_attn_d256(const __grid_constant__ CUtensorMap tm_sa, const __grid_constant__ C
                         ps0 += p0;
                         ps1 += p1;
                         pk[i >> 1] = pack_bf16x2(p0, p1);
+                    }
+                    if (it > 0 && __any_sync(0xffffffffu, grow)) {
+                        // O is rescaled once the previous block's accumulation has landed (its W is spent then, too)
+                        ok = warp_wait(bar_accstep, (itc - 1) & 1, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+#pragma unroll
+                        for (int c = 0; c < kD; c += 32) {
+                            uint32_t orow[32];
+                            tmem_ld32(t_acc + c, orow);
+                            tmem_ld_wait();
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) orow[i] = __float_as_uint(__uint_as_float(orow[i]) * factor);
+                            tmem_st32(t_acc + c, orow);
+                        }
                     }
                     l_sum += ps0 + ps1;
                 } else {
@@ -419,6 +444,11 @@ k_attn_d256(const __grid_constant__ CUtensorMap tm_sa, const __grid_constant__ C
                             pk[i >> 1] = pack_bf16x2(pf[i] * (__uint_as_float(dp[i]) - d0), pf[i + 1] * (__uint_as_float(dp[i + 1]) - d1));
                         }
                     }
+                }
+                if (itc > 0) {   // the previous accumulating GEMM has consumed W
+                    ok = warp_wait(bar_accstep, (itc - 1) & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
                 }
                 tmem_st16(t_w, pk);
                 tmem_st16(t_w + 16, pk + 16);

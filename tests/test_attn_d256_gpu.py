@@ -141,3 +141,42 @@ def test_sampled_rows_of_a_long_sample():
         assert np.abs(got_dk[c] - dk_ref[x]).max() <= TOL_G * max(np.abs(dk_ref[x]).max(), 1e-2), ("dk", int(c))
         assert np.abs(got_dv[c] - dv_ref[x]).max() <= TOL_G * max(np.abs(dv_ref[x]).max(), 1e-2), ("dv", int(c))
     plan.destroy()
+
+
+def test_give_up_path_of_the_256_wide_kernel():
+    """Producer stall injected on a healthy GPU (no loads are issued, a flag nothing sets): every pass reports
+    TIMEOUT through the status words and returns; with the injection off the same plan gives correct results."""
+    from paper_2607_23250_b200 import binding as lb
+    lengths = [300, 200, 524]
+    hq, hkv = 4, 2
+    cu_np = pools.cu_seqlens(lengths)
+    t = pools.make_tensors(int(cu_np[-1]), hq, hkv, D, seed=12)
+    q, k, v, dout = (t[n].cuda() for n in ("q", "k", "v", "dout"))
+    plan = lb.libra_plan_tiles(torch.from_numpy(cu_np).cuda(), hq, 256, tile_kv=128, n_heads_kv=hkv)
+    good_out, good_lse = lb.libra_attn_pool_fwd(q, k, v, plan)
+    plan.busy_times(lb.KERNEL_FWD)
+    plan.set_wait_limit_ns(200_000)
+    plan.inject_stall(True)
+    lb.libra_attn_pool_fwd(q, k, v, plan)
+    with pytest.raises(lb.LibraError) as err:
+        plan.busy_times(lb.KERNEL_FWD)
+    assert err.value.code == lb.ERR_TIMEOUT
+    lb.libra_attn_pool_bwd(q, k, v, good_out, good_lse, dout, plan)
+    for kern in (lb.KERNEL_BWD_DKDV, lb.KERNEL_BWD_DQ):
+        with pytest.raises(lb.LibraError) as err:
+            plan.busy_times(kern)
+        assert err.value.code == lb.ERR_TIMEOUT
+    plan.inject_stall(False)
+    plan.set_wait_limit_ns(0)
+    out, lse = lb.libra_attn_pool_fwd(q, k, v, plan)
+    dq, dk, dv = lb.libra_attn_pool_bwd(q, k, v, out, lse, dout, plan)
+    torch.cuda.synchronize()
+    for kern in (lb.KERNEL_FWD, lb.KERNEL_BWD_DKDV, lb.KERNEL_BWD_DQ):
+        plan.busy_times(kern)
+    assert torch.equal(out, good_out) and torch.equal(lse, good_lse)
+    f = {n: t[n].float().numpy() for n in t}
+    o_ref, l_ref = oracle.attn_fwd(f["q"], f["k"], f["v"], cu_np)
+    ref = oracle.attn_bwd(f["q"], f["k"], f["v"], o_ref, l_ref, f["dout"], cu_np)
+    for g, r in zip((dq, dk, dv), ref):
+        assert np.abs(g.float().cpu().numpy() - r).max() <= TOL_G * np.abs(r).max()
+    plan.destroy()
