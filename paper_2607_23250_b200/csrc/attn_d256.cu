@@ -14,8 +14,10 @@
 // three passes and recomputes S (eight GEMMs per cell for the five of the definition).
 // TMEM: X1 (2 x 64, double-buffered) | X2 (64) | W (32: the bf16 result of the element-wise step, A operand of the
 // last GEMM) | acc (256).
-// Roles (192 threads): warps 0-3 compute (one stationary row per thread), warp 4 one TMA thread, warp 5 one MMA
-// thread.  Per streamed block: X1 (and X2) are issued, the compute warps turn them into W, the accumulating GEMM
+// Roles (320 threads): warps 0-7 compute, warp 8 one TMA thread, warp 9 one MMA thread.  In the gradient passes two
+// threads share a stationary row (32 of the block's 64 columns each; warps w and w + 4 reach the same TMEM lanes); the
+// forward keeps one thread per row, because the running maximum and sum of a row live in its registers (warps 4-7
+// idle there).  Per streamed block: X1 (and X2) are issued, the compute warps turn them into W, the accumulating GEMM
 // is issued; X1 of the next block is issued ahead, so it runs under the element-wise step of the current one.
 // Tiles are prefetched through a ring of 32 KB slots.  Masks follow the sample bounds per element.
 #include <math.h>
@@ -26,8 +28,8 @@
 namespace libra {
 namespace d256 {
 
-constexpr int kThreads = 192;
-constexpr int kTmaWarp = 4, kMmaWarp = 5;
+constexpr int kThreads = 320;
+constexpr int kTmaWarp = 8, kMmaWarp = 9;
 constexpr int kRows = 128;       // stationary rows per unit
 constexpr int kBlk = 64;         // streamed rows per block
 constexpr int kD = 256;
@@ -40,6 +42,8 @@ template <int MODE>
 struct Cfg {
     static constexpr bool kKeyStationary = (MODE == DV || MODE == DK);
     static constexpr bool kHasX2 = (MODE == DK || MODE == DQ);
+    static constexpr int kGroups = MODE == FWD ? 1 : 2;      // compute threads per stationary row
+    static constexpr int kCols = 64 / kGroups;               // columns of a streamed block per compute thread
     static constexpr int kStationary = kHasX2 ? 2 : 1;       // resident 64 KB tiles
     static constexpr int kSlots = kHasX2 ? 3 : 4;            // ring of 32 KB tiles
     static constexpr int kBig = 65536, kBigHalf = 16384;     // 128 x 256 bf16: four column halves of 128 rows x 128 B
@@ -179,9 +183,9 @@ k_attn_d256(const __grid_constant__ CUtensorMap tm_sa, const __grid_constant__ C
         mbar_init(&bar_x1full[0], 1);
         mbar_init(&bar_x1full[1], 1);
         mbar_init(bar_x2full, 1);
-        mbar_init(bar_wready, kRows);
+        mbar_init(bar_wready, kRows * L::kGroups);
         mbar_init(bar_accdone, 1);
-        mbar_init(bar_accfree, kRows);
+        mbar_init(bar_accfree, kRows * L::kGroups);
         mbar_init(bar_drain, 1);
         mbar_init(bar_accstep, 1);
         abort_flag[0] = 0;
@@ -317,14 +321,18 @@ k_attn_d256(const __grid_constant__ CUtensorMap tm_sa, const __grid_constant__ C
             }
         }
         __syncwarp();
-    } else {
-        // ---------------- compute warps: thread r owns stationary row r (TMEM lane r) ----------------
-        const int r = warp * 32 + lane;
-        const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
-        const uint32_t t_x1 = tmem_base + lane_addr + kColX1;
-        const uint32_t t_x2 = tmem_base + lane_addr + kColX2;
-        const uint32_t t_w = tmem_base + lane_addr + kColW;
-        const uint32_t t_acc = tmem_base + lane_addr + kColAcc;
+    } else if (warp < 4 * L::kGroups) {
+        // ---------------- compute warps: thread (r, grp) owns stationary row r (TMEM lane r) and the columns
+        // [col0, col0 + kCols) of every streamed block ----------------
+        constexpr int NC = L::kCols;
+        const int grp = warp >> 2;
+        const int col0 = grp * NC;
+        const int r = (warp & 3) * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t t_x1 = tmem_base + lane_addr + kColX1 + col0;
+        const uint32_t t_x2 = tmem_base + lane_addr + kColX2 + col0;
+        const uint32_t t_w = tmem_base + lane_addr + kColW + col0 / 2;
+        const uint32_t t_acc = tmem_base + lane_addr + kColAcc + grp * (kD / L::kGroups);
         Units<MODE> u(p, cta);
         uint32_t uc = 0, itc = 0;
         bool ok = true;
@@ -350,10 +358,11 @@ k_attn_d256(const __grid_constant__ CUtensorMap tm_sa, const __grid_constant__ C
             }
             for (int it = 0; it < u.n_it && ok; ++it, ++itc) {
                 const int64_t b0 = u.stream_row(it);
-                const int c_lo = (int)(lo_abs - b0 > kBlk ? kBlk : lo_abs - b0);
-                const int c_hi = (int)(hi_abs - b0 < -1 ? -1 : hi_abs - b0);
+                // first and last visible column, counted from this thread's first column
+                const int c_lo = (int)(lo_abs - b0 > kBlk ? kBlk : lo_abs - b0) - col0;
+                const int c_hi = (int)(hi_abs - b0 < -1 ? -1 : hi_abs - b0) - col0;
                 const uint32_t s1 = L::slot1(itc);
-                const float* st = reinterpret_cast<const float*>(smem + L::kStatOff + s1 * 512);
+                const float* st = reinterpret_cast<const float*>(smem + L::kStatOff + s1 * 512) + col0;
                 if (L::kStatBytes > 0) {   // the streamed rows' statistics arrive with their first tile
                     ok = warp_wait(&bar_full[s1], L::phase1(itc), abort_flag);
                     if (!ok) break;
@@ -361,12 +370,12 @@ k_attn_d256(const __grid_constant__ CUtensorMap tm_sa, const __grid_constant__ C
                 ok = warp_wait(&bar_x1full[itc & 1], (itc >> 1) & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                uint32_t sr[kBlk];
-                tmem_ld32(t_x1 + (itc & 1) * 64, sr);
-                tmem_ld32(t_x1 + (itc & 1) * 64 + 32, sr + 32);
+                uint32_t sr[NC];
+#pragma unroll
+                for (int c = 0; c < NC; c += 32) tmem_ld32(t_x1 + (itc & 1) * 64 + c, sr + c);
                 tmem_ld_wait();
-                uint32_t pk[kBlk / 2];
-                if (MODE == FWD) {
+                uint32_t pk[NC / 2];
+                if constexpr (MODE == FWD) {
 #pragma unroll
                     for (int i = 0; i < kBlk; ++i)
                         if (i < c_lo || i > c_hi) sr[i] = 0xff800000u;  // -inf
@@ -419,26 +428,26 @@ k_attn_d256(const __grid_constant__ CUtensorMap tm_sa, const __grid_constant__ C
                     l_sum += ps0 + ps1;
                 } else {
                     // P = exp2(S c - LSE) on the visible elements, 0 elsewhere
-                    float pf[kBlk];
+                    float pf[NC];
 #pragma unroll
-                    for (int i = 0; i < kBlk; ++i) {
+                    for (int i = 0; i < NC; ++i) {
                         const float l2 = L::kKeyStationary ? st[i] : lse2r;
                         const float e = ex2_approx(fmaf(__uint_as_float(sr[i]), p.scale_log2, -l2));
                         pf[i] = (i < c_lo || i > c_hi) ? 0.f : e;
                     }
                     if (MODE == DV) {
 #pragma unroll
-                        for (int i = 0; i < kBlk; i += 2) pk[i >> 1] = pack_bf16x2(pf[i], pf[i + 1]);
+                        for (int i = 0; i < NC; i += 2) pk[i >> 1] = pack_bf16x2(pf[i], pf[i + 1]);
                     } else {
                         ok = warp_wait(bar_x2full, itc & 1, abort_flag);
                         if (!ok) break;
                         tc_fence_after();
-                        uint32_t dp[kBlk];
-                        tmem_ld32(t_x2, dp);
-                        tmem_ld32(t_x2 + 32, dp + 32);
+                        uint32_t dp[NC];
+#pragma unroll
+                        for (int c = 0; c < NC; c += 32) tmem_ld32(t_x2 + c, dp + c);
                         tmem_ld_wait();
 #pragma unroll
-                        for (int i = 0; i < kBlk; i += 2) {
+                        for (int i = 0; i < NC; i += 2) {
                             const float d0 = L::kKeyStationary ? st[64 + i] : dvecr;
                             const float d1 = L::kKeyStationary ? st[64 + i + 1] : dvecr;
                             pk[i >> 1] = pack_bf16x2(pf[i] * (__uint_as_float(dp[i]) - d0), pf[i + 1] * (__uint_as_float(dp[i + 1]) - d1));
@@ -450,8 +459,8 @@ k_attn_d256(const __grid_constant__ CUtensorMap tm_sa, const __grid_constant__ C
                     if (!ok) break;
                     tc_fence_after();
                 }
-                tmem_st16(t_w, pk);
-                tmem_st16(t_w + 16, pk + 16);
+#pragma unroll
+                for (int c = 0; c < NC / 2; c += 16) tmem_st16(t_w + c, pk + c);
                 tmem_st_wait();
                 tc_fence_before();
                 mbar_arrive(bar_wready);
@@ -466,9 +475,9 @@ k_attn_d256(const __grid_constant__ CUtensorMap tm_sa, const __grid_constant__ C
             if (MODE == DK || MODE == DQ) mul = p.scale;
             const int n_heads = L::kKeyStationary ? p.hkv : p.hq;
             const int head = L::kKeyStationary ? u.kvh : u.h;
-            __nv_bfloat16* dst_row = p.out + ((size_t)row * n_heads + head) * kD;
+            __nv_bfloat16* dst_row = p.out + ((size_t)row * n_heads + head) * kD + grp * (kD / L::kGroups);
 #pragma unroll
-            for (int c = 0; c < kD; c += 32) {
+            for (int c = 0; c < kD / L::kGroups; c += 32) {
                 uint32_t v[32];
                 tmem_ld32(t_acc + c, v);
                 tmem_ld_wait();
