@@ -37,8 +37,13 @@ from paper_2607_23250_b200 import pools, sharding  # noqa: E402
 METRIC = "useful attention TFLOP/s fwd+bwd (sum of per-sample causal FLOPs)"
 
 
-def kernel_ids(lb, fused):
+def kernel_ids(lb, fused, d=128):
     """name -> library kernel id of the launches of one step, and the names that keep per-CTA busy times."""
+    if d == 256:   # forward pass, row statistics, dV + dK passes, dQ pass (+ rounding of dK / dV with a pair-tile plan)
+        ids = {"fwd": lb.KERNEL_FWD, "bwd_prep": lb.KERNEL_BWD_PREP, "bwd_dkdv": lb.KERNEL_BWD_DKDV, "bwd_dq": lb.KERNEL_BWD_DQ}
+        if fused:
+            ids["bwd_post"] = lb.KERNEL_BWD_POST
+        return ids, ("fwd", "bwd_dkdv", "bwd_dq")
     if fused:
         return ({"fwd": lb.KERNEL_FWD, "bwd_prep": lb.KERNEL_BWD_PREP, "bwd_fused": lb.KERNEL_BWD_FUSED,
                  "bwd_post": lb.KERNEL_BWD_POST}, ("fwd", "bwd_fused"))
@@ -167,7 +172,8 @@ class Pool:
     def __init__(self, lb, spec, dev, shard=None, weight_model="pairs", heads=0, seed=0, fused=True):
         import torch
         self.lb, self.spec, self.dev, self.shard = lb, spec, dev, shard
-        self.fused = fused and spec.head_dim == 128      # the fused backward exists for head_dim 128
+        self.fused = fused and spec.head_dim in (128, 256)   # a pair-tile plan: fused backward at head_dim 128,
+                                                             # dV / dK passes over pair tiles at head_dim 256
         self.lengths = pools.pool_lengths(spec)
         cu_np = pools.cu_seqlens(self.lengths)
         T, d = spec.total_tokens, spec.head_dim
@@ -228,7 +234,7 @@ class Pool:
             self.step(plan)
         barrier()
         plan.set_timing(True)                          # fresh record: only the timed steps below
-        ids, with_busy = kernel_ids(lb, self.fused)
+        ids, with_busy = kernel_ids(lb, self.fused, self.d)
         n0 = lb.launch_count()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
@@ -242,7 +248,8 @@ class Pool:
         plan.set_timing(False)
         busy = {}
         for n in with_busy:
-            b = plan.busy_times(ids[n]).astype(np.float64)
+            which = lb.KERNEL_BWD_FUSED if (n == "bwd_dkdv" and self.fused) else ids[n]   # the lists the passes walked
+            b = plan.busy_times(which).astype(np.float64)
             b = b[b > 0]
             busy[n] = round(float(b.max() / b.mean()), 4)
         return ms, kern, busy
@@ -437,7 +444,7 @@ def headline(args, world, spec, pool, value, ms_per_step, ms_local, kern, busy, 
     # of the gradient (S, dP, dV, dK, dQ = 10 d flops per causal pair per query head, all of them useful); of the
     # dK/dV kernel of the two-kernel form: the four GEMMs it owns (8 d).  It is timed inside the timed region; that
     # region's length decides which measured peak applies (burst under a second, else sustained).
-    if pool.fused:
+    if pool.fused and d == 128:
         dom, dom_ms, fa = "k_attn_bwd_fused", kern["bwd_fused"], fb
         executed = {"fused (10 d per pair)": round(fb / kern["bwd_fused"] / 1e9, 1)}
         ratio = "14 d / 14 d per causal pair (every GEMM of the gradient is computed once)"
@@ -465,8 +472,9 @@ def headline(args, world, spec, pool, value, ms_per_step, ms_local, kern, busy, 
                                f"{len(pool.lengths)} samples (log-normal median 644, sigma 1.6), Hq {hq} / Hkv {hkv} / d {d}, "
                                f"causal per sample, fwd+bwd; plan built once and reused",
                    "backward": ("fused: one kernel over pair tiles (key block x %d-token query chunk x kv head), fp32 "
-                                "accumulators" % pool.plan.export_pairs()[2]) if pool.fused else
-                               ("three passes of the 256-wide kernel (dV, dK, dQ)" if d == 256 else "two kernels (dK/dV, dQ)"),
+                                "accumulators" % pool.plan.export_pairs()[2]) if (pool.fused and d == 128) else
+                               (("three passes of the 256-wide kernel (dV, dK, dQ)" + (", dV and dK over pair tiles with fp32 "
+                                 "accumulators" if pool.fused else "")) if d == 256 else "two kernels (dK/dV, dQ)"),
                    "tile_q": 256, "tile_kv": 128, "head_shards": pool.heads, "n_workers": pool.plan.info()["n_workers"],
                    "tile_weight": "blocks (time proxy)" if pool.blocks else "causal pairs (Eq. 6)",
                    "l2": "inputs larger than L2 (Q alone is %.2f GB per rank)" % (pool.inp["q"].numel() * 2 / 1e9),

@@ -603,15 +603,16 @@ static BwdWorkspace bwd_workspace(int64_t T, int hq, int hkv = 0, int d = 0, boo
     w.total = 2 * w.stat_bytes;
     w.dq_acc_bytes = w.dkv_acc_bytes = 0;
     if (fused) {
-        w.dq_acc_bytes = ((size_t)T * hq * d * sizeof(float) + 255) & ~(size_t)255;
+        if (d == 128) w.dq_acc_bytes = ((size_t)T * hq * d * sizeof(float) + 255) & ~(size_t)255;
         w.dkv_acc_bytes = ((size_t)T * hkv * d * sizeof(float) + 255) & ~(size_t)255;
         w.total += w.dq_acc_bytes + 2 * w.dkv_acc_bytes;
     }
     return w;
 }
-// The fused backward runs when the plan carries pair tiles and the head dimension is 128.
+// A plan with pair tiles selects the accumulating forms: at head_dim 128 the fused kernel (dQ, dK, dV accumulated in
+// fp32), at head_dim 256 the dV and dK passes over pair tiles (dK, dV accumulated in fp32; the dQ pass is unchanged).
 static bool use_fused(const libra_plan_t* plan, const libra_dims* dims) {
-    return plan->dir[2].enabled && dims->head_dim == 128;
+    return plan->dir[2].enabled && (dims->head_dim == 128 || dims->head_dim == 256);
 }
 
 template <typename Kernel>
@@ -728,6 +729,12 @@ extern "C" int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const v
     const PlanDir& dkv_dir = plan->dir[1];
     const bool fused = use_fused(plan, dims);
     if (plan->T != dims->total_tokens) return LIBRA_ERR_PLAN_MISMATCH;
+    if (fused && dims->head_dim == 256) {   // the dQ pass walks the query-major lists
+        const PlanDir& pd = plan->dir[2];
+        if (!dq_dir.enabled || dq_dir.tile != 2 * kBlk || dims->hq % dq_dir.H) return LIBRA_ERR_PLAN_MISMATCH;
+        if (pd.tile != kBlk || pd.H != dims->hkv) return LIBRA_ERR_PLAN_MISMATCH;
+        if (pd.W > plan->sm_count || dq_dir.W > plan->sm_count) return LIBRA_ERR_UNSUPPORTED;
+    }
     if (!fused) {
         if (!dq_dir.enabled || !dkv_dir.enabled) return LIBRA_ERR_PLAN_MISMATCH;
         if (dkv_dir.tile != kBlk || dq_dir.tile != 2 * kBlk) return LIBRA_ERR_UNSUPPORTED;
@@ -758,7 +765,25 @@ extern "C" int libra_attn_pool_bwd(const void* q_dev, const void* k_dev, const v
             (const __nv_bfloat16*)out_dev, (const __nv_bfloat16*)dout_dev, lse_dev, T, ws.Tpad, dims->hq, dvec, lse2);
         count_launch();
         time_end(mp256, 3, s);
-        return launch_bwd_d256(q_dev, k_dev, v_dev, dout_dev, dq_dev, dk_dev, dv_dev, lse2, dvec, ws.Tpad, plan, dims, scale, s);
+        float* dk_acc = nullptr;
+        float* dv_acc = nullptr;
+        if (fused) {
+            dk_acc = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(workspace_dev) + 2 * ws.stat_bytes);
+            dv_acc = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(workspace_dev) + 2 * ws.stat_bytes + ws.dkv_acc_bytes);
+            cudaMemsetAsync(dk_acc, 0, 2 * ws.dkv_acc_bytes, s);
+        }
+        int rc256 = launch_bwd_d256(q_dev, k_dev, v_dev, dout_dev, dq_dev, dk_dev, dv_dev, lse2, dvec, ws.Tpad, dk_acc,
+                                    dv_acc, plan, dims, scale, s);
+        if (rc256 == LIBRA_OK && fused) {
+            time_begin(mp256, 5, s);
+            const int64_t nk8 = T * dims->hkv * 256 / 8;
+            k_bwd_fused_finish<<<(unsigned)((nk8 + 255) / 256), 256, 0, s>>>(dk_acc, (__nv_bfloat16*)dk_dev, nk8, scale);
+            k_bwd_fused_finish<<<(unsigned)((nk8 + 255) / 256), 256, 0, s>>>(dv_acc, (__nv_bfloat16*)dv_dev, nk8, 1.0f);
+            time_end(mp256, 5, s);
+            count_launch(2);
+            if (cudaGetLastError() != cudaSuccess) rc256 = LIBRA_ERR_CUDA;
+        }
+        return rc256;
     }
     CUtensorMap tq, tk, tv, tdo, tdq;
     int rc = make_thd_map(&tq, q_dev, T, dims->hq, D, kBlk);

@@ -79,6 +79,13 @@ struct Params {
     const int32_t* tok_end;
     int64_t T, Tpad;
     int hq, hkv, H;         // H: head shards of the query-major lists (FWD, DQ)
+    // key-stationary passes over pair tiles (key block x query chunk x kv head) instead of key-major tiles: the
+    // accumulator of a unit is added to acc32 [T, Hkv, 256] (fp32) and rounded by a later kernel
+    float* acc32;           // null: key-major tiles, results stored as bf16 by the pass itself
+    const int32_t* u_blk;   // [NU] key block of pair-block u
+    const int32_t* u_chunk; // [NU] query chunk of pair-block u
+    int64_t NU;
+    int R;                  // 128-row blocks per query chunk
     float scale, scale_log2;
     int* status;
     const int* plan_status;
@@ -111,12 +118,25 @@ struct Units {
         if constexpr (Cfg<MODE>::kKeyStationary) {
             if (++idx >= end) return false;
             const int t = p.cta_tiles[idx];
-            kvh = t % p.hkv;
+            if (p.acc32) {   // pair tile: the query blocks of one chunk only
+                const int pb = (int)(t % p.NU);
+                kvh = (int)(t / p.NU);
+                const int j = p.u_blk[pb], c = p.u_chunk[pb];
+                r0 = (int64_t)j * kRows;
+                const int64_t last_key = r0 + kRows - 1 < p.T ? r0 + kRows - 1 : p.T - 1;
+                const int last64 = (p.tok_end[last_key] - 1) / kBlk;
+                const int lo128 = c * p.R > j ? c * p.R : j;
+                const int hi64 = 2 * (c * p.R + p.R - 1) + 1;
+                b_lo = 2 * lo128;
+                n_blk = (hi64 < last64 ? hi64 : last64) - b_lo + 1;
+            } else {
+                kvh = t % p.hkv;
+                r0 = (int64_t)(t / p.hkv) * kRows;
+                const int64_t last_key = r0 + kRows - 1 < p.T ? r0 + kRows - 1 : p.T - 1;
+                b_lo = (int)(r0 / kBlk);
+                n_blk = (p.tok_end[last_key] - 1) / kBlk - b_lo + 1;
+            }
             h = kvh * G;
-            r0 = (int64_t)(t / p.hkv) * kRows;
-            const int64_t last_key = r0 + kRows - 1 < p.T ? r0 + kRows - 1 : p.T - 1;
-            b_lo = (int)(r0 / kBlk);
-            n_blk = (p.tok_end[last_key] - 1) / kBlk - b_lo + 1;
             n_it = G * n_blk;
             return true;
         } else {
@@ -476,12 +496,23 @@ k_attn_d256(const __grid_constant__ CUtensorMap tm_sa, const __grid_constant__ C
             const int n_heads = L::kKeyStationary ? p.hkv : p.hq;
             const int head = L::kKeyStationary ? u.kvh : u.h;
             __nv_bfloat16* dst_row = p.out + ((size_t)row * n_heads + head) * kD + grp * (kD / L::kGroups);
+            float* acc_row = L::kKeyStationary && p.acc32
+                                 ? p.acc32 + ((size_t)row * n_heads + head) * kD + grp * (kD / L::kGroups) : nullptr;
 #pragma unroll
             for (int c = 0; c < kD / L::kGroups; c += 32) {
                 uint32_t v[32];
                 tmem_ld32(t_acc + c, v);
                 tmem_ld_wait();
-                if (row_ok) {
+                if (acc_row) {   // a key block meets several query chunks: its partial sums are added up in fp32
+                    if (row_ok) {
+#pragma unroll
+                        for (int i = 0; i < 32; i += 4)
+                            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(acc_row + c + i),
+                                         "f"(__uint_as_float(v[i])), "f"(__uint_as_float(v[i + 1])),
+                                         "f"(__uint_as_float(v[i + 2])), "f"(__uint_as_float(v[i + 3]))
+                                         : "memory");
+                    }
+                } else if (row_ok) {
                     uint4* dst = reinterpret_cast<uint4*>(dst_row + c);
 #pragma unroll
                     for (int i = 0; i < 32; i += 8) {
@@ -557,11 +588,12 @@ int launch_fwd_d256(const void* q, const void* k, const void* v, void* out, floa
 // Backward at head_dim 256: the dV and dK passes over the key-major lists, the dQ pass over the query-major lists.
 // lse2 / dvec are the row statistics [Hq, Tpad] the caller has computed on the same stream.
 int launch_bwd_d256(const void* q, const void* k, const void* v, const void* dout, void* dq, void* dk, void* dv,
-                    const float* lse2, const float* dvec, int64_t Tpad, const libra_plan* plan, const libra_dims* dims,
-                    float scale, cudaStream_t s) {
+                    const float* lse2, const float* dvec, int64_t Tpad, float* dk_acc, float* dv_acc,
+                    const libra_plan* plan, const libra_dims* dims, float scale, cudaStream_t s) {
     using namespace d256;
     const PlanDir& dq_dir = plan->dir[0];
-    const PlanDir& kv_dir = plan->dir[1];
+    const bool pairs = dk_acc != nullptr;            // key-stationary passes over pair tiles, fp32 accumulators
+    const PlanDir& kv_dir = plan->dir[pairs ? 2 : 1];
     CUtensorMap q128, do128, k128, v128, q64, do64, k64, v64;
     int rc = make_thd_map(&q128, q, plan->T, dims->hq, kD, kRows);
     if (rc == LIBRA_OK) rc = make_thd_map(&do128, dout, plan->T, dims->hq, kD, kRows);
@@ -585,12 +617,16 @@ int launch_bwd_d256(const void* q, const void* k, const void* v, const void* dou
     libra_plan* mp = const_cast<libra_plan*>(plan);
     // dV and dK: key-major lists
     prm.cta_offsets = kv_dir.d_cta_offsets; prm.cta_tiles = kv_dir.d_cta_exec; prm.busy = kv_dir.d_busy;
+    if (pairs) { prm.u_blk = kv_dir.d_u_blk; prm.u_chunk = kv_dir.d_u_chunk; prm.NU = kv_dir.NB; prm.R = kv_dir.chunk / kv_dir.tile; }
     time_begin(mp, 1, s);
     prm.out = reinterpret_cast<__nv_bfloat16*>(dv);
+    prm.acc32 = dv_acc;
     rc = launch<DV>(k128, k128, q64, do64, prm, kv_dir.W, s);
     prm.out = reinterpret_cast<__nv_bfloat16*>(dk);
+    prm.acc32 = dk_acc;
     if (rc == LIBRA_OK) rc = launch<DK>(k128, v128, q64, do64, prm, kv_dir.W, s);
     time_end(mp, 1, s);
+    prm.acc32 = nullptr;
     if (rc != LIBRA_OK) return rc;
     // dQ: query-major lists
     prm.cta_offsets = dq_dir.d_cta_offsets; prm.cta_tiles = dq_dir.d_cta_exec; prm.busy = dq_dir.d_busy2;

@@ -88,9 +88,11 @@ int make_f32_3d_map(CUtensorMap* m, const void* base, int64_t T, int H, int d, i
 // its key-major (dV, dK) and query-major (dQ) lists, given the row statistics lse2 / dvec [Hq, Tpad].
 int launch_fwd_d256(const void* q, const void* k, const void* v, void* out, float* lse, const libra_plan* plan,
                     const libra_dims* dims, float scale, cudaStream_t s);
+// dk_acc / dv_acc: fp32 accumulators [T, Hkv, 256], zero on entry, when the dV and dK passes are to walk the plan's
+// pair tiles (the caller rounds them afterwards); null: key-major tiles, dk / dv written directly.
 int launch_bwd_d256(const void* q, const void* k, const void* v, const void* dout, void* dq, void* dk, void* dv,
-                    const float* lse2, const float* dvec, int64_t Tpad, const libra_plan* plan, const libra_dims* dims,
-                    float scale, cudaStream_t s);
+                    const float* lse2, const float* dvec, int64_t Tpad, float* dk_acc, float* dv_acc,
+                    const libra_plan* plan, const libra_dims* dims, float scale, cudaStream_t s);
 }  // namespace libra
 
 // setmaxnreg moves registers inside the pool the CTA got at launch (registers per thread as compiled x

@@ -1,4 +1,5 @@
-"""head_dim 256 (the micro-benchmark head shape, Table 1): forward and backward against the CPU oracle."""
+"""head_dim 256 (the micro-benchmark head shape, Table 1): forward and backward against the CPU oracle.  `pairs` runs
+the dV and dK passes over the plan's pair tiles (fp32 accumulators) instead of its key-major tiles."""
 import numpy as np
 import pytest
 import torch
@@ -13,14 +14,16 @@ TOL_O, TOL_G, TOL_LSE = 2e-2, 5e-2, 1e-3
 D = 256
 
 
-def _run(lengths, hq, hkv, seed=0, W=0, H=0, qscale=1.0, backward=True):
+def _run(lengths, hq, hkv, seed=0, W=0, H=0, qscale=1.0, backward=True, pairs=False, chunk=0):
     from paper_2607_23250_b200 import binding as lb
     cu_np = pools.cu_seqlens(lengths)
     T = int(cu_np[-1])
     t = pools.make_tensors(T, hq, hkv, D, seed=seed, scale=qscale)
     q, k, v, dout = (t[n].cuda() for n in ("q", "k", "v", "dout"))
     cu = torch.from_numpy(cu_np).cuda()
-    plan = lb.libra_plan_tiles(cu, H or hq, 256, n_workers=W, tile_kv=128, n_heads_kv=hkv)
+    directions = lb.LIBRA_DIR_Q | (lb.LIBRA_DIR_PAIR if pairs else lb.LIBRA_DIR_KV)
+    plan = lb.libra_plan_tiles(cu, H or hq, 256, n_workers=W, directions=directions, tile_kv=128, n_heads_kv=hkv,
+                               pair_chunk=chunk)
     assert plan.status() == 0
     out, lse = lb.libra_attn_pool_fwd(q, k, v, plan)
     torch.cuda.synchronize()
@@ -32,7 +35,7 @@ def _run(lengths, hq, hkv, seed=0, W=0, H=0, qscale=1.0, backward=True):
     if backward:
         dq, dk, dv = lb.libra_attn_pool_bwd(q, k, v, out, lse, dout, plan)
         torch.cuda.synchronize()
-        plan.busy_times(lb.KERNEL_BWD_DKDV)
+        plan.busy_times(lb.KERNEL_BWD_FUSED if pairs else lb.KERNEL_BWD_DKDV)
         plan.busy_times(lb.KERNEL_BWD_DQ)
         got.update(dq=dq.float().cpu().numpy(), dk=dk.float().cpu().numpy(), dv=dv.float().cpu().numpy())
         ref.update(zip(("dq", "dk", "dv"), oracle.attn_bwd(f["q"], f["k"], f["v"], o_ref, l_ref, f["dout"], cu_np)))
@@ -55,32 +58,38 @@ def test_one_block():
     _check(*_run([64], 1, 1, seed=1))
 
 
-def test_single_sample_multi_tile():
-    _check(*_run([1000], 2, 1, seed=2))
+@pytest.mark.parametrize("pairs", [False, True])
+def test_single_sample_multi_tile(pairs):
+    _check(*_run([1000], 2, 1, seed=2, pairs=pairs, chunk=256))
 
 
-def test_tiny_layout():
+@pytest.mark.parametrize("pairs", [False, True])
+def test_tiny_layout(pairs):
     spec = pools.config(1)      # the 4096-token layout of the full-parity config, at this head width
-    _check(*_run(pools.pool_lengths(spec), 4, 2, seed=3))
+    _check(*_run(pools.pool_lengths(spec), 4, 2, seed=3, pairs=pairs))
 
 
+@pytest.mark.parametrize("pairs", [False, True])
 @pytest.mark.parametrize("seed", range(5))
-def test_random_small_pools(seed):
+def test_random_small_pools(seed, pairs):
     rng = np.random.default_rng(200 + seed)
     T = int(rng.integers(100, 2500))
     lengths = pools.random_layout(rng, T, int(rng.choice([3, 60, 300, 1200])))
     hkv = int(rng.choice([1, 2]))
     hq = hkv * int(rng.choice([1, 2, 4]))
-    _check(*_run(lengths, hq, hkv, seed=seed, W=int(rng.choice([0, 3, 37]))))
+    _check(*_run(lengths, hq, hkv, seed=seed, W=int(rng.choice([0, 3, 37])), pairs=pairs,
+                 chunk=int(rng.choice([0, 128, 512]))))
 
 
-def test_boundary_lengths_and_ragged_end():
-    _check(*_run([1, 63, 64, 65, 127, 128, 129, 255, 257, 1, 1, 40, 50, 60, 300, 5], 4, 2, seed=4))
+@pytest.mark.parametrize("pairs", [False, True])
+def test_boundary_lengths_and_ragged_end(pairs):
+    _check(*_run([1, 63, 64, 65, 127, 128, 129, 255, 257, 1, 1, 40, 50, 60, 300, 5], 4, 2, seed=4, pairs=pairs))
 
 
-def test_microbenchmark_head_shape():
+@pytest.mark.parametrize("pairs", [False, True])
+def test_microbenchmark_head_shape(pairs):
     """Hq 128 / Hkv 4: thirty-two query heads per kv head."""
-    _check(*_run([700, 1, 300, 129, 411], 128, 4, seed=5))
+    _check(*_run([700, 1, 300, 129, 411], 128, 4, seed=5, pairs=pairs))
 
 
 def test_head_shards_wider_than_one_head():
@@ -98,7 +107,8 @@ def test_single_token_pool():
     assert rel_to_max(got["out"], ref["out"]) <= TOL_O
 
 
-def test_sampled_rows_of_a_long_sample():
+@pytest.mark.parametrize("pairs", [False, True])
+def test_sampled_rows_of_a_long_sample(pairs):
     """A 32768-token sample beside short ones: sampled rows of O / LSE / dQ and key columns of dK / dV recomputed by
     the oracle one by one (the whole sample would take it minutes)."""
     from paper_2607_23250_b200 import binding as lb
@@ -108,11 +118,12 @@ def test_sampled_rows_of_a_long_sample():
     T = int(cu_np[-1])
     t = pools.make_tensors(T, hq, hkv, D, seed=9, device="cuda")
     cu = torch.from_numpy(cu_np).cuda()
-    plan = lb.libra_plan_tiles(cu, hq, 256, tile_kv=128, n_heads_kv=hkv)
+    plan = lb.libra_plan_tiles(cu, hq, 256, directions=lb.LIBRA_DIR_Q | (lb.LIBRA_DIR_PAIR if pairs else lb.LIBRA_DIR_KV),
+                               tile_kv=128, n_heads_kv=hkv)
     out, lse = lb.libra_attn_pool_fwd(t["q"], t["k"], t["v"], plan)
     dq, dk, dv = lb.libra_attn_pool_bwd(t["q"], t["k"], t["v"], out, lse, t["dout"], plan)
     torch.cuda.synchronize()
-    for kern in (lb.KERNEL_FWD, lb.KERNEL_BWD_DKDV, lb.KERNEL_BWD_DQ):
+    for kern in (lb.KERNEL_FWD, lb.KERNEL_BWD_FUSED if pairs else lb.KERNEL_BWD_DKDV, lb.KERNEL_BWD_DQ):
         plan.busy_times(kern)
     s, e, n = int(cu_np[1]), int(cu_np[2]), lengths[1]
     G = hq // hkv
