@@ -205,7 +205,10 @@ size_t libra_attn_pool_bwd_workspace_bytes(const libra_plan_t* plan, const libra
  *   bit for bit.  The other directions of the plan are not used by this form.
  *   At head_dim 256 the two-kernel form takes three passes of one kernel after the row statistics (dV and dK
  *   over the key-major lists, dQ over the query-major lists; S is recomputed by each: eight GEMMs per cell), because
- *   the accumulators of dK and dV together would fill the tensor memory.  Same plan, results and determinism.
+ *   the accumulators of dK and dV together would fill the tensor memory.  Same plan, results and determinism.  With a
+ *   pair-tile plan the dV and dK passes walk the pair tiles instead and add their partial sums to fp32 accumulators
+ *   in the workspace (T * hkv * 256 floats each), rounded once at the end; like the fused form, those results agree
+ *   to rounding from run to run, not bit for bit.
  * `workspace_dev` must hold libra_attn_pool_bwd_workspace_bytes bytes, 256-byte aligned; every byte the call reads
  * is written (or cleared) inside the call.  Errors: INVALID_ARG, UNSUPPORTED, PLAN_MISMATCH, CUDA.
  */
