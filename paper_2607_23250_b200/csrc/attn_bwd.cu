@@ -546,9 +546,8 @@ namespace libra {
 // ---- prep kernel ------------------------------------------------------------------------------
 
 // D = <dO, O> per (token, head) and LSE in log2 units; rows in [T, Tpad) get zeros.
-// One warp per (head, 32 consecutive tokens): a row is read by the whole warp (one contiguous 2 D bytes), lane i
-// keeps the sum of row i, so the two statistics leave as one coalesced 128-byte store each.  Rows are taken
-// four at a time to keep several loads in flight.
+// One warp per (head, 32 consecutive tokens): D / 8 lanes read a row with 16-byte loads, lane i ends up with the sum
+// of row i, so the two statistics leave as one coalesced 128-byte store each.  Eight steps' loads are issued at a time.
 template <int D>
 __global__ void k_bwd_prep(const __nv_bfloat16* __restrict__ out, const __nv_bfloat16* __restrict__ dout,
                            const float* __restrict__ lse, int64_t T, int64_t Tpad, int hq, float* __restrict__ dvec,
@@ -559,31 +558,38 @@ __global__ void k_bwd_prep(const __nv_bfloat16* __restrict__ out, const __nv_bfl
     if (w >= groups * hq) return;
     const int h = (int)(w / groups);
     const int64_t t0 = (w % groups) * 32;
-    constexpr int kPer = D / 32;  // 2 or 4 elements per lane
+    // 16-byte loads: D / 8 lanes cover a row, so a warp reads 32 / (D / 8) rows per step; eight steps' loads are
+    // issued before the first is used
+    constexpr int LPR = D / 8, RPS = 32 / LPR, STEPS = 32 / RPS, UNR = STEPS < 8 ? STEPS : 8;
+    const int sub = lane / LPR, part = lane % LPR;
     float mine = 0.f;
-#pragma unroll 2
-    for (int i0 = 0; i0 < 32; i0 += 4) {
-        float acc[4];
+    for (int s0 = 0; s0 < STEPS; s0 += UNR) {
+        uint4 a[UNR], b[UNR];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int64_t t = t0 + i0 + u;
-            acc[u] = 0.f;
+        for (int u = 0; u < UNR; ++u) {
+            const int64_t t = t0 + (s0 + u) * RPS + sub;
+            a[u] = b[u] = make_uint4(0, 0, 0, 0);
             if (t < T) {
-                const __nv_bfloat16* o = out + ((size_t)t * hq + h) * D + lane * kPer;
-                const __nv_bfloat16* g = dout + ((size_t)t * hq + h) * D + lane * kPer;
-#pragma unroll
-                for (int i = 0; i < kPer; i += 2) {
-                    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(o + i));
-                    const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(g + i));
-                    acc[u] += a.x * b.x + a.y * b.y;
-                }
+                a[u] = __ldg(reinterpret_cast<const uint4*>(out + ((size_t)t * hq + h) * D) + part);
+                b[u] = __ldg(reinterpret_cast<const uint4*>(dout + ((size_t)t * hq + h) * D) + part);
             }
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < UNR; ++u) {
+            const uint32_t* x = reinterpret_cast<const uint32_t*>(&a[u]);
+            const uint32_t* y = reinterpret_cast<const uint32_t*>(&b[u]);
+            float acc = 0.f;
 #pragma unroll
-            for (int off = 16; off > 0; off >>= 1) acc[u] += __shfl_xor_sync(0xffffffffu, acc[u], off);
-            if (lane == i0 + u) mine = acc[u];
+            for (int i = 0; i < 4; ++i) {
+                const float2 fa = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&x[i]));
+                const float2 fb = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&y[i]));
+                acc += fa.x * fb.x + fa.y * fb.y;
+            }
+#pragma unroll
+            for (int off = LPR / 2; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+            // row (s0 + u) * RPS + sub of the warp's 32 goes to the lane of that number
+            const float got = __shfl_sync(0xffffffffu, acc, (lane % RPS) * LPR);
+            if (lane / RPS == s0 + u) mine = got;
         }
     }
     const int64_t t = t0 + lane;
