@@ -118,45 +118,38 @@ __global__ void k_rank_blocks(const int64_t* __restrict__ weight_blk, int64_t NB
     if (b < NB) blk_order[rank] = (int32_t)b;
 }
 
-// Sequential placement by one warp.  Worker r's load lives in lane r / PER, register r % PER, so among equal
-// loads the lowest worker index is the lowest slot of the lowest lane.  Per tile: one warp reduction finds the
-// lightest load, a ballot finds the lowest lane that holds it, and that lane adds the weight to its lightest slot
-// and picks its new lightest.  The reduction runs on 32-bit loads relative to a moving base (the loads of a greedy
-// placement never spread by more than the heaviest tile, which is checked to be below 2^31 first; the base follows
-// the minimum whenever that passes 2^30), exact 64-bit loads are kept beside them.  With a heavier tile than that the
-// same steps run on the 64-bit loads themselves (two reductions per tile).
-template <int PER>
+// Sequential placement by one warp (Algorithm 2's greedy rule: the next tile goes to the least-loaded worker, lowest
+// index among equals).  The workers are kept as ONE sorted array of keys (load << 10 | worker) in shared memory; loads
+// stay below 2^53 (checked on the host from the weight total) and there are at most 1024 workers, so a key fits 64 bits.
+//   * Consecutive tiles of EQUAL weight w (the H head shards of a block; the interior pair tiles of a chunk) are placed
+//     in waves.  The first pick takes key[0] and puts it back w heavier; every key below that new key is picked before
+//     any key that has been put back, in array order.  So the next c tiles, c = number of keys below key[0] + w (at most
+//     32 are looked at), go to the first c workers of the array, one each, all at once; their keys come back w heavier,
+//     still in order, and are merged with the rest of the array (every key finds its place by a binary search in the
+//     other sequence).  The result is tile for tile what the one-by-one rule gives.
+//   * When fewer than kWaveMin tiles can go at once, one tile takes the first key and re-inserts it: the warp counts
+//     the keys below the new one and shifts that part of the array down by one.
+constexpr int kPlaceMaxW = 1024;
+constexpr int kWaveMin = 4;
+
+template <int PER>   // PER * 32 >= W
 __global__ void __launch_bounds__(32) k_place(const int64_t* __restrict__ weight_blk,
                                               const int32_t* __restrict__ blk_order /* null: tiles in id order, id =
                                               head * NB + block */, int64_t NB, int64_t NT, int H, int W,
                                               int32_t* __restrict__ cta_of_tile, int32_t* __restrict__ pos,
                                               int32_t* __restrict__ cta_offsets, int64_t* __restrict__ loads) {
+    __shared__ uint64_t key_a[kPlaceMaxW], key_b[kPlaceMaxW];   // the sorted array and its next version
+    __shared__ uint64_t back[32];                               // keys put back by a wave, in order
+    __shared__ int32_t cnt[kPlaceMaxW];                         // tiles per worker so far
     const int lane = threadIdx.x;
-    int64_t wmax = 0;
-    for (int64_t b = lane; b < NB; b += 32) wmax = weight_blk[b] > wmax ? weight_blk[b] : wmax;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        const int64_t other = __shfl_xor_sync(0xffffffffu, wmax, o);
-        wmax = other > wmax ? other : wmax;
-    }
-    const bool narrow = wmax < ((int64_t)1 << 31);
-    int64_t load[PER];      // exact loads of workers lane * PER + k
-    uint32_t rel[PER];      // narrow form: load - base; all ones: no such worker
-    int32_t cnt[PER];
-#pragma unroll
-    for (int k = 0; k < PER; ++k) {
-        load[k] = 0;
-        cnt[k] = 0;
-        rel[k] = (lane * PER + k < W) ? 0u : 0xffffffffu;
-    }
-    // the lane's lightest slot (lowest slot among equals)
-    uint32_t best = rel[0];
-    int64_t best64 = rel[0] == 0xffffffffu ? INT64_MAX : 0;
-    int slot = 0;
+    uint64_t* cur = key_a;
+    uint64_t* nxt = key_b;
+    for (int r = lane; r < W; r += 32) { cur[r] = (uint64_t)r; cnt[r] = 0; }
+    __syncwarp();
     for (int64_t x0 = 0; x0 < NT; x0 += 32) {
-        // each lane fetches one upcoming tile, then they are broadcast one by one
+        // each lane fetches one upcoming tile
         const int64_t xl = x0 + lane;
-        int64_t w_l = 0;
+        int64_t w_l = -1;
         int32_t t_l = 0;
         if (xl < NT) {
             if (blk_order) {
@@ -169,54 +162,94 @@ __global__ void __launch_bounds__(32) k_place(const int64_t* __restrict__ weight
             }
         }
         const int lim = (int)((NT - x0 < 32) ? NT - x0 : 32);
-        for (int i = 0; i < lim; ++i) {
+        int i = 0;
+        while (i < lim) {
             const int64_t w = __shfl_sync(0xffffffffu, w_l, i);
-            const int32_t t = __shfl_sync(0xffffffffu, t_l, i);
-            unsigned tie;
-            if (narrow) {
-                uint32_t m = __reduce_min_sync(0xffffffffu, best);
-                if (m > (1u << 30)) {   // move the base up to the minimum (uniform branch)
-#pragma unroll
-                    for (int k = 0; k < PER; ++k)
-                        if (rel[k] != 0xffffffffu) rel[k] -= m;
-                    if (best != 0xffffffffu) best -= m;
-                    m = 0;
-                }
-                tie = __ballot_sync(0xffffffffu, best == m);
-            } else {
-                const uint32_t hi = (uint32_t)((uint64_t)best64 >> 32), lo = (uint32_t)best64;
-                const uint32_t mhi = __reduce_min_sync(0xffffffffu, hi);
-                const uint32_t mlo = __reduce_min_sync(0xffffffffu, hi == mhi ? lo : 0xffffffffu);
-                tie = __ballot_sync(0xffffffffu, hi == mhi && lo == mlo);
+            // length of the run of equal weights that starts at tile i of this batch
+            const unsigned same = __ballot_sync(0xffffffffu, w_l == w) >> i;
+            int n = (~same == 0u) ? 32 : __ffs(~same) - 1;
+            if (n > lim - i) n = lim - i;
+            if (w == 0) {
+                // weightless tiles all go to the first worker and change nothing else
+                const int r0 = (int)(cur[0] & 1023u);
+                const int base = cnt[r0];
+                __syncwarp();
+                if (lane >= i && lane < i + n) { cta_of_tile[t_l] = r0; pos[t_l] = base + (lane - i); }
+                if (lane == 0) cnt[r0] = base + n;
+                __syncwarp();
+                i += n;
+                continue;
             }
-            if (lane == __ffs(tie) - 1) {
-                int32_t my_pos = 0;
+            // tiles that can go at once: keys below the first key put back (a prefix of the sorted array)
+            const uint64_t add = (uint64_t)w << 10;
+            const uint64_t first = cur[0];
+            const uint64_t mine_k = lane < W ? cur[lane] : ~0ull;
+            int take = __popc(__ballot_sync(0xffffffffu, mine_k < first + add));
+            if (take > n) take = n;
+            if (take < kWaveMin) {
+                // one tile: the first key, put back w heavier at its new place
+                const uint64_t k1 = first + add;
+                const int r0 = (int)(first & 1023u);
+                int below = 0;                                    // keys of cur[1..W) below the new key
+                uint64_t mine[PER];
 #pragma unroll
-                for (int k = 0; k < PER; ++k) {
-                    if (k == slot) { load[k] += w; rel[k] += (uint32_t)w; my_pos = cnt[k]++; }
+                for (int u = 0; u < PER; ++u) {
+                    const int idx = 1 + lane + 32 * u;
+                    mine[u] = idx < W ? cur[idx] : ~0ull;
+                    below += (idx < W && mine[u] < k1) ? 1 : 0;
                 }
-                cta_of_tile[t] = lane * PER + slot;
-                pos[t] = my_pos;
-                if (narrow) {
-                    best = rel[0];
-                    slot = 0;
 #pragma unroll
-                    for (int k = 1; k < PER; ++k)
-                        if (rel[k] < best) { best = rel[k]; slot = k; }
-                } else {
-                    best64 = INT64_MAX;
+                for (int o = 16; o > 0; o >>= 1) below += __shfl_xor_sync(0xffffffffu, below, o);
+                __syncwarp();
 #pragma unroll
-                    for (int k = PER - 1; k >= 0; --k)
-                        if (lane * PER + k < W && load[k] <= best64) { best64 = load[k]; slot = k; }
+                for (int u = 0; u < PER; ++u) {
+                    const int idx = 1 + lane + 32 * u;
+                    if (idx <= below) cur[idx - 1] = mine[u];     // the keys below the new one move down by one
                 }
+                if (lane == 0) cur[below] = k1;
+                const int32_t t = __shfl_sync(0xffffffffu, t_l, i);
+                if (lane == 0) { cta_of_tile[t] = r0; pos[t] = cnt[r0]; cnt[r0] += 1; }
+                __syncwarp();
+                i += 1;
+                continue;
             }
+            // ---- a wave: tile i + s goes to the worker of key[s], s < take; the workers are distinct ----
+            {
+                const int32_t t = __shfl_sync(0xffffffffu, t_l, (i + lane) & 31);
+                if (lane < take) {
+                    const int r = (int)(mine_k & 1023u);
+                    cta_of_tile[t] = r;
+                    pos[t] = cnt[r];
+                    cnt[r] += 1;
+                    back[lane] = mine_k + add;
+                }
+                __syncwarp();
+                // the rest of the array and the keys put back, merged into the new sorted array
+                const int na = W - take;
+                for (int idx = lane; idx < na; idx += 32) {       // a key of the array: keys put back that are below it
+                    const uint64_t k = cur[take + idx];
+                    int lo = 0, hi = take;
+                    while (lo < hi) { const int mid = (lo + hi) >> 1; if (back[mid] < k) lo = mid + 1; else hi = mid; }
+                    nxt[idx + lo] = k;
+                }
+                if (lane < take) {                                 // a key put back: keys of the array below it
+                    const uint64_t k = back[lane];
+                    int lo = 0, hi = na;
+                    while (lo < hi) { const int mid = (lo + hi) >> 1; if (cur[take + mid] < k) lo = mid + 1; else hi = mid; }
+                    nxt[lane + lo] = k;
+                }
+                __syncwarp();
+                uint64_t* tmp = cur; cur = nxt; nxt = tmp;
+            }
+            i += take;
         }
     }
-#pragma unroll
-    for (int k = 0; k < PER; ++k) {
-        const int r = lane * PER + k;
-        if (r < W) { loads[r] = load[k]; cta_offsets[r + 1] = cnt[k]; }
+    __syncwarp();
+    for (int idx = lane; idx < W; idx += 32) {
+        const uint64_t k = cur[idx];
+        loads[k & 1023u] = (int64_t)(k >> 10);
     }
+    for (int r = lane; r < W; r += 32) cta_offsets[r + 1] = cnt[r];
     __syncwarp();
     if (lane == 0) {  // counts -> offsets
         cta_offsets[0] = 0;
