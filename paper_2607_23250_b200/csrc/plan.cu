@@ -121,12 +121,12 @@ __global__ void k_rank_blocks(const int64_t* __restrict__ weight_blk, int64_t NB
 // Sequential placement by one warp (Algorithm 2's greedy rule: the next tile goes to the least-loaded worker, lowest
 // index among equals).  The workers are kept as ONE sorted array of keys (load << 10 | worker) in shared memory; loads
 // stay below 2^53 (checked on the host from the weight total) and there are at most 1024 workers, so a key fits 64 bits.
-//   * Consecutive tiles of EQUAL weight w (the H head shards of a block; the interior pair tiles of a chunk) are placed
-//     in waves.  The first pick takes key[0] and puts it back w heavier; every key below that new key is picked before
-//     any key that has been put back, in array order.  So the next c tiles, c = number of keys below key[0] + w (at most
-//     32 are looked at), go to the first c workers of the array, one each, all at once; their keys come back w heavier,
-//     still in order, and are merged with the rest of the array (every key finds its place by a binary search in the
-//     other sequence).  The result is tile for tile what the one-by-one rule gives.
+//   * Consecutive tiles are placed in waves.  Tile s of a batch goes to key[s], the s-th worker of the array, as long
+//     as key[s] lies below every key put back by the tiles before it (key[s'] + w[s'], s' < s): nothing put back can
+//     then overtake it.  The longest such prefix (at most 32 tiles) is placed at once, one tile per worker; the keys
+//     put back are ranked among themselves and merged with the rest of the array (every key finds its place by a
+//     binary search in the other sequence).  With equal weights (the H head shards of a block) the condition is
+//     key[s] < key[0] + w.  The result is tile for tile what the one-by-one rule gives.
 //   * When fewer than kWaveMin tiles can go at once, one tile takes the first key and re-inserts it: the warp counts
 //     the keys below the new one and shifts that part of the array down by one.
 constexpr int kPlaceMaxW = 1024;
@@ -140,6 +140,7 @@ __global__ void __launch_bounds__(32) k_place(const int64_t* __restrict__ weight
                                               int32_t* __restrict__ cta_offsets, int64_t* __restrict__ loads) {
     __shared__ uint64_t key_a[kPlaceMaxW], key_b[kPlaceMaxW];   // the sorted array and its next version
     __shared__ uint64_t back[32];                               // keys put back by a wave, in order
+    __shared__ uint64_t put_raw[32];                            // the same in tile order
     __shared__ int32_t cnt[kPlaceMaxW];                         // tiles per worker so far
     const int lane = threadIdx.x;
     uint64_t* cur = key_a;
@@ -165,12 +166,11 @@ __global__ void __launch_bounds__(32) k_place(const int64_t* __restrict__ weight
         int i = 0;
         while (i < lim) {
             const int64_t w = __shfl_sync(0xffffffffu, w_l, i);
-            // length of the run of equal weights that starts at tile i of this batch
-            const unsigned same = __ballot_sync(0xffffffffu, w_l == w) >> i;
-            int n = (~same == 0u) ? 32 : __ffs(~same) - 1;
-            if (n > lim - i) n = lim - i;
             if (w == 0) {
                 // weightless tiles all go to the first worker and change nothing else
+                const unsigned same = __ballot_sync(0xffffffffu, w_l == 0) >> i;
+                int n = (~same == 0u) ? 32 : __ffs(~same) - 1;
+                if (n > lim - i) n = lim - i;
                 const int r0 = (int)(cur[0] & 1023u);
                 const int base = cnt[r0];
                 __syncwarp();
@@ -180,12 +180,23 @@ __global__ void __launch_bounds__(32) k_place(const int64_t* __restrict__ weight
                 i += n;
                 continue;
             }
-            // tiles that can go at once: keys below the first key put back (a prefix of the sorted array)
-            const uint64_t add = (uint64_t)w << 10;
+            // lane s looks at tile i + s of the batch and at key[s]
+            const int64_t w_s = __shfl_sync(0xffffffffu, w_l, (i + lane) & 31);
+            const bool live = i + lane < lim && lane < W && w_s > 0;
             const uint64_t first = cur[0];
+            const uint64_t add = (uint64_t)w << 10;
             const uint64_t mine_k = lane < W ? cur[lane] : ~0ull;
-            int take = __popc(__ballot_sync(0xffffffffu, mine_k < first + add));
-            if (take > n) take = n;
+            const uint64_t put = live ? mine_k + ((uint64_t)w_s << 10) : ~0ull;
+            uint64_t before = put;                                // min of the keys put back by the lanes below this one
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint64_t other = __shfl_up_sync(0xffffffffu, before, o);
+                if (lane >= o && other < before) before = other;
+            }
+            before = __shfl_up_sync(0xffffffffu, before, 1);
+            if (lane == 0) before = ~0ull;
+            const unsigned fits = __ballot_sync(0xffffffffu, live && mine_k < before);
+            const int take = (~fits == 0u) ? 32 : __ffs(~fits) - 1;
             if (take < kWaveMin) {
                 // one tile: the first key, put back w heavier at its new place
                 const uint64_t k1 = first + add;
@@ -221,7 +232,13 @@ __global__ void __launch_bounds__(32) k_place(const int64_t* __restrict__ weight
                     cta_of_tile[t] = r;
                     pos[t] = cnt[r];
                     cnt[r] += 1;
-                    back[lane] = mine_k + add;
+                    put_raw[lane] = put;
+                }
+                __syncwarp();
+                if (lane < take) {   // the keys put back, ranked among themselves (all keys differ)
+                    int rank = 0;
+                    for (int j = 0; j < take; ++j) rank += put_raw[j] < put ? 1 : 0;
+                    back[rank] = put;
                 }
                 __syncwarp();
                 // the rest of the array and the keys put back, merged into the new sorted array
