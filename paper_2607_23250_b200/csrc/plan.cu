@@ -132,12 +132,31 @@ __global__ void k_rank_blocks(const int64_t* __restrict__ weight_blk, int64_t NB
 constexpr int kPlaceMaxW = 1024;
 constexpr int kWaveMin = 4;
 
+struct PlaceJob {
+    const int64_t* weight_blk;
+    const int32_t* blk_order;   // null: tiles in id order, id = head * NB + block
+    int64_t NB, NT;
+    int H, W;
+    int32_t* cta_of_tile;
+    int32_t* pos;
+    int32_t* cta_offsets;
+    int64_t* loads;
+};
+struct PlaceJobs {
+    PlaceJob job[3];            // the directions of a plan are independent: one block (one warp) each
+};
+
 template <int PER>   // PER * 32 >= W
-__global__ void __launch_bounds__(32) k_place(const int64_t* __restrict__ weight_blk,
-                                              const int32_t* __restrict__ blk_order /* null: tiles in id order, id =
-                                              head * NB + block */, int64_t NB, int64_t NT, int H, int W,
-                                              int32_t* __restrict__ cta_of_tile, int32_t* __restrict__ pos,
-                                              int32_t* __restrict__ cta_offsets, int64_t* __restrict__ loads) {
+__global__ void __launch_bounds__(32) k_place(const PlaceJobs jobs) {
+    const PlaceJob& jb = jobs.job[blockIdx.x];
+    const int64_t* __restrict__ weight_blk = jb.weight_blk;
+    const int32_t* __restrict__ blk_order = jb.blk_order;
+    const int64_t NB = jb.NB, NT = jb.NT;
+    const int H = jb.H, W = jb.W;
+    int32_t* __restrict__ cta_of_tile = jb.cta_of_tile;
+    int32_t* __restrict__ pos = jb.pos;
+    int32_t* __restrict__ cta_offsets = jb.cta_offsets;
+    int64_t* __restrict__ loads = jb.loads;
     __shared__ uint64_t key_a[kPlaceMaxW], key_b[kPlaceMaxW];   // the sorted array and its next version
     __shared__ uint64_t back[32];                               // keys put back by a wave, in order
     __shared__ uint64_t put_raw[32];                            // the same in tile order
@@ -417,7 +436,8 @@ static int count_pair_blocks(libra_plan* p, PlanDir& d, PairTables& tb) {
     }
 }
 
-static int build_dir(libra_plan* p, PlanDir& d, int key_major, const libra_plan_opts& o, bool pairs = false) {
+// First half of a direction: sizes, allocations, weights and block order; fills the placement job.
+static int build_dir(libra_plan* p, PlanDir& d, int key_major, const libra_plan_opts& o, bool pairs, PlaceJob* job) {
     const int64_t T = p->T;
     PairTables tb;
     if (pairs) {
@@ -465,24 +485,38 @@ static int build_dir(libra_plan* p, PlanDir& d, int key_major, const libra_plan_
     else
         k_block_weights<<<grid_for(d.NB, 128), 128, 0, s>>>(p->d_tok_start, p->d_tok_end, T, d.tile, d.NB, key_major,
                                                             d.d_weight_blk);
-    const int32_t* ord = pairs ? nullptr : d.d_blk_order;   // pair tiles are placed in id order
     if (!pairs) k_rank_blocks<<<grid_for(d.NB, 256), 256, 0, s>>>(d.d_weight_blk, d.NB, d.d_blk_order);
-    if (d.W <= 160)
-        k_place<5><<<1, 32, 0, s>>>(d.d_weight_blk, ord, d.NB, d.NT, d.H, d.W, d.d_cta_of_tile, d.d_pos,
-                                    d.d_cta_offsets, d.d_loads);
-    else if (d.W <= 320)
-        k_place<10><<<1, 32, 0, s>>>(d.d_weight_blk, ord, d.NB, d.NT, d.H, d.W, d.d_cta_of_tile, d.d_pos,
-                                     d.d_cta_offsets, d.d_loads);
+    job->weight_blk = d.d_weight_blk;
+    job->blk_order = pairs ? nullptr : d.d_blk_order;   // pair tiles are placed in id order
+    job->NB = d.NB; job->NT = d.NT; job->H = d.H; job->W = d.W;
+    job->cta_of_tile = d.d_cta_of_tile; job->pos = d.d_pos; job->cta_offsets = d.d_cta_offsets; job->loads = d.d_loads;
+    count_launch(2);
+    return cudaGetLastError() == cudaSuccess ? LIBRA_OK : LIBRA_ERR_CUDA;
+}
+
+// The placements of all directions in one launch (a block of one warp per direction).
+static int place_all(const PlaceJobs& jobs, int n, int max_w, cudaStream_t s) {
+    if (n == 0) return LIBRA_OK;
+    if (max_w <= 160)
+        k_place<5><<<n, 32, 0, s>>>(jobs);
+    else if (max_w <= 320)
+        k_place<10><<<n, 32, 0, s>>>(jobs);
     else
-        k_place<32><<<1, 32, 0, s>>>(d.d_weight_blk, ord, d.NB, d.NT, d.H, d.W, d.d_cta_of_tile, d.d_pos,
-                                     d.d_cta_offsets, d.d_loads);
+        k_place<32><<<n, 32, 0, s>>>(jobs);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? LIBRA_OK : LIBRA_ERR_CUDA;
+}
+
+// Second half of a direction: the per-worker lists from the placement.
+static int finish_dir(libra_plan* p, PlanDir& d, bool pairs) {
+    cudaStream_t s = p->stream;
     k_scatter_lists<<<grid_for(d.NT, 256), 256, 0, s>>>(d.d_cta_of_tile, d.d_pos, d.d_cta_offsets, d.NT,
                                                         d.d_cta_tiles);
     if (pairs)   // placed in id order: the lists already are in execution order
         cudaMemcpyAsync(d.d_cta_exec, d.d_cta_tiles, sizeof(int32_t) * d.NT, cudaMemcpyDeviceToDevice, s);
     else
         k_exec_order<<<d.W, 256, 0, s>>>(d.d_cta_offsets, d.d_cta_tiles, d.H, d.NB, d.d_cta_exec);
-    count_launch(5);
+    count_launch(2);
     d.enabled = 1;
     return cudaGetLastError() == cudaSuccess ? LIBRA_OK : LIBRA_ERR_CUDA;
 }
@@ -533,22 +567,32 @@ extern "C" int libra_plan_tiles(const int32_t* cu_seqlens_dev, int n_samples, in
         count_launch(2);
         const int dirs = o.directions ? o.directions : (LIBRA_DIR_Q | LIBRA_DIR_KV);
         const int W = o.n_workers ? o.n_workers : sms;
+        PlaceJobs jobs = {};
+        int n_jobs = 0;
+        bool built[3] = {false, false, false};
         if (dirs & LIBRA_DIR_Q) {
             PlanDir& d = p->dir[0];
             d.tile = tile_q; d.H = n_heads; d.W = W;
-            rc = build_dir(p, d, 0, o);
+            rc = build_dir(p, d, 0, o, false, &jobs.job[n_jobs]);
+            if (rc == LIBRA_OK) { built[0] = true; ++n_jobs; }
         }
         if (rc == LIBRA_OK && (dirs & LIBRA_DIR_KV)) {
             PlanDir& d = p->dir[1];
             d.tile = o.tile_kv ? o.tile_kv : 128; d.H = o.n_heads_kv ? o.n_heads_kv : n_heads; d.W = W;
-            rc = build_dir(p, d, 1, o);
+            rc = build_dir(p, d, 1, o, false, &jobs.job[n_jobs]);
+            if (rc == LIBRA_OK) { built[1] = true; ++n_jobs; }
         }
         if (rc == LIBRA_OK && (dirs & LIBRA_DIR_PAIR)) {
             PlanDir& d = p->dir[2];
             d.tile = o.tile_kv ? o.tile_kv : 128; d.H = o.n_heads_kv ? o.n_heads_kv : n_heads; d.W = W;
             d.chunk = o.pair_chunk ? o.pair_chunk : 2048;
-            rc = d.chunk % d.tile ? LIBRA_ERR_INVALID_ARG : build_dir(p, d, 1, o, true);
+            rc = d.chunk % d.tile ? LIBRA_ERR_INVALID_ARG : build_dir(p, d, 1, o, true, &jobs.job[n_jobs]);
+            if (rc == LIBRA_OK) { built[2] = true; ++n_jobs; }
         }
+        // the directions are independent: their placements run side by side, one warp each
+        if (rc == LIBRA_OK) rc = place_all(jobs, n_jobs, W, s);
+        for (int k = 0; k < 3 && rc == LIBRA_OK; ++k)
+            if (built[k]) rc = finish_dir(p, p->dir[k], k == 2);
     }
     if (rc != LIBRA_OK) {
         libra_plan_destroy(p);
