@@ -49,3 +49,34 @@ def test_head_slices_reproduce_the_unsharded_call(hq, hkv, world):
     if shared:     # partial sums over the query heads of a kv head, added as the sub-group all-reduce would
         for got, want in ((dk_sum, dk.float()), (dv_sum, dv.float())):
             assert float((got - want).abs().max()) <= 2e-2 * float(want.abs().max())
+
+
+def test_head_slices_with_the_fused_backward():
+    """The same with pair-tile plans, i.e. the fused backward the benchmark runs per rank: its fp32 accumulation order
+    varies from run to run, so the slices agree with the unsharded call to rounding (forward still bit for bit)."""
+    from paper_2607_23250_b200 import binding as lb
+    lengths = [700, 1, 300, 129, 411, 260]
+    hq, hkv, world = 8, 4, 4
+    cu_np = pools.cu_seqlens(lengths)
+    t = pools.make_tensors(int(cu_np[-1]), hq, hkv, 128, seed=43, device="cuda")
+    cu = torch.from_numpy(cu_np).cuda()
+
+    def run(q, k, v, dout):
+        plan = lb.libra_plan_tiles(cu, q.shape[1], 256, directions=lb.LIBRA_DIR_Q | lb.LIBRA_DIR_PAIR, tile_kv=128,
+                                   n_heads_kv=k.shape[1])
+        out, lse = lb.libra_attn_pool_fwd(q, k, v, plan)
+        dq, dk, dv = lb.libra_attn_pool_bwd(q, k, v, out, lse, dout, plan)
+        torch.cuda.synchronize()
+        plan.busy_times(lb.KERNEL_BWD_FUSED)
+        plan.destroy()
+        return out, lse, dq, dk, dv
+
+    out, lse, dq, dk, dv = run(t["q"], t["k"], t["v"], t["dout"])
+    for r in range(world):
+        s = sharding.head_groups(hq, hkv, world, r)
+        qs, ks, vs, dos = sharding.slice_heads(s, t["q"], t["k"], t["v"], t["dout"])
+        o_r, l_r, dq_r, dk_r, dv_r = run(qs, ks, vs, dos)
+        qh, kh = list(s.q_heads), list(s.kv_heads)
+        assert torch.equal(o_r, out[:, qh]) and torch.equal(l_r, lse[qh])
+        for got, want in ((dq_r, dq[:, qh]), (dk_r, dk[:, kh]), (dv_r, dv[:, kh])):
+            assert float((got.float() - want.float()).abs().max()) <= 2.0 ** -7 * float(want.float().abs().max())
