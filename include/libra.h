@@ -82,7 +82,7 @@ typedef struct {
     int     unit_cost_q;   /* LIBRA_WEIGHT_BLOCKS: added per row chunk of a query-major tile, in
                               eighths of a block (>= 0)                                             */
     int     unit_cost_kv;  /* same per key chunk of a key-major tile                                */
-    int     pair_chunk;    /* LIBRA_DIR_PAIR: tokens per query chunk, a multiple of the key block; 0 = 2048
+    int     pair_chunk;    /* LIBRA_DIR_PAIR: tokens per query chunk, a multiple of the key block; 0 = 4096
                               (doubled by the planner while there are more than 262144 pair-blocks)    */
 } libra_plan_opts;
 

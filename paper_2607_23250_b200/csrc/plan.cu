@@ -585,7 +585,7 @@ extern "C" int libra_plan_tiles(const int32_t* cu_seqlens_dev, int n_samples, in
         if (rc == LIBRA_OK && (dirs & LIBRA_DIR_PAIR)) {
             PlanDir& d = p->dir[2];
             d.tile = o.tile_kv ? o.tile_kv : 128; d.H = o.n_heads_kv ? o.n_heads_kv : n_heads; d.W = W;
-            d.chunk = o.pair_chunk ? o.pair_chunk : 2048;
+            d.chunk = o.pair_chunk ? o.pair_chunk : 4096;
             rc = d.chunk % d.tile ? LIBRA_ERR_INVALID_ARG : build_dir(p, d, 1, o, true, &jobs.job[n_jobs]);
             if (rc == LIBRA_OK) { built[2] = true; ++n_jobs; }
         }
