@@ -254,6 +254,25 @@ class Pool:
             busy[n] = round(float(b.max() / b.mean()), 4)
         return ms, kern, busy
 
+    def tile_time_corr(self, plan=None):
+        """Pearson correlation between the plan's tile weights and the time the last launch spent on each tile
+        (forward: query-major tiles; fused backward: pair tiles); the paper notes that a FLOPs-balanced assignment
+        need not be time-balanced."""
+        lb, plan = self.lb, plan or self.plan
+        out = {}
+        legs = [("fwd", lb.KERNEL_FWD, lb.LIBRA_DIR_Q)]
+        if self.fused and self.d == 128:
+            legs.append(("bwd_fused", lb.KERNEL_BWD_FUSED, lb.LIBRA_DIR_PAIR))
+        if self.d == 256:
+            return out                                 # the 256-wide kernel keeps no per-tile times
+        for name, kern, direction in legs:
+            ns = plan.tile_times(kern).astype(np.float64)
+            w = plan.export(direction)["weight"].astype(np.float64)
+            ran = ns > 0
+            if ran.sum() > 2 and w[ran].std() > 0 and ns[ran].std() > 0:
+                out[name] = round(float(np.corrcoef(w[ran], ns[ran])[0, 1]), 4)
+        return out
+
     def destroy(self):
         if self.plan is not None:
             self.plan.destroy()
@@ -312,6 +331,7 @@ def run_ours(args):
         sampler.start()
     ms_local, kern, busy = pool.timed(args.steps, max(args.warmup, 3), barrier)
     launches = pool.launches
+    corr = pool.tile_time_corr()
     clocks = sampler.stop() if rank == 0 else None
     ms_per_step, work = sharding.aggregate(ms_local, float(pool.ff + pool.fb), device=dev)
     value = work / (ms_per_step * 1e-3) / 1e12
@@ -324,7 +344,7 @@ def run_ours(args):
         ms2, _, busy2 = pool.timed(args.steps, 3, barrier, plan=plan2)
         alt = {"tile_weight": "blocks (time proxy)" if other else "causal pairs (Eq. 6)",
                "value": round((pool.ff + pool.fb) / (ms2 * 1e-3) / 1e12, 2), "unit": "TFLOP/s",
-               "busy_max_over_mean": busy2}
+               "busy_max_over_mean": busy2, "tile_time_weight_corr": pool.tile_time_corr(plan2)}
         plan2.destroy()
 
     e2e = None
@@ -335,6 +355,7 @@ def run_ours(args):
     if rank == 0:
         line = headline(args, world, spec, pool, value, ms_per_step, ms_local, kern, busy, clocks, launches, e2e,
                         plan_ms, alt, shard)
+        line["tile_time_weight_corr"] = corr
     pool.destroy()
     del pool
     torch.cuda.empty_cache()
@@ -364,6 +385,7 @@ def skewed_pools(args, lb, dev, barrier):
         pool.build()
         ms, kern, busy = pool.timed(steps, 1 if cfg == 4 else 2, barrier)
         rec = pool_line(pool, ms, kern, busy)
+        rec["tile_time_weight_corr"] = pool.tile_time_corr()
         rec.update(steps=steps, samples=len(pool.lengths), max_sample=int(max(pool.lengths)), tokens=spec.total_tokens,
                    heads=f"Hq {spec.hq} / Hkv {spec.hkv}")
         out[name] = rec

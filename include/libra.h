@@ -343,6 +343,15 @@ int libra_tap_schedule(const int32_t* cu_seqlens_dev, int n_samples, const int32
  * cu_seqlens was malformed and the kernels therefore did no work. */
 int libra_busy_times(const libra_plan_t* plan, int which, uint64_t* ns_host);
 
+/* Time each tile took in the most recent launch of the forward kernel (which = LIBRA_KERNEL_FWD, tiles of the
+ * query-major direction) or of the fused backward kernel (LIBRA_KERNEL_BWD_FUSED, pair tiles): nanoseconds of the
+ * global timer from the moment a compute thread of the CTA turns to the tile until it has finished the tile's
+ * last output, indexed by tile id; 0 for a tile that was not run.  With the plan's weights (libra_plan_export)
+ * this shows how well the tile weight predicts time: the paper notes that a FLOPs-balanced assignment need not
+ * be time-balanced (Section 3.2).  Copies n_tiles values to ns_host (HOST) and synchronises the device.
+ * Errors: INVALID_ARG (another kernel id), PLAN_MISMATCH (the plan lacks the direction), CUDA. */
+int libra_tile_times(const libra_plan_t* plan, int which, uint32_t* ns_host);
+
 /* Budget of one device-side wait of the attention kernels launched with this plan, in nanoseconds
  * (0 restores the default of 2 s, the maximum is 4 s).  Every wait on a barrier inside the kernels
  * is bounded: a wait that outlives the budget makes its CTA stop issuing work, let the copies and

@@ -29,7 +29,7 @@ ERR_SCRATCH_TOO_SMALL = -9
 EXPORTS = ["libra_plan_tiles", "libra_plan_info", "libra_plan_status", "libra_plan_export",
            "libra_plan_export_pairs", "libra_plan_destroy", "libra_attn_pool_fwd", "libra_attn_pool_bwd_workspace_bytes",
            "libra_attn_pool_bwd", "libra_attn_pool_bwd_noalloc_max_bytes", "libra_attn_pool_bwd_noalloc",
-           "libra_tap_schedule", "libra_busy_times", "libra_plan_set_wait_limit_ns", "libra_plan_inject_stall", "libra_plan_set_timing", "libra_kernel_time_ms", "libra_kernel_times_ms", "libra_selftest_wait_timeout", "libra_launch_count",
+           "libra_tap_schedule", "libra_busy_times", "libra_tile_times", "libra_plan_set_wait_limit_ns", "libra_plan_inject_stall", "libra_plan_set_timing", "libra_kernel_time_ms", "libra_kernel_times_ms", "libra_selftest_wait_timeout", "libra_launch_count",
            "libra_strerror"]
 
 
@@ -144,6 +144,14 @@ class Plan:
         ms = ctypes.c_float()
         _check(_lib.libra_kernel_time_ms(self._h, which, ctypes.byref(ms)), "libra_kernel_time_ms")
         return float(ms.value)
+
+    def tile_times(self, which=KERNEL_FWD):
+        """Nanoseconds each tile took in the last launch of the forward (query-major tiles) or the fused backward
+        (pair tiles), indexed by tile id (uint32 numpy array)."""
+        nt = self.info(LIBRA_DIR_PAIR if which == KERNEL_BWD_FUSED else LIBRA_DIR_Q)["n_tiles"]
+        out = np.zeros(nt, dtype=np.uint32)
+        _check(_lib.libra_tile_times(self._h, which, _np(out)), "libra_tile_times")
+        return out
 
     def kernel_times_ms(self, which=KERNEL_FWD, capacity=64):
         """Durations (ms) of the most recent recorded launches of kernel `which`, oldest first."""

@@ -708,6 +708,7 @@ static int launch_fused(const void* q_dev, const void* k_dev, const void* v_dev,
     fp.status = plan->d_status + 2; fp.plan_status = plan->d_status;
     fp.wait_limit_ns = plan->wait_limit_ns; fp.inject_stall = plan->inject_stall;
     fp.busy = d.d_busy;
+    fp.tile_ns = d.d_tile_ns;
     time_begin(mp, 4, s);
     cudaMemsetAsync(dq_acc, 0, ws.dq_acc_bytes + 2 * ws.dkv_acc_bytes, s);   // the three accumulators are contiguous
     k_attn_bwd_fused<<<d.W, kFusedThreads, FusedSmem::kBytes, s>>>(tq, tk, tv, tdo, tacc, fp);

@@ -72,6 +72,7 @@ struct FusedParams {
     uint32_t wait_limit_ns;
     int inject_stall;
     uint64_t* busy;
+    uint32_t* tile_ns;        // [tiles] time spent on each pair tile (first exp thread), ns
 };
 
 // The row blocks [i0, i1] a pair tile walks for every head of its group.
@@ -453,6 +454,7 @@ k_attn_bwd_fused(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         uint32_t ucnt = 0, it_all = 0;
         bool ok = true;
         for (int idx = unit_begin; idx < unit_end && ok; ++idx) {
+            const uint64_t tile_t0 = threadIdx.x == 0 ? globaltimer_ns() : 0;
             const FusedUnit u = fused_unit(p, p.cta_tiles[idx]);
             const int n_it = G * u.n_blk;
             const int64_t key = u.k0 + r;
@@ -567,6 +569,7 @@ k_attn_bwd_fused(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             }
             tc_fence_before();
             mbar_arrive(bar_dkvempty);
+            if (threadIdx.x == 0) p.tile_ns[p.cta_tiles[idx]] = (uint32_t)(globaltimer_ns() - tile_t0);
         }
         // every bulk reduce this warp issued has completed before the CTA leaves
         if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");

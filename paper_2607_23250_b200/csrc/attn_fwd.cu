@@ -61,6 +61,7 @@ struct FwdParams {
     uint32_t wait_limit_ns;  // budget of one device-side wait
     int inject_stall;        // test aid: the producer issues no loads, so the consumers' waits run out
     uint64_t* busy;    // [2 * gridDim.x]
+    uint32_t* tile_ns; // [tiles] time spent on each tile (slot 0's first softmax thread), ns
 };
 
 // Range of key blocks slot g of a tile sees; empty (lo > hi) if the slot lies past T.
@@ -309,6 +310,7 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
             const int64_t qs = (int64_t)(t / p.H) * (2 * kBM) + g * kBM;
             const SlotRange rg = slot_range(p.tok_start, p.T, qs);
             if (rg.lo > rg.hi) continue;  // slot past the end of the pool
+            const uint64_t tile_t0 = threadIdx.x == 0 ? globaltimer_ns() : 0;
             const int64_t row = qs + row_in_tile;
             const bool row_ok = row < p.T;
             const int kstart = row_ok ? p.tok_start[row] : 0;
@@ -441,6 +443,7 @@ k_attn_fwd(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUt
                 // after this group's next p_ready arrival, which follows in program order
                 tc_fence_before();
             }
+            if (threadIdx.x == 0 && ok) p.tile_ns[t] = (uint32_t)(globaltimer_ns() - tile_t0);
         }
     }
 
@@ -580,6 +583,7 @@ extern "C" int libra_attn_pool_fwd(const void* q_dev, const void* k_dev, const v
     prm.wait_limit_ns = plan->wait_limit_ns;
     prm.inject_stall = plan->inject_stall;
     prm.busy = d.d_busy;
+    prm.tile_ns = d.d_tile_ns;
     cudaMemsetAsync(plan->d_status + 1, 0, sizeof(int), s);   // the word reports the most recent launch
     time_begin(mp, 0, s);
     rc = dims->head_dim == 128 ? launch_fwd<128>(tq, tk, tv, prm, d.W, s) : launch_fwd<64>(tq, tk, tv, prm, d.W, s);

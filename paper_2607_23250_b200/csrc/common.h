@@ -28,6 +28,7 @@ struct PlanDir {
     int64_t* d_loads = nullptr;        // [W]
     uint64_t* d_busy = nullptr;        // [2*W] (start, end) global-timer stamps of the last run
     uint64_t* d_busy2 = nullptr;       // [2*W] same, for the second kernel that walks this direction (dQ)
+    uint32_t* d_tile_ns = nullptr;     // [NT] time the last run spent on each tile (forward / fused backward), ns
     // pair tiles only (key block x query chunk x head): the "blocks" above are pair-blocks
     int chunk = 0;                     // tokens per query chunk
     int32_t* d_u_blk = nullptr;        // [NB] key block of pair-block u

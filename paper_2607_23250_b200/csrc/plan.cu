@@ -402,7 +402,7 @@ static inline unsigned grid_for(int64_t n, int block) { return (unsigned)((n + b
 
 static void free_dir(PlanDir& d) {
     cudaFree(d.d_weight_blk); cudaFree(d.d_blk_order); cudaFree(d.d_cta_of_tile); cudaFree(d.d_pos);
-    cudaFree(d.d_cta_offsets); cudaFree(d.d_cta_tiles); cudaFree(d.d_cta_exec); cudaFree(d.d_loads); cudaFree(d.d_busy); cudaFree(d.d_busy2);
+    cudaFree(d.d_cta_offsets); cudaFree(d.d_cta_tiles); cudaFree(d.d_cta_exec); cudaFree(d.d_loads); cudaFree(d.d_busy); cudaFree(d.d_busy2); cudaFree(d.d_tile_ns);
     cudaFree(d.d_u_blk); cudaFree(d.d_u_chunk);
     d = PlanDir();
 }
@@ -464,6 +464,7 @@ static int build_dir(libra_plan* p, PlanDir& d, int key_major, const libra_plan_
     A((void**)&d.d_loads, sizeof(int64_t) * d.W);
     A((void**)&d.d_busy, sizeof(uint64_t) * 2 * d.W);
     A((void**)&d.d_busy2, sizeof(uint64_t) * 2 * d.W);
+    A((void**)&d.d_tile_ns, sizeof(uint32_t) * d.NT);
     if (pairs) {
         A((void**)&d.d_u_blk, sizeof(int32_t) * d.NB);
         A((void**)&d.d_u_chunk, sizeof(int32_t) * d.NB);
@@ -472,6 +473,7 @@ static int build_dir(libra_plan* p, PlanDir& d, int key_major, const libra_plan_
     cudaStream_t s = p->stream;
     cudaMemsetAsync(d.d_busy, 0, sizeof(uint64_t) * 2 * d.W, s);
     cudaMemsetAsync(d.d_busy2, 0, sizeof(uint64_t) * 2 * d.W, s);
+    cudaMemsetAsync(d.d_tile_ns, 0, sizeof(uint32_t) * d.NT, s);
     if (pairs) {
         k_pair_fill<<<(unsigned)tb.NC, 128, 0, s>>>(p->d_tok_end, T, d.tile, d.chunk / d.tile, tb.NC, tb.first_j, tb.count,
                                                     tb.base, d.d_u_blk, d.d_u_chunk, d.d_weight_blk);
@@ -719,6 +721,16 @@ extern "C" int libra_busy_times(const libra_plan_t* plan, int which, uint64_t* n
     delete[] tmp;
     if (e != cudaSuccess) return LIBRA_ERR_CUDA;
     return st[which == LIBRA_KERNEL_FWD ? 1 : 2];
+}
+
+extern "C" int libra_tile_times(const libra_plan_t* plan, int which, uint32_t* ns_host) {
+    if (!plan || !ns_host) return LIBRA_ERR_INVALID_ARG;
+    if (which != LIBRA_KERNEL_FWD && which != LIBRA_KERNEL_BWD_FUSED) return LIBRA_ERR_INVALID_ARG;
+    PlanDir* d = dir_of(plan, which == LIBRA_KERNEL_BWD_FUSED ? LIBRA_DIR_PAIR : LIBRA_DIR_Q);
+    if (!d) return LIBRA_ERR_PLAN_MISMATCH;
+    if (cudaDeviceSynchronize() != cudaSuccess) return LIBRA_ERR_CUDA;
+    return cudaMemcpy(ns_host, d->d_tile_ns, sizeof(uint32_t) * d->NT, cudaMemcpyDeviceToHost) == cudaSuccess
+               ? LIBRA_OK : LIBRA_ERR_CUDA;
 }
 
 extern "C" int libra_plan_set_timing(libra_plan_t* plan, int enabled) {

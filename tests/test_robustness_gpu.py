@@ -172,3 +172,29 @@ def test_fused_backward_gives_up_cleanly_when_its_producer_stalls():
     for g, r in zip((dq, dk, dv), ref):
         assert np.abs(g.float().cpu().numpy() - r).max() <= 5e-2 * np.abs(r).max()
     plan.destroy()
+
+
+def test_tile_times_cover_every_tile_that_ran():
+    """Per-tile times of the forward (query-major tiles) and of the fused backward (pair tiles): every tile of the
+    plan has run, so every entry is positive, and no tile took longer than the CTA that ran it was busy."""
+    from paper_2607_23250_b200 import binding as lb
+    lengths = [700, 1, 300, 129, 411, 2000]
+    hq, hkv, d = 4, 2, 128
+    cu_np = pools.cu_seqlens(lengths)
+    t = pools.make_tensors(int(cu_np[-1]), hq, hkv, d, seed=5)
+    q, k, v, dout = (t[n].cuda() for n in ("q", "k", "v", "dout"))
+    plan = lb.libra_plan_tiles(torch.from_numpy(cu_np).cuda(), hq, 256, directions=lb.LIBRA_DIR_Q | lb.LIBRA_DIR_PAIR,
+                               tile_kv=128, n_heads_kv=hkv)
+    out, lse = lb.libra_attn_pool_fwd(q, k, v, plan)
+    lb.libra_attn_pool_bwd(q, k, v, out, lse, dout, plan)
+    torch.cuda.synchronize()
+    for kern, direction in ((lb.KERNEL_FWD, lb.LIBRA_DIR_Q), (lb.KERNEL_BWD_FUSED, lb.LIBRA_DIR_PAIR)):
+        ns = plan.tile_times(kern)
+        busy = plan.busy_times(kern)
+        ex = plan.export(direction)
+        assert len(ns) == plan.info(direction)["n_tiles"] and (ns > 0).all()
+        assert (ns.astype(np.int64) <= busy[ex["cta_of_tile"]].astype(np.int64)).all()
+    with pytest.raises(lb.LibraError) as err:
+        plan.tile_times(lb.KERNEL_BWD_DQ)
+    assert err.value.code == lb.ERR_INVALID_ARG
+    plan.destroy()
