@@ -199,7 +199,7 @@ size_t libra_attn_pool_bwd_workspace_bytes(const libra_plan_t* plan, const libra
  *   Fused form (plan with LIBRA_DIR_PAIR, tile_kv == 128, n_heads_kv == hkv, and head_dim 128): row statistics, one
  *   kernel that walks the pair-tile lists and computes S, dP, dV, dK and dQ of a cell together (five GEMMs per
  *   cell), and a conversion pass.  dK and dV of a pair tile accumulate on chip and are added to fp32 accumulators
- *   in the workspace when the tile ends; dQ of every cell is added to its fp32 accumulator by bulk reduce-adds.
+ *   in the workspace when the tile ends; dQ of every cell is added to its fp32 accumulator; all by bulk reduce-adds.
  *   The accumulators are rounded to bf16 once, at the end, so the result is at least as accurate as the two-kernel
  *   form's, but the order of the floating-point additions varies from run to run: results agree to rounding, not
  *   bit for bit.  The other directions of the plan are not used by this form.

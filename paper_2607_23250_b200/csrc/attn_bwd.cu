@@ -679,12 +679,14 @@ static int launch_fused(const void* q_dev, const void* k_dev, const void* v_dev,
     float* dq_acc = reinterpret_cast<float*>(ws_dev + 2 * ws.stat_bytes);
     float* dk_acc = reinterpret_cast<float*>(ws_dev + 2 * ws.stat_bytes + ws.dq_acc_bytes);
     float* dv_acc = reinterpret_cast<float*>(ws_dev + 2 * ws.stat_bytes + ws.dq_acc_bytes + ws.dkv_acc_bytes);
-    CUtensorMap tq, tk, tv, tdo, tacc;
+    CUtensorMap tq, tk, tv, tdo, tacc, tdkacc, tdvacc;
     int rc = make_thd_map(&tq, q_dev, T, dims->hq, 128, kBlk);
     if (rc == LIBRA_OK) rc = make_thd_map(&tk, k_dev, T, dims->hkv, 128, kBlk);
     if (rc == LIBRA_OK) rc = make_thd_map(&tv, v_dev, T, dims->hkv, 128, kBlk);
     if (rc == LIBRA_OK) rc = make_thd_map(&tdo, dout_dev, T, dims->hq, 128, kBlk);
     if (rc == LIBRA_OK) rc = make_f32_thd_map(&tacc, dq_acc, T, dims->hq);
+    if (rc == LIBRA_OK) rc = make_f32_thd_map(&tdkacc, dk_acc, T, dims->hkv);
+    if (rc == LIBRA_OK) rc = make_f32_thd_map(&tdvacc, dv_acc, T, dims->hkv);
     if (rc != LIBRA_OK) return rc;
     if (!cfg_done(4)) {
         if (set_smem(k_attn_bwd_fused, FusedSmem::kBytes) != LIBRA_OK) return LIBRA_ERR_CUDA;
@@ -711,7 +713,7 @@ static int launch_fused(const void* q_dev, const void* k_dev, const void* v_dev,
     fp.tile_ns = d.d_tile_ns;
     time_begin(mp, 4, s);
     cudaMemsetAsync(dq_acc, 0, ws.dq_acc_bytes + 2 * ws.dkv_acc_bytes, s);   // the three accumulators are contiguous
-    k_attn_bwd_fused<<<d.W, kFusedThreads, FusedSmem::kBytes, s>>>(tq, tk, tv, tdo, tacc, fp);
+    k_attn_bwd_fused<<<d.W, kFusedThreads, FusedSmem::kBytes, s>>>(tq, tk, tv, tdo, tacc, tdkacc, tdvacc, fp);
     time_end(mp, 4, s);
     time_begin(mp, 5, s);
     const int64_t nq8 = T * dims->hq * 128 / 8, nk8 = T * dims->hkv * 128 / 8;

@@ -138,7 +138,8 @@ __device__ __forceinline__ void fused_stage_dq(const CUtensorMap* tm, uint8_t* s
 __global__ void __launch_bounds__(kFusedThreads, 1)
 k_attn_bwd_fused(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                  const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do,
-                 const __grid_constant__ CUtensorMap tm_dqacc, const FusedParams p) {
+                 const __grid_constant__ CUtensorMap tm_dqacc, const __grid_constant__ CUtensorMap tm_dkacc,
+                 const __grid_constant__ CUtensorMap tm_dvacc, const FusedParams p) {
     using L = FusedSmem;
     constexpr int D = 128, QS = L::kQStages;
     extern __shared__ __align__(1024) uint8_t smem[];
@@ -210,6 +211,8 @@ k_attn_bwd_fused(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
         prefetch_tmap(&tm_v);
         prefetch_tmap(&tm_do);
         prefetch_tmap(&tm_dqacc);
+        prefetch_tmap(&tm_dkacc);
+        prefetch_tmap(&tm_dvacc);
     }
     tc_fence_before();
     __syncthreads();
@@ -548,23 +551,17 @@ k_attn_bwd_fused(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             tc_fence_after();
             const uint32_t t_dk = tmem_base + lane_addr + kColDK + c0;
             const uint32_t t_dv = tmem_base + lane_addr + kColDV + c0;
-            const size_t gofs = ((size_t)key * p.hkv + u.kvh) * D + c0;
+            // through the warp's staging tile, like dQ: bulk reduce-adds of 32 key rows x 32 head-dim columns (rows
+            // past the end of the pool are dropped by the hardware)
 #pragma unroll
             for (int which = 0; which < 2; ++which) {
-                float* gdst = (which == 0 ? p.dk_acc : p.dv_acc) + gofs;
 #pragma unroll
                 for (int cc = 0; cc < 64; cc += 32) {
                     uint32_t v[32];
                     tmem_ld32((which == 0 ? t_dk : t_dv) + cc, v);
                     tmem_ld_wait();
-                    if (key_ok) {
-#pragma unroll
-                        for (int i = 0; i < 32; i += 4)
-                            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(gdst + cc + i),
-                                         "f"(__uint_as_float(v[i])), "f"(__uint_as_float(v[i + 1])),
-                                         "f"(__uint_as_float(v[i + 2])), "f"(__uint_as_float(v[i + 3]))
-                                         : "memory");
-                    }
+                    fused_stage_dq(which == 0 ? &tm_dkacc : &tm_dvacc, stage, v, lane, c0 + cc, u.kvh,
+                                   (int)u.k0 + (warp & 3) * 32);
                 }
             }
             tc_fence_before();
