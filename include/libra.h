@@ -72,7 +72,7 @@ typedef struct libra_plan libra_plan_t;   /* opaque, library-owned */
 
 typedef struct {
     int     n_workers;     /* persistent CTAs to place onto; 0 = one per SM of the current device */
-    int     directions;    /* LIBRA_DIR_Q | LIBRA_DIR_KV; 0 = both                                  */
+    int     directions;    /* any of LIBRA_DIR_Q | LIBRA_DIR_KV | LIBRA_DIR_PAIR; 0 = Q and KV      */
     int     tile_kv;       /* key-major block size in tokens; 0 = 128                              */
     int     n_heads_kv;    /* key-major head shards; 0 = same as n_heads                           */
     int64_t total_tokens;  /* T if the caller knows it; 0 = read cu_seqlens[n] back (one 4-byte
