@@ -397,3 +397,51 @@ class Worker:
                     dv[tok0 - self.t0:tok0 - self.t0 + ntok, kvh] += f[pos + n:pos + 2 * n].reshape(ntok, L.head_dim)
                     pos += 2 * n
         return handles, finish
+
+
+def library_attention(device="cuda"):
+    """Attention callables for Worker that run the library's kernels on `device`.
+
+    The Worker hands a fragment (rows at sample positions a .. a + rows of a sample whose K / V prefix it has
+    assembled from local and received rows) in the worker's own memory; the fragment is copied to the device, the
+    query side is padded with zero rows in front so that it becomes one whole sample of a one-sample pool, and the
+    library plans and runs it.  Zero query rows with zero upstream gradient contribute nothing to dK / dV, so the
+    padded call returns exactly the fragment's partial sums.  Planning a pool per fragment is the simple form: it
+    serves to run the exchange with the real kernels; a production executor would batch a worker's fragments into
+    one pool per chunk."""
+    import torch
+    from . import binding as lb
+
+    def _plan(n, hq, hkv):
+        cu = torch.tensor([0, n], dtype=torch.int32, device=device)
+        return lb.libra_plan_tiles(cu, hq, 256, tile_kv=128, n_heads_kv=hkv, total_tokens=n)
+
+    def _dev(x, n=None, a=0):
+        y = x.to(device=device, dtype=torch.bfloat16)
+        if n is None:
+            return y.contiguous()
+        full = torch.zeros((n,) + tuple(x.shape[1:]), dtype=torch.bfloat16, device=device)
+        full[a:] = y
+        return full
+
+    def fwd(qf, k, v, a):
+        n = k.shape[0]
+        plan = _plan(n, qf.shape[1], k.shape[1])
+        out, lse = lb.libra_attn_pool_fwd(_dev(qf, n, a), _dev(k), _dev(v), plan)
+        torch.cuda.synchronize()
+        plan.busy_times(lb.KERNEL_FWD)
+        plan.destroy()
+        return out[a:].to("cpu", qf.dtype), lse[:, a:].cpu()
+
+    def bwd(qf, k, v, o, lse, do, a):
+        n = k.shape[0]
+        plan = _plan(n, qf.shape[1], k.shape[1])
+        lse_full = torch.zeros((qf.shape[1], n), dtype=torch.float32, device=device)
+        lse_full[:, a:] = lse.to(device)
+        dq, dk, dv = lb.libra_attn_pool_bwd(_dev(qf, n, a), _dev(k), _dev(v), _dev(o, n, a), lse_full, _dev(do, n, a), plan)
+        torch.cuda.synchronize()
+        plan.busy_times(lb.KERNEL_BWD_DQ)
+        plan.destroy()
+        return dq[a:].to("cpu", qf.dtype), dk.to("cpu", qf.dtype), dv.to("cpu", qf.dtype)
+
+    return fwd, bwd
