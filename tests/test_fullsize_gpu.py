@@ -30,10 +30,10 @@ def _rel(got, want, floor=1e-3):
 @pytest.fixture(scope="module",
                 params=[(2, 0.0, False), (2, 0.0, True), (3, 0.0, False), (3, 0.0, True), (4, 0.0, False), (4, 0.0, True),
                         (5, 0.0, False), (5, 0.25, False), (5, 0.5, False), (5, 1.0, False), (5, 1.0, True),
-                        (6, 0.0, False)],
+                        (6, 0.0, False), (6, 0.0, True)],
                 ids=["config2", "config2_fused", "config3", "config3_fused", "config4", "config4_fused",
                      "config5_skew0", "config5_skew0.25", "config5_skew0.5", "config5_skew1", "config5_skew1_fused",
-                     "config6_d256"])
+                     "config6_d256", "config6_d256_pairs"])
 def run(request):
     from paper_2607_23250_b200 import binding as lb
     fused = request.param[2]
@@ -52,6 +52,8 @@ def run(request):
     torch.cuda.synchronize()
     for kern in (lb.KERNEL_FWD,) + ((lb.KERNEL_BWD_FUSED,) if fused else (lb.KERNEL_BWD_DKDV, lb.KERNEL_BWD_DQ)):
         plan.busy_times(kern)
+    if fused and d == 256:
+        plan.busy_times(lb.KERNEL_BWD_DQ)       # at this width the dQ pass still walks the query-major lists
     res = dict(fused=fused, spec=spec, lengths=lengths, cu=cu_np, t=t, out=out, lse=lse, dq=dq, dk=dk, dv=dv, plan=plan, lb=lb)
     yield res
     plan.destroy()
